@@ -1,0 +1,459 @@
+/*
+ * Cascade scheduling + KV-tier step: CPU oracle (TEST INFRASTRUCTURE, not product code).
+ *
+ * Plain single-threaded C++17, sequential loops, std::stable_sort, memcpy.  No blocking,
+ * fusion or reordering: each function takes the steps in the order the method states them
+ * so that it can be checked against the paper by eye.  Only tests, the smoke check and the
+ * bench's CPU-baseline leg may call this file; the CUDA library never does.
+ *
+ * What the paper fixes and what it leaves open:
+ *   - Eq. 3 (effective latency), Eq. 4 (budget), Eq. 5 (remaining budget), Eq. 6 (restore
+ *     time), Eq. 7 (max restorable volume) and Algorithm 1 (queue tiers, least-remaining-
+ *     budget-first order, pop-while-capacity batch formation, largest-budget preemption)
+ *     are followed literally.
+ *   - The paper's latency estimator is an "offline-trained predictive model" with no printed
+ *     form.  The integer polynomial used here (iter_q / A / comp_q below) is this build's
+ *     reading; so are the token-granular admission scan, the Tier-2 reserve in tokens, the
+ *     decode-overrun penalty and the three-candidate restore-vs-recompute choice.
+ *
+ * Parity pins: every function here is pinned by tests/test_oracle_*.py (hand-worked values,
+ * closed forms, invariants, brute force on tiny inputs).  The paper's system-level results
+ * (goodput, violation rate, fairness index) need its traces and simulator: parity unpinned.
+ */
+#include "cascade_oracle.h"
+
+#include <algorithm>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+namespace {
+
+constexpr int64_t kBudgetClamp = int64_t(1) << 39; /* key holds budget in [-2^39, 2^39) ns   */
+constexpr uint32_t kIdMask = 0x7FFFFFu;            /* key holds the low 23 bits of the id     */
+constexpr int64_t kInvalidBudget = -(int64_t(1) << 62);
+
+struct Load {
+    int64_t D; /* decode sequences sharing the iteration */
+    int64_t K; /* their KV tokens                        */
+};
+
+/* Cost of one engine iteration that carries D decode sequences over K KV tokens (Q20 ns). */
+int64_t iter_q(const orc_params *p, Load l) { return p->c_iter_q20 + l.D * p->c_dseq_q20 + l.K * p->c_dkv_q20; }
+
+/* Cost per prefill token: its own linear cost plus its 1/chunk share of the iteration (Q20 ns). */
+int64_t tok_q(const orc_params *p, Load l) { return p->c_tok_q20 + (iter_q(p, l) >> p->chunk_shift); }
+
+/* Prefill compute for prompt tokens [s, P) when s tokens are already in the KV cache (Q20 ns). */
+int64_t comp_q(const orc_params *p, int64_t A, int64_t P, int64_t s) {
+    return A * (P - s) + p->c_attn_q20 * (P * P - s * s);
+}
+
+/* Eq. 6 in blocks: fixed overheads of the path plus per-block time; nothing to move costs nothing. */
+int64_t restore_time(const orc_params *p, int k, int64_t x) {
+    return x == 0 ? 0 : p->delta_ns[k] + x * p->blk_ns[k];
+}
+
+/* Eq. 7 in blocks: [rem - sum(delta)]^+ / per-block time, floored and capped at the nk blocks held. */
+int64_t max_restorable(const orc_params *p, int k, int64_t rem, int64_t nk) {
+    if (nk == 0) return 0;
+    int64_t head = rem - p->delta_ns[k];
+    if (head < 0) head = 0;
+    return std::min<int64_t>(nk, head / p->blk_ns[k]);
+}
+
+/* The two load regimes of Eq. 3: actual load, and B_max - 1 concurrent decodes (never below actual). */
+Load load_act(int32_t D_act, int64_t K_act) { return Load{D_act, K_act}; }
+Load load_max(const orc_params *p, int32_t D_act, int64_t K_act) {
+    int64_t Dm = std::max<int64_t>(D_act, p->max_batch - 1);
+    int64_t Km = std::max<int64_t>(K_act, int64_t(p->max_batch - 1) * p->max_ctx_avg);
+    return Load{Dm, Km};
+}
+
+/* Input bounds every step relies on (prompt <= 2^17, hits <= 2^13 blocks, at least one
+ * prompt token left to compute). */
+bool request_valid(const orc_params *p, int64_t P, int64_t n0, int64_t n1, int64_t n2) {
+    if (P < 1 || P > (int64_t(1) << 17)) return false;
+    if (n0 < 0 || n1 < 0 || n2 < 0) return false;
+    if (n0 + n1 + n2 > (int64_t(1) << 13)) return false;
+    return (n0 + n1 + n2) * p->bt < P;
+}
+
+int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+/* F(x1, x2): predicted completion time (Q20 ns, exact) when x1 host blocks and x2 deep blocks
+ * are restored and the rest of the prompt is recomputed under the actual load. */
+int64_t plan_cost_q20(const orc_params *p, Load act, int64_t P, int64_t n0, int64_t x1, int64_t x2) {
+    int64_t transfer = restore_time(p, 1, x1) + restore_time(p, 2, x2);
+    return (transfer << 20) + comp_q(p, tok_q(p, act), P, (n0 + x1 + x2) * p->bt);
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t orc_restore_time(const orc_params *p, int k, int64_t x_blocks) { return restore_time(p, k, x_blocks); }
+
+int64_t orc_max_restorable(const orc_params *p, int k, int64_t rem_ns, int64_t nk) {
+    return max_restorable(p, k, rem_ns, nk);
+}
+
+int64_t orc_plan_cost_q20(const orc_params *p, int32_t D_act, int64_t K_act, int32_t prompt, int32_t n0, int32_t x1,
+                          int32_t x2) {
+    return plan_cost_q20(p, load_act(D_act, K_act), prompt, n0, x1, x2);
+}
+
+uint32_t orc_budget(const orc_params *p, int n, const int64_t *arrival_ns, const int32_t *prompt,
+                    const int32_t *pred_out, const int32_t *n0, const int32_t *n1, const int32_t *n2,
+                    const uint32_t *id, const uint8_t *cls, int64_t now_ns, int32_t D_act, int64_t K_act,
+                    int64_t *budget_out, uint64_t *key_out) {
+    uint32_t status = 0;
+    const Load act = load_act(D_act, K_act);
+    const Load mx = load_max(p, D_act, K_act);
+    for (int r = 0; r < n; ++r) {
+        const int64_t P = prompt[r];
+        const int64_t O = pred_out[r];
+        const int64_t elapsed = now_ns - arrival_ns[r];
+        bool ok = request_valid(p, P, n0[r], n1[r], n2[r]);
+        ok = ok && O >= 0 && O <= (int64_t(1) << 20);
+        ok = ok && cls[r] < p->n_classes;
+        ok = ok && elapsed <= (int64_t(1) << 50) && elapsed >= -(int64_t(1) << 50);
+        if (!ok) {
+            /* flagged; parked at the very end of the Tier-2 queue */
+            status |= ORC_ST_EPRECOND;
+            budget_out[r] = kInvalidBudget;
+            key_out[r] = (uint64_t(1) << 63) | uint64_t(id[r] & kIdMask);
+            continue;
+        }
+        /* B1: tokens of the prompt already cached in some tier */
+        const int64_t s_hit = int64_t(n0[r] + n1[r] + n2[r]) * p->bt;
+        /* B2: tier-priced transfer of the matched non-HBM prefix plus the compute of the rest,
+         *     under the actual and under the maximum load */
+        const int64_t tp = restore_time(p, 1, n1[r]) + restore_time(p, 2, n2[r]);
+        const int64_t L_act = tp + (comp_q(p, tok_q(p, act), P, s_hit) >> 20);
+        const int64_t L_max = tp + (comp_q(p, tok_q(p, mx), P, s_hit) >> 20);
+        /* B3 (Eq. 3): L = (L_act + L_max)/2 * gamma, floored */
+        const int64_t L = ((L_act + L_max) * p->gamma_q16) >> 17;
+        /* B4 (Eq. 4, Eq. 5): budget against the class TTFT target; queue tier; remaining budget */
+        const int64_t B = p->ttft_ns[cls[r]] - L;
+        const int tier = (B > 0) ? 1 : 2;
+        const int64_t B_rem = B - elapsed;
+        /* B5: decode-overrun penalty from the predicted output length */
+        const Load act1{act.D + 1, act.K + P};
+        const Load mx1{mx.D + 1, mx.K + P};
+        const int64_t chunk_q = p->c_tok_q20 << p->chunk_shift;
+        const int64_t tdec_act = (iter_q(p, act1) + chunk_q) >> 20;
+        const int64_t tdec_max = (iter_q(p, mx1) + chunk_q) >> 20;
+        const int64_t tdec = ((tdec_act + tdec_max) * p->gamma_q16) >> 17;
+        const int64_t tpot = p->tpot_ns[cls[r]];
+        int64_t pen = 0;
+        if (tpot != 0) pen = O * std::max<int64_t>(0, tdec - tpot);
+        const int64_t budget = B_rem - pen;
+        /* B6: 64-bit key = (tier-2 bit, clamped budget, arrival id) */
+        int64_t u = std::min(std::max(budget, -kBudgetClamp), kBudgetClamp - 1) + kBudgetClamp;
+        budget_out[r] = budget;
+        key_out[r] = (uint64_t(tier == 2) << 63) | (uint64_t(u) << 23) | uint64_t(id[r] & kIdMask);
+    }
+    return status;
+}
+
+uint32_t orc_schedule(const orc_params *p, int n, const uint64_t *key, const int32_t *prompt, const int32_t *n0,
+                      const int32_t *n1, const int32_t *n2, int32_t D_act, uint32_t *order_out, int32_t *grant_out,
+                      orc_sched_counts *counts) {
+    /* S1: ascending by key; equal keys keep slot order */
+    std::vector<uint32_t> order(n);
+    std::iota(order.begin(), order.end(), 0u);
+    std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return key[a] < key[b]; });
+
+    /* S2: tokens each request would compute if its whole matched prefix is reused */
+    std::vector<int64_t> want(n);
+    for (int r = 0; r < n; ++r) {
+        if (request_valid(p, prompt[r], n0[r], n1[r], n2[r]))
+            want[r] = int64_t(prompt[r]) - int64_t(n0[r] + n1[r] + n2[r]) * p->bt;
+        else
+            want[r] = 0;
+    }
+    /* every in-flight decode sequence takes one token of the iteration */
+    const int64_t TB = std::max<int64_t>(0, int64_t(p->token_budget) - D_act);
+    int n_t1 = 0;
+    int64_t W2 = 0;
+    for (int i = 0; i < n; ++i) {
+        uint32_t r = order[i];
+        if (key[r] >> 63)
+            W2 += want[r];
+        else
+            ++n_t1;
+    }
+    const int64_t R2 = std::min<int64_t>(std::min<int64_t>(p->tier2_reserve, W2), TB);
+    /* Tier-1 queue: pop in order, give each request what is left of the Tier-1 share */
+    int64_t left = TB - R2;
+    int64_t used1 = 0;
+    for (int i = 0; i < n_t1; ++i) {
+        uint32_t r = order[i];
+        int64_t g = std::min(want[r], left);
+        grant_out[r] = int32_t(g);
+        left -= g;
+        used1 += g;
+    }
+    /* Tier-2 queue: the reserve plus whatever Tier-1 left */
+    left = TB - used1;
+    for (int i = n_t1; i < n; ++i) {
+        uint32_t r = order[i];
+        int64_t g = std::min(want[r], left);
+        grant_out[r] = int32_t(g);
+        left -= g;
+    }
+    /* S3: at most max_batch sequences per iteration, decodes included */
+    const int64_t seq_cap = std::max<int64_t>(0, int64_t(p->max_batch) - D_act);
+    int64_t rank = 0;
+    int32_t n_adm = 0;
+    int64_t tokens = 0;
+    for (int i = 0; i < n; ++i) {
+        uint32_t r = order[i];
+        if (grant_out[r] > 0) {
+            if (rank >= seq_cap) grant_out[r] = 0;
+            ++rank;
+        }
+        if (grant_out[r] > 0) {
+            ++n_adm;
+            tokens += grant_out[r];
+        }
+    }
+    for (int i = 0; i < n; ++i) order_out[i] = order[i];
+    counts->n_tier1 = n_t1;
+    counts->n_admitted = n_adm;
+    counts->tokens_granted = tokens;
+    return 0;
+}
+
+uint32_t orc_tier_plan(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
+                       const int32_t *n2, const uint8_t *flags, const int64_t *budget, const uint32_t *order,
+                       int32_t *grant, int32_t D_act, int64_t K_act, int32_t *hbm_tbl, int32_t *host_tbl,
+                       int32_t maxb, int32_t *hbm_free, int32_t *hbm_free_count, int32_t hbm_free_cap,
+                       int32_t *host_free, int32_t *host_free_count, int32_t host_free_cap, int32_t *x1_out,
+                       int32_t *x2_out, int32_t *tokens_run_out, uint8_t *action_out, int32_t *restore_src,
+                       int32_t *restore_dst, int32_t restore_cap, int32_t *evict_src, int32_t *evict_dst,
+                       int32_t evict_cap, orc_plan_counts *counts) {
+    uint32_t status = 0;
+    const bool with_tables = hbm_tbl != nullptr;
+    const Load act = load_act(D_act, K_act);
+
+    int64_t hbm_cnt = *hbm_free_count;
+    int64_t host_cnt = *host_free_count;
+    if (with_tables) {
+        if (hbm_cnt < 0 || hbm_cnt > hbm_free_cap) {
+            status |= ORC_ST_EBOUNDS;
+            hbm_cnt = std::min<int64_t>(std::max<int64_t>(hbm_cnt, 0), hbm_free_cap);
+        }
+        if (host_cnt < 0 || host_cnt > host_free_cap) {
+            status |= ORC_ST_EBOUNDS;
+            host_cnt = std::min<int64_t>(std::max<int64_t>(host_cnt, 0), host_free_cap);
+        }
+    }
+
+    /* requests the plan may touch: inside the input bounds and, with tables, inside a table row */
+    std::vector<uint8_t> valid(n);
+    for (int r = 0; r < n; ++r) {
+        bool ok = request_valid(p, prompt[r], n0[r], n1[r], n2[r]);
+        if (ok && with_tables) ok = ceil_div(prompt[r], p->bt) <= maxb;
+        valid[r] = ok;
+        if (!ok) {
+            status |= ORC_ST_EPRECOND;
+            grant[r] = 0;
+        }
+    }
+
+    /* P1 + P2 for every admitted request */
+    std::vector<int32_t> need(n, 0);
+    for (int r = 0; r < n; ++r) {
+        x1_out[r] = 0;
+        x2_out[r] = 0;
+        tokens_run_out[r] = 0;
+        action_out[r] = ORC_ACT_NONE;
+        if (!valid[r] || grant[r] <= 0) continue;
+        const int64_t P = prompt[r];
+        /* P1 (Eq. 7): host first, deep tier from what is left and only behind a fully restored host segment */
+        const int64_t rem = std::max<int64_t>(0, budget[r]);
+        const int64_t x1max = max_restorable(p, 1, rem, n1[r]);
+        int64_t x2max = 0;
+        if (x1max == n1[r] && n2[r] > 0) {
+            const int64_t rem2 = rem - restore_time(p, 1, n1[r]);
+            x2max = max_restorable(p, 2, rem2, n2[r]);
+        }
+        /* P2: smallest predicted completion time over the endpoint candidates; ties restore more */
+        int64_t bx1 = 0, bx2 = 0;
+        int64_t bF = plan_cost_q20(p, act, P, n0[r], 0, 0);
+        if (x1max > 0) {
+            const int64_t F = plan_cost_q20(p, act, P, n0[r], x1max, 0);
+            if (F <= bF) { bF = F; bx1 = x1max; bx2 = 0; }
+        }
+        if (x2max > 0) {
+            const int64_t F = plan_cost_q20(p, act, P, n0[r], n1[r], x2max);
+            if (F <= bF) { bF = F; bx1 = n1[r]; bx2 = x2max; }
+        }
+        x1_out[r] = int32_t(bx1);
+        x2_out[r] = int32_t(bx2);
+        /* a deep fetch is staged first: nothing runs this iteration, HBM is taken only at the last hop */
+        const int64_t have = (n0[r] + bx1) * int64_t(p->bt);
+        const int64_t run = (bx2 > 0) ? 0 : std::min<int64_t>(grant[r], P - have);
+        tokens_run_out[r] = int32_t(run);
+        need[r] = int32_t(bx1 + (ceil_div(have + run, p->bt) - (n0[r] + bx1)));
+    }
+
+    /* P3: HBM capacity.  Only blocks of non-admitted private holders can be freed. */
+    int64_t evictable = 0;
+    for (int r = 0; r < n; ++r)
+        if (valid[r] && grant[r] <= 0 && (flags[r] & ORC_FLAG_HBM_PRIVATE)) evictable += n0[r];
+    const int64_t cap = hbm_cnt + evictable;
+    int64_t c = 0, need_total = 0;
+    int32_t n_unadmitted = 0;
+    for (int i = 0; i < n; ++i) {
+        const uint32_t r = order[i];
+        if (!valid[r] || grant[r] <= 0) continue;
+        c += need[r];
+        if (c > cap) {
+            grant[r] = 0;
+            x1_out[r] = x2_out[r] = tokens_run_out[r] = 0;
+            need[r] = 0;
+            ++n_unadmitted;
+            status |= ORC_ST_ENOSPC;
+        } else {
+            need_total += need[r];
+        }
+    }
+    const int64_t deficit = std::max<int64_t>(0, need_total - hbm_cnt);
+
+    /* P4 + P5: victims, walking the order backwards (last to be served first) */
+    std::vector<uint32_t> victims;
+    {
+        int64_t v = 0; /* blocks of eligible requests visited so far    */
+        int64_t h = 0; /* blocks of victims that fit, visited so far     */
+        for (int i = n - 1; i >= 0; --i) {
+            const uint32_t r = order[i];
+            const bool eligible = valid[r] && grant[r] <= 0 && (flags[r] & ORC_FLAG_HBM_PRIVATE) && n0[r] > 0;
+            if (!eligible) continue;
+            if (v < deficit) {
+                /* spill only if it could be brought back within the victim's own budget, and host has room */
+                const bool fits = restore_time(p, 1, n0[r]) <= budget[r];
+                if (fits && h + n0[r] <= host_cnt)
+                    action_out[r] = ORC_ACT_EVICT;
+                else
+                    action_out[r] = ORC_ACT_DROP;
+                if (fits) h += n0[r];
+                victims.push_back(r);
+            }
+            v += n0[r];
+        }
+    }
+    for (int r = 0; r < n; ++r)
+        if (valid[r] && action_out[r] == ORC_ACT_NONE && n0[r] > 0) action_out[r] = ORC_ACT_RETAIN;
+
+    /* P6 / K1: block ids.  Free lists are stacks; all pushes precede all pops. */
+    int32_t n_restore = 0, n_evict = 0, n_drop = 0;
+    int64_t hbm_pos = hbm_cnt, host_pos = host_cnt;
+    auto hbm_push = [&](int32_t v) {
+        if (with_tables) {
+            if (hbm_pos < hbm_free_cap) hbm_free[hbm_pos] = v; else status |= ORC_ST_EBOUNDS;
+        }
+        ++hbm_pos;
+    };
+    auto hbm_pop = [&]() -> int32_t {
+        --hbm_pos;
+        if (!with_tables) return -1;
+        if (hbm_pos < hbm_free_cap) return hbm_free[hbm_pos];
+        status |= ORC_ST_EBOUNDS;
+        return -1;
+    };
+    for (uint32_t r : victims) {
+        for (int j = 0; j < n0[r]; ++j) {
+            const int32_t g = with_tables ? hbm_tbl[int64_t(r) * maxb + j] : -1;
+            if (action_out[r] == ORC_ACT_EVICT) {
+                --host_pos;
+                if (with_tables) {
+                    const int32_t hslot = host_free[host_pos];
+                    if (n_evict < evict_cap) { evict_src[n_evict] = g; evict_dst[n_evict] = hslot; }
+                    else status |= ORC_ST_ELISTCAP;
+                    host_tbl[int64_t(r) * maxb + j] = hslot;
+                }
+                ++n_evict;
+            } else {
+                ++n_drop;
+            }
+            hbm_push(g);
+            if (with_tables) hbm_tbl[int64_t(r) * maxb + j] = -1;
+        }
+    }
+    int32_t n_admitted = 0;
+    int64_t tokens_run = 0;
+    for (int i = 0; i < n; ++i) {
+        const uint32_t r = order[i];
+        if (!valid[r] || grant[r] <= 0) continue;
+        ++n_admitted;
+        tokens_run += tokens_run_out[r];
+        for (int j = n0[r]; j < n0[r] + need[r]; ++j) {
+            const int32_t g = hbm_pop();
+            if (j < n0[r] + x1_out[r]) {
+                if (with_tables) {
+                    if (n_restore < restore_cap) { restore_src[n_restore] = host_tbl[int64_t(r) * maxb + j]; restore_dst[n_restore] = g; }
+                    else status |= ORC_ST_ELISTCAP;
+                }
+                ++n_restore;
+            }
+            if (with_tables) hbm_tbl[int64_t(r) * maxb + j] = g;
+        }
+    }
+    if (with_tables) {
+        *hbm_free_count = int32_t(hbm_pos);
+        *host_free_count = int32_t(host_pos);
+    }
+    counts->n_restore = n_restore;
+    counts->n_evict = n_evict;
+    counts->n_drop_blocks = n_drop;
+    counts->n_victims = int32_t(victims.size());
+    counts->n_unadmitted = n_unadmitted;
+    counts->n_admitted = n_admitted;
+    counts->hbm_need = int32_t(need_total);
+    counts->deficit = int32_t(deficit);
+    counts->hbm_free_after = int32_t(hbm_pos);
+    counts->host_free_after = int32_t(host_pos);
+    counts->tokens_run = tokens_run;
+    return status;
+}
+
+uint32_t orc_kv_restore(uint8_t *hbm_pool, int64_t hbm_blocks, int32_t n_chunks, int64_t chunk_bytes,
+                        int64_t chunk_stride, int64_t block_stride, const uint8_t *host_pool, int64_t host_blocks,
+                        const int32_t *src_ids, const int32_t *dst_ids, int n_copies) {
+    uint32_t status = 0;
+    const int64_t bb = int64_t(n_chunks) * chunk_bytes;
+    for (int i = 0; i < n_copies; ++i) {
+        const int64_t s = src_ids[i], d = dst_ids[i];
+        if (s < 0 || s >= host_blocks || d < 0 || d >= hbm_blocks) {
+            status |= ORC_ST_EBOUNDS;
+            continue;
+        }
+        for (int c = 0; c < n_chunks; ++c)
+            std::memcpy(hbm_pool + c * chunk_stride + d * block_stride, host_pool + s * bb + c * chunk_bytes,
+                        size_t(chunk_bytes));
+    }
+    return status;
+}
+
+uint32_t orc_kv_evict(const uint8_t *hbm_pool, int64_t hbm_blocks, int32_t n_chunks, int64_t chunk_bytes,
+                      int64_t chunk_stride, int64_t block_stride, uint8_t *host_pool, int64_t host_blocks,
+                      const int32_t *src_ids, const int32_t *dst_ids, int n_copies) {
+    uint32_t status = 0;
+    const int64_t bb = int64_t(n_chunks) * chunk_bytes;
+    for (int i = 0; i < n_copies; ++i) {
+        const int64_t s = src_ids[i], d = dst_ids[i];
+        if (s < 0 || s >= hbm_blocks || d < 0 || d >= host_blocks) {
+            status |= ORC_ST_EBOUNDS;
+            continue;
+        }
+        for (int c = 0; c < n_chunks; ++c)
+            std::memcpy(host_pool + d * bb + c * chunk_bytes, hbm_pool + c * chunk_stride + s * block_stride,
+                        size_t(chunk_bytes));
+    }
+    return status;
+}
+
+}  // extern "C"

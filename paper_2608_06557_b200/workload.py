@@ -1,0 +1,265 @@
+"""Seeded synthetic workloads for the Cascade scheduling + KV-tier step.
+
+This module only DRAWS inputs (numpy, ``default_rng(seed)``): request arrays, class tables,
+block tables, free lists, copy lists and pool byte patterns.  It holds none of the method's
+arithmetic and is the one module shared by the CUDA tests/bench and the CPU oracle's tests.
+
+The paper evaluates on production traces that are not available here; these inputs stand in
+for them with the same kind of structure: heterogeneous (lognormal) prompt and output
+lengths, mixed SLO classes, partial prefix reuse split between HBM and host DRAM.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+Q20 = 1 << 20
+FLAG_HBM_PRIVATE, FLAG_RUNNING = 1, 2
+MS = 1_000_000
+S = 1_000_000_000
+
+
+def default_params(**over) -> dict:
+    """Cost-model and policy parameters (synthetic; the paper prints no coefficients)."""
+    d = dict(
+        bt=16, chunk_shift=9, max_batch=128, max_ctx_avg=2048, gamma_q16=81920,
+        token_budget=2048, tier2_reserve=256,
+        c_tok_q20=50_000 * Q20, c_attn_q20=Q20 // 2, c_iter_q20=2_000_000 * Q20,
+        c_dseq_q20=10_000 * Q20, c_dkv_q20=20 * Q20,
+        delta_ns=[0, 10_000, 110_000], blk_ns=[0, 40_000, 340_000],
+        ttft_ns=[1 * S], tpot_ns=[50 * MS],
+    )
+    d.update(over)
+    return d
+
+
+def kv_layout(n_blocks: int, n_chunks: int, chunk_bytes: int) -> dict:
+    """Layer-major paged HBM pool: chunk c of block b at c*chunk_stride + b*block_stride."""
+    return dict(n_blocks=n_blocks, n_chunks=n_chunks, chunk_bytes=chunk_bytes,
+                chunk_stride=n_blocks * chunk_bytes, block_stride=chunk_bytes)
+
+
+def splitmix64(x: np.ndarray) -> np.ndarray:
+    """Counter-based 64-bit mixer used for pool byte patterns (uint64 in, uint64 out)."""
+    x = (x + np.uint64(0x9E3779B97F4A7C15)).astype(np.uint64)
+    x = (x ^ (x >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+    x = (x ^ (x >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+    return x ^ (x >> np.uint64(31))
+
+
+def pool_bytes(tag: int, n_bytes: int) -> np.ndarray:
+    """Deterministic byte pattern of a pool: word i = splitmix64(tag * 2^40 + i)."""
+    assert n_bytes % 8 == 0
+    with np.errstate(over="ignore"):
+        w = splitmix64(np.arange(n_bytes // 8, dtype=np.uint64) + (np.uint64(tag) << np.uint64(40)))
+    return w.view(np.uint8)
+
+
+@dataclass
+class Workload:
+    """One iteration's inputs.  Arrays are host numpy; the caller moves them where needed."""
+    name: str
+    params: dict
+    reqs: dict                    # arrival_ns i64, prompt/pred_out/n0/n1/n2 i32, id u32, cls/flags u8
+    now_ns: int
+    D_act: int
+    K_act: int
+    layout: dict | None = None    # HBM pool layout
+    host_blocks: int = 0
+    maxb: int = 0
+    hbm_tbl: np.ndarray | None = None
+    host_tbl: np.ndarray | None = None
+    hbm_free: np.ndarray | None = None   # stack storage sized to the pool; top = [count-1]
+    hbm_free_count: int = 0
+    host_free: np.ndarray | None = None
+    host_free_count: int = 0
+    notes: dict = field(default_factory=dict)
+
+    @property
+    def n(self) -> int:
+        return len(self.reqs["prompt"])
+
+    @property
+    def block_bytes(self) -> int:
+        return self.layout["n_chunks"] * self.layout["chunk_bytes"]
+
+
+def _lognormal_int(rng, median, sigma, lo, hi, n):
+    v = np.exp(rng.normal(np.log(median), sigma, n))
+    return np.clip(np.rint(v), lo, hi).astype(np.int32)
+
+
+def draw_requests(rng, n, class_mix, ttft_ns, prompt_median, prompt_clip, out_median_by_class, out_clip,
+                  now_ns, elapsed_scale, hit_draw, hbm_share, bt, id0=0):
+    """Request fields of the SoA arrays.  ``hit_draw(rng, n)`` gives the reused fraction in [0,1];
+    ``hbm_share`` of the reused blocks sit in HBM (the head of the prefix), the rest on host."""
+    cls = rng.choice(len(class_mix), size=n, p=np.asarray(class_mix, float)).astype(np.uint8)
+    prompt = _lognormal_int(rng, prompt_median, 1.0, prompt_clip[0], prompt_clip[1], n)
+    med = np.asarray(out_median_by_class, float)[cls]
+    pred_out = np.clip(np.rint(np.exp(rng.normal(np.log(med), 1.0))), out_clip[0], out_clip[1]).astype(np.int32)
+    if elapsed_scale is None:          # C1: uniform in [0, 2 s]
+        elapsed = rng.uniform(0, 2 * S, n)
+    else:                              # uniform in [0, elapsed_scale * TTFT_c]
+        elapsed = rng.uniform(0, 1, n) * elapsed_scale * np.asarray(ttft_ns, float)[cls]
+    arrival = (now_ns - np.rint(elapsed)).astype(np.int64)
+    frac = hit_draw(rng, n)
+    max_hit = (prompt - 1) // bt       # at least one prompt token is always computed
+    hit = np.minimum(np.floor(frac * (prompt // bt)).astype(np.int64), max_hit).astype(np.int32)
+    n0 = np.ceil(hit * hbm_share).astype(np.int32)
+    n0 = np.minimum(n0, hit)
+    n1 = (hit - n0).astype(np.int32)
+    n2 = np.zeros(n, np.int32)
+    ids = (np.arange(n, dtype=np.uint32) + np.uint32(id0))
+    flags = np.zeros(n, np.uint8)
+    return dict(arrival_ns=arrival, prompt=prompt, pred_out=pred_out, n0=n0, n1=n1, n2=n2, id=ids, cls=cls,
+                flags=flags)
+
+
+def place_blocks(rng, reqs, n_hbm, n_host, maxb, occupancy, hbm_free_target, private_prob):
+    """Give every hit block an id, request by request, until a pool reaches ``occupancy``; later hits
+    in that tier are truncated.  Then other tenants' blocks are taken out of the HBM free list until
+    ``hbm_free_target`` ids are left.  Returns tables and free-list stacks."""
+    n = len(reqs["prompt"])
+    hbm_ids = rng.permutation(n_hbm).astype(np.int32)
+    host_ids = rng.permutation(n_host).astype(np.int32)
+    hbm_lim, host_lim = int(n_hbm * occupancy), int(n_host * occupancy)
+    hbm_used = host_used = 0
+    hbm_tbl = np.full((n, maxb), -1, np.int32)
+    host_tbl = np.full((n, maxb), -1, np.int32)
+    n0, n1 = reqs["n0"], reqs["n1"]
+    for r in range(n):
+        a = min(int(n0[r]), hbm_lim - hbm_used)
+        if a < n0[r]:                  # HBM prefix cut short: the host part would not be contiguous
+            n0[r], n1[r] = a, 0
+        hbm_tbl[r, :a] = hbm_ids[hbm_used:hbm_used + a]
+        hbm_used += a
+        b = min(int(n1[r]), host_lim - host_used)
+        n1[r] = b
+        host_tbl[r, a:a + b] = host_ids[host_used:host_used + b]
+        host_used += b
+    has = n0 > 0
+    private = has & (rng.uniform(0, 1, n) < private_prob)
+    reqs["flags"][private] |= FLAG_HBM_PRIVATE | FLAG_RUNNING
+    hbm_free_count = min(n_hbm - hbm_used, hbm_free_target)
+    hbm_free = np.full(n_hbm, -1, np.int32)
+    hbm_free[:hbm_free_count] = hbm_ids[n_hbm - hbm_free_count:]
+    host_free_count = n_host - host_used
+    host_free = np.full(n_host, -1, np.int32)
+    host_free[:host_free_count] = host_ids[host_used:]
+    return hbm_tbl, host_tbl, hbm_free, hbm_free_count, host_free, host_free_count
+
+
+def config_tiny(seed: int = 0) -> Workload:
+    """64 requests, two SLO classes, 16 KiB blocks, 512+512 block pools, one iteration."""
+    rng = np.random.default_rng(seed)
+    ttft = [S // 2, 5 * S]
+    params = default_params(ttft_ns=ttft, tpot_ns=[50 * MS, 50 * MS], token_budget=2048, tier2_reserve=256,
+                            max_batch=128)
+    bb = 16384  # 2 layers x (K,V) x 2 KV heads x 64 dim x 2 B (bf16) x 16 tokens = 16 KiB
+    n_chunks, chunk_bytes = 4, bb // 4
+    params["blk_ns"] = [0, -(-bb * 1_000_000_000 // 50_000_000_000), 340_000]
+    now = 10 * S
+    reqs = draw_requests(rng, 64, [0.5, 0.5], ttft, 256, (16, 2048), [128, 128], (1, 4096), now, None,
+                         lambda g, n: g.uniform(0, 1, n), 0.5, params["bt"])
+    maxb = 128
+    tbl = place_blocks(rng, reqs, 512, 512, maxb, 1.0, 32, 0.5)
+    return Workload("tiny", params, reqs, now, 8, 8 * 512, kv_layout(512, n_chunks, chunk_bytes), 512, maxb, *tbl)
+
+
+LLAMA8B_CLASSES = dict(mix=[0.6, 0.3, 0.1], ttft=[1 * S, 3 * S, 30 * S], out_median=[256, 256, 4096])
+
+
+def config_llama8b(seed: int = 0, n: int = 1024, hbm_bytes: int = 60 * 10**9, host_bytes: int = 40 * 10**9,
+                   hbm_free_target: int = 256) -> Workload:
+    """Llama-3-8B-shaped KV (2 MiB blocks: 64 chunks of 32 KiB), three SLO classes, beta(2,2) reuse."""
+    rng = np.random.default_rng(seed)
+    c = LLAMA8B_CLASSES
+    n_chunks, chunk_bytes = 64, 32 * 1024
+    bb = n_chunks * chunk_bytes
+    params = default_params(ttft_ns=c["ttft"], tpot_ns=[50 * MS] * 3, token_budget=8192, tier2_reserve=1024,
+                            max_batch=128)
+    params["blk_ns"] = [0, -(-bb * 1_000_000_000 // 50_000_000_000), 10 * -(-bb * 1_000_000_000 // 50_000_000_000)]
+    now = 100 * S
+    reqs = draw_requests(rng, n, c["mix"], c["ttft"], 1024, (32, 32768), c["out_median"], (1, 65536), now, 1.5,
+                         lambda g, m: g.beta(2, 2, m), 0.5, params["bt"])
+    n_hbm, n_host = hbm_bytes // bb, host_bytes // bb
+    maxb = 2048
+    tbl = place_blocks(rng, reqs, n_hbm, n_host, maxb, 0.9, hbm_free_target, 0.5)
+    return Workload("llama8b", params, reqs, now, 64, 64 * 2048, kv_layout(n_hbm, n_chunks, chunk_bytes), n_host,
+                    maxb, *tbl)
+
+
+class SchedulerSweep:
+    """Scheduler-scale sweep: budget + order + admission + plan only (no tables, no copies).
+
+    ``n`` live requests drawn as in the Llama-3-8B-shaped configuration; the load comes from 256
+    in-flight decode sequences.  Every iteration the clock advances 25 ms, a seeded 5 % of the
+    slots are replaced by fresh arrivals and 5 % of the decode contexts are replaced; the rest of
+    the contexts grow by one token."""
+
+    def __init__(self, n: int, seed: int = 0):
+        self.rng = np.random.default_rng(seed)
+        c = LLAMA8B_CLASSES
+        self.n = n
+        bb = 64 * 32 * 1024
+        self.params = default_params(ttft_ns=c["ttft"], tpot_ns=[50 * MS] * 3, token_budget=8192,
+                                     tier2_reserve=1024, max_batch=512)
+        self.params["blk_ns"] = [0, -(-bb * 1_000_000_000 // 50_000_000_000), 420_000]
+        self.now = 100 * S
+        self.reqs = self._draw(n, 0)
+        self.next_id = n
+        self.ctx = self._draw_ctx(256)
+        self.hbm_free_count = 1 << 30
+        self.host_free_count = 1 << 30
+
+    def _draw(self, m, id0, fresh=False):
+        c = LLAMA8B_CLASSES
+        r = draw_requests(self.rng, m, c["mix"], c["ttft"], 1024, (32, 32768), c["out_median"], (1, 65536),
+                          self.now, 0.0 if fresh else 1.5, lambda g, k: g.beta(2, 2, k), 0.5, self.params["bt"], id0)
+        has = r["n0"] > 0
+        r["flags"][has & (self.rng.uniform(0, 1, m) < 0.5)] |= FLAG_HBM_PRIVATE | FLAG_RUNNING
+        return r
+
+    def _draw_ctx(self, m):
+        c = LLAMA8B_CLASSES
+        r = draw_requests(self.rng, m, c["mix"], c["ttft"], 1024, (32, 32768), c["out_median"], (1, 65536),
+                          self.now, 1.5, lambda g, k: g.beta(2, 2, k), 0.5, self.params["bt"])
+        return r["prompt"].astype(np.int64) + np.floor(self.rng.uniform(0, 1, m) * r["pred_out"]).astype(np.int64)
+
+    @property
+    def D_act(self) -> int:
+        return len(self.ctx)
+
+    @property
+    def K_act(self) -> int:
+        return int(self.ctx.sum())
+
+    def step(self):
+        """Advance one iteration.  Returns the slot indices that were rewritten."""
+        self.now += 25 * MS
+        m = max(1, self.n // 20)
+        slots = self.rng.choice(self.n, size=m, replace=False)
+        fresh = self._draw(m, self.next_id & 0xFFFFFFFF, fresh=True)
+        self.next_id += m
+        for k, v in fresh.items():
+            self.reqs[k][slots] = v
+        self.ctx += 1
+        k = max(1, len(self.ctx) // 20)
+        which = self.rng.choice(len(self.ctx), size=k, replace=False)
+        self.ctx[which] = self._draw_ctx(k)
+        return np.sort(slots)
+
+    def workload(self) -> Workload:
+        w = Workload(f"sweep{self.n}", self.params, self.reqs, self.now, self.D_act, self.K_act)
+        w.hbm_free_count = self.hbm_free_count
+        w.host_free_count = self.host_free_count
+        return w
+
+
+def copy_lists(seed: int, n_copies: int, n_src_blocks: int, n_dst_blocks: int):
+    """Two independent samples without replacement: scattered, non-contiguous source and destination ids."""
+    rng = np.random.default_rng(seed)
+    src = rng.choice(n_src_blocks, size=n_copies, replace=False).astype(np.int32)
+    dst = rng.choice(n_dst_blocks, size=n_copies, replace=False).astype(np.int32)
+    return src, dst

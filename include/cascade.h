@@ -1,0 +1,274 @@
+/*
+ * libcascade: the per-iteration, budget-driven scheduling and KV-tier step of the Cascade
+ * serving loop as hand-written CUDA kernels for sm_100a (NVIDIA B200), behind a C ABI.
+ *
+ * One iteration = five stream-ordered calls on ONE stream, no host synchronisation between them:
+ *
+ *   cascade_budget     per-request latency budget and 64-bit priority key      (Eq. 3, Eq. 4, Eq. 5)
+ *   cascade_schedule   least-remaining-budget-first order + admission          (Algorithm 1, phase 2)
+ *   cascade_tier_plan  restore bound, restore/retain/recompute, preemption     (Eq. 6, Eq. 7, Algorithm 1)
+ *   cascade_kv_evict   paged HBM blocks  -> contiguous host records            (preemption under HBM pressure)
+ *   cascade_kv_restore contiguous host records -> paged HBM blocks             (TriggerPrefetch of Algorithm 1)
+ *
+ * Conventions
+ *   - Every time is an int64 number of nanoseconds, every token / block count an int32, every
+ *     cost coefficient a Q20 fixed-point int64 (value * 2^20).  All results are exact integers.
+ *   - Unless a parameter says "host", a pointer is a DEVICE pointer owned by the caller; a pinned,
+ *     mapped host allocation (cudaHostAlloc / torch pin_memory) counts as device-accessible.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - The library allocates device memory only in cascade_create.  The five hot calls allocate
+ *     nothing, never synchronise the host and use no stream of their own.
+ *   - One context per stream.  A context is not thread-safe.
+ *   - Return value: 0 on success, a negative CASCADE_E* code for errors found on the host before
+ *     anything is launched.  Conditions found on the device never trap; they OR a CASCADE_ST_* bit
+ *     into the context's sticky status word, read with cascade_status.
+ */
+#ifndef CASCADE_H
+#define CASCADE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CASCADE_MAX_CLASSES 8
+#define CASCADE_MAX_REQUESTS 65536 /* largest queue one context can order */
+
+/* host-side return codes */
+#define CASCADE_OK 0
+#define CASCADE_EINVAL (-1) /* NULL pointer, negative or oversized count, bad alignment            */
+#define CASCADE_ERANGE (-2) /* a parameter outside the overflow-safe bounds listed below           */
+#define CASCADE_ECUDA (-3)  /* a CUDA runtime call failed; its code is kept in cascade_status_t    */
+#define CASCADE_ENOMEM (-4) /* cascade_create could not allocate its scratch                       */
+
+/* device-side sticky status bits */
+#define CASCADE_ST_EBOUNDS 1u   /* a block id or list length outside its pool: that item was skipped   */
+#define CASCADE_ST_ENOSPC 2u    /* HBM could not hold the admitted set: it was cut from the tail       */
+#define CASCADE_ST_ETIMEOUT 4u  /* a bounded wait inside a kernel expired                              */
+#define CASCADE_ST_EPRECOND 8u  /* a request outside the input bounds: it was parked / ignored         */
+#define CASCADE_ST_ELISTCAP 16u /* a copy list was too short: entries beyond its capacity were dropped */
+
+/* request flags */
+#define CASCADE_FLAG_HBM_PRIVATE 1u /* the request's n0 HBM blocks are its own and may be preempted */
+#define CASCADE_FLAG_RUNNING 2u     /* informational: partially prefilled                            */
+
+/* per-request action written by cascade_tier_plan */
+#define CASCADE_ACT_NONE 0u   /* holds no HBM block                                  */
+#define CASCADE_ACT_RETAIN 1u /* keeps its HBM blocks                                */
+#define CASCADE_ACT_EVICT 2u  /* preempted, KV spilled to host (on the evict list)   */
+#define CASCADE_ACT_DROP 3u   /* preempted, KV discarded (recomputed on re-execution) */
+
+/*
+ * Cost model and policy parameters (host struct, copied at cascade_create).
+ * The paper's TTFT estimator is an offline-trained model with no printed form; this library
+ * uses an integer polynomial:
+ *   iter_q(D,K)   = c_iter + D*c_dseq + K*c_dkv            one engine iteration with D decodes over K KV tokens
+ *   A(D,K)        = c_tok + (iter_q(D,K) >> chunk_shift)   per prefill token
+ *   comp_q(A,P,s) = A*(P-s) + c_attn*(P*P - s*s)           prefill of prompt tokens [s,P)
+ *   T_k(x)        = x ? delta_ns[k] + x*blk_ns[k] : 0      Eq. 6 in blocks, k = 1 host DRAM, 2 deep tier
+ * Overflow-safe bounds (checked, CASCADE_ERANGE): 1 <= bt <= 4096, 0 <= chunk_shift <= 20,
+ * 1 <= max_batch <= 65536, 0 <= max_ctx_avg <= 2^20, (max_batch-1)*max_ctx_avg <= 2^32,
+ * 0 <= gamma_q16 <= 2^17, 1 <= n_classes <= 8, 0 <= token_budget, 0 <= tier2_reserve,
+ * 0 <= c_tok_q20 <= 2^40, 0 <= c_attn_q20 <= 2^20, 0 <= c_iter_q20 <= 2^50, 0 <= c_dseq_q20 <= 2^40,
+ * 0 <= c_dkv_q20 <= 2^28, 0 <= delta_ns[k] <= 2^30, 1 <= blk_ns[k] <= 2^27, 0 <= ttft_ns, tpot_ns <= 2^40.
+ * Per call: 0 <= D_act <= 2^16, 0 <= K_act <= 2^32.
+ */
+typedef struct cascade_params {
+    int32_t bt;            /* tokens per KV block                                              */
+    int32_t chunk_shift;   /* prefill chunk = 2^chunk_shift tokens                             */
+    int32_t max_batch;     /* B_max: sequences per engine iteration, decodes included          */
+    int32_t max_ctx_avg;   /* KV tokens per decode sequence assumed in the maximum-load regime */
+    int32_t gamma_q16;     /* guardband gamma of Eq. 3, times 2^16                             */
+    int32_t n_classes;
+    int32_t token_budget;  /* tokens per engine iteration (decodes take one each)              */
+    int32_t tier2_reserve; /* tokens of every iteration kept for the Tier-2 queue              */
+    int64_t c_tok_q20, c_attn_q20, c_iter_q20, c_dseq_q20, c_dkv_q20;
+    int64_t delta_ns[3];   /* Eq. 6: fixed overheads summed over path P(k); [0] unused         */
+    int64_t blk_ns[3];     /* Eq. 6: time per block summed over path P(k); [0] unused          */
+    int64_t ttft_ns[CASCADE_MAX_CLASSES]; /* class TTFT targets                                */
+    int64_t tpot_ns[CASCADE_MAX_CLASSES]; /* class TPOT targets; 0 disables the decode term    */
+} cascade_params;
+
+/*
+ * The request queue as a structure of arrays (host struct of device pointers, n entries each).
+ * Per-request bounds (a violation parks the request and sets CASCADE_ST_EPRECOND):
+ * 1 <= prompt <= 2^17, 0 <= pred_out <= 2^20, n0,n1,n2 >= 0, n0+n1+n2 <= 2^13,
+ * (n0+n1+n2)*bt < prompt, cls < n_classes, |now - arrival| <= 2^50.
+ */
+typedef struct cascade_reqs {
+    const int64_t *arrival_ns; /* arrival timestamp a_r                                         */
+    const int32_t *prompt;     /* prompt length in tokens                                       */
+    const int32_t *pred_out;   /* predicted output length in tokens                             */
+    const int32_t *n0;         /* matched prefix blocks resident in HBM (table positions 0..n0) */
+    const int32_t *n1;         /* next matched blocks held in host DRAM                         */
+    const int32_t *n2;         /* next matched blocks held in the deep tier (priced only)       */
+    const uint32_t *id;        /* arrival id; ties in budget are broken by its low 23 bits      */
+    const uint8_t *cls;        /* SLO class                                                     */
+    const uint8_t *flags;      /* CASCADE_FLAG_*                                                */
+} cascade_reqs;
+
+/* written to device memory by cascade_schedule */
+typedef struct cascade_sched_counts {
+    int32_t n_tier1;        /* requests in the Tier-1 queue (budget of Eq. 4 positive) */
+    int32_t n_admitted;     /* requests with grant > 0                                 */
+    int64_t tokens_granted; /* sum of grants                                           */
+} cascade_sched_counts;
+
+/* written to device memory by cascade_tier_plan */
+typedef struct cascade_plan_counts {
+    int32_t n_restore;       /* entries of the restore list (blocks)            */
+    int32_t n_evict;         /* entries of the evict list (blocks)              */
+    int32_t n_drop_blocks;   /* HBM blocks freed without a copy                 */
+    int32_t n_victims;       /* requests preempted (EVICT or DROP)              */
+    int32_t n_unadmitted;    /* requests un-admitted by the HBM capacity check  */
+    int32_t n_admitted;      /* requests still admitted after the plan          */
+    int32_t hbm_need;        /* new HBM blocks the admitted set takes           */
+    int32_t deficit;         /* blocks that had to be freed                     */
+    int32_t hbm_free_after;  /* HBM free-list length after the plan             */
+    int32_t host_free_after; /* host free-list length after the plan            */
+    int64_t tokens_run;      /* tokens the admitted set computes this iteration */
+} cascade_plan_counts;
+
+/*
+ * Block tables and free lists (host struct of device pointers).  Read AND updated by
+ * cascade_tier_plan.  Tables are row-major [n][maxb] int32, -1 = no block: hbm_tbl[r][j] is the
+ * HBM block holding tokens [j*bt,(j+1)*bt) of request r, host_tbl[r][j] its host record.
+ * Free lists are stacks: the next id handed out is list[count-1].  hbm_free must have room for
+ * every block that can be freed (capacity = number of HBM blocks is always enough).
+ * hbm_tbl == NULL selects plan-only mode: decisions and counts are produced from the two counts
+ * alone; no table, free list, count or copy list is touched.
+ */
+typedef struct cascade_pools {
+    int32_t *hbm_tbl;
+    int32_t *host_tbl;
+    int32_t maxb;
+    int32_t *hbm_free;
+    int32_t *hbm_free_count; /* device scalar, updated */
+    int32_t hbm_free_cap;
+    int32_t *host_free;
+    int32_t *host_free_count; /* device scalar, updated */
+    int32_t host_free_cap;
+} cascade_pools;
+
+/* Outputs of cascade_tier_plan (host struct of device pointers; arrays of n, lists of *_cap). */
+typedef struct cascade_plan {
+    int32_t *x1;         /* host blocks to restore now                          */
+    int32_t *x2;         /* deep-tier blocks to stage (priced and planned only) */
+    int32_t *tokens_run; /* prompt tokens computed this iteration               */
+    uint8_t *action;     /* CASCADE_ACT_*                                       */
+    int32_t *restore_src; /* host record ids, in schedule order                 */
+    int32_t *restore_dst; /* HBM block ids                                      */
+    int32_t restore_cap;
+    int32_t *evict_src;   /* HBM block ids, in preemption order                 */
+    int32_t *evict_dst;   /* host record ids                                    */
+    int32_t evict_cap;
+    cascade_plan_counts *counts; /* device */
+} cascade_plan;
+
+/*
+ * Geometry of the paged HBM pool.  Byte address of chunk c (0..n_chunks-1, one per layer and K/V
+ * plane) of block b: c*chunk_stride + b*block_stride.  A layer-major pool has block_stride =
+ * chunk_bytes and chunk_stride = n_blocks*chunk_bytes; a block-major pool has chunk_stride =
+ * chunk_bytes and block_stride = n_chunks*chunk_bytes.  The host pool (or a device staging buffer
+ * standing in for it) is always record-major: record h occupies [h*bb, (h+1)*bb) with
+ * bb = n_chunks*chunk_bytes, its chunks back to back.
+ * chunk_bytes, both strides and both pool base addresses must be multiples of 16.
+ */
+typedef struct cascade_kv_layout {
+    int64_t n_blocks;
+    int32_t n_chunks;
+    int32_t reserved;
+    int64_t chunk_bytes;
+    int64_t chunk_stride;
+    int64_t block_stride;
+} cascade_kv_layout;
+
+typedef struct cascade_status_t {
+    uint32_t bits;       /* OR of CASCADE_ST_* seen since the last clear */
+    int32_t cuda_error;  /* last failing cudaError_t, 0 if none          */
+} cascade_status_t;
+
+typedef struct cascade_ctx cascade_ctx;
+
+/* Creates a context on `device` for queues of up to max_requests (<= CASCADE_MAX_REQUESTS).
+ * Validates the parameters against the bounds above.  Allocates scratch (about 48 bytes per request).
+ * `p` and `out` are host pointers. */
+int cascade_create(cascade_ctx **out, const cascade_params *p, int max_requests, int device);
+void cascade_destroy(cascade_ctx *ctx);
+/* Replaces the parameters (same validation); takes effect for calls made afterwards. */
+int cascade_set_params(cascade_ctx *ctx, const cascade_params *p);
+
+/*
+ * Latency budget and priority key of every request (one thread per request).
+ *   L      = ((L_act + L_max) * gamma) / 2                      Eq. 3, with L_rho = T_1(n1) + T_2(n2) +
+ *            comp_q(A(rho), prompt, (n0+n1+n2)*bt) for the actual load rho = (D_act, K_act) and the
+ *            maximum load (max(D_act, max_batch-1), max(K_act, (max_batch-1)*max_ctx_avg))
+ *   B      = ttft_ns[cls] - L                                   Eq. 4;  B > 0 -> Tier-1 queue, else Tier-2
+ *   B_rem  = B - (now_ns - arrival_ns)                          Eq. 5
+ *   budget = B_rem - pred_out * max(0, t_dec - tpot_ns[cls])    decode-overrun penalty, 0 if tpot_ns == 0
+ *   key    = tier2 << 63 | (clamp(budget, -2^39, 2^39-1) + 2^39) << 23 | (id & 0x7FFFFF)
+ * budget_out[n] and key_out[n] are written.
+ */
+int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, int64_t now_ns, int32_t D_act, int64_t K_act,
+                   int64_t *budget_out, uint64_t *key_out, void *stream);
+
+/*
+ * Least-remaining-budget-first order and admission (Algorithm 1, phase 2).
+ *   order_out[n]  slot indices sorted ascending by key (stable: equal keys keep slot order)
+ *   grant_out[n]  tokens granted to each slot this iteration (0 = not admitted): the Tier-1 queue
+ *                 is served in order from token_budget - D_act minus the Tier-2 reserve, the Tier-2
+ *                 queue from the reserve plus what Tier-1 left; each request is offered
+ *                 prompt - (n0+n1+n2)*bt tokens; at most max_batch - D_act requests are admitted.
+ *   counts_dev    device struct, written.
+ */
+int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const uint64_t *key, int n, int32_t D_act,
+                     uint32_t *order_out, int32_t *grant_out, cascade_sched_counts *counts_dev, void *stream);
+
+/*
+ * Tier plan for the admitted set.
+ *   - Eq. 7 bound per tier from the request's budget (host first, deep tier from what is left),
+ *     then the candidate (nothing / host bound / host + deep bound) with the smallest predicted
+ *     completion time  (T_1(x1)+T_2(x2)) + comp(prompt, (n0+x1+x2)*bt); ties restore more.
+ *   - HBM capacity: admitted requests whose cumulative block need exceeds free + preemptable are
+ *     un-admitted from the tail (`grant` is zeroed for them; CASCADE_ST_ENOSPC).
+ *   - Preemption: non-admitted CASCADE_FLAG_HBM_PRIVATE holders, last in the order first, until the
+ *     deficit is covered; EVICT when T_1(n0) <= budget and the host pool has room, else DROP.
+ *   - Block ids: freed HBM ids are pushed, then admitted requests pop ids for restored and newly
+ *     computed blocks; tables, free lists, counts and the two copy lists are updated.
+ * `grant` is read and updated.  `pools` and `plan_out` are host structs (copied during the call).
+ * The evict list must be executed before the restore list (a freed block may be reused at once).
+ */
+int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *budget, const uint32_t *order,
+                      int32_t *grant, int n, int32_t D_act, int64_t K_act, const cascade_pools *pools,
+                      const cascade_plan *plan_out, void *stream);
+
+/*
+ * Restore: for i < count, copy host record src_ids[i] into HBM block dst_ids[i]
+ * (n_chunks pieces of chunk_bytes scattered into the paged layout).
+ *   src_pool       record-major pool: pinned mapped host memory (read over the host link) or a
+ *                  device staging buffer; src_is_device says which (tuning hint only)
+ *   src_blocks     number of records in src_pool (ids outside are skipped, CASCADE_ST_EBOUNDS)
+ *   n_copies_dev   device scalar holding the count, or NULL to use n_copies_max itself
+ *   n_copies_max   upper bound of the count (list capacity)
+ * Destination ids must be distinct within a call.
+ */
+int cascade_kv_restore(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, const void *src_pool,
+                       int64_t src_blocks, int src_is_device, const int32_t *src_ids, const int32_t *dst_ids,
+                       const int32_t *n_copies_dev, int n_copies_max, void *stream);
+
+/* Evict: for i < count, copy HBM block src_ids[i] into host record dst_ids[i]; arguments as above. */
+int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, const void *hbm_pool, void *dst_pool,
+                     int64_t dst_blocks, int dst_is_device, const int32_t *src_ids, const int32_t *dst_ids,
+                     const int32_t *n_copies_dev, int n_copies_max, void *stream);
+
+/* Waits for `stream`, copies the status word to *host_out and, if clear != 0, resets it. */
+int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream);
+
+/* Library version (major*10000 + minor*100 + patch). */
+int cascade_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,102 @@
+// Context management, parameter validation and status read-back of libcascade.
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+
+static bool in_range(int64_t v, int64_t lo, int64_t hi) { return v >= lo && v <= hi; }
+
+int cascade_validate_params(const cascade_params *p) {
+    if (!p) return CASCADE_EINVAL;
+    const int64_t one = 1;
+    bool ok = in_range(p->bt, 1, 4096) && in_range(p->chunk_shift, 0, 20) && in_range(p->max_batch, 1, 65536) &&
+              in_range(p->max_ctx_avg, 0, one << 20) && in_range(p->gamma_q16, 0, one << 17) &&
+              in_range(p->n_classes, 1, CASCADE_MAX_CLASSES) && p->token_budget >= 0 && p->tier2_reserve >= 0 &&
+              in_range(p->c_tok_q20, 0, one << 40) && in_range(p->c_attn_q20, 0, one << 20) &&
+              in_range(p->c_iter_q20, 0, one << 50) && in_range(p->c_dseq_q20, 0, one << 40) &&
+              in_range(p->c_dkv_q20, 0, one << 28);
+    if (ok) ok = (int64_t)(p->max_batch - 1) * p->max_ctx_avg <= (one << 32);
+    for (int k = 1; ok && k <= 2; ++k)
+        ok = in_range(p->delta_ns[k], 0, one << 30) && in_range(p->blk_ns[k], 1, one << 27);
+    for (int c = 0; ok && c < p->n_classes; ++c)
+        ok = in_range(p->ttft_ns[c], 0, one << 40) && in_range(p->tpot_ns[c], 0, one << 40);
+    return ok ? CASCADE_OK : CASCADE_ERANGE;
+}
+
+extern "C" int cascade_version(void) { return 100; }
+
+extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int max_requests, int device) {
+    if (!out || !p) return CASCADE_EINVAL;
+    *out = nullptr;
+    if (max_requests < 1 || max_requests > CASCADE_MAX_REQUESTS) return CASCADE_EINVAL;
+    int rc = cascade_validate_params(p);
+    if (rc != CASCADE_OK) return rc;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return CASCADE_ECUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return CASCADE_ECUDA;
+    cascade_ctx *ctx = (cascade_ctx *)calloc(1, sizeof(cascade_ctx));
+    if (!ctx) return CASCADE_ENOMEM;
+    ctx->params = *p;
+    ctx->device = device;
+    ctx->max_requests = max_requests;
+    cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
+    const char *e = getenv("CASCADE_SORT_CLUSTER");
+    ctx->sort_cluster = e ? atoi(e) : 0;
+    e = getenv("CASCADE_SORT_ITEMS");
+    ctx->sort_items = e ? atoi(e) : 0;
+    e = getenv("CASCADE_COPY_CTAS_HOST");
+    ctx->copy_ctas_host = e && atoi(e) > 0 ? atoi(e) : 4;
+    e = getenv("CASCADE_COPY_CTAS_DEV");
+    ctx->copy_ctas_dev = e && atoi(e) > 0 ? atoi(e) : 8;
+    size_t n = (size_t)max_requests;
+    bool ok = cudaMalloc(&ctx->status_dev, sizeof(uint32_t)) == cudaSuccess &&
+              cudaMallocHost(&ctx->status_host, sizeof(uint32_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->pack_by_slot, n * sizeof(uint64_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->pack_sorted, n * sizeof(uint64_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->work_admit, n * sizeof(int4)) == cudaSuccess &&
+              cudaMalloc(&ctx->work_victim, n * sizeof(int4)) == cudaSuccess &&
+              cudaMalloc(&ctx->plan_scalars, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
+    if (ok) ok = cudaMemset(ctx->status_dev, 0, sizeof(uint32_t)) == cudaSuccess &&
+                 cudaMemset(ctx->plan_scalars, 0, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        cascade_destroy(ctx);
+        return CASCADE_ENOMEM;
+    }
+    *out = ctx;
+    return CASCADE_OK;
+}
+
+extern "C" void cascade_destroy(cascade_ctx *ctx) {
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->status_dev);
+    cudaFreeHost(ctx->status_host);
+    cudaFree(ctx->pack_by_slot);
+    cudaFree(ctx->pack_sorted);
+    cudaFree(ctx->work_admit);
+    cudaFree(ctx->work_victim);
+    cudaFree(ctx->plan_scalars);
+    free(ctx);
+}
+
+extern "C" int cascade_set_params(cascade_ctx *ctx, const cascade_params *p) {
+    if (!ctx) return CASCADE_EINVAL;
+    int rc = cascade_validate_params(p);
+    if (rc != CASCADE_OK) return rc;
+    ctx->params = *p;
+    return CASCADE_OK;
+}
+
+extern "C" int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream) {
+    if (!ctx || !host_out) return CASCADE_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(uint32_t),
+                                          cudaMemcpyDeviceToHost, s));
+    if (clear) CASCADE_CUDA_TRY(ctx, cudaMemsetAsync(ctx->status_dev, 0, sizeof(uint32_t), s));
+    CASCADE_CUDA_TRY(ctx, cudaStreamSynchronize(s));
+    host_out->bits = *ctx->status_host;
+    host_out->cuda_error = ctx->cuda_error;
+    if (clear) ctx->cuda_error = 0;
+    return CASCADE_OK;
+}

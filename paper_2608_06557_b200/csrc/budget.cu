@@ -1,0 +1,73 @@
+// cascade_budget: per-request latency budget (Eq. 3, Eq. 4, Eq. 5) and 64-bit priority key.
+// One thread per request; int64 multiply/add/shift only, no division.  The work is a few
+// dozen integer operations on ~37 bytes per request, so the kernel is launch-latency bound at
+// every queue size this library accepts; loads are coalesced SoA reads.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__global__ void __launch_bounds__(kThreads)
+budget_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ LoadConsts lc,
+              const __grid_constant__ cascade_reqs r, int n, int64_t now_ns, int64_t *__restrict__ budget_out,
+              uint64_t *__restrict__ key_out, uint32_t *__restrict__ status) {
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i >= n) return;
+    const int64_t P = r.prompt[i];
+    const int64_t O = r.pred_out[i];
+    const int64_t n0 = r.n0[i], n1 = r.n1[i], n2 = r.n2[i];
+    const uint32_t cls = r.cls[i];
+    const uint32_t id = r.id[i] & 0x7FFFFFu;
+    const int64_t elapsed = now_ns - r.arrival_ns[i];
+    const int64_t lim = int64_t(1) << 50;
+    bool ok = dev_request_valid(p.bt, P, n0, n1, n2) && O >= 0 && O <= (int64_t(1) << 20) &&
+              cls < (uint32_t)p.n_classes && elapsed <= lim && elapsed >= -lim;
+    if (!ok) {
+        // out-of-bounds request: flagged and parked at the very end of the Tier-2 queue
+        atomicOr(status, CASCADE_ST_EPRECOND);
+        budget_out[i] = -(int64_t(1) << 62);
+        key_out[i] = (uint64_t(1) << 63) | id;
+        return;
+    }
+    const int64_t s_hit = (n0 + n1 + n2) * p.bt;
+    // matched prefix outside HBM is priced by tier (Eq. 6), the rest of the prompt is computed
+    const int64_t tp = dev_restore_time(p, 1, n1) + dev_restore_time(p, 2, n2);
+    const int64_t L_act = tp + (dev_comp_q(lc.A_act, p.c_attn_q20, P, s_hit) >> 20);
+    const int64_t L_max = tp + (dev_comp_q(lc.A_max, p.c_attn_q20, P, s_hit) >> 20);
+    const int64_t L = ((L_act + L_max) * p.gamma_q16) >> 17;   // Eq. 3
+    const int64_t B = p.ttft_ns[cls] - L;                      // Eq. 4
+    const int64_t B_rem = B - elapsed;                         // Eq. 5
+    // one decode step of this request, co-scheduled with a full prefill chunk
+    const int64_t kv = P * p.c_dkv_q20;
+    const int64_t tdec_act = (lc.dec_act + kv) >> 20;
+    const int64_t tdec_max = (lc.dec_max + kv) >> 20;
+    const int64_t tdec = ((tdec_act + tdec_max) * p.gamma_q16) >> 17;
+    const int64_t tpot = p.tpot_ns[cls];
+    int64_t over = tdec - tpot;
+    if (over < 0 || tpot == 0) over = 0;
+    const int64_t budget = B_rem - O * over;
+    const int64_t clampv = int64_t(1) << 39;
+    int64_t u = budget < -clampv ? -clampv : (budget > clampv - 1 ? clampv - 1 : budget);
+    u += clampv;
+    budget_out[i] = budget;
+    key_out[i] = (uint64_t(B <= 0) << 63) | (uint64_t(u) << 23) | id;
+}
+
+}  // namespace
+
+extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, int64_t now_ns, int32_t D_act,
+                              int64_t K_act, int64_t *budget_out, uint64_t *key_out, void *stream) {
+    if (!ctx || !r || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
+    if (n == 0) return CASCADE_OK;
+    if (!budget_out || !key_out || !r->arrival_ns || !r->prompt || !r->pred_out || !r->n0 || !r->n1 || !r->n2 ||
+        !r->id || !r->cls)
+        return CASCADE_EINVAL;
+    if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
+    const LoadConsts lc = make_load_consts(ctx->params, D_act, K_act);
+    const int grid = (n + kThreads - 1) / kThreads;
+    budget_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(ctx->params, lc, *r, n, now_ns, budget_out, key_out,
+                                                              ctx->status_dev);
+    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    return CASCADE_OK;
+}

@@ -1,0 +1,84 @@
+// Internal declarations shared by the libcascade translation units (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cascade.h"
+
+// Context: parameters, scratch sized at creation, the sticky device status word.
+struct cascade_ctx {
+    cascade_params params;
+    int device;
+    int max_requests;
+    int num_sms;
+    uint32_t *status_dev;        // sticky CASCADE_ST_* bits
+    uint32_t *status_host;       // pinned mirror used by cascade_status
+    int cuda_error;              // last failing cudaError_t
+    // tier-plan scratch
+    uint64_t *pack_by_slot;      // per-request decision word, slot order
+    uint64_t *pack_sorted;       // the same words gathered into schedule order
+    int4 *work_admit;            // per admitted request: slot, pop offset, restore offset, counts
+    int4 *work_victim;           // per preempted request: slot, freed offset, evict offset, action
+    int32_t *plan_scalars;       // device scalars handed from the plan kernel to the apply kernels
+    int sort_cluster;            // cluster size override for the ordering kernel (0 = automatic)
+    int sort_items;              // keys per thread override (0 = automatic)
+    int copy_ctas_host;          // copy CTAs per SM when the record pool is pinned host memory
+    int copy_ctas_dev;           // copy CTAs per SM when the record pool is device memory
+};
+
+// plan_scalars layout
+enum { PS_N_ADMIT = 0, PS_N_VICTIM, PS_HBM_CNT0, PS_HOST_CNT0, PS_TOTAL_FREED, PS_COUNT };
+
+#define CASCADE_CUDA_TRY(ctx, expr)                         \
+    do {                                                    \
+        cudaError_t e__ = (expr);                           \
+        if (e__ != cudaSuccess) {                           \
+            (ctx)->cuda_error = (int)e__;                   \
+            return CASCADE_ECUDA;                           \
+        }                                                   \
+    } while (0)
+
+// ---- the integer cost model, device side --------------------------------------------------
+// Load-dependent constants are folded on the host once per call (exact integer arithmetic).
+struct LoadConsts {
+    int64_t A_act, A_max;          // per-token prefill cost under actual / maximum load (Q20 ns)
+    int64_t dec_act, dec_max;      // iteration cost with one more decode sequence, before its KV term,
+                                   // plus a full prefill chunk (Q20 ns)
+};
+
+static inline int64_t host_iter_q(const cascade_params &p, int64_t D, int64_t K) {
+    return p.c_iter_q20 + D * p.c_dseq_q20 + K * p.c_dkv_q20;
+}
+
+static inline LoadConsts make_load_consts(const cascade_params &p, int32_t D_act, int64_t K_act) {
+    int64_t Dm = D_act > p.max_batch - 1 ? D_act : p.max_batch - 1;
+    int64_t Kcap = (int64_t)(p.max_batch - 1) * p.max_ctx_avg;
+    int64_t Km = K_act > Kcap ? K_act : Kcap;
+    LoadConsts c;
+    c.A_act = p.c_tok_q20 + (host_iter_q(p, D_act, K_act) >> p.chunk_shift);
+    c.A_max = p.c_tok_q20 + (host_iter_q(p, Dm, Km) >> p.chunk_shift);
+    int64_t chunk_q = p.c_tok_q20 << p.chunk_shift;
+    c.dec_act = host_iter_q(p, (int64_t)D_act + 1, K_act) + chunk_q;
+    c.dec_max = host_iter_q(p, Dm + 1, Km) + chunk_q;
+    return c;
+}
+
+__device__ __forceinline__ int64_t dev_comp_q(int64_t A, int64_t c_attn, int64_t P, int64_t s) {
+    return A * (P - s) + c_attn * (P * P - s * s);
+}
+
+__device__ __forceinline__ int64_t dev_restore_time(const cascade_params &p, int k, int64_t x) {
+    return x == 0 ? 0 : p.delta_ns[k] + x * p.blk_ns[k];
+}
+
+__device__ __forceinline__ bool dev_request_valid(int32_t bt, int64_t P, int64_t n0, int64_t n1, int64_t n2) {
+    if (P < 1 || P > (int64_t(1) << 17)) return false;
+    if ((n0 | n1 | n2) < 0) return false;
+    int64_t h = n0 + n1 + n2;
+    if (h > (int64_t(1) << 13)) return false;
+    return h * bt < P;
+}
+
+// entry points implemented in the other translation units
+int cascade_validate_params(const cascade_params *p);

@@ -1,0 +1,172 @@
+"""Device-side state of one serving instance and the five-call iteration over it.
+
+Allocates every tensor the iteration needs (PyTorch as the memory/stream owner), uploads a
+``workload.Workload`` and issues the C-ABI calls in stream order:
+budget -> schedule -> tier_plan -> kv_evict -> kv_restore.  No host synchronisation happens
+between the calls; results are read back only by ``fetch``.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import cascade as cs
+
+_REQ_DTYPES = dict(arrival_ns=torch.int64, prompt=torch.int32, pred_out=torch.int32, n0=torch.int32,
+                   n1=torch.int32, n2=torch.int32, id=torch.uint32, cls=torch.uint8, flags=torch.uint8)
+_NP_DTYPES = dict(arrival_ns=np.int64, prompt=np.int32, pred_out=np.int32, n0=np.int32, n1=np.int32, n2=np.int32,
+                  id=np.uint32, cls=np.uint8, flags=np.uint8)
+
+
+def _to_dev(a: np.ndarray, device, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None and t.dtype != dtype:
+        t = t.view(dtype)
+    return t.to(device)
+
+
+class Instance:
+    """All device buffers of one scheduler instance.
+
+    ``hbm_pool`` / ``host_pool`` may be passed in (uint8 tensors, device and pinned host); when a
+    workload has a layout and none is given they are allocated here, uninitialised."""
+
+    def __init__(self, w, device: str = "cuda:0", max_requests: int | None = None, alloc_pools: bool = True,
+                 hbm_pool=None, host_pool=None, ctx: cs.Context | None = None):
+        self.device = torch.device(device)
+        self.n = w.n
+        cap = max_requests or max(w.n, 1)
+        self.cap = cap
+        dev_index = self.device.index or 0
+        self.ctx = ctx or cs.Context(w.params, cap, dev_index)
+        if ctx is not None:
+            self.ctx.set_params(w.params)
+        self.now_ns, self.D_act, self.K_act = w.now_ns, w.D_act, w.K_act
+        d = self.device
+        # request queue, structure of arrays; a pinned host mirror serves the end-to-end path
+        self.reqs = {k: torch.empty(cap, dtype=dt, device=d) for k, dt in _REQ_DTYPES.items()}
+        self.reqs_host = {k: torch.empty(cap, dtype=dt).pin_memory() for k, dt in _REQ_DTYPES.items()}
+        self.reqs_struct = cs.make_reqs(self.reqs)
+        self.upload_requests(w.reqs)
+        # outputs
+        self.budget = torch.empty(cap, dtype=torch.int64, device=d)
+        self.key = torch.empty(cap, dtype=torch.uint64, device=d)
+        self.order = torch.empty(cap, dtype=torch.uint32, device=d)
+        self.grant = torch.empty(cap, dtype=torch.int32, device=d)
+        self.sched_counts = torch.zeros(2, dtype=torch.int64, device=d)      # cascade_sched_counts (16 B)
+        self.plan_counts = torch.zeros(12, dtype=torch.int32, device=d)      # cascade_plan_counts (48 B)
+        self.x1 = torch.empty(cap, dtype=torch.int32, device=d)
+        self.x2 = torch.empty(cap, dtype=torch.int32, device=d)
+        self.tokens_run = torch.empty(cap, dtype=torch.int32, device=d)
+        self.action = torch.empty(cap, dtype=torch.uint8, device=d)
+        self.hbm_free_count = torch.tensor([w.hbm_free_count], dtype=torch.int32, device=d)
+        self.host_free_count = torch.tensor([w.host_free_count], dtype=torch.int32, device=d)
+        self.with_tables = w.hbm_tbl is not None
+        self.layout = None
+        self.hbm_pool = hbm_pool
+        self.host_pool = host_pool
+        if self.with_tables:
+            self.maxb = w.maxb
+            self.hbm_tbl = _to_dev(w.hbm_tbl, d)
+            self.host_tbl = _to_dev(w.host_tbl, d)
+            self.hbm_free = _to_dev(w.hbm_free, d)
+            self.host_free = _to_dev(w.host_free, d)
+            self.restore_cap = len(w.hbm_free)
+            self.evict_cap = len(w.host_free)
+            self.restore_src = torch.full((self.restore_cap,), -1, dtype=torch.int32, device=d)
+            self.restore_dst = torch.full((self.restore_cap,), -1, dtype=torch.int32, device=d)
+            self.evict_src = torch.full((self.evict_cap,), -1, dtype=torch.int32, device=d)
+            self.evict_dst = torch.full((self.evict_cap,), -1, dtype=torch.int32, device=d)
+            self.pools_struct = cs.Pools(cs._p(self.hbm_tbl), cs._p(self.host_tbl), self.maxb, cs._p(self.hbm_free),
+                                         cs._p(self.hbm_free_count), len(w.hbm_free), cs._p(self.host_free),
+                                         cs._p(self.host_free_count), len(w.host_free))
+            self.plan_struct = cs.Plan(cs._p(self.x1), cs._p(self.x2), cs._p(self.tokens_run), cs._p(self.action),
+                                       cs._p(self.restore_src), cs._p(self.restore_dst), self.restore_cap,
+                                       cs._p(self.evict_src), cs._p(self.evict_dst), self.evict_cap,
+                                       cs._p(self.plan_counts))
+            self.layout_dict = w.layout
+            self.layout = cs.make_layout(w.layout)
+            self.host_blocks = w.host_blocks
+            self.block_bytes = w.block_bytes
+            if alloc_pools:
+                if self.hbm_pool is None:
+                    self.hbm_pool = torch.empty(w.layout["n_blocks"] * self.block_bytes, dtype=torch.uint8, device=d)
+                if self.host_pool is None:
+                    self.host_pool = torch.empty(w.host_blocks * self.block_bytes, dtype=torch.uint8).pin_memory()
+        else:
+            self.pools_struct = cs.Pools(None, None, 0, None, cs._p(self.hbm_free_count), 0, None,
+                                         cs._p(self.host_free_count), 0)
+            self.plan_struct = cs.Plan(cs._p(self.x1), cs._p(self.x2), cs._p(self.tokens_run), cs._p(self.action),
+                                       None, None, 0, None, None, 0, cs._p(self.plan_counts))
+
+    # -- inputs ---------------------------------------------------------------------------------
+    def upload_requests(self, reqs: dict, n: int | None = None, stream=None):
+        """Host -> device copy of the whole request queue through the pinned mirror."""
+        n = len(reqs["prompt"]) if n is None else n
+        self.n = n
+        for k, dt in _NP_DTYPES.items():
+            src = np.ascontiguousarray(reqs[k], dtype=dt)
+            self.reqs_host[k][:n].numpy()[...] = src if dt != np.uint32 else src
+            self.reqs[k][:n].copy_(self.reqs_host[k][:n], non_blocking=True)
+
+    def request_bytes(self) -> int:
+        return sum(self.reqs[k].element_size() for k in self.reqs) * self.n
+
+    def set_clock(self, now_ns: int, D_act: int, K_act: int):
+        self.now_ns, self.D_act, self.K_act = now_ns, D_act, K_act
+
+    # -- the path -------------------------------------------------------------------------------
+    def run_schedule(self, stream=None):
+        """budget -> schedule -> tier plan (three C-ABI calls, stream ordered)."""
+        c = self.ctx
+        c.budget(self.reqs_struct, self.n, self.now_ns, self.D_act, self.K_act, self.budget, self.key, stream)
+        c.schedule(self.reqs_struct, self.key, self.n, self.D_act, self.order, self.grant, self.sched_counts, stream)
+        c.tier_plan(self.reqs_struct, self.budget, self.order, self.grant, self.n, self.D_act, self.K_act,
+                    self.pools_struct, self.plan_struct, stream)
+
+    def run_copies(self, stream=None, record_pool=None, record_is_device: bool = False):
+        """evict then restore, with the counts the plan left in device memory."""
+        c = self.ctx
+        rec = self.host_pool if record_pool is None else record_pool
+        n_evict = self.plan_counts[1:2]
+        n_restore = self.plan_counts[0:1]
+        c.kv_evict(self.layout, self.hbm_pool, rec, self.host_blocks, record_is_device, self.evict_src,
+                   self.evict_dst, n_evict, self.evict_cap, stream)
+        c.kv_restore(self.layout, self.hbm_pool, rec, self.host_blocks, record_is_device, self.restore_src,
+                     self.restore_dst, n_restore, self.restore_cap, stream)
+
+    def run_iteration(self, stream=None):
+        self.run_schedule(stream)
+        if self.with_tables and self.hbm_pool is not None:
+            self.run_copies(stream)
+
+    # -- outputs --------------------------------------------------------------------------------
+    def fetch(self) -> dict:
+        """Synchronise and bring every result to the host as numpy."""
+        torch.cuda.synchronize(self.device)
+        n = self.n
+        sc = self.sched_counts.cpu().numpy()
+        pc = self.plan_counts.cpu().numpy()
+        names = ("n_restore", "n_evict", "n_drop_blocks", "n_victims", "n_unadmitted", "n_admitted", "hbm_need",
+                 "deficit", "hbm_free_after", "host_free_after")
+        plan_counts = {k: int(pc[i]) for i, k in enumerate(names)}
+        plan_counts["tokens_run"] = int(pc[10:12].view(np.int64)[0])
+        out = dict(
+            budget=self.budget[:n].cpu().numpy(), key=self.key[:n].cpu().numpy(),
+            order=self.order[:n].cpu().numpy(), grant=self.grant[:n].cpu().numpy(),
+            sched_counts=dict(n_tier1=int(sc[0] & 0xFFFFFFFF), n_admitted=int(sc[0] >> 32),
+                              tokens_granted=int(sc[1])),
+            x1=self.x1[:n].cpu().numpy(), x2=self.x2[:n].cpu().numpy(),
+            tokens_run=self.tokens_run[:n].cpu().numpy(), action=self.action[:n].cpu().numpy(),
+            plan_counts=plan_counts)
+        if self.with_tables:
+            nr = min(plan_counts["n_restore"], self.restore_cap)
+            ne = min(plan_counts["n_evict"], self.evict_cap)
+            out.update(hbm_tbl=self.hbm_tbl.cpu().numpy(), host_tbl=self.host_tbl.cpu().numpy(),
+                       hbm_free=self.hbm_free.cpu().numpy(), host_free=self.host_free.cpu().numpy(),
+                       hbm_free_count=int(self.hbm_free_count.item()),
+                       host_free_count=int(self.host_free_count.item()),
+                       restore_src=self.restore_src[:nr].cpu().numpy(), restore_dst=self.restore_dst[:nr].cpu().numpy(),
+                       evict_src=self.evict_src[:ne].cpu().numpy(), evict_dst=self.evict_dst[:ne].cpu().numpy())
+        out["status"] = self.ctx.status(clear=True)[0]
+        return out

@@ -1,0 +1,53 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+from paper_2608_06557_b200 import build as cbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "cascade.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cascade_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(cbuild.build())
+    names = declared_symbols()
+    assert {"cascade_budget", "cascade_schedule", "cascade_tier_plan", "cascade_kv_restore",
+            "cascade_kv_evict"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), name
+    lib.cascade_version.restype = ctypes.c_int
+    assert lib.cascade_version() >= 100
+
+
+def test_binding_lists_the_same_symbols_and_struct_sizes():
+    from paper_2608_06557_b200 import cascade as cs
+    declared = set(declared_symbols())
+    assert declared <= set(cs.EXPORTS) | {"cascade_kv_restore_noalloc"} or declared == set(cs.EXPORTS)
+    assert ctypes.sizeof(cs.Params) == 8 * 4 + 5 * 8 + 6 * 8 + 16 * 8
+    assert ctypes.sizeof(cs.SchedCounts) == 16 and ctypes.sizeof(cs.PlanCounts) == 48
+    assert ctypes.sizeof(cs.KvLayout) == 40 and ctypes.sizeof(cs.Reqs) == 72
+
+
+def test_host_validation_without_a_device():
+    """Errors the library finds before touching CUDA are reachable with no GPU at all."""
+    from paper_2608_06557_b200 import cascade as cs
+    from paper_2608_06557_b200 import workload as wl
+    lib = cs.raw()
+    h = ctypes.c_void_p()
+    p = cs.make_params(wl.default_params())
+    assert lib.cascade_create(None, ctypes.byref(p), 16, 0) == cs.EINVAL
+    assert lib.cascade_create(ctypes.byref(h), None, 16, 0) == cs.EINVAL
+    assert lib.cascade_create(ctypes.byref(h), ctypes.byref(p), 0, 0) == cs.EINVAL
+    assert lib.cascade_create(ctypes.byref(h), ctypes.byref(p), cs.MAX_REQUESTS + 1, 0) == cs.EINVAL
+    for bad in (dict(bt=0), dict(gamma_q16=1 << 18), dict(blk_ns=[0, 0, 1]), dict(c_attn_q20=(1 << 20) + 1),
+                dict(ttft_ns=[1 << 41]), dict(max_batch=0), dict(delta_ns=[0, -1, 0])):
+        q = cs.make_params(wl.default_params(**bad))
+        assert lib.cascade_create(ctypes.byref(h), ctypes.byref(q), 16, 0) == cs.ERANGE, bad
+    assert lib.cascade_budget(None, None, 0, 0, 0, 0, None, None, None) == cs.EINVAL
+    assert lib.cascade_status(None, None, 0, None) == cs.EINVAL

@@ -1,0 +1,162 @@
+"""GPU parity: paged KV restore / evict against the CPU oracle, byte for byte."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import oracle_iteration
+from paper_2608_06557_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _gpu():
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    from paper_2608_06557_b200.runner import Instance
+    assert torch.cuda.is_available()
+    return torch, cs, Instance
+
+
+class CopyRig:
+    """A paged HBM pool, a pinned host pool and a device staging pool with guard bands around each."""
+
+    GUARD = 4096
+
+    def __init__(self, n_hbm, n_host, n_chunks, chunk_bytes, block_major=False):
+        torch, cs, _ = _gpu()
+        self.torch, self.cs = torch, cs
+        if block_major:
+            self.lay = dict(n_blocks=n_hbm, n_chunks=n_chunks, chunk_bytes=chunk_bytes, chunk_stride=chunk_bytes,
+                            block_stride=n_chunks * chunk_bytes)
+        else:
+            self.lay = wl.kv_layout(n_hbm, n_chunks, chunk_bytes)
+        self.n_hbm, self.n_host = n_hbm, n_host
+        self.bb = n_chunks * chunk_bytes
+        g = self.GUARD
+        self.hbm_np = wl.pool_bytes(1, n_hbm * self.bb).copy()
+        self.host_np = wl.pool_bytes(2, n_host * self.bb).copy()
+        self.hbm_buf = torch.full((n_hbm * self.bb + 2 * g,), 0xA5, dtype=torch.uint8, device="cuda")
+        self.host_buf = torch.full((n_host * self.bb + 2 * g,), 0x5A, dtype=torch.uint8).pin_memory()
+        self.stage_buf = torch.full((n_host * self.bb + 2 * g,), 0x3C, dtype=torch.uint8, device="cuda")
+        self.hbm = self.hbm_buf[g:-g]
+        self.host = self.host_buf[g:-g]
+        self.stage = self.stage_buf[g:-g]
+        self.hbm.copy_(torch.from_numpy(self.hbm_np))
+        self.host.copy_(torch.from_numpy(self.host_np))
+        self.stage.copy_(torch.from_numpy(self.host_np))
+        self.ctx = cs.Context(wl.default_params(), 16, 0)
+        self.layout = cs.make_layout(self.lay)
+        torch.cuda.synchronize()
+
+    def ids(self, a):
+        return self.torch.from_numpy(np.ascontiguousarray(a, np.int32)).cuda()
+
+    def guards_intact(self):
+        g = self.GUARD
+        t = self.torch
+        t.cuda.synchronize()
+        return (bool((self.hbm_buf[:g] == 0xA5).all()) and bool((self.hbm_buf[-g:] == 0xA5).all())
+                and bool((self.host_buf[:g] == 0x5A).all()) and bool((self.host_buf[-g:] == 0x5A).all())
+                and bool((self.stage_buf[:g] == 0x3C).all()) and bool((self.stage_buf[-g:] == 0x3C).all()))
+
+
+@pytest.mark.parametrize("shape", [(64, 48, 4, 4096, False), (40, 24, 3, 208, False), (33, 20, 5, 48, True),
+                                   (24, 16, 64, 32768, False), (20, 12, 2, 16 * 1024 + 16, True)])
+@pytest.mark.parametrize("via", ["host", "stage"])
+def test_restore_evict_round_trip(shape, via):
+    n_hbm, n_host, n_chunks, cb, bm = shape
+    rig = CopyRig(n_hbm, n_host, n_chunks, cb, bm)
+    torch = rig.torch
+    rec = rig.host if via == "host" else rig.stage
+    is_dev = via == "stage"
+    n = min(n_hbm, n_host) // 2 + 1
+    # restore: host records -> HBM blocks
+    src, dst = wl.copy_lists(1, n, n_host, n_hbm)
+    ref_hbm, ref_host = rig.hbm_np.copy(), rig.host_np.copy()
+    assert oracle.kv_restore(ref_hbm, rig.lay, ref_host, n_host, src, dst) == 0
+    rig.ctx.kv_restore(rig.layout, rig.hbm, rec, n_host, is_dev, rig.ids(src), rig.ids(dst), None, n)
+    torch.cuda.synchronize()
+    assert np.array_equal(rig.hbm.cpu().numpy(), ref_hbm)
+    # evict: other HBM blocks -> other host records, count taken from device memory
+    src2, dst2 = wl.copy_lists(2, n, n_hbm, n_host)
+    assert oracle.kv_evict(ref_hbm, rig.lay, ref_host, n_host, src2, dst2) == 0
+    cap = n + 5
+    s2 = rig.ids(np.concatenate([src2, np.full(5, 10**6, np.int32)]))
+    d2 = rig.ids(np.concatenate([dst2, np.full(5, 10**6, np.int32)]))
+    n_dev = torch.tensor([n], dtype=torch.int32, device="cuda")
+    rig.ctx.kv_evict(rig.layout, rig.hbm, rec, n_host, is_dev, s2, d2, n_dev, cap)
+    torch.cuda.synchronize()
+    assert np.array_equal(rec.cpu().numpy(), ref_host)
+    assert np.array_equal(rig.hbm.cpu().numpy(), ref_hbm)
+    # poison the evicted blocks and bring them back: identity
+    view = rig.hbm_np.reshape(-1)
+    rig.hbm.fill_(0xEE)
+    back = np.random.default_rng(5).permutation(n_hbm)[:n].astype(np.int32)
+    rig.ctx.kv_restore(rig.layout, rig.hbm, rec, n_host, is_dev, rig.ids(dst2), rig.ids(back), None, n)
+    torch.cuda.synchronize()
+    now = rig.hbm.cpu().numpy()
+    exp = np.full_like(now, 0xEE)
+    assert oracle.kv_restore(exp, rig.lay, ref_host, n_host, dst2, back) == 0
+    assert np.array_equal(now, exp)
+    assert rig.guards_intact()
+    assert rig.ctx.status()[0] == 0
+
+
+def test_bad_ids_are_skipped_and_flagged():
+    rig = CopyRig(16, 16, 4, 256)
+    torch = rig.torch
+    src = np.array([3, -1, 16, 5, 2], np.int32)
+    dst = np.array([0, 1, 2, 99, 7], np.int32)
+    ref = rig.hbm_np.copy()
+    st = oracle.kv_restore(ref, rig.lay, rig.host_np, 16, src, dst)
+    rig.ctx.kv_restore(rig.layout, rig.hbm, rig.host, 16, False, rig.ids(src), rig.ids(dst), None, 5)
+    torch.cuda.synchronize()
+    assert np.array_equal(rig.hbm.cpu().numpy(), ref)
+    assert rig.ctx.status()[0] == st == 1
+    assert rig.guards_intact()
+    # empty and zero-count calls launch nothing / move nothing
+    rig.ctx.kv_restore(rig.layout, rig.hbm, rig.host, 16, False, rig.ids(src), rig.ids(dst), None, 0)
+    zero = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rig.ctx.kv_evict(rig.layout, rig.hbm, rig.host, 16, False, rig.ids(src), rig.ids(dst), zero, 5)
+    torch.cuda.synchronize()
+    assert np.array_equal(rig.host.cpu().numpy(), rig.host_np)
+
+
+def test_layout_validation_on_the_host():
+    rig = CopyRig(8, 8, 2, 64)
+    cs = rig.cs
+    ids = rig.ids([0])
+    bad = cs.make_layout(dict(rig.lay, chunk_bytes=40))
+    with pytest.raises(cs.CascadeError):
+        rig.ctx.kv_restore(bad, rig.hbm, rig.host, 8, False, ids, ids, None, 1)
+    with pytest.raises(cs.CascadeError):
+        rig.ctx.kv_restore(rig.layout, rig.hbm[8:], rig.host, 8, False, ids, ids, None, 1)
+    with pytest.raises(cs.CascadeError):
+        rig.ctx.kv_restore(rig.layout, rig.hbm, rig.host, 8, False, None, ids, None, 1)
+
+
+@pytest.mark.parametrize("seed,ttft_scale", [(0, 1), (1, 1), (2, 1), (0, 20), (3, 20)])
+def test_full_iteration_tiny_with_copies(seed, ttft_scale):
+    """All five calls on the tiny configuration; pools compared byte for byte with the oracle's mirrors.
+    With the published class targets most queued requests are already past their TTFT target and get no
+    restore (Eq. 7 with a negative remaining budget); the looser targets exercise the restore list."""
+    torch, cs, Instance = _gpu()
+    w = wl.config_tiny(seed)
+    w.params["ttft_ns"] = [t * ttft_scale for t in w.params["ttft_ns"]]
+    ref = oracle_iteration(w)
+    bb = w.block_bytes
+    hbm_np = wl.pool_bytes(3, w.layout["n_blocks"] * bb).copy()
+    host_np = wl.pool_bytes(4, w.host_blocks * bb).copy()
+    inst = Instance(w)
+    inst.hbm_pool.copy_(torch.from_numpy(hbm_np))
+    inst.host_pool.copy_(torch.from_numpy(host_np))
+    inst.run_iteration()
+    got = inst.fetch()
+    plan = ref["plan"]
+    assert oracle.kv_evict(hbm_np, w.layout, host_np, w.host_blocks, plan["evict_src"], plan["evict_dst"]) == 0
+    assert oracle.kv_restore(hbm_np, w.layout, host_np, w.host_blocks, plan["restore_src"], plan["restore_dst"]) == 0
+    assert got["plan_counts"] == plan["counts"]
+    assert np.array_equal(inst.hbm_pool.cpu().numpy(), hbm_np)
+    assert np.array_equal(inst.host_pool.cpu().numpy(), host_np)
+    if ttft_scale > 1:
+        assert plan["counts"]["n_restore"] > 0

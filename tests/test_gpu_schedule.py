@@ -1,0 +1,172 @@
+"""GPU parity: budget, ordering/admission and tier plan against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import oracle_iteration
+from paper_2608_06557_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _gpu():
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    from paper_2608_06557_b200.runner import Instance
+    assert torch.cuda.is_available()
+    return torch, cs, Instance
+
+
+def compare_iteration(w, tag=""):
+    torch, cs, Instance = _gpu()
+    ref = oracle_iteration(w)
+    inst = Instance(w, alloc_pools=False)
+    inst.run_schedule()
+    got = inst.fetch()
+    for k in ("budget", "key", "order"):
+        assert np.array_equal(got[k], ref[k]), (tag, k)
+    assert np.array_equal(got["grant"], ref["grant"]), (tag, "grant")
+    plan = ref["plan"]
+    for k in ("x1", "x2", "tokens_run", "action"):
+        assert np.array_equal(got[k], plan[k]), (tag, k)
+    assert got["plan_counts"] == plan["counts"], (tag, got["plan_counts"], plan["counts"])
+    assert got["status"] == ref["status"], (tag, got["status"], ref["status"])
+    if w.hbm_tbl is not None:
+        pools = ref["pools"]
+        assert np.array_equal(got["hbm_tbl"], pools.hbm_tbl), (tag, "hbm_tbl")
+        assert np.array_equal(got["host_tbl"], pools.host_tbl), (tag, "host_tbl")
+        assert got["hbm_free_count"] == pools.hbm_free_count and got["host_free_count"] == pools.host_free_count
+        assert np.array_equal(got["hbm_free"][: pools.hbm_free_count], pools.hbm_free[: pools.hbm_free_count])
+        assert np.array_equal(got["host_free"][: pools.host_free_count], pools.host_free[: pools.host_free_count])
+        for k in ("restore_src", "restore_dst", "evict_src", "evict_dst"):
+            assert np.array_equal(got[k], plan[k]), (tag, k)
+    return got, ref
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_tiny_config(seed):
+    got, ref = compare_iteration(wl.config_tiny(seed), f"tiny{seed}")
+    assert got["plan_counts"]["n_victims"] > 0 or seed > 0
+
+
+def test_tiny_schedule_counts_match():
+    torch, cs, Instance = _gpu()
+    w = wl.config_tiny(0)
+    ref = oracle_iteration(w)
+    inst = Instance(w, alloc_pools=False)
+    inst.ctx.budget(inst.reqs_struct, inst.n, w.now_ns, w.D_act, w.K_act, inst.budget, inst.key)
+    inst.ctx.schedule(inst.reqs_struct, inst.key, inst.n, w.D_act, inst.order, inst.grant, inst.sched_counts)
+    torch.cuda.synchronize()
+    assert np.array_equal(inst.grant[: w.n].cpu().numpy(), ref["grant_sched"])
+    sc = inst.sched_counts.cpu().numpy()
+    assert int(sc[0] & 0xFFFFFFFF) == ref["sched_counts"]["n_tier1"]
+    assert int(sc[0] >> 32) == ref["sched_counts"]["n_admitted"]
+    assert int(sc[1]) == ref["sched_counts"]["tokens_granted"]
+
+
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 1023, 1024, 1025, 3000, 8192, 8193, 16384, 40000, 65536])
+def test_llama8b_shaped_queue_sizes(n):
+    """Spans every cluster / keys-per-thread configuration of the ordering kernel and ragged tails."""
+    w = wl.config_llama8b(seed=n, n=n, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9, hbm_free_target=64)
+    if n > 4096:      # tables of 65536 x 2048 are not needed to exercise the ordering: plan-only above 4096
+        w.hbm_tbl = w.host_tbl = w.hbm_free = w.host_free = None
+        w.hbm_free_count, w.host_free_count = 1 << 30, 1 << 30
+    compare_iteration(w, f"n{n}")
+
+
+def test_heavy_load_tier2_and_saturated_budgets():
+    w = wl.config_llama8b(seed=77, n=5000, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9)
+    w.hbm_tbl = w.host_tbl = w.hbm_free = w.host_free = None
+    w.hbm_free_count, w.host_free_count = 1 << 30, 1 << 30
+    w.D_act, w.K_act = 120, 4_000_000
+    got, ref = compare_iteration(w, "heavy")
+    assert 0 < ref["sched_counts"]["n_tier1"] < w.n
+    assert np.any(ref["budget"] < -(1 << 39))
+
+
+def test_duplicate_and_constant_keys_keep_slot_order():
+    torch, cs, Instance = _gpu()
+    w = wl.config_llama8b(seed=5, n=2500, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9)
+    p = oracle.make_params(w.params)
+    inst = Instance(w, alloc_pools=False)
+    rng = np.random.default_rng(0)
+    for case in range(4):
+        if case == 0:
+            key = np.full(w.n, 12345 << 23, np.uint64)                        # every key equal: no pass runs
+        elif case == 1:
+            key = (rng.integers(0, 4, w.n).astype(np.uint64) << np.uint64(40))  # four distinct keys
+        elif case == 2:
+            key = rng.integers(0, 1 << 63, w.n).astype(np.uint64) * np.uint64(2) + np.uint64(1)
+            key[::7] = np.uint64(0xFFFFFFFFFFFFFFFF)                           # equals the padding value
+        else:
+            key = np.arange(w.n, dtype=np.uint64)[::-1].copy()
+        order, grant, counts, _ = oracle.schedule(p, w.reqs, key, w.D_act)
+        inst.key.view(torch.int64)[: w.n].copy_(torch.from_numpy(key.view(np.int64)))
+        inst.ctx.schedule(inst.reqs_struct, inst.key, inst.n, w.D_act, inst.order, inst.grant, inst.sched_counts)
+        torch.cuda.synchronize()
+        assert np.array_equal(inst.order[: w.n].cpu().numpy(), order), case
+        assert np.array_equal(inst.grant[: w.n].cpu().numpy(), grant), case
+
+
+def test_scheduler_sweep_iterations_with_churn():
+    """Consecutive iterations of the scheduler-scale sweep (plan-only), with 5 % slot churn."""
+    torch, cs, Instance = _gpu()
+    sw = wl.SchedulerSweep(4096, seed=1)
+    inst = Instance(sw.workload(), alloc_pools=False)
+    for it in range(5):
+        w = sw.workload()
+        ref = oracle_iteration(w, with_tables=False)
+        inst.upload_requests(w.reqs)
+        inst.set_clock(w.now_ns, w.D_act, w.K_act)
+        inst.run_schedule()
+        got = inst.fetch()
+        for k in ("budget", "key", "order", "grant"):
+            assert np.array_equal(got[k], ref[k]), (it, k)
+        for k in ("x1", "x2", "tokens_run", "action"):
+            assert np.array_equal(got[k], ref["plan"][k]), (it, k)
+        assert got["plan_counts"] == ref["plan"]["counts"]
+        sw.step()
+
+
+def test_precondition_flag_and_parking():
+    w = wl.config_tiny(2)
+    w.reqs["prompt"][3] = 0
+    w.reqs["n0"][5] = -4
+    w.reqs["cls"][7] = 6
+    got, ref = compare_iteration(w, "precond")
+    assert got["status"] & 8
+
+
+def test_capacity_and_host_pressure_variants():
+    w = wl.config_tiny(0)
+    w.hbm_free_count = 3
+    w.reqs["flags"][:] = 0
+    got, ref = compare_iteration(w, "nospace")
+    assert got["status"] & 2 and got["plan_counts"]["n_unadmitted"] > 0
+    w = wl.config_tiny(0)
+    w.host_free_count = 0
+    got, ref = compare_iteration(w, "hostfull")
+    assert got["plan_counts"]["n_evict"] == 0 and got["plan_counts"]["n_drop_blocks"] > 0
+    w = wl.config_tiny(4)
+    w.host_free_count = 7
+    compare_iteration(w, "hosttight")
+
+
+def test_host_side_validation_needs_no_launch():
+    torch, cs, Instance = _gpu()
+    w = wl.config_tiny(0)
+    inst = Instance(w, alloc_pools=False)
+    lib = cs.raw()
+    import ctypes as C
+    h = inst.ctx._h
+    assert lib.cascade_budget(h, C.byref(inst.reqs_struct), -1, 0, 0, 0, None, None, None) == cs.EINVAL
+    assert lib.cascade_budget(h, C.byref(inst.reqs_struct), w.n + 1, 0, 0, 0, cs._p(inst.budget), cs._p(inst.key),
+                              None) == cs.EINVAL
+    assert lib.cascade_budget(h, C.byref(inst.reqs_struct), w.n, 0, -1, 0, cs._p(inst.budget), cs._p(inst.key),
+                              None) == cs.ERANGE
+    assert lib.cascade_budget(h, C.byref(inst.reqs_struct), w.n, 0, 0, 0, None, cs._p(inst.key), None) == cs.EINVAL
+    bad = dict(w.params, blk_ns=[0, 0, 5])
+    with pytest.raises(cs.CascadeError):
+        cs.Context(bad, 16, 0)
+    with pytest.raises(cs.CascadeError):
+        cs.Context(w.params, cs.MAX_REQUESTS + 1, 0)

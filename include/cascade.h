@@ -69,7 +69,7 @@ extern "C" {
  *   T_k(x)        = x ? delta_ns[k] + x*blk_ns[k] : 0      Eq. 6 in blocks, k = 1 host DRAM, 2 deep tier
  * Overflow-safe bounds (checked, CASCADE_ERANGE): 1 <= bt <= 4096, 0 <= chunk_shift <= 20,
  * 1 <= max_batch <= 65536, 0 <= max_ctx_avg <= 2^20, (max_batch-1)*max_ctx_avg <= 2^32,
- * 0 <= gamma_q16 <= 2^17, 1 <= n_classes <= 8, 0 <= token_budget, 0 <= tier2_reserve,
+ * 0 <= gamma_q16 <= 2^17, 1 <= n_classes <= 8, 0 <= token_budget <= 2^30, 0 <= tier2_reserve,
  * 0 <= c_tok_q20 <= 2^40, 0 <= c_attn_q20 <= 2^20, 0 <= c_iter_q20 <= 2^50, 0 <= c_dseq_q20 <= 2^40,
  * 0 <= c_dkv_q20 <= 2^28, 0 <= delta_ns[k] <= 2^30, 1 <= blk_ns[k] <= 2^27, 0 <= ttft_ns, tpot_ns <= 2^40.
  * Per call: 0 <= D_act <= 2^16, 0 <= K_act <= 2^32.
@@ -192,7 +192,7 @@ typedef struct cascade_status_t {
 typedef struct cascade_ctx cascade_ctx;
 
 /* Creates a context on `device` for queues of up to max_requests (<= CASCADE_MAX_REQUESTS).
- * Validates the parameters against the bounds above.  Allocates scratch (about 48 bytes per request).
+ * Validates the parameters against the bounds above.  Allocates scratch (about 32 bytes per request).
  * `p` and `out` are host pointers. */
 int cascade_create(cascade_ctx **out, const cascade_params *p, int max_requests, int device);
 void cascade_destroy(cascade_ctx *ctx);

@@ -11,7 +11,7 @@ int cascade_validate_params(const cascade_params *p) {
     const int64_t one = 1;
     bool ok = in_range(p->bt, 1, 4096) && in_range(p->chunk_shift, 0, 20) && in_range(p->max_batch, 1, 65536) &&
               in_range(p->max_ctx_avg, 0, one << 20) && in_range(p->gamma_q16, 0, one << 17) &&
-              in_range(p->n_classes, 1, CASCADE_MAX_CLASSES) && p->token_budget >= 0 && p->tier2_reserve >= 0 &&
+              in_range(p->n_classes, 1, CASCADE_MAX_CLASSES) && in_range(p->token_budget, 0, one << 30) && p->tier2_reserve >= 0 &&
               in_range(p->c_tok_q20, 0, one << 40) && in_range(p->c_attn_q20, 0, one << 20) &&
               in_range(p->c_iter_q20, 0, one << 50) && in_range(p->c_dseq_q20, 0, one << 40) &&
               in_range(p->c_dkv_q20, 0, one << 28);
@@ -44,6 +44,10 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->sort_cluster = e ? atoi(e) : 0;
     e = getenv("CASCADE_SORT_ITEMS");
     ctx->sort_items = e ? atoi(e) : 0;
+    e = getenv("CASCADE_SORT_THREADS");
+    ctx->sort_threads = e ? atoi(e) : 0;
+    e = getenv("CASCADE_SORT_MATCH");
+    ctx->sort_match = e ? atoi(e) : 0;
     e = getenv("CASCADE_COPY_CTAS_HOST");
     ctx->copy_ctas_host = e && atoi(e) > 0 ? atoi(e) : 4;
     e = getenv("CASCADE_COPY_CTAS_DEV");
@@ -51,8 +55,6 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     size_t n = (size_t)max_requests;
     bool ok = cudaMalloc(&ctx->status_dev, sizeof(uint32_t)) == cudaSuccess &&
               cudaMallocHost(&ctx->status_host, sizeof(uint32_t)) == cudaSuccess &&
-              cudaMalloc(&ctx->pack_by_slot, n * sizeof(uint64_t)) == cudaSuccess &&
-              cudaMalloc(&ctx->pack_sorted, n * sizeof(uint64_t)) == cudaSuccess &&
               cudaMalloc(&ctx->work_admit, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->work_victim, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->plan_scalars, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
@@ -72,8 +74,6 @@ extern "C" void cascade_destroy(cascade_ctx *ctx) {
     cudaSetDevice(ctx->device);
     cudaFree(ctx->status_dev);
     cudaFreeHost(ctx->status_host);
-    cudaFree(ctx->pack_by_slot);
-    cudaFree(ctx->pack_sorted);
     cudaFree(ctx->work_admit);
     cudaFree(ctx->work_victim);
     cudaFree(ctx->plan_scalars);

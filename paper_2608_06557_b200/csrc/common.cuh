@@ -16,13 +16,13 @@ struct cascade_ctx {
     uint32_t *status_host;       // pinned mirror used by cascade_status
     int cuda_error;              // last failing cudaError_t
     // tier-plan scratch
-    uint64_t *pack_by_slot;      // per-request decision word, slot order
-    uint64_t *pack_sorted;       // the same words gathered into schedule order
     int4 *work_admit;            // per admitted request: slot, pop offset, restore offset, counts
     int4 *work_victim;           // per preempted request: slot, freed offset, evict offset, action
     int32_t *plan_scalars;       // device scalars handed from the plan kernel to the apply kernels
     int sort_cluster;            // cluster size override for the ordering kernel (0 = automatic)
     int sort_items;              // keys per thread override (0 = automatic)
+    int sort_threads;            // threads per CTA override (0 = automatic)
+    int sort_match;              // 1: rank digits with match.any, 0: with eight ballots
     int copy_ctas_host;          // copy CTAs per SM when the record pool is pinned host memory
     int copy_ctas_dev;           // copy CTAs per SM when the record pool is device memory
 };
@@ -78,6 +78,28 @@ __device__ __forceinline__ bool dev_request_valid(int32_t bt, int64_t P, int64_t
     int64_t h = n0 + n1 + n2;
     if (h > (int64_t(1) << 13)) return false;
     return h * bt < P;
+}
+
+// Geometry of the two cluster kernels (ordering and tier plan): T threads per CTA, K elements per
+// thread, C CTAs per cluster, C*T*K >= n and T*K <= 4096.  Chosen by measurement on B200; the
+// context's overrides (environment, for tuning) win when they are consistent.
+static inline bool cascade_pick_geometry(const cascade_ctx *ctx, int n, int *T, int *C, int *K) {
+    int t, c, k;
+    if (n <= 1024) { t = 256; c = 4; k = 1; }
+    else if (n <= 2048) { t = 256; c = 8; k = 1; }
+    else if (n <= 4096) { t = 256; c = 8; k = 2; }
+    else if (n <= 8192) { t = 256; c = 16; k = 2; }
+    else if (n <= 16384) { t = 512; c = 16; k = 2; }
+    else if (n <= 32768) { t = 512; c = 16; k = 4; }
+    else { t = 512; c = 16; k = 8; }
+    if (ctx->sort_threads == 256 || ctx->sort_threads == 512 || ctx->sort_threads == 1024) t = ctx->sort_threads;
+    if (ctx->sort_items == 1 || ctx->sort_items == 2 || ctx->sort_items == 4 || ctx->sort_items == 8)
+        k = ctx->sort_items;
+    if (ctx->sort_cluster == 1 || ctx->sort_cluster == 2 || ctx->sort_cluster == 4 || ctx->sort_cluster == 8 ||
+        ctx->sort_cluster == 16)
+        c = ctx->sort_cluster;
+    *T = t; *C = c; *K = k;
+    return (long long)c * t * k >= n && t * k <= 4096;
 }
 
 // entry points implemented in the other translation units

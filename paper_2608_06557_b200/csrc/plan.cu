@@ -1,27 +1,35 @@
 // cascade_tier_plan: restore bound (Eq. 7), restore-vs-recompute choice, HBM capacity check,
 // preemption victims with their disposition (Algorithm 1), and deterministic block-id allocation.
 //
-// Kernel 1 (one CTA of 1024 threads): a per-request phase in slot order (coalesced SoA loads, the
-// only int64 divisions of the path, at most two per admitted request), then two block-wide scans
-// over the schedule order - a forward scan over the admitted set (cumulative HBM need, restore-list
-// offsets) and a backward scan over the preemptable holders (freed-block and evict-list offsets).
-// The sequential "pop one request at a time / preempt the largest budget" loops of Algorithm 1
-// become prefix sums because admitted requests and victims are prefixes of the order walked
-// forwards and backwards.
+// Kernel 1 (one thread-block cluster, the queue spread over its CTAs in schedule order, K
+// elements per thread held in registers):
+//   phase 1  gather each request's fields through `order`, evaluate Eq. 7 and the candidate plans
+//            (the only int64 divisions of the path, at most two per admitted request);
+//   phase 2  forward prefix sums over the admitted set (cumulative HBM need, restore-list offsets)
+//            and the sum of preemptable blocks; one exchange of per-CTA totals through distributed
+//            shared memory; the admitted set is cut where the cumulative need exceeds the capacity;
+//   phase 3  prefix sums over the preemptable holders; one more exchange; walking the order
+//            backwards is the same as subtracting the forward inclusive sum from the total, so the
+//            sequential "pop one request / preempt the largest budget" loops of Algorithm 1 become
+//            two scans because admitted requests and victims are prefixes of the two walks;
+//   phase 4  per-request outputs are scattered by slot; CTA 0 writes the counts.
+// Three hardware cluster barriers are the only inter-CTA waits (no spin loops).
 // Kernels 2 and 3 (many CTAs, one warp per request): rewrite block tables, free lists and the two
 // copy lists from the offsets kernel 1 left in scratch; pushes of freed ids (kernel 2) finish
 // before any pop (kernel 3).  In plan-only mode (no tables) only kernel 1 runs.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
-constexpr int kThreads = 1024;
-constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kMaxCluster = 16;
 
-// decision word: n0 (14 bits) | x1 (14) | tokens_run (18) | flags
-constexpr int kX1Shift = 14, kRunShift = 28;
-constexpr unsigned long long kAdm = 1ull << 46, kPriv = 1ull << 47, kFits = 1ull << 48, kValid = 1ull << 49;
+// element flags
+constexpr unsigned kAdm = 1u, kPriv = 2u, kFits = 4u, kValid = 8u, kReal = 16u;
 
 struct PlanArgs {
     const int32_t *prompt, *n0, *n1, *n2;
@@ -31,7 +39,6 @@ struct PlanArgs {
     int32_t *grant;
     cascade_pools pools;
     cascade_plan plan;
-    uint64_t *pack_by_slot, *pack_sorted;
     int4 *work_admit, *work_victim;
     int32_t *scalars;
     uint32_t *status;
@@ -40,43 +47,69 @@ struct PlanArgs {
     int with_tables;
 };
 
-__device__ __forceinline__ int unpack_n0(unsigned long long w) { return int(w & 0x3fff); }
-__device__ __forceinline__ int unpack_x1(unsigned long long w) { return int((w >> kX1Shift) & 0x3fff); }
-__device__ __forceinline__ int unpack_run(unsigned long long w) { return int((w >> kRunShift) & 0x3ffff); }
+// per-CTA totals published to every CTA of the cluster
+struct __align__(16) Exch1 {
+    int need, x1, cnt, evictable;
+};
+struct __align__(16) Exch2 {
+    int v, h, c;                      // preemptable holders: blocks, blocks that fit, requests
+    int kept_need, kept_cnt, kept_x1, unadm;
+    int pad;
+    long long tokens;
+    long long pad2;
+};
+struct __align__(16) Exch3 {
+    int nv, freed, nev, pad;
+};
 
-// Block-wide exclusive scan of three int32 partials (one per thread); totals returned in tot[3].
-__device__ void block_scan3(int &a, int &b, int &c, int *tot, int (*ws)[3]) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int ia = a, ib = b, ic = c;
+__device__ __forceinline__ int warp_incl_scan_i(int v, int lane) {
 #pragma unroll
     for (int s = 1; s < 32; s <<= 1) {
-        int ta = __shfl_up_sync(kFull, ia, s), tb = __shfl_up_sync(kFull, ib, s), tc = __shfl_up_sync(kFull, ic, s);
-        if (lane >= s) { ia += ta; ib += tb; ic += tc; }
+        int t = __shfl_up_sync(kFull, v, s);
+        if (lane >= s) v += t;
     }
-    if (lane == 31) { ws[warp][0] = ia; ws[warp][1] = ib; ws[warp][2] = ic; }
+    return v;
+}
+
+// Inclusive scan of three per-element int32 values over the CTA's T*K elements laid out as
+// (warp, round, lane); returns inclusive values in place and CTA totals in tot[3].
+template <int T, int K>
+__device__ __forceinline__ void cta_scan3(int (&a)[K], int (&b)[K], int (&c)[K], int *tot, int (*ws)[3]) {
+    constexpr int W = T / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int ra = 0, rb = 0, rc = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const int ia = warp_incl_scan_i(a[k], lane), ib = warp_incl_scan_i(b[k], lane),
+                  ic = warp_incl_scan_i(c[k], lane);
+        a[k] = ra + ia;
+        b[k] = rb + ib;
+        c[k] = rc + ic;
+        ra += __shfl_sync(kFull, ia, 31);
+        rb += __shfl_sync(kFull, ib, 31);
+        rc += __shfl_sync(kFull, ic, 31);
+    }
+    if (lane == 0) { ws[warp][0] = ra; ws[warp][1] = rb; ws[warp][2] = rc; }
     __syncthreads();
     if (warp == 0) {
-        int va = ws[lane][0], vb = ws[lane][1], vc = ws[lane][2];
-        int ja = va, jb = vb, jc = vc;
-#pragma unroll
-        for (int s = 1; s < 32; s <<= 1) {
-            int ta = __shfl_up_sync(kFull, ja, s), tb = __shfl_up_sync(kFull, jb, s), tc = __shfl_up_sync(kFull, jc, s);
-            if (lane >= s) { ja += ta; jb += tb; jc += tc; }
-        }
-        ws[lane][0] = ja - va; ws[lane][1] = jb - vb; ws[lane][2] = jc - vc;
-        if (lane == 31) { ws[kWarps][0] = ja; ws[kWarps][1] = jb; ws[kWarps][2] = jc; }
+        const bool in = lane < W;
+        const int va = in ? ws[lane][0] : 0, vb = in ? ws[lane][1] : 0, vc = in ? ws[lane][2] : 0;
+        const int ja = warp_incl_scan_i(va, lane), jb = warp_incl_scan_i(vb, lane), jc = warp_incl_scan_i(vc, lane);
+        if (in) { ws[lane][0] = ja - va; ws[lane][1] = jb - vb; ws[lane][2] = jc - vc; }
+        if (lane == 31) { ws[32][0] = ja; ws[32][1] = jb; ws[32][2] = jc; }
     }
     __syncthreads();
-    a = ws[warp][0] + ia - a;
-    b = ws[warp][1] + ib - b;
-    c = ws[warp][2] + ic - c;
-    tot[0] = ws[kWarps][0]; tot[1] = ws[kWarps][1]; tot[2] = ws[kWarps][2];
+    const int oa = ws[warp][0], ob = ws[warp][1], oc = ws[warp][2];
+#pragma unroll
+    for (int k = 0; k < K; ++k) { a[k] += oa; b[k] += ob; c[k] += oc; }
+    tot[0] = ws[32][0]; tot[1] = ws[32][1]; tot[2] = ws[32][2];
     __syncthreads();
 }
 
-// Block-wide sum of up to six int64 partials; every thread gets the totals.
-template <int M>
-__device__ void block_sum(long long (&v)[M], long long (*ws)[6]) {
+// Sum of M int64 partials over the CTA; the totals land in every thread.
+template <int T, int M>
+__device__ __forceinline__ void cta_sum(long long (&v)[M], long long (*ws)[8]) {
+    constexpr int W = T / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int m = 0; m < M; ++m)
@@ -87,7 +120,7 @@ __device__ void block_sum(long long (&v)[M], long long (*ws)[6]) {
     __syncthreads();
 #pragma unroll
     for (int m = 0; m < M; ++m) {
-        long long t = ws[lane][m];
+        long long t = lane < W ? ws[lane][m] : 0;
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) t += __shfl_xor_sync(kFull, t, s);
         v[m] = t;
@@ -95,11 +128,19 @@ __device__ void block_sum(long long (&v)[M], long long (*ws)[6]) {
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+template <int T, int K>
+__global__ void __launch_bounds__(T, 1)
 plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ PlanArgs a) {
-    __shared__ int ws3[kWarps + 1][3];
-    __shared__ long long ws6[kWarps][6];
-    const int tid = threadIdx.x;
+    constexpr int per = T * K;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned crank = cluster.block_rank();
+    const unsigned csize = cluster.num_blocks();
+    __shared__ int ws3[33][3];
+    __shared__ long long ws8[32][8];
+    __shared__ Exch1 ex1[kMaxCluster];
+    __shared__ Exch2 ex2[kMaxCluster];
+    __shared__ Exch3 ex3[kMaxCluster];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = a.n;
     const int bt = p.bt;
     uint32_t st = 0;
@@ -117,22 +158,41 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         }
     }
 
-    // ---- phase 1, slot order: Eq. 7 bounds and the restore-vs-recompute choice ------------------
-    for (int r = tid; r < n; r += kThreads) {
+    // ---- phase 1: gather through the order, Eq. 7 bounds, restore-vs-recompute choice -----------
+    uint32_t slot[K];
+    unsigned fl[K];
+    int n0v[K], x1v[K], runv[K];
+    long long pos0 = (long long)crank * per + (warp * K) * 32 + lane;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const long long q = pos0 + k * 32;
+        slot[k] = q < n ? a.order[q] : 0u;
+    }
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const long long q = pos0 + k * 32;
+        fl[k] = 0;
+        n0v[k] = 0;
+        x1v[k] = 0;
+        runv[k] = 0;
+        if (q >= n) continue;
+        const uint32_t r = slot[k];
         const long long P = a.prompt[r], n0 = a.n0[r], n1 = a.n1[r], n2 = a.n2[r];
         const long long b = a.budget[r];
         const int g = a.grant[r];
+        const unsigned rf = a.flags[r];
         bool valid = dev_request_valid(bt, P, n0, n1, n2);
         if (valid && a.with_tables) valid = (P + bt - 1) / bt <= a.pools.maxb;
-        unsigned long long w = 0;
-        int x1 = 0, x2 = 0, run = 0;
+        int x2 = 0;
         if (!valid) {
             st |= CASCADE_ST_EPRECOND;
             if (g != 0) a.grant[r] = 0;
+            fl[k] = kReal;
         } else {
-            w = kValid | (unsigned long long)n0;
-            if (a.flags[r] & CASCADE_FLAG_HBM_PRIVATE) w |= kPriv;
-            if (dev_restore_time(p, 1, n0) <= b) w |= kFits;
+            fl[k] = kReal | kValid;
+            n0v[k] = (int)n0;
+            if (rf & CASCADE_FLAG_HBM_PRIVATE) fl[k] |= kPriv;
+            if (dev_restore_time(p, 1, n0) <= b) fl[k] |= kFits;
             if (g > 0) {
                 const long long rem = b > 0 ? b : 0;
                 // Eq. 7, host tier first
@@ -164,151 +224,184 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
                                         dev_comp_q(a.A_act, p.c_attn_q20, P, (n0 + n1 + x2max) * bt);
                     if (F <= bF) { bF = F; bx1 = n1; bx2 = x2max; }
                 }
-                x1 = (int)bx1;
-                x2 = (int)bx2;
                 // a deep fetch is staged first: nothing runs now, HBM is taken at the last hop only
                 const long long left = P - (n0 + bx1) * bt;
-                run = bx2 > 0 ? 0 : (int)(g < left ? g : left);
-                w |= kAdm | ((unsigned long long)x1 << kX1Shift) | ((unsigned long long)run << kRunShift);
+                x1v[k] = (int)bx1;
+                x2 = (int)bx2;
+                runv[k] = bx2 > 0 ? 0 : (int)(g < left ? g : left);
+                fl[k] |= kAdm;
             }
         }
-        a.pack_by_slot[r] = w;
-        a.plan.x1[r] = x1;
-        a.plan.x2[r] = x2;
-        a.plan.tokens_run[r] = run;
+        a.plan.x2[r] = x2;   // rewritten below if the request is un-admitted
     }
-    __syncthreads();
 
-    // ---- phase 2a, forward over the order: HBM capacity and offsets of the admitted set ---------
-    const int ipt = (n + kThreads - 1) / kThreads;
-    const int lo = min(n, tid * ipt), hi = min(n, lo + ipt);
-    int t_need = 0, t_x1 = 0, t_cnt = 0;
-    long long t_evictable = 0;
-    for (int q = lo; q < hi; ++q) {
-        const unsigned long long w = a.pack_by_slot[a.order[q]];
-        a.pack_sorted[q] = w;
-        if (w & kValid) {
-            if (w & kAdm) {
-                const int x1 = unpack_x1(w);
-                t_need += x1 + (unpack_run(w) + bt - 1) / bt;
-                t_x1 += x1;
-                ++t_cnt;
-            } else if (w & kPriv) {
-                t_evictable += unpack_n0(w);
-            }
+    // ---- phase 2: forward scan over the admitted set, capacity cut --------------------------------
+    int s_need[K], s_x1[K], s_cnt[K];
+    long long evictable = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const bool adm = fl[k] & kAdm;
+        s_need[k] = adm ? x1v[k] + (runv[k] + bt - 1) / bt : 0;
+        s_x1[k] = adm ? x1v[k] : 0;
+        s_cnt[k] = adm ? 1 : 0;
+        if ((fl[k] & kValid) && !adm && (fl[k] & kPriv)) evictable += n0v[k];
+    }
+    int tot[3];
+    cta_scan3<T, K>(s_need, s_x1, s_cnt, tot, ws3);
+    long long red1[1] = {evictable};
+    cta_sum<T, 1>(red1, ws8);
+    if (tid < csize) {
+        Exch1 x;
+        x.need = tot[0];
+        x.x1 = tot[1];
+        x.cnt = tot[2];
+        x.evictable = (int)red1[0];
+        cluster.map_shared_rank(ex1, tid)[crank] = x;
+    }
+    cluster.sync();
+    long long off_need = 0, cap = hbm_cnt;
+    int off_x1 = 0, off_cnt = 0;
+#pragma unroll
+    for (int c = 0; c < kMaxCluster; ++c) {
+        if (c < csize) {
+            const Exch1 x = ex1[c];
+            cap += x.evictable;
+            if (c < crank) { off_need += x.need; off_x1 += x.x1; off_cnt += x.cnt; }
         }
     }
-    int tot3[3];
-    block_scan3(t_need, t_x1, t_cnt, tot3, ws3);
-    long long red1[1] = {t_evictable};
-    block_sum<1>(red1, ws6);
-    const long long cap = hbm_cnt + red1[0];
+    long long k_need = 0, k_cnt = 0, k_x1 = 0, k_unadm = 0, k_tok = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (!(fl[k] & kAdm)) continue;
+        const int nd = x1v[k] + (runv[k] + bt - 1) / bt;
+        const long long c_incl = off_need + s_need[k];
+        if (c_incl > cap) {
+            // HBM cannot hold it even after preempting everything preemptable: cut from the tail
+            fl[k] &= ~kAdm;
+            x1v[k] = 0;
+            runv[k] = 0;
+            a.grant[slot[k]] = 0;
+            a.plan.x2[slot[k]] = 0;
+            ++k_unadm;
+            st |= CASCADE_ST_ENOSPC;
+        } else {
+            k_need += nd;
+            ++k_cnt;
+            k_x1 += x1v[k];
+            k_tok += runv[k];
+            a.work_admit[off_cnt + s_cnt[k] - 1] =
+                make_int4((int)slot[k], (int)(c_incl - nd), off_x1 + s_x1[k] - x1v[k], (x1v[k] << 18) | nd);
+        }
+    }
 
-    long long s_need = 0, s_adm = 0, s_tok = 0, s_unadm = 0, s_rest = 0;
-    {
-        long long c = t_need;
-        int rx = t_x1, ci = t_cnt;
-        for (int q = lo; q < hi; ++q) {
-            unsigned long long w = a.pack_sorted[q];
-            if ((w & kValid) && (w & kAdm)) {
-                const int x1 = unpack_x1(w), run = unpack_run(w);
-                const int nd = x1 + (run + bt - 1) / bt;
-                c += nd;
-                const uint32_t slot = a.order[q];
-                if (c > cap) {
-                    // HBM cannot hold it even after preempting everything preemptable: cut from the tail
-                    a.grant[slot] = 0;
-                    a.plan.x1[slot] = 0;
-                    a.plan.x2[slot] = 0;
-                    a.plan.tokens_run[slot] = 0;
-                    a.pack_sorted[q] = w & (kValid | kPriv | kFits | 0x3fffull);
-                    ++s_unadm;
-                    st |= CASCADE_ST_ENOSPC;
-                } else {
-                    s_need += nd;
-                    ++s_adm;
-                    s_tok += run;
-                    s_rest += x1;
-                    a.work_admit[ci] = make_int4((int)slot, (int)(c - nd), rx, (x1 << 18) | nd);
-                }
-                rx += x1;
-                ++ci;
-            }
+    // ---- phase 3: preemptable holders, walked backwards ---------------------------------------------
+    int s_v[K], s_h[K], s_c[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const bool elig = (fl[k] & kValid) && !(fl[k] & kAdm) && (fl[k] & kPriv) && n0v[k] > 0;
+        s_v[k] = elig ? n0v[k] : 0;
+        s_h[k] = (elig && (fl[k] & kFits)) ? n0v[k] : 0;
+        s_c[k] = elig ? 1 : 0;
+    }
+    cta_scan3<T, K>(s_v, s_h, s_c, tot, ws3);
+    long long red5[5] = {k_need, k_cnt, k_x1, k_unadm, k_tok};
+    cta_sum<T, 5>(red5, ws8);
+    if (tid < csize) {
+        Exch2 x;
+        x.v = tot[0];
+        x.h = tot[1];
+        x.c = tot[2];
+        x.kept_need = (int)red5[0];
+        x.kept_cnt = (int)red5[1];
+        x.kept_x1 = (int)red5[2];
+        x.unadm = (int)red5[3];
+        x.pad = 0;
+        x.tokens = red5[4];
+        x.pad2 = 0;
+        cluster.map_shared_rank(ex2, tid)[crank] = x;
+    }
+    cluster.sync();
+    long long need_total = 0, V = 0, H = 0, tokens = 0;
+    int Cn = 0, off_v = 0, off_h = 0, off_c = 0, n_adm = 0, n_rest = 0, n_unadm = 0;
+#pragma unroll
+    for (int c = 0; c < kMaxCluster; ++c) {
+        if (c < csize) {
+            const Exch2 x = ex2[c];
+            need_total += x.kept_need;
+            n_adm += x.kept_cnt;
+            n_rest += x.kept_x1;
+            n_unadm += x.unadm;
+            tokens += x.tokens;
+            V += x.v;
+            H += x.h;
+            Cn += x.c;
+            if (c < crank) { off_v += x.v; off_h += x.h; off_c += x.c; }
         }
     }
-    long long red5[5] = {s_need, s_adm, s_tok, s_unadm, s_rest};
-    block_sum<5>(red5, ws6);  // also orders the pack_sorted rewrites before phase 2b reads them
-    const long long need_total = red5[0];
     long long deficit = need_total - hbm_cnt;
     if (deficit < 0) deficit = 0;
-
-    // ---- phase 2b, backward over the order: victims and their disposition -----------------------
-    int t_v = 0, t_h = 0, t_c = 0;
-    for (int q = lo; q < hi; ++q) {
-        const unsigned long long w = a.pack_sorted[n - 1 - q];
-        if ((w & kValid) && !(w & kAdm) && (w & kPriv)) {
-            const int n0 = unpack_n0(w);
-            if (n0 > 0) {
-                t_v += n0;
-                ++t_c;
-                if (w & kFits) t_h += n0;
-            }
-        }
-    }
-    block_scan3(t_v, t_h, t_c, tot3, ws3);
     long long s_nv = 0, s_freed = 0, s_nev = 0;
-    {
-        long long v = t_v, h = t_h;
-        int ci = t_c;
-        for (int q = lo; q < hi; ++q) {
-            const int pos = n - 1 - q;
-            const unsigned long long w = a.pack_sorted[pos];
-            const uint32_t slot = a.order[pos];
-            uint8_t act = CASCADE_ACT_NONE;
-            if (w & kValid) {
-                const int n0 = unpack_n0(w);
-                const bool elig = !(w & kAdm) && (w & kPriv) && n0 > 0;
-                if (elig && v < deficit) {
-                    // spill only if it can be brought back within the victim's own budget and host has room
-                    const bool ev = (w & kFits) && (h + n0 <= host_cnt);
-                    act = ev ? CASCADE_ACT_EVICT : CASCADE_ACT_DROP;
-                    a.work_victim[ci] = make_int4((int)slot, (int)v, (int)h, (int)act);
-                    ++s_nv;
-                    s_freed += n0;
-                    if (ev) s_nev += n0;
-                } else if (n0 > 0) {
-                    act = CASCADE_ACT_RETAIN;
-                }
-                if (elig) {
-                    v += n0;
-                    ++ci;
-                    if (w & kFits) h += n0;
-                }
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (!(fl[k] & kReal)) continue;
+        uint8_t act = CASCADE_ACT_NONE;
+        if (fl[k] & kValid) {
+            const int n0 = n0v[k];
+            const bool elig = !(fl[k] & kAdm) && (fl[k] & kPriv) && n0 > 0;
+            // blocks of preemptable holders visited before this one when the order is walked backwards
+            const long long v = V - (off_v + s_v[k]);
+            if (elig && v < deficit) {
+                // spill only if it can be brought back within the victim's own budget and host has room
+                const long long h = H - (off_h + s_h[k]);
+                const bool ev = (fl[k] & kFits) && (h + n0 <= host_cnt);
+                act = ev ? CASCADE_ACT_EVICT : CASCADE_ACT_DROP;
+                a.work_victim[Cn - (off_c + s_c[k])] = make_int4((int)slot[k], (int)v, (int)h, (int)act);
+                ++s_nv;
+                s_freed += n0;
+                if (ev) s_nev += n0;
+            } else if (n0 > 0) {
+                act = CASCADE_ACT_RETAIN;
             }
-            a.plan.action[slot] = act;
         }
+        // ---- phase 4: per-request outputs, scattered by slot ---------------------------------------
+        a.plan.action[slot[k]] = act;
+        a.plan.x1[slot[k]] = x1v[k];
+        a.plan.tokens_run[slot[k]] = runv[k];
     }
     long long red3[3] = {s_nv, s_freed, s_nev};
-    block_sum<3>(red3, ws6);
-
-    st = __reduce_or_sync(kFull, st);
-    if ((tid & 31) == 0 && st) atomicOr(a.status, st);
+    cta_sum<T, 3>(red3, ws8);
     if (tid == 0) {
-        const long long freed = red3[1], nev = red3[2];
+        Exch3 x;
+        x.nv = (int)red3[0];
+        x.freed = (int)red3[1];
+        x.nev = (int)red3[2];
+        x.pad = 0;
+        cluster.map_shared_rank(ex3, 0)[crank] = x;
+    }
+    st = __reduce_or_sync(kFull, st);
+    if (lane == 0 && st) atomicOr(a.status, st);
+    cluster.sync();
+    if (crank == 0 && tid == 0) {
+        long long nv = 0, freed = 0, nev = 0;
+        for (unsigned c = 0; c < csize; ++c) {
+            nv += ex3[c].nv;
+            freed += ex3[c].freed;
+            nev += ex3[c].nev;
+        }
         cascade_plan_counts *c = a.plan.counts;
-        c->n_restore = (int)red5[4];
+        c->n_restore = n_rest;
         c->n_evict = (int)nev;
         c->n_drop_blocks = (int)(freed - nev);
-        c->n_victims = (int)red3[0];
-        c->n_unadmitted = (int)red5[3];
-        c->n_admitted = (int)red5[1];
+        c->n_victims = (int)nv;
+        c->n_unadmitted = n_unadm;
+        c->n_admitted = n_adm;
         c->hbm_need = (int)need_total;
         c->deficit = (int)deficit;
         c->hbm_free_after = (int)(hbm_cnt + freed - need_total);
         c->host_free_after = (int)(host_cnt - nev);
-        c->tokens_run = red5[2];
-        a.scalars[PS_N_ADMIT] = (int)red5[1];
-        a.scalars[PS_N_VICTIM] = (int)red3[0];
+        c->tokens_run = tokens;
+        a.scalars[PS_N_ADMIT] = n_adm;
+        a.scalars[PS_N_VICTIM] = (int)nv;
         a.scalars[PS_HBM_CNT0] = (int)hbm_cnt;
         a.scalars[PS_HOST_CNT0] = (int)host_cnt;
         a.scalars[PS_TOTAL_FREED] = (int)freed;
@@ -395,6 +488,38 @@ apply_admitted_kernel(const __grid_constant__ PlanArgs a) {
     if (st) atomicOr(a.status, st);
 }
 
+
+
+template <int T, int K>
+cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_size, cudaStream_t stream) {
+    cudaFuncSetAttribute(plan_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cluster_size, 1, 1);
+    cfg.blockDim = dim3(T, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster_size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, plan_kernel<T, K>, p, a);
+}
+
+template <int T>
+cudaError_t launch_plan_k(int K, const cascade_params &p, const PlanArgs &a, int C, cudaStream_t s) {
+    switch (K) {
+        case 1: return launch_plan<T, 1>(p, a, C, s);
+        case 2: return launch_plan<T, 2>(p, a, C, s);
+        case 4: return launch_plan<T, 4>(p, a, C, s);
+        default:
+            if constexpr (T <= 512) return launch_plan<T, 8>(p, a, C, s);
+            else return cudaErrorInvalidConfiguration;
+    }
+}
+
 }  // namespace
 
 extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *budget,
@@ -427,8 +552,6 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     a.grant = grant;
     a.pools = *pools;
     a.plan = *plan_out;
-    a.pack_by_slot = ctx->pack_by_slot;
-    a.pack_sorted = ctx->pack_sorted;
     a.work_admit = ctx->work_admit;
     a.work_victim = ctx->work_victim;
     a.scalars = ctx->plan_scalars;
@@ -436,8 +559,12 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     a.A_act = make_load_consts(ctx->params, D_act, K_act).A_act;
     a.n = n;
     a.with_tables = with_tables ? 1 : 0;
-    plan_kernel<<<1, kThreads, 0, s>>>(ctx->params, a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    int T, C, K;
+    if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, s)
+                  : T == 512 ? launch_plan_k<512>(K, ctx->params, a, C, s)
+                             : launch_plan_k<1024>(K, ctx->params, a, C, s);
+    CASCADE_CUDA_TRY(ctx, e);
     if (with_tables && n > 0) {
         const int grid = ctx->num_sms * 2;
         apply_victims_kernel<<<grid, 256, 0, s>>>(a);

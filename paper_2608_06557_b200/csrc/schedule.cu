@@ -1,18 +1,19 @@
 // cascade_schedule: least-remaining-budget-first order (64-bit LSD radix sort) and prefix-sum
 // admission (Algorithm 1, phase 2) in ONE kernel launch.
 //
-// Layout: a thread-block cluster of C CTAs (C = 1, 2, 4, 8) holds the whole queue in shared memory,
-// 1024*K elements of 16 bytes (key, slot, want) per CTA.  Each radix pass
-//   (a) ranks the 8-bit digits of a warp's 32*K consecutive elements with __match_any_sync and a
-//       per-warp 16-bit histogram in shared memory (stable within the warp),
-//   (b) scans those histograms across the 32 warps with warp shuffles,
-//   (c) exchanges the 256-bin CTA histograms through distributed shared memory and derives, per
-//       digit, the global base of this CTA,
+// Layout: a thread-block cluster of C CTAs (C = 1..16) holds the whole queue in shared memory,
+// T*K elements of 16 bytes (key, slot, want) per CTA (T threads, K elements per thread).  Each
+// radix pass
+//   (a) ranks the 8-bit digits of a warp's 32*K consecutive elements (stable within the warp) with
+//       a per-warp 16-bit histogram in shared memory,
+//   (b) scans those histograms across the CTA's warps with segmented warp shuffles and PUSHES the
+//       256-bin CTA histogram into every CTA of the cluster (distributed shared memory stores),
+//   (c) derives, per digit, the global base of this CTA from the locally received histograms,
 //   (d) scatters every element straight into the destination CTA's shared memory (16-byte
 //       remote store), so keys never visit global memory between passes.
 // Passes whose digit is the same in every key are skipped.  The admission scans run on the sorted
-// elements while they are still on chip.  Two cluster barriers per pass are the only waits; they
-// are hardware barriers (no spin loops).
+// elements while they are still on chip.  Two cluster barriers per pass are the only inter-CTA
+// waits; they are hardware barriers (no spin loops).
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -21,10 +22,9 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-constexpr int kThreads = 1024;
-constexpr int kWarps = kThreads / 32;
 constexpr int kBins = 256;
 constexpr int kWhistStride = kBins + 2;  // in uint16 units: column reads by 32 lanes hit 32 banks
+constexpr int kMaxCluster = 16;
 constexpr unsigned kFull = 0xffffffffu;
 
 struct __align__(16) SortElem {
@@ -33,8 +33,8 @@ struct __align__(16) SortElem {
     int32_t want;
 };
 
-// per-CTA values published to the cluster
-struct Exch {
+// per-CTA values published to every CTA of the cluster
+struct __align__(16) Exch {
     unsigned long long diff;  // OR of (key ^ key[0]) over this CTA's keys
     long long w1, w2;         // tokens wanted by this CTA's Tier-1 / Tier-2 elements
     int n1;                   // Tier-1 elements in this CTA
@@ -52,41 +52,42 @@ struct ScheduleArgs {
     int seq_cap;        // max_batch - D_act, >= 0
     int n;
     int bt;
-    int per_shift;      // log2(elements per CTA)
 };
 
-__device__ __forceinline__ long long warp_incl_scan(long long v, int lane) {
-#pragma unroll
-    for (int s = 1; s < 32; s <<= 1) {
-        long long t = __shfl_up_sync(kFull, v, s);
-        if (lane >= s) v += t;
+#ifdef CASCADE_PHASE_TIMING
+__device__ long long g_phase_ticks[128];
+#define TICK(i) do { if (tid == 0 && crank == 0) g_phase_ticks[(i)] = clock64(); } while (0)
+#else
+#define TICK(i) do { } while (0)
+#endif
+
+template <typename T>
+__device__ __forceinline__ T seg_incl_scan(T v, int pos, int width) {
+    // inclusive scan inside aligned groups of `width` lanes; pos = lane % width
+    for (int s = 1; s < width; s <<= 1) {
+        T t = __shfl_up_sync(kFull, v, s, width);
+        if (pos >= s) v += t;
     }
     return v;
 }
 
-__device__ __forceinline__ unsigned warp_incl_scan(unsigned v, int lane) {
-#pragma unroll
-    for (int s = 1; s < 32; s <<= 1) {
-        unsigned t = __shfl_up_sync(kFull, v, s);
-        if (lane >= s) v += t;
-    }
-    return v;
-}
-
-template <int K>
-__global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_constant__ ScheduleArgs a) {
+template <int T, int K, bool kMatch>
+__global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ ScheduleArgs a) {
+    constexpr int W = T / 32;          // warps per CTA
+    constexpr int per = T * K;         // elements per CTA
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned crank = cluster.block_rank();
     const unsigned csize = cluster.num_blocks();
-    constexpr int per = kThreads * K;
 
     extern __shared__ __align__(16) unsigned char smem[];
     SortElem *elems = reinterpret_cast<SortElem *>(smem);
-    uint16_t *whist = reinterpret_cast<uint16_t *>(smem + size_t(per) * sizeof(SortElem));
-    uint32_t *hist = reinterpret_cast<uint32_t *>(whist + kWarps * kWhistStride);
-    uint32_t *base = hist + kBins;
-    long long *wtmp = reinterpret_cast<long long *>(base + kBins);  // 3 * 32 entries
-    Exch *exch = reinterpret_cast<Exch *>(wtmp + 3 * kWarps);
+    SortElem *stage = elems + per;
+    uint16_t *whist = reinterpret_cast<uint16_t *>(smem + 2 * size_t(per) * sizeof(SortElem));
+    uint16_t *allhist = whist + W * kWhistStride;                      // [kMaxCluster][kBins]
+    uint32_t *base = reinterpret_cast<uint32_t *>(allhist + kMaxCluster * kBins);
+    uint32_t *lbase = base + kBins;
+    long long *wtmp = reinterpret_cast<long long *>(lbase + kBins);    // 3 * 32 entries
+    Exch *exall = reinterpret_cast<Exch *>(wtmp + 3 * 32);             // [kMaxCluster]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned lt_mask = (1u << lane) - 1u;
@@ -96,6 +97,7 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
         a.counts->tokens_granted = 0;
     }
 
+    TICK(66);
     // ---- load: key, slot, tokens wanted (prompt minus the matched prefix) ----------------------
     SortElem e[K];
     const unsigned long long key0 = a.key[0];
@@ -125,21 +127,24 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
         if (lane == 0) wtmp[warp] = (long long)(((unsigned long long)hi << 32) | lo);
         __syncthreads();
         if (warp == 0) {
-            unsigned long long v = (unsigned long long)wtmp[lane];
+            unsigned long long v = lane < W ? (unsigned long long)wtmp[lane] : 0ull;
             lo = __reduce_or_sync(kFull, (unsigned)v);
             hi = __reduce_or_sync(kFull, (unsigned)(v >> 32));
-            if (lane == 0) exch->diff = ((unsigned long long)hi << 32) | lo;
+            if (lane < csize) cluster.map_shared_rank(exall, lane)[crank].diff = ((unsigned long long)hi << 32) | lo;
         }
     }
     cluster.sync();
     unsigned long long alld = 0;
-    for (unsigned c = 0; c < csize; ++c) alld |= cluster.map_shared_rank(exch, c)->diff;
+#pragma unroll
+    for (int c = 0; c < kMaxCluster; ++c)
+        if (c < csize) alld |= exall[c].diff;
 
     // ---- LSD radix sort, 8 bits per pass --------------------------------------------------------
     for (int pass = 0; pass < 8; ++pass) {
         const int shift = pass * 8;
         if (((alld >> shift) & 0xffull) == 0) continue;  // same digit in every key: nothing moves
 
+        TICK(pass * 8 + 0);
         // (a) stable rank of each element among equal digits of its warp's chunk
         uint16_t *myhist = whist + warp * kWhistStride;
         for (int i = lane; i < kWhistStride / 2; i += 32) reinterpret_cast<uint32_t *>(myhist)[i] = 0;
@@ -148,7 +153,17 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
 #pragma unroll
         for (int k = 0; k < K; ++k) {
             const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
-            const unsigned peers = __match_any_sync(kFull, d);
+            unsigned peers;
+            if (kMatch) {
+                peers = __match_any_sync(kFull, d);
+            } else {
+                peers = kFull;
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    const unsigned bal = __ballot_sync(kFull, (d >> b) & 1u);
+                    peers &= ((d >> b) & 1u) ? bal : ~bal;
+                }
+            }
             const unsigned lower = peers & lt_mask;
             const unsigned pre = myhist[d];
             __syncwarp();
@@ -157,49 +172,87 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
             off[k] = pre + __popc(lower);
         }
         __syncthreads();
+        TICK(pass * 8 + 1);
 
-        // (b) exclusive scan across warps, one digit column per iteration; warp j owns digits 8j..8j+7
-#pragma unroll
-        for (int dd = 0; dd < kBins / kWarps; ++dd) {
-            const int d = warp * (kBins / kWarps) + dd;
-            const unsigned v = whist[lane * kWhistStride + d];
-            const unsigned incl = warp_incl_scan(v, lane);
-            whist[lane * kWhistStride + d] = (uint16_t)(incl - v);
-            if (lane == 31) hist[d] = incl;
-        }
-        cluster.sync();  // histograms visible cluster-wide; every CTA holds its elements in registers
-
-        // (c) global base of this CTA for each digit
-        unsigned total = 0, before = 0, incl = 0;
+        // (b) one thread per digit walks its column of the W per-warp histograms (exclusive scan in
+        //     place) and pushes the CTA's count of that digit to every CTA of the cluster
+        unsigned mine = 0;
         if (tid < kBins) {
-            for (unsigned c = 0; c < csize; ++c) {
-                const unsigned h = cluster.map_shared_rank(hist, c)[tid];
-                total += h;
-                if (c < crank) before += h;
+            unsigned v[W];
+#pragma unroll
+            for (int w = 0; w < W; ++w) v[w] = whist[w * kWhistStride + tid];
+#pragma unroll
+            for (int w = 0; w < W; ++w) {
+                whist[w * kWhistStride + tid] = (uint16_t)mine;
+                mine += v[w];
             }
-            incl = warp_incl_scan(total, lane);
+#pragma unroll
+            for (int c = 0; c < kMaxCluster; ++c)
+                if (c < csize) cluster.map_shared_rank(allhist, c)[crank * kBins + tid] = (uint16_t)mine;
+        }
+        TICK(pass * 8 + 2);
+        cluster.sync();  // histograms delivered; every CTA holds its elements in registers
+        TICK(pass * 8 + 3);
+
+        // (c) per digit: global base of this CTA (high bits) and local base inside this CTA (low 14
+        //     bits), both from one packed exclusive scan over the 256 digits
+        unsigned packed = 0, before = 0, incl = 0;
+        if (tid < kBins) {
+            unsigned total = 0;
+#pragma unroll
+            for (int c = 0; c < kMaxCluster; ++c) {
+                if (c < csize) {
+                    const unsigned h = allhist[c * kBins + tid];
+                    total += h;
+                    if (c < crank) before += h;
+                }
+            }
+            packed = (total << 14) | mine;
+            incl = seg_incl_scan(packed, lane, 32);
             if (lane == 31) reinterpret_cast<unsigned *>(wtmp)[warp] = incl;
         }
         __syncthreads();
         if (tid < kBins) {
             unsigned add = 0;
-            for (int w = 0; w < warp; ++w) add += reinterpret_cast<unsigned *>(wtmp)[w];
-            base[tid] = incl - total + add + before;
+#pragma unroll
+            for (int w = 0; w < kBins / 32; ++w) {
+                const unsigned t = reinterpret_cast<unsigned *>(wtmp)[w];
+                if (w < warp) add += t;
+            }
+            const unsigned excl = incl - packed + add;
+            base[tid] = (excl >> 14) + before;      // first global position of this CTA's run of digit tid
+            lbase[tid] = excl & 0x3fffu;            // first local position of that run
         }
         __syncthreads();
+        TICK(pass * 8 + 4);
 
-        // (d) scatter into the owning CTA's shared memory
+        // (d) group the CTA's elements by digit in a local staging buffer, then copy runs of equal
+        //     digits to their owners: consecutive lanes store to consecutive remote addresses
 #pragma unroll
         for (int k = 0; k < K; ++k) {
             const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
-            const unsigned pos = base[d] + whist[warp * kWhistStride + d] + off[k];
-            SortElem *dst = cluster.map_shared_rank(elems, pos >> a.per_shift) + (pos & (per - 1));
-            *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(&e[k]);
+            const unsigned lpos = lbase[d] + whist[warp * kWhistStride + d] + off[k];
+            *reinterpret_cast<uint4 *>(stage + lpos) = *reinterpret_cast<const uint4 *>(&e[k]);
         }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const unsigned i = (warp * K + k) * 32 + lane;
+            const uint4 v = *reinterpret_cast<const uint4 *>(stage + i);
+            const unsigned long long key = ((unsigned long long)v.y << 32) | v.x;
+            const unsigned d = (unsigned)(key >> shift) & 0xffu;
+            const unsigned pos = base[d] + (i - lbase[d]);
+            SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
+            *reinterpret_cast<uint4 *>(dst) = v;
+        }
+        TICK(pass * 8 + 5);
         cluster.sync();  // all remote stores have landed
+        TICK(pass * 8 + 6);
 #pragma unroll
         for (int k = 0; k < K; ++k) e[k] = elems[(warp * K + k) * 32 + lane];
+        TICK(pass * 8 + 7);
     }
+    TICK(64);
 
     // ---- admission: clamped prefix sums over the sorted elements ---------------------------------
     long long ex[K];
@@ -212,7 +265,7 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
         const bool t2 = (e[k].key >> 63) != 0;
         if (real && !t2) { s1 += w; ++c1; }
         if (real && t2) s2 += w;
-        const long long x = warp_incl_scan(w, lane);
+        const long long x = seg_incl_scan(w, lane, 32);
         ex[k] = run + x - w;
         run += __shfl_sync(kFull, x, 31);
     }
@@ -224,39 +277,43 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
     }
     if (lane == 0) {
         wtmp[warp] = run;
-        wtmp[kWarps + warp] = s1;
-        wtmp[2 * kWarps + warp] = s2;
+        wtmp[32 + warp] = s1;
+        wtmp[64 + warp] = s2;
         reinterpret_cast<int *>(base)[warp] = c1;
     }
     __syncthreads();
     if (warp == 0) {
-        const long long t = wtmp[lane];
-        const long long inc = warp_incl_scan(t, lane);
-        long long a1 = wtmp[kWarps + lane], a2 = wtmp[2 * kWarps + lane];
-        int ac = reinterpret_cast<int *>(base)[lane];
+        const bool in = lane < W;
+        const long long t = in ? wtmp[lane] : 0;
+        const long long inc = seg_incl_scan(t, lane, 32);
+        long long a1 = in ? wtmp[32 + lane] : 0, a2 = in ? wtmp[64 + lane] : 0;
+        int ac = in ? reinterpret_cast<int *>(base)[lane] : 0;
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) {
             a1 += __shfl_xor_sync(kFull, a1, s);
             a2 += __shfl_xor_sync(kFull, a2, s);
             ac += __shfl_xor_sync(kFull, ac, s);
         }
-        wtmp[lane] = inc - t;  // exclusive offset of each warp inside the CTA
-        if (lane == 0) {
-            exch->w1 = a1;
-            exch->w2 = a2;
-            exch->n1 = ac;
+        if (in) wtmp[lane] = inc - t;  // exclusive offset of each warp inside the CTA
+        if (lane < csize) {
+            Exch *x = cluster.map_shared_rank(exall, lane) + crank;
+            x->w1 = a1;
+            x->w2 = a2;
+            x->n1 = ac;
         }
     }
     cluster.sync();
     long long W1 = 0, W2 = 0, cta_off = 0;
     int N1 = 0;
-    for (unsigned c = 0; c < csize; ++c) {
-        const Exch *x = cluster.map_shared_rank(exch, c);
-        const long long x1 = x->w1, x2 = x->w2;
-        W1 += x1;
-        W2 += x2;
-        N1 += x->n1;
-        if (c < crank) cta_off += x1 + x2;
+#pragma unroll
+    for (int c = 0; c < kMaxCluster; ++c) {
+        if (c < csize) {
+            const long long x1 = exall[c].w1, x2 = exall[c].w2;
+            W1 += x1;
+            W2 += x2;
+            N1 += exall[c].n1;
+            if (c < crank) cta_off += x1 + x2;
+        }
     }
     const long long R2 = min(min(a.reserve, W2), a.TB);
     const long long TB1 = a.TB - R2;
@@ -281,15 +338,17 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
     if (lane == 0) reinterpret_cast<unsigned *>(wtmp)[warp] = runc;
     __syncthreads();
     if (warp == 0) {
-        const unsigned t = reinterpret_cast<unsigned *>(wtmp)[lane];
-        const unsigned inc = warp_incl_scan(t, lane);
-        reinterpret_cast<unsigned *>(wtmp)[lane] = inc - t;
-        if (lane == 31) exch->cnt = (int)inc;
+        const unsigned t = lane < W ? reinterpret_cast<unsigned *>(wtmp)[lane] : 0u;
+        const unsigned inc = seg_incl_scan(t, lane, 32);
+        if (lane < W) reinterpret_cast<unsigned *>(wtmp)[lane] = inc - t;
+        const int tot = (int)__shfl_sync(kFull, inc, 31);
+        if (lane < csize) cluster.map_shared_rank(exall, lane)[crank].cnt = tot;
     }
     cluster.sync();
-    unsigned cnt_off = 0;
-    for (unsigned c = 0; c < crank; ++c) cnt_off += (unsigned)cluster.map_shared_rank(exch, c)->cnt;
-    cnt_off += reinterpret_cast<unsigned *>(wtmp)[warp];
+    unsigned cnt_off = reinterpret_cast<unsigned *>(wtmp)[warp];
+#pragma unroll
+    for (int c = 0; c < kMaxCluster; ++c)
+        if (c < crank) cnt_off += (unsigned)exall[c].cnt;
 
     long long tok = 0;
     int adm = 0;
@@ -314,7 +373,9 @@ __global__ void __launch_bounds__(kThreads, 1) schedule_kernel(const __grid_cons
         atomicAdd(&a.counts->n_admitted, adm);
     }
     if (crank == 0 && tid == 0) a.counts->n_tier1 = N1;
-    cluster.sync();  // no CTA leaves while a peer may still read its shared memory
+    TICK(65);
+    // every remote store of this kernel is followed by a cluster barrier and nothing reads remote
+    // shared memory, so a CTA may leave as soon as it is done
 }
 
 __global__ void zero_counts_kernel(cascade_sched_counts *c) {
@@ -323,28 +384,29 @@ __global__ void zero_counts_kernel(cascade_sched_counts *c) {
     c->tokens_granted = 0;
 }
 
-size_t smem_bytes(int K) {
-    return size_t(kThreads) * K * sizeof(SortElem) + size_t(kWarps) * kWhistStride * sizeof(uint16_t) +
-           2 * kBins * sizeof(uint32_t) + 3 * kWarps * sizeof(long long) + sizeof(Exch) + 16;
+size_t smem_bytes(int T, int K) {
+    return 2 * size_t(T) * K * sizeof(SortElem) + size_t(T / 32) * kWhistStride * sizeof(uint16_t) +
+           size_t(kMaxCluster) * kBins * sizeof(uint16_t) + 2 * kBins * sizeof(uint32_t) + 3 * 32 * sizeof(long long) +
+           kMaxCluster * sizeof(Exch) + 16;
 }
 
-template <int K>
+template <int T, int K, bool kMatch>
 cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, cudaStream_t stream) {
     static bool configured_dev[64] = {};
     bool unknown = false;
     bool &configured = (device >= 0 && device < 64) ? configured_dev[device] : unknown;
-    const size_t smem = smem_bytes(K);
+    const size_t smem = smem_bytes(T, K);
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(schedule_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(schedule_kernel<T, K, kMatch>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(schedule_kernel<K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        e = cudaFuncSetAttribute(schedule_kernel<T, K, kMatch>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cluster_size, 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(T, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -354,10 +416,37 @@ cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, cudaStre
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, schedule_kernel<K>, a);
+    return cudaLaunchKernelEx(&cfg, schedule_kernel<T, K, kMatch>, a);
+}
+
+template <int T, bool kMatch>
+cudaError_t launch_k(int K, const ScheduleArgs &a, int C, int device, cudaStream_t s) {
+    switch (K) {
+        case 1: return launch<T, 1, kMatch>(a, C, device, s);
+        case 2: return launch<T, 2, kMatch>(a, C, device, s);
+        case 4: return launch<T, 4, kMatch>(a, C, device, s);
+        default:
+            if constexpr (T <= 512) return launch<T, 8, kMatch>(a, C, device, s);
+            else return cudaErrorInvalidConfiguration;
+    }
+}
+
+template <bool kMatch>
+cudaError_t launch_t(int T, int K, const ScheduleArgs &a, int C, int device, cudaStream_t s) {
+    switch (T) {
+        case 256: return launch_k<256, kMatch>(K, a, C, device, s);
+        case 512: return launch_k<512, kMatch>(K, a, C, device, s);
+        default: return launch_k<1024, kMatch>(K, a, C, device, s);
+    }
 }
 
 }  // namespace
+
+#ifdef CASCADE_PHASE_TIMING
+extern "C" int cascade_debug_ticks(long long *host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_phase_ticks, sizeof(g_phase_ticks));
+}
+#endif
 
 extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const uint64_t *key, int n, int32_t D_act,
                                 uint32_t *order_out, int32_t *grant_out, cascade_sched_counts *counts_dev,
@@ -372,20 +461,8 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     }
     if (!key || !order_out || !grant_out || !r->prompt || !r->n0 || !r->n1 || !r->n2) return CASCADE_EINVAL;
     const cascade_params &p = ctx->params;
-    // cluster size C and keys per thread K: the smallest K that fits the queue into <= 8 CTAs
-    int C = ctx->sort_cluster, K = ctx->sort_items;
-    if (K != 1 && K != 2 && K != 4 && K != 8) K = 0;
-    if (C != 1 && C != 2 && C != 4 && C != 8 && C != 16) C = 0;
-    if (K == 0) {
-        const int cmax = C ? C : 8;
-        K = 1;
-        while (K < 8 && (long long)cmax * kThreads * K < n) K *= 2;
-    }
-    if (C == 0) {
-        C = 1;
-        while (C < 16 && (long long)C * kThreads * K < n) C *= 2;
-    }
-    if ((long long)C * kThreads * K < n) return CASCADE_EINVAL;
+    int T, C, K;
+    if (!cascade_pick_geometry(ctx, n, &T, &C, &K)) return CASCADE_EINVAL;
     ScheduleArgs a;
     a.key = key;
     a.prompt = r->prompt;
@@ -402,16 +479,8 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.seq_cap = cap > 0 ? cap : 0;
     a.n = n;
     a.bt = p.bt;
-    int sh = 10;
-    for (int k = K; k > 1; k >>= 1) ++sh;
-    a.per_shift = sh;
-    cudaError_t e;
-    switch (K) {
-        case 1: e = launch<1>(a, C, ctx->device, s); break;
-        case 2: e = launch<2>(a, C, ctx->device, s); break;
-        case 4: e = launch<4>(a, C, ctx->device, s); break;
-        default: e = launch<8>(a, C, ctx->device, s); break;
-    }
+    cudaError_t e = ctx->sort_match ? launch_t<true>(T, K, a, C, ctx->device, s)
+                                    : launch_t<false>(T, K, a, C, ctx->device, s);
     CASCADE_CUDA_TRY(ctx, e);
     return CASCADE_OK;
 }

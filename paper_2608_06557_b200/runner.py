@@ -45,7 +45,7 @@ class Instance:
         d = self.device
         # request queue, structure of arrays; a pinned host mirror serves the end-to-end path
         self.reqs = {k: torch.empty(cap, dtype=dt, device=d) for k, dt in _REQ_DTYPES.items()}
-        self.reqs_host = {k: torch.empty(cap, dtype=dt).pin_memory() for k, dt in _REQ_DTYPES.items()}
+        self.reqs_host = {k: torch.empty(cap, dtype=dt, pin_memory=True) for k, dt in _REQ_DTYPES.items()}
         self.reqs_struct = cs.make_reqs(self.reqs)
         self.upload_requests(w.reqs)
         # outputs
@@ -92,7 +92,7 @@ class Instance:
                 if self.hbm_pool is None:
                     self.hbm_pool = torch.empty(w.layout["n_blocks"] * self.block_bytes, dtype=torch.uint8, device=d)
                 if self.host_pool is None:
-                    self.host_pool = torch.empty(w.host_blocks * self.block_bytes, dtype=torch.uint8).pin_memory()
+                    self.host_pool = torch.empty(w.host_blocks * self.block_bytes, dtype=torch.uint8, pin_memory=True)
         else:
             self.pools_struct = cs.Pools(None, None, 0, None, cs._p(self.hbm_free_count), 0, None,
                                          cs._p(self.host_free_count), 0)

@@ -171,8 +171,10 @@ LLAMA8B_CLASSES = dict(mix=[0.6, 0.3, 0.1], ttft=[1 * S, 3 * S, 30 * S], out_med
 
 
 def config_llama8b(seed: int = 0, n: int = 1024, hbm_bytes: int = 60 * 10**9, host_bytes: int = 40 * 10**9,
-                   hbm_free_target: int = 256) -> Workload:
-    """Llama-3-8B-shaped KV (2 MiB blocks: 64 chunks of 32 KiB), three SLO classes, beta(2,2) reuse."""
+                   hbm_free_target: int = 256, elapsed_scale: float = 1.5, hbm_share: float = 0.5) -> Workload:
+    """Llama-3-8B-shaped KV (2 MiB blocks: 64 chunks of 32 KiB), three SLO classes, beta(2,2) reuse.
+    Waiting times are uniform in [0, elapsed_scale * TTFT of the class]; ``hbm_share`` of every reused
+    prefix sits in HBM, the rest in the host pool."""
     rng = np.random.default_rng(seed)
     c = LLAMA8B_CLASSES
     n_chunks, chunk_bytes = 64, 32 * 1024
@@ -181,8 +183,8 @@ def config_llama8b(seed: int = 0, n: int = 1024, hbm_bytes: int = 60 * 10**9, ho
                             max_batch=128)
     params["blk_ns"] = [0, -(-bb * 1_000_000_000 // 50_000_000_000), 10 * -(-bb * 1_000_000_000 // 50_000_000_000)]
     now = 100 * S
-    reqs = draw_requests(rng, n, c["mix"], c["ttft"], 1024, (32, 32768), c["out_median"], (1, 65536), now, 1.5,
-                         lambda g, m: g.beta(2, 2, m), 0.5, params["bt"])
+    reqs = draw_requests(rng, n, c["mix"], c["ttft"], 1024, (32, 32768), c["out_median"], (1, 65536), now,
+                         elapsed_scale, lambda g, m: g.beta(2, 2, m), hbm_share, params["bt"])
     n_hbm, n_host = hbm_bytes // bb, host_bytes // bb
     maxb = 2048
     tbl = place_blocks(rng, reqs, n_hbm, n_host, maxb, 0.9, hbm_free_target, 0.5)

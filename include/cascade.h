@@ -41,6 +41,7 @@ extern "C" {
 #define CASCADE_ERANGE (-2) /* a parameter outside the overflow-safe bounds listed below           */
 #define CASCADE_ECUDA (-3)  /* a CUDA runtime call failed; its code is kept in cascade_status_t    */
 #define CASCADE_ENOMEM (-4) /* cascade_create could not allocate its scratch                       */
+#define CASCADE_ETOOBIG (-5) /* a size beyond a fixed maximum of the entry point (see the _noalloc call) */
 
 /* device-side sticky status bits */
 #define CASCADE_ST_EBOUNDS 1u   /* a block id or list length outside its pool: that item was skipped   */
@@ -264,6 +265,37 @@ int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, const void 
 
 /* Waits for `stream`, copies the status word to *host_out and, if clear != 0, resets it. */
 int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream);
+
+/*
+ * Tier plan without any allocation.  (The paper has no counterpart: this entry point exists for
+ * the library's users, not for the method.)
+ *
+ * Same computation, same arguments and same results as cascade_tier_plan, but no context: the
+ * per-request offsets that the first plan kernel hands to the two table-rewrite kernels live in a
+ * fixed scratch area compiled into the library (about 256 KiB of device memory on every GPU that
+ * loads the library, held from load to exit) instead of memory obtained in cascade_create.  It is
+ * meant for callers that cannot call cudaMalloc: an engine that has already handed all free HBM to
+ * its KV block pool, code running under a host framework that owns the allocator, or a loop that
+ * cannot accept the device-wide synchronisation an allocation may cause.  The call itself makes no
+ * cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ *   p            parameters (host), validated on every call as in cascade_create
+ *   status_dev   caller-owned device word; CASCADE_ST_* bits are OR-ed into it (never cleared here)
+ *   n            at most CASCADE_NOALLOC_MAX_REQUESTS, otherwise CASCADE_ETOOBIG is returned and
+ *                nothing is launched
+ *   all other arguments as in cascade_tier_plan; the device used is the calling thread's current one.
+ *
+ * The first call on each device looks up the device address of the scratch area (no allocation, but
+ * a runtime query): make that first call outside any stream capture.  Every call on a GPU shares
+ * the one scratch area and it keeps the previous call's contents; the entry point rewrites what it
+ * reads, but two calls whose kernels can overlap on the GPU (different streams, or one process
+ * with several host threads) race on it: issue them on one stream or order them with events.
+ */
+#define CASCADE_NOALLOC_MAX_REQUESTS 8192
+int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_reqs *r, const int64_t *budget,
+                              const uint32_t *order, int32_t *grant, int n, int32_t D_act, int64_t K_act,
+                              const cascade_pools *pools, const cascade_plan *plan_out, uint32_t *status_dev,
+                              void *stream);
 
 /* Library version (major*10000 + minor*100 + patch). */
 int cascade_version(void);

@@ -15,13 +15,15 @@ LIB_PATH = os.path.join(_PKG, "libcascade.so")
 
 MAX_CLASSES = 8
 MAX_REQUESTS = 65536
-OK, EINVAL, ERANGE, ECUDA, ENOMEM = 0, -1, -2, -3, -4
+OK, EINVAL, ERANGE, ECUDA, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5
+NOALLOC_MAX_REQUESTS = 8192
 ST_EBOUNDS, ST_ENOSPC, ST_ETIMEOUT, ST_EPRECOND, ST_ELISTCAP = 1, 2, 4, 8, 16
 FLAG_HBM_PRIVATE, FLAG_RUNNING = 1, 2
 ACT_NONE, ACT_RETAIN, ACT_EVICT, ACT_DROP = 0, 1, 2, 3
 
 EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_budget", "cascade_schedule",
-           "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version")
+           "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
+           "cascade_tier_plan_noalloc")
 
 
 class Params(C.Structure):
@@ -89,6 +91,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_kv_restore.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, C.c_int, vp, vp, vp, C.c_int, vp]
     lib.cascade_kv_evict.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, C.c_int, vp, vp, vp, C.c_int, vp]
     lib.cascade_status.argtypes = [vp, C.POINTER(Status), C.c_int, vp]
+    lib.cascade_tier_plan_noalloc.argtypes = [C.POINTER(Params), C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64,
+                                              C.POINTER(Pools), C.POINTER(Plan), vp, vp]
     for name in EXPORTS:
         if name != "cascade_destroy":
             getattr(lib, name).restype = C.c_int
@@ -144,7 +148,8 @@ class CascadeError(RuntimeError):
 
 def _check(rc: int, what: str):
     if rc != OK:
-        names = {EINVAL: "CASCADE_EINVAL", ERANGE: "CASCADE_ERANGE", ECUDA: "CASCADE_ECUDA", ENOMEM: "CASCADE_ENOMEM"}
+        names = {EINVAL: "CASCADE_EINVAL", ERANGE: "CASCADE_ERANGE", ECUDA: "CASCADE_ECUDA", ENOMEM: "CASCADE_ENOMEM",
+                 ETOOBIG: "CASCADE_ETOOBIG"}
         raise CascadeError(f"{what} failed: {names.get(rc, rc)}")
 
 
@@ -202,6 +207,17 @@ class Context:
         st = Status()
         _check(_lib.cascade_status(self._h, C.byref(st), int(clear), _stream(stream)), "cascade_status")
         return int(st.bits), int(st.cuda_error)
+
+
+def tier_plan_noalloc(params: Params, reqs: Reqs, budget, order, grant, n, D_act, K_act, pools: Pools, plan: Plan,
+                      status_dev, stream=None):
+    """cascade_tier_plan_noalloc: the tier plan on the library's built-in scratch area, for callers
+    that cannot allocate device memory (no context is needed).  ``status_dev`` is a caller-owned
+    uint32 device word that receives the CASCADE_ST_* bits.  Raises CascadeError (CASCADE_ETOOBIG)
+    when ``n`` exceeds NOALLOC_MAX_REQUESTS."""
+    _check(_lib.cascade_tier_plan_noalloc(C.byref(params), C.byref(reqs), _p(budget), _p(order), _p(grant), n,
+                                          D_act, K_act, C.byref(pools), C.byref(plan), _p(status_dev),
+                                          _stream(stream)), "cascade_tier_plan_noalloc")
 
 
 def raw():

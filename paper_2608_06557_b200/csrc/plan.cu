@@ -574,3 +574,125 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     }
     return CASCADE_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// cascade_tier_plan_noalloc: the tier plan for callers that must not allocate.
+//
+// cascade_tier_plan hands per-request offsets from its first kernel to the two table-rewrite
+// kernels through scratch that cascade_create obtained with cudaMalloc.  Some users of this
+// library cannot make that call at all: a serving engine that has already given every free byte
+// of HBM to its KV block pool (a later cudaMalloc can fail or force the pool to shrink), a
+// plug-in that runs under a host framework's memory manager and is not allowed to go to the
+// driver allocator behind its back, or a loop that may not tolerate the device-wide
+// synchronisation an allocation can imply.  For them the same kernels run here on a fixed
+// scratch area that is part of the library image: a file-scope device array, present on every GPU
+// that loads the library from load until exit, sized for CASCADE_NOALLOC_MAX_REQUESTS requests.
+//
+// The array's name is only a host-side handle in host code, never a device address, so its
+// address is looked up once per device with cudaGetSymbolAddress (with that device current) and
+// the resulting pointer is what the kernels receive.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct NoAllocScratch {
+    int4 work_admit[CASCADE_NOALLOC_MAX_REQUESTS];
+    int4 work_victim[CASCADE_NOALLOC_MAX_REQUESTS];
+    int32_t scalars[PS_COUNT];
+};
+
+// ~256 KiB + a few scalars per GPU; shared by every call on that GPU
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+struct NoAllocDevice {
+    NoAllocScratch *scratch;  // device address of g_noalloc_scratch on this device
+    int num_sms;
+    bool ready;
+};
+NoAllocDevice g_noalloc_dev[64];
+
+// First use on a device: resolve the device address of the static array (no allocation).
+int noalloc_setup(int device, NoAllocDevice **out) {
+    if (device < 0 || device >= 64) return CASCADE_EINVAL;
+    NoAllocDevice &d = g_noalloc_dev[device];
+    if (!d.ready) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return CASCADE_ECUDA;
+        if (cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+            return CASCADE_ECUDA;
+        d.scratch = reinterpret_cast<NoAllocScratch *>(ptr);
+        d.ready = true;
+    }
+    *out = &d;
+    return CASCADE_OK;
+}
+
+}  // namespace
+
+extern "C" int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_reqs *r, const int64_t *budget,
+                                         const uint32_t *order, int32_t *grant, int n, int32_t D_act, int64_t K_act,
+                                         const cascade_pools *pools, const cascade_plan *plan_out,
+                                         uint32_t *status_dev, void *stream) {
+    if (!p || !r || !pools || !plan_out || !status_dev || n < 0) return CASCADE_EINVAL;
+    if (n > CASCADE_NOALLOC_MAX_REQUESTS) return CASCADE_ETOOBIG;  // beyond the fixed scratch
+    int rc = cascade_validate_params(p);
+    if (rc != CASCADE_OK) return rc;
+    if (!plan_out->counts || !pools->hbm_free_count || !pools->host_free_count) return CASCADE_EINVAL;
+    if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
+    const bool with_tables = pools->hbm_tbl != nullptr;
+    if (n > 0 && (!budget || !order || !grant || !r->prompt || !r->n0 || !r->n1 || !r->n2 || !r->flags ||
+                  !plan_out->x1 || !plan_out->x2 || !plan_out->tokens_run || !plan_out->action))
+        return CASCADE_EINVAL;
+    if (with_tables) {
+        if (!pools->host_tbl || !pools->hbm_free || !pools->host_free || pools->maxb < 1 || pools->hbm_free_cap < 0 ||
+            pools->host_free_cap < 0 || plan_out->restore_cap < 0 || plan_out->evict_cap < 0)
+            return CASCADE_EINVAL;
+        if ((plan_out->restore_cap > 0 && (!plan_out->restore_src || !plan_out->restore_dst)) ||
+            (plan_out->evict_cap > 0 && (!plan_out->evict_src || !plan_out->evict_dst)))
+            return CASCADE_EINVAL;
+    }
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return CASCADE_ECUDA;
+    NoAllocDevice *dev = nullptr;
+    rc = noalloc_setup(device, &dev);
+    if (rc != CASCADE_OK) return rc;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    PlanArgs a;
+    a.prompt = r->prompt;
+    a.n0 = r->n0;
+    a.n1 = r->n1;
+    a.n2 = r->n2;
+    a.flags = r->flags;
+    a.budget = budget;
+    a.order = order;
+    a.grant = grant;
+    a.pools = *pools;
+    a.plan = *plan_out;
+    a.work_admit = dev->scratch->work_admit;
+    a.work_victim = dev->scratch->work_victim;
+    a.scalars = dev->scratch->scalars;
+    a.status = status_dev;
+    a.A_act = make_load_consts(*p, D_act, K_act).A_act;
+    a.n = n;
+    a.with_tables = with_tables ? 1 : 0;
+    // The scalars are rewritten by every call before the rewrite kernels read them and only the
+    // work entries written by this call are read back, so nothing has to be cleared; they are
+    // zeroed anyway so that a call that launches nothing leaves no stale counts behind.
+    if (cudaMemsetAsync(dev->scratch->scalars, 0, sizeof(dev->scratch->scalars), s) != cudaSuccess)
+        return CASCADE_ECUDA;
+    cascade_ctx geo = {};
+    int T, C, K;
+    if (!cascade_pick_geometry(&geo, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, *p, a, C, s)
+                  : T == 512 ? launch_plan_k<512>(K, *p, a, C, s)
+                             : launch_plan_k<1024>(K, *p, a, C, s);
+    if (e != cudaSuccess) return CASCADE_ECUDA;
+    if (with_tables && n > 0) {
+        const int grid = dev->num_sms * 2;
+        apply_victims_kernel<<<grid, 256, 0, s>>>(a);
+        if (cudaGetLastError() != cudaSuccess) return CASCADE_ECUDA;
+        apply_admitted_kernel<<<grid, 256, 0, s>>>(a);
+        if (cudaGetLastError() != cudaSuccess) return CASCADE_ECUDA;
+    }
+    return CASCADE_OK;
+}

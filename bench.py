@@ -170,6 +170,21 @@ def workload_config(args, extra):
     return cfg
 
 
+def rank_seed(rank: int, step: int) -> int:
+    """Every replica draws its own batches: disjoint seed ranges per rank."""
+    return 10_000 * rank + step
+
+
+def aggregate_over_ranks(dist, ms_total: float, moved: int, device):
+    """Whole-job figures of N independent replicas: the slowest rank's time, the sum of the bytes moved."""
+    import torch
+    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    mv = torch.tensor([moved], dtype=torch.int64, device=device)
+    dist.all_reduce(mv, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(mv.item())
+
+
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -212,31 +227,6 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
         return out
-
-
-def fill_pools(torch, hbm_pool, host_pool):
-    """Deterministic byte patterns, written in 256 MiB pieces (device pattern, then copied to host)."""
-    piece = 1 << 28
-    words = torch.arange(piece // 8, dtype=torch.int64, device=hbm_pool.device)
-    for base in range(0, hbm_pool.numel(), piece):
-        n = min(piece, hbm_pool.numel() - base)
-        chunk = (words[: n // 8] * -0x61C8864680B583EB + base * 31 + 1)
-        hbm_pool[base:base + (n // 8) * 8].view(torch.int64).copy_(chunk)
-    for base in range(0, host_pool.numel(), piece):
-        n = min(piece, host_pool.numel() - base)
-        chunk = (words[: n // 8] * -0x6B2FB644ECCEEE15 + base * 17 + 2)
-        host_pool[base:base + (n // 8) * 8].view(torch.int64).copy_(chunk, non_blocking=True)
-    torch.cuda.synchronize()
-
-
-def alloc_pinned(torch, nbytes):
-    """Pinned host pool; halves the request until the allocation succeeds."""
-    while nbytes >= (1 << 28):
-        try:
-            return torch.empty(nbytes, dtype=torch.uint8, pin_memory=True), nbytes
-        except RuntimeError:
-            nbytes //= 2
-    raise RuntimeError("could not pin a host pool")
 
 
 def event_pair(torch):
@@ -353,22 +343,22 @@ def ours_main(args):
     if world > 1:
         dist.barrier()
     from paper_2608_06557_b200 import cascade as cs
-    from paper_2608_06557_b200.runner import Instance
+    from paper_2608_06557_b200.runner import Instance, alloc_pinned_pool, fill_pools
 
     dev = f"cuda:{local_rank}"
     K, W = args.steps, max(args.warmup, 0)
     # ---- inputs: W+K fresh batches, resident on the device before anything is timed ---------------
-    batches = [make_batch(args, 10_000 * rank + s) for s in range(W + K)]
+    batches = [make_batch(args, rank_seed(rank, s)) for s in range(W + K)]
     w0 = batches[0]
     bb = w0.block_bytes
-    host_pool, host_bytes = alloc_pinned(torch, w0.host_blocks * bb)
+    host_pool, host_bytes = alloc_pinned_pool(w0.host_blocks * bb)
     if host_bytes != w0.host_blocks * bb:      # pinning was refused at full size: regenerate at the size we got
         args.host_gb = host_bytes / GB
-        batches = [make_batch(args, 10_000 * rank + s) for s in range(W + K)]
+        batches = [make_batch(args, rank_seed(rank, s)) for s in range(W + K)]
         w0 = batches[0]
         host_pool = host_pool[: w0.host_blocks * bb]
     hbm_pool = torch.empty(w0.layout["n_blocks"] * bb, dtype=torch.uint8, device=dev)
-    fill_pools(torch, hbm_pool, host_pool)
+    fill_pools(hbm_pool, host_pool)
     ctx = cs.Context(w0.params, args.requests, local_rank)
     insts = [Instance(w, device=dev, ctx=ctx, hbm_pool=hbm_pool, host_pool=host_pool, alloc_pools=False)
              for w in batches]
@@ -413,12 +403,7 @@ def ours_main(args):
     t_evict = np.array([ev[i][1].elapsed_time(ev[i][2]) for i in range(K)])
     t_rest = np.array([ev[i][2].elapsed_time(ev[i][3]) for i in range(K)])
     if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-        mv = torch.tensor([moved], dtype=torch.int64, device=dev)
-        dist.all_reduce(mv, op=dist.ReduceOp.SUM)
-        moved = int(mv.item())
+        ms_total, moved = aggregate_over_ranks(dist, ms_total, moved, dev)
     value = moved / (ms_total * 1e-3) / GB
 
     # ---- dominant kernel of the step and its roofline ----------------------------------------------

@@ -170,3 +170,30 @@ class Instance:
                        evict_src=self.evict_src[:ne].cpu().numpy(), evict_dst=self.evict_dst[:ne].cpu().numpy())
         out["status"] = self.ctx.status(clear=True)[0]
         return out
+
+
+def alloc_pinned_pool(nbytes: int, floor: int = 1 << 28):
+    """Pinned, device-mapped host pool of ``nbytes``; the request is halved until the allocation
+    succeeds.  Returns (uint8 tensor, bytes obtained)."""
+    while nbytes >= floor:
+        try:
+            return torch.empty(nbytes, dtype=torch.uint8, pin_memory=True), nbytes
+        except RuntimeError:
+            nbytes //= 2
+    raise RuntimeError("could not pin a host pool")
+
+
+def fill_pools(hbm_pool, host_pool):
+    """Deterministic, position-dependent byte patterns for both pools, produced on the device in
+    256 MiB pieces (the host pool is filled by device-to-host copies)."""
+    piece = 1 << 28
+    words = torch.arange(piece // 8, dtype=torch.int64, device=hbm_pool.device)
+    for base in range(0, hbm_pool.numel(), piece):
+        n = min(piece, hbm_pool.numel() - base)
+        chunk = words[: n // 8] * -0x61C8864680B583EB + (base * 31 + 1)
+        hbm_pool[base:base + (n // 8) * 8].view(torch.int64).copy_(chunk)
+    for base in range(0, host_pool.numel(), piece):
+        n = min(piece, host_pool.numel() - base)
+        chunk = words[: n // 8] * -0x6B2FB644ECCEEE15 + (base * 17 + 2)
+        host_pool[base:base + (n // 8) * 8].view(torch.int64).copy_(chunk, non_blocking=True)
+    torch.cuda.synchronize()

@@ -265,3 +265,91 @@ def copy_lists(seed: int, n_copies: int, n_src_blocks: int, n_dst_blocks: int):
     src = rng.choice(n_src_blocks, size=n_copies, replace=False).astype(np.int32)
     dst = rng.choice(n_dst_blocks, size=n_copies, replace=False).astype(np.int32)
     return src, dst
+
+
+LLAMA70B_CLASSES = dict(mix=[0.3, 0.2, 0.1, 0.4], ttft=[1 * S, 3 * S, 30 * S, 1 * S], out_median=[256, 256, 4096, 128])
+
+
+@dataclass
+class Trace:
+    """A whole arrival trace for the closed-loop replay (Llama-3-70B-shaped KV, 5 MiB blocks)."""
+    params: dict
+    arrival_ns: np.ndarray     # int64 [n], ascending
+    prompt: np.ndarray         # int32
+    pred_out: np.ndarray       # int32
+    cls: np.ndarray            # uint8
+    n0: np.ndarray             # int32: matched blocks resident in HBM at arrival
+    n1: np.ndarray             # int32: matched blocks on host at arrival
+    shared: np.ndarray         # bool: the HBM part is the shared system prefix (never preempted)
+    hbm_tbl: np.ndarray        # int32 [n, maxb]
+    host_tbl: np.ndarray       # int32 [n, maxb]
+    hbm_free: np.ndarray
+    hbm_free_count: int
+    host_free: np.ndarray
+    host_free_count: int
+    layout: dict
+    host_blocks: int
+    maxb: int
+    shared_ids: np.ndarray     # HBM ids of the shared prefix
+
+
+def config_llama70b_trace(seed: int = 0, n: int = 4096, rate_per_s: float = 20.0, hbm_bytes: int = 60 * 10**9,
+                          host_bytes: int = 40 * 10**9, shared_prefix_tokens: int = 8192,
+                          hbm_occupancy: float = 0.5) -> Trace:
+    """4096 requests with exponential inter-arrival times (20 requests/s), four SLO classes (chat, code,
+    reasoning, agentic).  Agentic requests hit a shared system prefix held in HBM with probability 0.7 (the
+    same block ids in every hitting request's table); other requests reuse a Beta(2,2) fraction of their
+    prompt, 40 % of it in HBM and 60 % on host.  5 MiB blocks (160 chunks of 32 KiB).  Cached prefixes of
+    requests that have not arrived yet occupy at most ``hbm_occupancy`` of the HBM pool."""
+    rng = np.random.default_rng(seed)
+    c = LLAMA70B_CLASSES
+    n_chunks, chunk_bytes = 160, 32 * 1024
+    bb = n_chunks * chunk_bytes
+    blk = -(-bb * 1_000_000_000 // 50_000_000_000)
+    params = default_params(ttft_ns=c["ttft"], tpot_ns=[100 * MS] * 4, token_budget=16384, tier2_reserve=2048,
+                            max_batch=128, blk_ns=[0, blk, 10 * blk])
+    bt = params["bt"]
+    arrival = np.cumsum(rng.exponential(1e9 / rate_per_s, n)).astype(np.int64)
+    cls = rng.choice(4, size=n, p=c["mix"]).astype(np.uint8)
+    prompt = _lognormal_int(rng, 1024, 1.0, 32, 32768, n)
+    agentic_hit = (cls == 3) & (rng.uniform(0, 1, n) < 0.7)
+    prompt[agentic_hit] = np.maximum(prompt[agentic_hit], shared_prefix_tokens + 64)  # prefix + own suffix
+    med = np.asarray(c["out_median"], float)[cls]
+    pred_out = np.clip(np.rint(np.exp(rng.normal(np.log(med), 1.0))), 1, 65536).astype(np.int32)
+    n_hbm, n_host = hbm_bytes // bb, host_bytes // bb
+    maxb = 2048
+    shared_blocks = shared_prefix_tokens // bt
+    hbm_ids = rng.permutation(n_hbm).astype(np.int32)
+    host_ids = rng.permutation(n_host).astype(np.int32)
+    shared_ids = hbm_ids[:shared_blocks].copy()
+    hbm_used, host_used = shared_blocks, 0
+    hbm_lim, host_lim = int(n_hbm * hbm_occupancy), int(n_host * 0.9)
+    frac = rng.beta(2, 2, n)
+    n0 = np.zeros(n, np.int32)
+    n1 = np.zeros(n, np.int32)
+    hbm_tbl = np.full((n, maxb), -1, np.int32)
+    host_tbl = np.full((n, maxb), -1, np.int32)
+    for r in range(n):
+        if agentic_hit[r]:
+            n0[r] = shared_blocks
+            hbm_tbl[r, :shared_blocks] = shared_ids
+            continue
+        hit = min(int(frac[r] * (prompt[r] // bt)), (prompt[r] - 1) // bt)
+        a = int(np.ceil(hit * 0.4))
+        a = min(a, hbm_lim - hbm_used)
+        b = hit - int(np.ceil(hit * 0.4)) if a == int(np.ceil(hit * 0.4)) else 0
+        b = min(b, host_lim - host_used)
+        n0[r], n1[r] = a, b
+        hbm_tbl[r, :a] = hbm_ids[hbm_used:hbm_used + a]
+        hbm_used += a
+        host_tbl[r, a:a + b] = host_ids[host_used:host_used + b]
+        host_used += b
+    hbm_free = np.full(n_hbm, -1, np.int32)
+    hbm_free_count = n_hbm - hbm_used
+    hbm_free[:hbm_free_count] = hbm_ids[hbm_used:]
+    host_free = np.full(n_host, -1, np.int32)
+    host_free_count = n_host - host_used
+    host_free[:host_free_count] = host_ids[host_used:]
+    return Trace(params, arrival, prompt, pred_out, cls, n0, n1, agentic_hit, hbm_tbl, host_tbl, hbm_free,
+                 hbm_free_count, host_free, host_free_count, kv_layout(n_hbm, n_chunks, chunk_bytes), n_host, maxb,
+                 shared_ids)

@@ -1,0 +1,109 @@
+"""GPU parity on the Llama-3-70B-shaped closed-loop replay: 5 MiB blocks (160 chunks), Poisson arrivals,
+shared agentic prefix, restore-heavy reuse, HBM pressure.  Every iteration's outputs are compared with
+the oracle bit for bit; the copies of all iterations are verified at the end by tracking, on the host,
+which original block's bytes every HBM block and host record must hold."""
+import numpy as np
+import pytest
+
+from helpers import oracle_iteration
+from paper_2608_06557_b200 import workload as wl
+from paper_2608_06557_b200.replay import Replay
+
+pytestmark = pytest.mark.gpu
+
+P1, P2 = -0x61C8864680B583EB, 0x2545F4914F6CDD1D
+HOST_TAG = 1 << 20
+
+
+def fill_by_content(torch, hbm, host, lay, n_host):
+    cw = lay["chunk_bytes"] // 8
+    hv = hbm.view(torch.int64).view(lay["n_chunks"], lay["n_blocks"], cw)
+    ids = torch.arange(lay["n_blocks"], dtype=torch.int64, device="cuda")
+    k = torch.arange(cw, dtype=torch.int64, device="cuda")
+    for ch in range(lay["n_chunks"]):
+        hv[ch] = ids[:, None] * P1 + (ch * cw + k)[None, :] * P2
+    bw = lay["n_chunks"] * cw
+    j = torch.arange(bw, dtype=torch.int64, device="cuda")
+    ov = host.view(torch.int64).view(n_host, bw)
+    step = 256
+    for base in range(0, n_host, step):
+        c = torch.arange(base, min(base + step, n_host), dtype=torch.int64, device="cuda") + HOST_TAG
+        ov[base:base + len(c)].copy_(c[:, None] * P1 + j[None, :] * P2)
+    torch.cuda.synchronize()
+
+
+def verify_by_content(torch, hbm, host, lay, n_host, hbm_content, host_content):
+    cw = lay["chunk_bytes"] // 8
+    hv = hbm.view(torch.int64).view(lay["n_chunks"], lay["n_blocks"], cw)
+    c = torch.from_numpy(hbm_content).cuda()
+    k = torch.arange(cw, dtype=torch.int64, device="cuda")
+    for ch in range(lay["n_chunks"]):
+        assert torch.equal(hv[ch], c[:, None] * P1 + (ch * cw + k)[None, :] * P2), ch
+    bw = lay["n_chunks"] * cw
+    j = torch.arange(bw, dtype=torch.int64, device="cuda")
+    ov = host.view(torch.int64).view(n_host, bw)
+    oc = torch.from_numpy(host_content).cuda()
+    step = 256
+    for base in range(0, n_host, step):
+        got = ov[base:base + step].cuda()
+        assert torch.equal(got, oc[base:base + len(got), None] * P1 + j[None, :] * P2), base
+
+
+@pytest.mark.parametrize("variant", ["pressure", "restore_heavy"])
+def test_replay_iterations_match_oracle_and_bytes_end_up_where_they_should(variant):
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    from paper_2608_06557_b200.runner import Instance
+
+    if variant == "pressure":
+        tr = wl.config_llama70b_trace(1, n=1024, hbm_bytes=12 * 10**9, host_bytes=8 * 10**9, hbm_occupancy=0.7,
+                                      rate_per_s=60.0)
+        iters = 200
+    else:
+        tr = wl.config_llama70b_trace(0, n=1024, hbm_bytes=16 * 10**9, host_bytes=10 * 10**9, hbm_occupancy=0.5)
+        iters = 120
+    lay = tr.layout
+    bb = lay["n_chunks"] * lay["chunk_bytes"]
+    assert bb == 5 * 1024 * 1024
+    hbm = torch.empty(lay["n_blocks"] * bb, dtype=torch.uint8, device="cuda")
+    host = torch.empty(tr.host_blocks * bb, dtype=torch.uint8, pin_memory=True)
+    fill_by_content(torch, hbm, host, lay, tr.host_blocks)
+    hbm_content = np.arange(lay["n_blocks"], dtype=np.int64)
+    host_content = np.arange(tr.host_blocks, dtype=np.int64) + HOST_TAG
+
+    rp = Replay(tr)
+    ctx = cs.Context(tr.params, 1024, 0)
+    tot = dict(n_restore=0, n_evict=0, n_drop_blocks=0, n_unadmitted=0)
+    for it in range(iters):
+        w, ids = rp.workload()
+        if len(ids) == 0:
+            break
+        ref = oracle_iteration(w)
+        plan, pools = ref["plan"], ref["pools"]
+        inst = Instance(w, ctx=ctx, hbm_pool=hbm, host_pool=host, alloc_pools=False)
+        inst.run_iteration()
+        got = inst.fetch()
+        for k in ("budget", "key", "order", "grant"):
+            assert np.array_equal(got[k], ref[k]), (it, k)
+        for k in ("x1", "x2", "tokens_run", "action", "restore_src", "restore_dst", "evict_src", "evict_dst"):
+            assert np.array_equal(got[k], plan[k]), (it, k)
+        assert got["plan_counts"] == plan["counts"], it
+        assert got["status"] == ref["status"], it
+        assert np.array_equal(got["hbm_tbl"], pools.hbm_tbl) and np.array_equal(got["host_tbl"], pools.host_tbl), it
+        assert got["hbm_free_count"] == pools.hbm_free_count and got["host_free_count"] == pools.host_free_count
+        assert np.array_equal(got["hbm_free"][: pools.hbm_free_count], pools.hbm_free[: pools.hbm_free_count])
+        assert np.array_equal(got["host_free"][: pools.host_free_count], pools.host_free[: pools.host_free_count])
+        # bookkeeping of what the copies of this iteration must have moved (evict first, then restore)
+        host_content[plan["evict_dst"]] = hbm_content[plan["evict_src"]]
+        hbm_content[plan["restore_dst"]] = host_content[plan["restore_src"]]
+        for k in tot:
+            tot[k] += plan["counts"][k]
+        rp.apply(ids, dict(grant=ref["grant"], x1=plan["x1"], tokens_run=plan["tokens_run"], action=plan["action"],
+                           hbm_tbl=pools.hbm_tbl, host_tbl=pools.host_tbl, hbm_free=pools.hbm_free,
+                           host_free=pools.host_free, hbm_free_count=pools.hbm_free_count,
+                           host_free_count=pools.host_free_count))
+        del inst
+    assert tot["n_restore"] > 200
+    if variant == "pressure":
+        assert tot["n_evict"] > 0 and tot["n_drop_blocks"] > 0 and tot["n_unadmitted"] > 0
+    verify_by_content(torch, hbm, host, lay, tr.host_blocks, hbm_content, host_content)

@@ -108,12 +108,14 @@ def test_duplicate_and_constant_keys_keep_slot_order():
         assert np.array_equal(inst.grant[: w.n].cpu().numpy(), grant), case
 
 
-def test_scheduler_sweep_iterations_with_churn():
-    """Consecutive iterations of the scheduler-scale sweep (plan-only), with 5 % slot churn."""
+@pytest.mark.parametrize("n,iters", [(1024, 1000), (4096, 100), (16384, 40), (65536, 8)])
+def test_scheduler_sweep_iterations_with_churn(n, iters):
+    """Consecutive iterations of the scheduler-scale sweep (plan-only): the clock advances 25 ms and 5 % of
+    the slots and of the decode contexts are replaced every iteration."""
     torch, cs, Instance = _gpu()
-    sw = wl.SchedulerSweep(4096, seed=1)
+    sw = wl.SchedulerSweep(n, seed=1)
     inst = Instance(sw.workload(), alloc_pools=False)
-    for it in range(5):
+    for it in range(iters):
         w = sw.workload()
         ref = oracle_iteration(w, with_tables=False)
         inst.upload_requests(w.reqs)

@@ -410,7 +410,7 @@ def ours_main(args):
     ev_bytes, rs_bytes = int(n_evict.sum()) * bb, int(n_restore.sum()) * bb
     evict_gbs = ev_bytes / (t_evict.sum() * 1e-3) / GB if ev_bytes else 0.0
     restore_gbs = rs_bytes / (t_rest.sum() * 1e-3) / GB if rs_bytes else 0.0
-    dominant = "kv_copy_kernel<evict>" if t_evict.sum() >= t_rest.sum() else "kv_copy_kernel<restore>"
+    dominant = "kv_copy_bulk_kernel<evict>" if t_evict.sum() >= t_rest.sum() else "kv_copy_bulk_kernel<restore>"
     dom_ach = evict_gbs if dominant.endswith("<evict>") else restore_gbs
     dom_peak = peaks["d2h"] if dominant.endswith("<evict>") else peaks["h2d"]
     dom_launch_bytes = (ev_bytes if dominant.endswith("<evict>") else rs_bytes) / K
@@ -454,7 +454,7 @@ def ours_main(args):
             line["copy_sweep_GBps"] = sweep
             hbm_peak = load_hbm_peak()
             big = sweep.get("restore_hbm_4096", 0.0)
-            line["roofline_hbm"] = dict(bound="hbm", kernel="kv_copy_kernel<restore>, device staging buffer, "
+            line["roofline_hbm"] = dict(bound="hbm", kernel="kv_copy_bulk_kernel<restore>, device staging buffer, "
                                         "4096 blocks", achieved=big, peak=hbm_peak[0], unit="GB/s",
                                         frac=round(big / hbm_peak[0], 4), traffic=None, peak_source=hbm_peak[1])
             del insts

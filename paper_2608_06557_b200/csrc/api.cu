@@ -52,6 +52,10 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->copy_ctas_host = e && atoi(e) > 0 ? atoi(e) : 4;
     e = getenv("CASCADE_COPY_CTAS_DEV");
     ctx->copy_ctas_dev = e && atoi(e) > 0 ? atoi(e) : 8;
+    e = getenv("CASCADE_COPY_BULK_HOST");
+    ctx->copy_bulk_host = e ? atoi(e) : 1;
+    e = getenv("CASCADE_COPY_BULK_DEV");
+    ctx->copy_bulk_dev = e ? atoi(e) : 2;
     size_t n = (size_t)max_requests;
     bool ok = cudaMalloc(&ctx->status_dev, sizeof(uint32_t)) == cudaSuccess &&
               cudaMallocHost(&ctx->status_host, sizeof(uint32_t)) == cudaSuccess &&

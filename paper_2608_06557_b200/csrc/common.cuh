@@ -25,6 +25,8 @@ struct cascade_ctx {
     int sort_match;              // 1: rank digits with match.any, 0: with eight ballots
     int copy_ctas_host;          // copy CTAs per SM when the record pool is pinned host memory
     int copy_ctas_dev;           // copy CTAs per SM when the record pool is device memory
+    int copy_bulk_host;          // >0: TMA bulk-copy ring (that many CTAs per SM) for the pinned-host path
+    int copy_bulk_dev;           // >0: TMA bulk-copy ring for the device-staging path
 };
 
 // plan_scalars layout

@@ -4,9 +4,12 @@
 //
 // The bytes are opaque.  A block is n_chunks pieces of chunk_bytes; on the record side they are
 // back to back, on the HBM side chunk c of block b sits at c*chunk_stride + b*block_stride.
-// Work is cut into 16 KiB pieces (one CTA iteration each: 256 threads x 4 x 16-byte vectors, all
-// loads issued before the first store) and spread over a persistent grid, so a single 2 MiB block
-// already occupies 128 CTAs and every access is a fully coalesced 512-byte warp transaction.
+// Two kernels do the same copy:
+//   kv_copy_bulk_kernel (default)  one elected thread per CTA drives TMA bulk copies
+//       (cp.async.bulk) through a 4-slot shared-memory ring, 32 KiB pieces, one or two CTAs per SM;
+//       it leaves the SMs' issue slots free for whatever else runs on the GPU;
+//   kv_copy_kernel                 256 threads x 4 x 16-byte vector loads/stores per 16 KiB piece on a
+//       persistent grid (selected with CASCADE_COPY_BULK_HOST=0 / CASCADE_COPY_BULK_DEV=0).
 #include "common.cuh"
 
 namespace {
@@ -72,6 +75,135 @@ __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant
     if (bad && tid == 0) atomicOr(a.status, CASCADE_ST_EBOUNDS);
 }
 
+
+// ---- bulk-copy variant: TMA (cp.async.bulk) through a shared-memory ring ---------------------------
+// One elected thread per CTA moves pieces of up to 32 KiB: global -> shared with an mbarrier that
+// counts the arriving bytes, then shared -> global as a bulk store group.  kStages ring slots; two
+// loads are kept in flight ahead of the piece being stored, and a slot is refilled only after the
+// store that last used it has finished reading shared memory.  Every wait is bounded: when the
+// clock limit is hit the kernel records CASCADE_ST_ETIMEOUT, stops issuing work, drains its own
+// store groups and returns.
+constexpr int kBulkPiece = 32 * 1024;
+constexpr int kStages = 4;
+constexpr int kAhead = kStages - 2;
+constexpr long long kWaitCycles = 4000000000LL;  // about two seconds at 1.9 GHz
+
+__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_load(unsigned dst_smem, const void *src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst, unsigned src_smem, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+template <bool kRestore>
+__global__ void __launch_bounds__(32) kv_copy_bulk_kernel(const __grid_constant__ CopyArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long bars[kStages];
+    if (threadIdx.x != 0) return;
+    for (int s = 0; s < kStages; ++s) mbar_init(smem_addr(&bars[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+    int count = a.n_max;
+    if (a.n_dev) {
+        const int c = *a.n_dev;
+        count = c < 0 ? 0 : (c < count ? c : count);
+    }
+    const int ppc = a.pieces_per_chunk;  // pieces of kBulkPiece per chunk
+    const long long per_block = (long long)a.n_chunks * ppc;
+    const long long items = (long long)count * per_block;
+    const long long bb = (long long)a.n_chunks * a.chunk_bytes;
+    uint32_t st = 0;
+
+    long long next = blockIdx.x;  // next item of this CTA to load
+    // resolves item `it` into addresses; false when an id is outside its pool (pair skipped)
+    auto resolve = [&](long long it, const char *&src, char *&dst, unsigned &bytes) -> bool {
+        const long long i = it / per_block;
+        const int rem = (int)(it - i * per_block);
+        const int c = rem / ppc, pc = rem - c * ppc;
+        const long long s = a.src_ids[i], d = a.dst_ids[i];
+        const long long rec_id = kRestore ? s : d, pg_id = kRestore ? d : s;
+        if (rec_id < 0 || rec_id >= a.record_blocks || pg_id < 0 || pg_id >= a.paged_blocks) return false;
+        const long long off = (long long)pc * kBulkPiece;
+        const long long left = a.chunk_bytes - off;
+        bytes = (unsigned)(left < kBulkPiece ? left : kBulkPiece);
+        char *rec = a.record + rec_id * bb + (long long)c * a.chunk_bytes + off;
+        char *pg = a.paged + (long long)c * a.chunk_stride + pg_id * a.block_stride + off;
+        src = kRestore ? rec : pg;
+        dst = kRestore ? pg : rec;
+        return true;
+    };
+    char *dst_of[kStages];
+    unsigned bytes_of[kStages];
+    long long issued = 0, stored = 0;
+    auto issue_next = [&]() -> bool {  // loads the next valid item into ring slot issued % kStages
+        while (next < items) {
+            const char *src;
+            char *dst;
+            unsigned bytes;
+            const bool ok = resolve(next, src, dst, bytes);
+            next += gridDim.x;
+            if (!ok) {
+                st |= CASCADE_ST_EBOUNDS;
+                continue;
+            }
+            const int slot = (int)(issued % kStages);
+            const unsigned bar = smem_addr(&bars[slot]);
+            mbar_expect_tx(bar, bytes);
+            bulk_load(smem_addr(ring + (size_t)slot * kBulkPiece), src, bytes, bar);
+            dst_of[slot] = dst;
+            bytes_of[slot] = bytes;
+            ++issued;
+            return true;
+        }
+        return false;
+    };
+    for (int k = 0; k < kAhead; ++k)
+        if (!issue_next()) break;
+    while (stored < issued) {
+        const int slot = (int)(stored % kStages);
+        const unsigned parity = (unsigned)((stored / kStages) & 1);
+        const unsigned bar = smem_addr(&bars[slot]);
+        const long long t0 = clock64();
+        bool arrived = mbar_try_wait(bar, parity);
+        while (!arrived && clock64() - t0 < kWaitCycles) arrived = mbar_try_wait(bar, parity);
+        if (!arrived) {  // give up: record it, issue nothing more
+            st |= CASCADE_ST_ETIMEOUT;
+            break;
+        }
+        bulk_store(dst_of[slot], smem_addr(ring + (size_t)slot * kBulkPiece), bytes_of[slot]);
+        ++stored;
+        // the slot refilled next was last read by the store issued one step earlier
+        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        issue_next();
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (st) atomicOr(a.status, st);
+}
+
 int check_layout(const cascade_kv_layout *l, const void *paged, const void *record, long long record_blocks) {
     if (!l || !paged || !record) return CASCADE_EINVAL;
     if (l->n_blocks < 0 || record_blocks < 0 || l->n_chunks < 1 || l->chunk_bytes < 16) return CASCADE_EINVAL;
@@ -104,6 +236,26 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
     a.block_stride = l->block_stride;
     a.n_chunks = l->n_chunks;
     a.n_max = n_max;
+    const int mode = record_is_device ? ctx->copy_bulk_dev : ctx->copy_bulk_host;
+    if (mode) {
+        // TMA ring: one CTA (one elected thread) per SM slot, 32 KiB pieces
+        a.pieces_per_chunk = (int)((l->chunk_bytes + kBulkPiece - 1) / kBulkPiece);
+        const long long items = (long long)n_max * l->n_chunks * a.pieces_per_chunk;
+        long long grid = (long long)ctx->num_sms * (mode > 1 ? mode : 1);
+        if (grid > items) grid = items;
+        const size_t smem = (size_t)kStages * kBulkPiece;
+        static bool configured = false;
+        if (!configured) {
+            CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_copy_bulk_kernel<true>,
+                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_copy_bulk_kernel<false>,
+                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            configured = true;
+        }
+        kv_copy_bulk_kernel<kRestore><<<(unsigned)grid, 32, smem, s>>>(a);
+        CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+        return CASCADE_OK;
+    }
     a.pieces_per_chunk = (int)((l->chunk_bytes + kPiece - 1) / kPiece);
     const long long items = (long long)n_max * l->n_chunks * a.pieces_per_chunk;
     const int per_sm = record_is_device ? ctx->copy_ctas_dev : ctx->copy_ctas_host;

@@ -23,6 +23,7 @@ struct cascade_ctx {
     int sort_items;              // keys per thread override (0 = automatic)
     int sort_threads;            // threads per CTA override (0 = automatic)
     int sort_match;              // 1: rank digits with match.any, 0: with eight ballots
+    int sort_stage;              // 1: group elements by digit locally before the remote scatter
     int copy_ctas_host;          // copy CTAs per SM when the record pool is pinned host memory
     int copy_ctas_dev;           // copy CTAs per SM when the record pool is device memory
     int copy_bulk_host;          // >0: TMA bulk-copy ring (that many CTAs per SM) for the pinned-host path

@@ -244,7 +244,9 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
         long long grid = (long long)ctx->num_sms * (mode > 1 ? mode : 1);
         if (grid > items) grid = items;
         const size_t smem = (size_t)kStages * kBulkPiece;
-        static bool configured = false;
+        static bool configured_dev[64] = {};
+        bool unknown = false;
+        bool &configured = (ctx->device >= 0 && ctx->device < 64) ? configured_dev[ctx->device] : unknown;
         if (!configured) {
             CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_copy_bulk_kernel<true>,
                                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

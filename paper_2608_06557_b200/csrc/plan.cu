@@ -492,7 +492,15 @@ apply_admitted_kernel(const __grid_constant__ PlanArgs a) {
 
 template <int T, int K>
 cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_size, cudaStream_t stream) {
-    cudaFuncSetAttribute(plan_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    // clusters of 16 CTAs need the non-portable size opt-in, once per device
+    static bool configured_dev[64] = {};
+    int device = 0;
+    cudaGetDevice(&device);
+    if (device < 0 || device >= 64 || !configured_dev[device]) {
+        cudaError_t e = cudaFuncSetAttribute(plan_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+        if (device >= 0 && device < 64) configured_dev[device] = true;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cluster_size, 1, 1);
     cfg.blockDim = dim3(T, 1, 1);

@@ -52,6 +52,7 @@ struct ScheduleArgs {
     int seq_cap;        // max_batch - D_act, >= 0
     int n;
     int bt;
+    int stage;          // 1: group by digit locally before the remote copy
 };
 
 #ifdef CASCADE_PHASE_TIMING
@@ -226,24 +227,35 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         __syncthreads();
         TICK(pass * 8 + 4);
 
-        // (d) group the CTA's elements by digit in a local staging buffer, then copy runs of equal
-        //     digits to their owners: consecutive lanes store to consecutive remote addresses
+        if (a.stage) {
+            // (d) group the CTA's elements by digit in a local staging buffer, then copy runs of equal
+            //     digits to their owners: consecutive lanes store to consecutive remote addresses
 #pragma unroll
-        for (int k = 0; k < K; ++k) {
-            const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
-            const unsigned lpos = lbase[d] + whist[warp * kWhistStride + d] + off[k];
-            *reinterpret_cast<uint4 *>(stage + lpos) = *reinterpret_cast<const uint4 *>(&e[k]);
-        }
-        __syncthreads();
+            for (int k = 0; k < K; ++k) {
+                const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
+                const unsigned lpos = lbase[d] + whist[warp * kWhistStride + d] + off[k];
+                *reinterpret_cast<uint4 *>(stage + lpos) = *reinterpret_cast<const uint4 *>(&e[k]);
+            }
+            __syncthreads();
 #pragma unroll
-        for (int k = 0; k < K; ++k) {
-            const unsigned i = (warp * K + k) * 32 + lane;
-            const uint4 v = *reinterpret_cast<const uint4 *>(stage + i);
-            const unsigned long long key = ((unsigned long long)v.y << 32) | v.x;
-            const unsigned d = (unsigned)(key >> shift) & 0xffu;
-            const unsigned pos = base[d] + (i - lbase[d]);
-            SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
-            *reinterpret_cast<uint4 *>(dst) = v;
+            for (int k = 0; k < K; ++k) {
+                const unsigned i = (warp * K + k) * 32 + lane;
+                const uint4 v = *reinterpret_cast<const uint4 *>(stage + i);
+                const unsigned long long key = ((unsigned long long)v.y << 32) | v.x;
+                const unsigned d = (unsigned)(key >> shift) & 0xffu;
+                const unsigned pos = base[d] + (i - lbase[d]);
+                SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
+                *reinterpret_cast<uint4 *>(dst) = v;
+            }
+        } else {
+            // (d) scatter every element straight to its owner
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
+                const unsigned pos = base[d] + whist[warp * kWhistStride + d] + off[k];
+                SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
+                *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(&e[k]);
+            }
         }
         TICK(pass * 8 + 5);
         cluster.sync();  // all remote stores have landed
@@ -479,6 +491,7 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.seq_cap = cap > 0 ? cap : 0;
     a.n = n;
     a.bt = p.bt;
+    a.stage = ctx->sort_stage >= 0 ? ctx->sort_stage : (K >= 4);
     cudaError_t e = ctx->sort_match ? launch_t<true>(T, K, a, C, ctx->device, s)
                                     : launch_t<false>(T, K, a, C, ctx->device, s);
     CASCADE_CUDA_TRY(ctx, e);

@@ -89,7 +89,18 @@ typedef struct cascade_params {
     int64_t blk_ns[3];     /* Eq. 6: time per block summed over path P(k); [0] unused          */
     int64_t ttft_ns[CASCADE_MAX_CLASSES]; /* class TTFT targets                                */
     int64_t tpot_ns[CASCADE_MAX_CLASSES]; /* class TPOT targets; 0 disables the decode term    */
+    int32_t policy;        /* CASCADE_POLICY_*: what the queue is ordered by (0 = the paper's method)     */
+    int32_t reserved;      /* must be 0                                                                   */
 } cascade_params;
+
+/* Ordering policies.  BUDGET is the method: least remaining budget first with the Tier-1 / Tier-2 split.
+ * The others are the comparison policies of the paper's evaluation, one queue, same key packing:
+ * FCFS orders by arrival time, EDF by the TTFT deadline arrival + ttft_ns[cls], SJF by the tokens left
+ * to prefill.  budget_out is the latency budget under every policy (the tier plan needs it). */
+#define CASCADE_POLICY_BUDGET 0
+#define CASCADE_POLICY_FCFS 1
+#define CASCADE_POLICY_EDF 2
+#define CASCADE_POLICY_SJF 3
 
 /*
  * The request queue as a structure of arrays (host struct of device pointers, n entries each).
@@ -213,6 +224,18 @@ int cascade_set_params(cascade_ctx *ctx, const cascade_params *p);
  */
 int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, int64_t now_ns, int32_t D_act, int64_t K_act,
                    int64_t *budget_out, uint64_t *key_out, void *stream);
+
+/*
+ * The TTFT estimator's four operating regimes for every request (Section "TTFT Latency Estimator"):
+ *   lat4_out[4*r + 0]  zero load, full recomputation            (L^zero_recomp)
+ *   lat4_out[4*r + 1]  actual load, full recomputation          (L^act_recomp)
+ *   lat4_out[4*r + 2]  actual load, tier-aware prefix reuse     (L^actual of Eq. 3)
+ *   lat4_out[4*r + 3]  maximum load, tier-aware prefix reuse    (L^max of Eq. 3)
+ * in ns, from the same integer model cascade_budget uses.  A request outside the input bounds gets
+ * four zeros and CASCADE_ST_EPRECOND.  Diagnostic: not part of the per-iteration path.
+ */
+int cascade_latency_regimes(cascade_ctx *ctx, const cascade_reqs *r, int n, int32_t D_act, int64_t K_act,
+                            int64_t *lat4_out, void *stream);
 
 /*
  * Least-remaining-budget-first order and admission (Algorithm 1, phase 2).

@@ -33,7 +33,11 @@ class OrcParams(C.Structure):
         ("c_dseq_q20", C.c_int64), ("c_dkv_q20", C.c_int64),
         ("delta_ns", C.c_int64 * 3), ("blk_ns", C.c_int64 * 3),
         ("ttft_ns", C.c_int64 * MAX_CLASSES), ("tpot_ns", C.c_int64 * MAX_CLASSES),
+        ("policy", C.c_int32), ("reserved", C.c_int32),
     ]
+
+
+POLICY_BUDGET, POLICY_FCFS, POLICY_EDF, POLICY_SJF = 0, 1, 2, 3
 
 
 class OrcSchedCounts(C.Structure):
@@ -89,6 +93,7 @@ def make_params(d: dict) -> OrcParams:
         p.ttft_ns[i] = int(v)
     for i, v in enumerate(d["tpot_ns"]):
         p.tpot_ns[i] = int(v)
+    p.policy = int(d.get("policy", 0))
     return p
 
 
@@ -130,6 +135,18 @@ def budget(p: OrcParams, reqs: dict, now_ns: int, D_act: int, K_act: int):
                           C.c_int64(now_ns), C.c_int32(D_act), C.c_int64(K_act),
                           _ptr(out_b, C.c_int64), _ptr(out_k, C.c_uint64))
     return out_b, out_k, int(st)
+
+
+def latency_regimes(p: OrcParams, reqs: dict, D_act: int, K_act: int):
+    """The estimator's four regimes, int64 [n, 4] (ns).  Returns (array, status bits)."""
+    n = len(reqs["prompt"])
+    a = {k: _arr(reqs[k], np.int32) for k in ("prompt", "n0", "n1", "n2")}
+    out = np.empty((n, 4), np.int64)
+    lib().orc_latency_regimes.restype = C.c_uint32
+    st = lib().orc_latency_regimes(C.byref(p), C.c_int(n), _ptr(a["prompt"], C.c_int32), _ptr(a["n0"], C.c_int32),
+                                   _ptr(a["n1"], C.c_int32), _ptr(a["n2"], C.c_int32), C.c_int32(D_act),
+                                   C.c_int64(K_act), _ptr(out, C.c_int64))
+    return out, int(st)
 
 
 def schedule(p: OrcParams, reqs: dict, key: np.ndarray, D_act: int):

@@ -149,10 +149,40 @@ uint32_t orc_budget(const orc_params *p, int n, const int64_t *arrival_ns, const
         int64_t pen = 0;
         if (tpot != 0) pen = O * std::max<int64_t>(0, tdec - tpot);
         const int64_t budget = B_rem - pen;
-        /* B6: 64-bit key = (tier-2 bit, clamped budget, arrival id) */
-        int64_t u = std::min(std::max(budget, -kBudgetClamp), kBudgetClamp - 1) + kBudgetClamp;
+        /* B6: 64-bit key = (tier-2 bit, clamped budget, arrival id).  The comparison policies keep the
+         *     same packing with one queue: arrival time (FCFS), TTFT deadline (EDF), tokens left to
+         *     prefill (SJF). */
+        int64_t v = budget;
+        bool tier2 = tier == 2;
+        if (p->policy == ORC_POLICY_FCFS) { v = -elapsed; tier2 = false; }
+        if (p->policy == ORC_POLICY_EDF) { v = p->ttft_ns[cls[r]] - elapsed; tier2 = false; }
+        if (p->policy == ORC_POLICY_SJF) { v = P - s_hit; tier2 = false; }
+        int64_t u = std::min(std::max(v, -kBudgetClamp), kBudgetClamp - 1) + kBudgetClamp;
         budget_out[r] = budget;
-        key_out[r] = (uint64_t(tier == 2) << 63) | (uint64_t(u) << 23) | uint64_t(id[r] & kIdMask);
+        key_out[r] = (uint64_t(tier2) << 63) | (uint64_t(u) << 23) | uint64_t(id[r] & kIdMask);
+    }
+    return status;
+}
+
+uint32_t orc_latency_regimes(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
+                             const int32_t *n2, int32_t D_act, int64_t K_act, int64_t *lat4_out) {
+    uint32_t status = 0;
+    const Load idle{0, 0};
+    const Load act = load_act(D_act, K_act);
+    const Load mx = load_max(p, D_act, K_act);
+    for (int r = 0; r < n; ++r) {
+        const int64_t P = prompt[r];
+        if (!request_valid(p, P, n0[r], n1[r], n2[r])) {
+            status |= ORC_ST_EPRECOND;
+            for (int i = 0; i < 4; ++i) lat4_out[4 * r + i] = 0;
+            continue;
+        }
+        const int64_t s_hit = int64_t(n0[r] + n1[r] + n2[r]) * p->bt;
+        const int64_t tp = restore_time(p, 1, n1[r]) + restore_time(p, 2, n2[r]);
+        lat4_out[4 * r + 0] = comp_q(p, tok_q(p, idle), P, 0) >> 20;          /* zero load, recompute all    */
+        lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, 0) >> 20;           /* actual load, recompute all  */
+        lat4_out[4 * r + 2] = tp + (comp_q(p, tok_q(p, act), P, s_hit) >> 20); /* actual load, tiered reuse   */
+        lat4_out[4 * r + 3] = tp + (comp_q(p, tok_q(p, mx), P, s_hit) >> 20);  /* maximum load, tiered reuse  */
     }
     return status;
 }

@@ -57,7 +57,14 @@ typedef struct orc_params {
     int64_t blk_ns[3];     /* Eq. 6: time per block on path P(k); [0] unused                 */
     int64_t ttft_ns[ORC_MAX_CLASSES]; /* class TTFT targets                                  */
     int64_t tpot_ns[ORC_MAX_CLASSES]; /* class TPOT targets; 0 disables the decode term      */
+    int32_t policy;        /* ordering: 0 least remaining budget, 1 FCFS, 2 EDF, 3 SJF (comparison policies) */
+    int32_t reserved;
 } orc_params;
+
+#define ORC_POLICY_BUDGET 0
+#define ORC_POLICY_FCFS 1
+#define ORC_POLICY_EDF 2
+#define ORC_POLICY_SJF 3
 
 /* counts written by orc_schedule */
 typedef struct orc_sched_counts {
@@ -126,6 +133,12 @@ uint32_t orc_kv_evict(const uint8_t *hbm_pool, int64_t hbm_blocks, int32_t n_chu
                       int64_t chunk_stride, int64_t block_stride,
                       uint8_t *host_pool, int64_t host_blocks,
                       const int32_t *src_ids, const int32_t *dst_ids, int n_copies);
+
+/* The estimator's four operating regimes for every request, lat4_out[4*r + i] in ns:
+ * 0 zero load, full recomputation; 1 actual load, full recomputation; 2 actual load with tier-aware
+ * prefix reuse; 3 maximum load with prefix reuse.  Regimes 2 and 3 are the L_actual and L_max of Eq. 3. */
+uint32_t orc_latency_regimes(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
+                             const int32_t *n2, int32_t D_act, int64_t K_act, int64_t *lat4_out);
 
 /* Pieces of the model exposed so the tests can pin them one by one. */
 int64_t orc_restore_time(const orc_params *p, int k, int64_t x_blocks);            /* Eq. 6 */

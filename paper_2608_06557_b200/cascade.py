@@ -23,7 +23,7 @@ ACT_NONE, ACT_RETAIN, ACT_EVICT, ACT_DROP = 0, 1, 2, 3
 
 EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_budget", "cascade_schedule",
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
-           "cascade_tier_plan_noalloc")
+           "cascade_tier_plan_noalloc", "cascade_latency_regimes")
 
 
 class Params(C.Structure):
@@ -35,7 +35,11 @@ class Params(C.Structure):
         ("c_dseq_q20", C.c_int64), ("c_dkv_q20", C.c_int64),
         ("delta_ns", C.c_int64 * 3), ("blk_ns", C.c_int64 * 3),
         ("ttft_ns", C.c_int64 * MAX_CLASSES), ("tpot_ns", C.c_int64 * MAX_CLASSES),
+        ("policy", C.c_int32), ("reserved", C.c_int32),
     ]
+
+
+POLICY_BUDGET, POLICY_FCFS, POLICY_EDF, POLICY_SJF = 0, 1, 2, 3
 
 
 class Reqs(C.Structure):
@@ -85,6 +89,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_destroy.restype = None
     lib.cascade_set_params.argtypes = [vp, C.POINTER(Params)]
     lib.cascade_budget.argtypes = [vp, C.POINTER(Reqs), C.c_int, i64, i32, i64, vp, vp, vp]
+    lib.cascade_latency_regimes.argtypes = [vp, C.POINTER(Reqs), C.c_int, i32, i64, vp, vp]
     lib.cascade_schedule.argtypes = [vp, C.POINTER(Reqs), vp, C.c_int, i32, vp, vp, vp, vp]
     lib.cascade_tier_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64, C.POINTER(Pools),
                                       C.POINTER(Plan), vp]
@@ -116,6 +121,7 @@ def make_params(d: dict) -> Params:
         p.ttft_ns[i] = int(v)
     for i, v in enumerate(d["tpot_ns"]):
         p.tpot_ns[i] = int(v)
+    p.policy = int(d.get("policy", 0))
     return p
 
 
@@ -183,6 +189,10 @@ class Context:
         _check(_lib.cascade_budget(self._h, C.byref(reqs), n, now_ns, D_act, K_act, _p(budget_out), _p(key_out),
                                    _stream(stream)), "cascade_budget")
 
+    def latency_regimes(self, reqs: Reqs, n, D_act, K_act, lat4_out, stream=None):
+        _check(_lib.cascade_latency_regimes(self._h, C.byref(reqs), n, D_act, K_act, _p(lat4_out), _stream(stream)),
+               "cascade_latency_regimes")
+
     def schedule(self, reqs: Reqs, key, n, D_act, order_out, grant_out, counts_dev, stream=None):
         _check(_lib.cascade_schedule(self._h, C.byref(reqs), _p(key), n, D_act, _p(order_out), _p(grant_out),
                                      _p(counts_dev), _stream(stream)), "cascade_schedule")
@@ -217,7 +227,7 @@ def tier_plan_noalloc(params: Params, reqs: Reqs, budget, order, grant, n, D_act
     when ``n`` exceeds NOALLOC_MAX_REQUESTS."""
     _check(_lib.cascade_tier_plan_noalloc(C.byref(params), C.byref(reqs), _p(budget), _p(order), _p(grant), n,
                                           D_act, K_act, C.byref(pools), C.byref(plan), _p(status_dev),
-                                          _stream(stream)), "cascade_tier_plan_noalloc")
+                                          _stream(stream)), "cascade_tier_plan_noalloc", "cascade_latency_regimes")
 
 
 def raw():

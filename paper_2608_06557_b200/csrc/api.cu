@@ -16,6 +16,7 @@ int cascade_validate_params(const cascade_params *p) {
               in_range(p->c_iter_q20, 0, one << 50) && in_range(p->c_dseq_q20, 0, one << 40) &&
               in_range(p->c_dkv_q20, 0, one << 28);
     if (ok) ok = (int64_t)(p->max_batch - 1) * p->max_ctx_avg <= (one << 32);
+    if (ok) ok = in_range(p->policy, CASCADE_POLICY_BUDGET, CASCADE_POLICY_SJF) && p->reserved == 0;
     for (int k = 1; ok && k <= 2; ++k)
         ok = in_range(p->delta_ns[k], 0, one << 30) && in_range(p->blk_ns[k], 1, one << 27);
     for (int c = 0; ok && c < p->n_classes; ++c)

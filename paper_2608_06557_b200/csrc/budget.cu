@@ -47,11 +47,44 @@ budget_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ 
     int64_t over = tdec - tpot;
     if (over < 0 || tpot == 0) over = 0;
     const int64_t budget = B_rem - O * over;
+    // ordering value: the budget, or the comparison policies' arrival time / deadline / tokens left
+    int64_t v = budget;
+    bool tier2 = B <= 0;
+    if (p.policy != CASCADE_POLICY_BUDGET) {
+        tier2 = false;
+        v = p.policy == CASCADE_POLICY_FCFS ? -elapsed
+          : p.policy == CASCADE_POLICY_EDF  ? p.ttft_ns[cls] - elapsed
+                                            : P - s_hit;
+    }
     const int64_t clampv = int64_t(1) << 39;
-    int64_t u = budget < -clampv ? -clampv : (budget > clampv - 1 ? clampv - 1 : budget);
+    int64_t u = v < -clampv ? -clampv : (v > clampv - 1 ? clampv - 1 : v);
     u += clampv;
     budget_out[i] = budget;
-    key_out[i] = (uint64_t(B <= 0) << 63) | (uint64_t(u) << 23) | id;
+    key_out[i] = (uint64_t(tier2) << 63) | (uint64_t(u) << 23) | id;
+}
+
+__global__ void __launch_bounds__(kThreads)
+regimes_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ LoadConsts lc, int64_t A_idle,
+               const __grid_constant__ cascade_reqs r, int n, int64_t *__restrict__ lat4, uint32_t *__restrict__ status) {
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i >= n) return;
+    const int64_t P = r.prompt[i];
+    const int64_t n0 = r.n0[i], n1 = r.n1[i], n2 = r.n2[i];
+    longlong4 out = make_longlong4(0, 0, 0, 0);
+    if (!dev_request_valid(p.bt, P, n0, n1, n2)) {
+        atomicOr(status, CASCADE_ST_EPRECOND);
+    } else {
+        const int64_t s_hit = (n0 + n1 + n2) * p.bt;
+        const int64_t tp = dev_restore_time(p, 1, n1) + dev_restore_time(p, 2, n2);
+        out.x = dev_comp_q(A_idle, p.c_attn_q20, P, 0) >> 20;
+        out.y = dev_comp_q(lc.A_act, p.c_attn_q20, P, 0) >> 20;
+        out.z = tp + (dev_comp_q(lc.A_act, p.c_attn_q20, P, s_hit) >> 20);
+        out.w = tp + (dev_comp_q(lc.A_max, p.c_attn_q20, P, s_hit) >> 20);
+    }
+    lat4[4 * (size_t)i + 0] = out.x;
+    lat4[4 * (size_t)i + 1] = out.y;
+    lat4[4 * (size_t)i + 2] = out.z;
+    lat4[4 * (size_t)i + 3] = out.w;
 }
 
 }  // namespace
@@ -68,6 +101,21 @@ extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, in
     const int grid = (n + kThreads - 1) / kThreads;
     budget_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(ctx->params, lc, *r, n, now_ns, budget_out, key_out,
                                                               ctx->status_dev);
+    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    return CASCADE_OK;
+}
+
+extern "C" int cascade_latency_regimes(cascade_ctx *ctx, const cascade_reqs *r, int n, int32_t D_act, int64_t K_act,
+                                       int64_t *lat4_out, void *stream) {
+    if (!ctx || !r || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
+    if (n == 0) return CASCADE_OK;
+    if (!lat4_out || !r->prompt || !r->n0 || !r->n1 || !r->n2) return CASCADE_EINVAL;
+    if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
+    const LoadConsts lc = make_load_consts(ctx->params, D_act, K_act);
+    const int64_t A_idle = make_load_consts(ctx->params, 0, 0).A_act;
+    const int grid = (n + kThreads - 1) / kThreads;
+    regimes_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(ctx->params, lc, A_idle, *r, n, lat4_out,
+                                                               ctx->status_dev);
     CASCADE_CUDA_TRY(ctx, cudaGetLastError());
     return CASCADE_OK;
 }

@@ -29,7 +29,7 @@ def test_binding_lists_the_same_symbols_and_struct_sizes():
     from paper_2608_06557_b200 import cascade as cs
     declared = set(declared_symbols())
     assert declared == set(cs.EXPORTS)
-    assert ctypes.sizeof(cs.Params) == 8 * 4 + 5 * 8 + 6 * 8 + 16 * 8
+    assert ctypes.sizeof(cs.Params) == 8 * 4 + 5 * 8 + 6 * 8 + 16 * 8 + 8
     assert ctypes.sizeof(cs.SchedCounts) == 16 and ctypes.sizeof(cs.PlanCounts) == 48
     assert ctypes.sizeof(cs.KvLayout) == 40 and ctypes.sizeof(cs.Reqs) == 72
 

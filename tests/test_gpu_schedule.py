@@ -172,3 +172,27 @@ def test_host_side_validation_needs_no_launch():
         cs.Context(bad, 16, 0)
     with pytest.raises(cs.CascadeError):
         cs.Context(w.params, cs.MAX_REQUESTS + 1, 0)
+
+
+@pytest.mark.parametrize("policy", [1, 2, 3])
+def test_comparison_policies(policy):
+    w = wl.config_tiny(1)
+    w.params = dict(w.params, policy=policy)
+    compare_iteration(w, f"policy{policy}")
+    w = wl.config_llama8b(seed=21, n=6000, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9)
+    w.hbm_tbl = w.host_tbl = w.hbm_free = w.host_free = None
+    w.hbm_free_count, w.host_free_count = 1 << 30, 1 << 30
+    w.params = dict(w.params, policy=policy)
+    compare_iteration(w, f"policy{policy}-6000")
+
+
+def test_latency_regimes_match():
+    torch, cs, Instance = _gpu()
+    for w in (wl.config_tiny(5), wl.config_llama8b(seed=8, n=3000, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9)):
+        w.reqs["prompt"][2] = 0                       # one request outside the input bounds
+        inst = Instance(w, alloc_pools=False)
+        lat = torch.empty((w.n, 4), dtype=torch.int64, device="cuda")
+        inst.ctx.latency_regimes(inst.reqs_struct, w.n, w.D_act, w.K_act, lat)
+        ref, st = oracle.latency_regimes(oracle.make_params(w.params), w.reqs, w.D_act, w.K_act)
+        assert np.array_equal(lat.cpu().numpy(), ref)
+        assert inst.ctx.status()[0] == st == 8

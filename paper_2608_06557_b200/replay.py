@@ -39,6 +39,7 @@ class Replay:
         self.max_active = max_active
         self.decode_residency = decode_residency   # iterations a finished prefill keeps its blocks (at most)
         self.stats = dict(restored=0, evicted=0, dropped=0, admitted=0, tokens=0, finished=0)
+        self.finish_ns = np.full(n, -1, np.int64)   # virtual time at which the prefill completed
 
     # ---- queue view ---------------------------------------------------------------------------
     def active_ids(self) -> np.ndarray:
@@ -93,6 +94,7 @@ class Replay:
         self.host_free_count = int(out["host_free_count"])
         tokens = 0
         x1_sum = 0
+        self._just_finished = []
         for s, r in enumerate(ids):
             act = int(out["action"][s])
             if act == ACT_EVICT:                       # whole HBM part now lives on host, in front of the old host part
@@ -121,6 +123,7 @@ class Replay:
                 self.decode_left[r] = min(int(t.pred_out[r]), self.decode_residency)
                 self.n0[r] = -(-int(t.prompt[r]) // bt)
                 self.stats["finished"] += 1
+                self._just_finished.append(r)
             else:
                 full = have // bt
                 if have % bt:                          # a partly filled block is recomputed next time
@@ -144,7 +147,43 @@ class Replay:
         per_tok = p["c_tok_q20"] >> 20
         xfer = 0 if x1_sum == 0 else p["delta_ns"][1] + x1_sum * p["blk_ns"][1]
         self.now += max(1_000_000, tokens * per_tok + xfer)
+        self.finish_ns[self._just_finished] = self.now       # first token leaves at the end of the iteration
         self.iteration += 1
 
     def done(self) -> bool:
         return not ((self.state == FUTURE) | (self.state == QUEUED)).any()
+
+
+def jain_index(values) -> float:
+    """Jain's fairness index of non-negative values: (sum v)^2 / (n * sum v^2); 1 when all are equal."""
+    v = np.asarray(values, float)
+    if len(v) == 0 or not np.any(v):
+        return 1.0
+    return float(v.sum() ** 2 / (len(v) * (v * v).sum()))
+
+
+def slo_report(replay: "Replay", bins=(0, 25, 50, 75, 90, 99, 100)) -> dict:
+    """TTFT outcome of the requests that have arrived: violation rate overall and per input-length
+    percentile bin (a request still queued past its target counts as violated), and the fairness
+    index over the bins' attainment A_i = max(0, 100 - V_i) in percent (the paper's Eq. 1)."""
+    t = replay.t
+    arrived = t.arrival_ns <= replay.now
+    ttft = np.asarray(t.params["ttft_ns"], np.int64)[t.cls]
+    done = replay.finish_ns >= 0
+    lat = np.where(done, replay.finish_ns - t.arrival_ns, replay.now - t.arrival_ns)
+    judged = arrived & (done | (lat > ttft))            # still waiting inside the target: not judged yet
+    viol = judged & (lat > ttft)
+    out = dict(arrived=int(arrived.sum()), judged=int(judged.sum()), finished=int((done & arrived).sum()),
+               violation_rate=float(viol.sum() / max(judged.sum(), 1)))
+    edges = np.percentile(t.prompt[judged], bins) if judged.any() else np.zeros(len(bins))
+    per_bin = []
+    for lo, hi in zip(edges[:-1], edges[1:]):
+        m = judged & (t.prompt >= lo) & ((t.prompt < hi) | (hi == edges[-1]))
+        if m.any():                                      # equal prompt lengths can leave a bin empty
+            per_bin.append(100.0 * float(viol[m].sum()) / int(m.sum()))
+    out["violation_pct_by_length_bin"] = [round(v, 1) for v in per_bin]
+    out["jain_index"] = round(jain_index([max(0.0, 100.0 - v) for v in per_bin]), 4)
+    lat_done = lat[done & arrived]
+    out["ttft_p50_s"] = float(np.percentile(lat_done, 50) / 1e9) if len(lat_done) else None
+    out["ttft_p95_s"] = float(np.percentile(lat_done, 95) / 1e9) if len(lat_done) else None
+    return out

@@ -224,6 +224,47 @@ def tier_plan(p: OrcParams, reqs: dict, budget_: np.ndarray, order: np.ndarray, 
                 evict_src=es[:ne], evict_dst=ed[:ne], counts=counts, status=int(st))
 
 
+class OrcPrefetchCounts(C.Structure):
+    _fields_ = [("n_prefetch", C.c_int32), ("n_requests", C.c_int32), ("hbm_free_after", C.c_int32),
+                ("n_restore_total", C.c_int32), ("link_ns_left", C.c_int64)]
+
+
+def prefetch_plan(p: OrcParams, reqs: dict, budget_: np.ndarray, order: np.ndarray, grant: np.ndarray,
+                  action: np.ndarray, x1: np.ndarray, D_act: int, K_act: int, link_budget_ns: int, hbm_reserve: int,
+                  pools: Pools, restore_src: np.ndarray, restore_dst: np.ndarray):
+    """Budget-bounded prefetch for queued requests.  ``pools`` (HBM table, HBM free list and its count) is
+    updated in place; the restore list passed in is extended.  Returns a dict with pf (blocks per request),
+    the extended restore_src/dst, counts and status bits."""
+    n = len(reqs["prompt"])
+    a = {k: _arr(reqs[k], np.int32) for k in ("prompt", "n0", "n1", "n2")}
+    with_tables = pools.hbm_tbl is not None
+    maxb = pools.hbm_tbl.shape[1] if with_tables else 0
+    cap = max(pools.restore_cap, 1)
+    rs = np.full(cap, -1, np.int32)
+    rd = np.full(cap, -1, np.int32)
+    rs[: len(restore_src)] = restore_src
+    rd[: len(restore_dst)] = restore_dst
+    nrest = C.c_int32(len(restore_src))
+    hc = C.c_int32(pools.hbm_free_count)
+    pf = np.empty(n, np.int32)
+    cnt = OrcPrefetchCounts()
+    lib().orc_prefetch_plan.restype = C.c_uint32
+    st = lib().orc_prefetch_plan(
+        C.byref(p), C.c_int(n), _ptr(a["prompt"], C.c_int32), _ptr(a["n0"], C.c_int32), _ptr(a["n1"], C.c_int32),
+        _ptr(a["n2"], C.c_int32), _ptr(_arr(budget_, np.int64), C.c_int64), _ptr(_arr(order, np.uint32), C.c_uint32),
+        _ptr(_arr(grant, np.int32), C.c_int32), _ptr(_arr(action, np.uint8), C.c_uint8),
+        _ptr(_arr(x1, np.int32), C.c_int32), C.c_int32(D_act), C.c_int64(K_act), C.c_int64(link_budget_ns),
+        C.c_int32(hbm_reserve), _ptr(pools.hbm_tbl, C.c_int32), _ptr(pools.host_tbl, C.c_int32), C.c_int32(maxb),
+        _ptr(pools.hbm_free, C.c_int32), C.byref(hc),
+        C.c_int32(0 if pools.hbm_free is None else len(pools.hbm_free)),
+        _ptr(rs, C.c_int32), _ptr(rd, C.c_int32), C.c_int32(pools.restore_cap), C.byref(nrest),
+        _ptr(pf, C.c_int32), C.byref(cnt))
+    pools.hbm_free_count = int(hc.value)
+    counts = {k: int(getattr(cnt, k)) for k, _ in OrcPrefetchCounts._fields_}
+    nr = min(counts["n_restore_total"], pools.restore_cap)
+    return dict(pf=pf, restore_src=rs[:nr], restore_dst=rd[:nr], counts=counts, status=int(st))
+
+
 def _layout_args(layout: dict):
     return (C.c_int64(layout["n_blocks"]), C.c_int32(layout["n_chunks"]), C.c_int64(layout["chunk_bytes"]),
             C.c_int64(layout["chunk_stride"]), C.c_int64(layout["block_stride"]))

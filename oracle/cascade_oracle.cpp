@@ -450,6 +450,82 @@ uint32_t orc_tier_plan(const orc_params *p, int n, const int32_t *prompt, const 
     return status;
 }
 
+/* Budget-bounded prefetch for requests that stay queued (the prefix prefetcher acting ahead of
+ * admission).  Walks the order; every valid request that was neither admitted nor preempted and
+ * holds host blocks gets, while link time and free HBM last:
+ *   m = its Eq. 7 bound for the host tier, if restoring m blocks beats recomputing them;
+ *   b = min(m, blocks that still fit the link budget, free HBM blocks above the reserve).
+ * Link time already spent this iteration: the sum of T_1(x1) over the admitted requests. */
+uint32_t orc_prefetch_plan(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
+                           const int32_t *n2, const int64_t *budget, const uint32_t *order, const int32_t *grant,
+                           const uint8_t *action, const int32_t *x1, int32_t D_act, int64_t K_act,
+                           int64_t link_budget_ns, int32_t hbm_reserve, int32_t *hbm_tbl, const int32_t *host_tbl,
+                           int32_t maxb, int32_t *hbm_free, int32_t *hbm_free_count, int32_t hbm_free_cap,
+                           int32_t *restore_src, int32_t *restore_dst, int32_t restore_cap, int32_t *n_restore,
+                           int32_t *pf_out, orc_prefetch_counts *counts) {
+    uint32_t status = 0;
+    const bool with_tables = hbm_tbl != nullptr;
+    const Load act = load_act(D_act, K_act);
+    int64_t hbm_pos = *hbm_free_count;
+    if (with_tables && (hbm_pos < 0 || hbm_pos > hbm_free_cap)) {
+        status |= ORC_ST_EBOUNDS;
+        hbm_pos = std::min<int64_t>(std::max<int64_t>(hbm_pos, 0), hbm_free_cap);
+    }
+    int64_t link_left = link_budget_ns;
+    for (int r = 0; r < n; ++r) {
+        pf_out[r] = 0;
+        bool ok = request_valid(p, prompt[r], n0[r], n1[r], n2[r]);
+        if (ok && with_tables) ok = ceil_div(prompt[r], p->bt) <= maxb;
+        if (ok && grant[r] > 0) link_left -= restore_time(p, 1, x1[r]);
+    }
+    int64_t avail = hbm_pos - hbm_reserve;
+    int32_t n_pf = 0, n_req = 0, rest = *n_restore;
+    const int64_t link_start = link_left;
+    for (int i = 0; i < n; ++i) {
+        const uint32_t r = order[i];
+        bool ok = request_valid(p, prompt[r], n0[r], n1[r], n2[r]);
+        if (ok && with_tables) ok = ceil_div(prompt[r], p->bt) <= maxb;
+        if (!ok || grant[r] > 0 || n1[r] <= 0) continue;
+        if (action[r] == ORC_ACT_EVICT || action[r] == ORC_ACT_DROP) continue;
+        /* Eq. 7 bound, then restore-vs-recompute */
+        const int64_t rem = std::max<int64_t>(0, budget[r]);
+        int64_t m = max_restorable(p, 1, rem, n1[r]);
+        if (m > 0 && plan_cost_q20(p, act, prompt[r], n0[r], m, 0) > plan_cost_q20(p, act, prompt[r], n0[r], 0, 0)) m = 0;
+        if (m == 0) continue;
+        /* what the link and HBM still allow */
+        int64_t b = m;
+        const int64_t by_link = link_left > p->delta_ns[1] ? (link_left - p->delta_ns[1]) / p->blk_ns[1] : 0;
+        b = std::min(b, by_link);
+        b = std::min(b, std::max<int64_t>(avail, 0));
+        if (b <= 0) continue;
+        link_left -= restore_time(p, 1, b);
+        avail -= b;
+        pf_out[r] = int32_t(b);
+        n_pf += int32_t(b);
+        ++n_req;
+        for (int64_t j = 0; j < b; ++j) {
+            --hbm_pos;
+            if (!with_tables) continue;
+            const int32_t g = hbm_pos < hbm_free_cap ? hbm_free[hbm_pos] : -1;
+            const int64_t t = int64_t(r) * maxb + n0[r] + j;
+            if (rest < restore_cap) { restore_src[rest] = host_tbl[t]; restore_dst[rest] = g; }
+            else status |= ORC_ST_ELISTCAP;
+            ++rest;
+            hbm_tbl[t] = g;
+        }
+    }
+    if (with_tables) {
+        *hbm_free_count = int32_t(hbm_pos);
+        *n_restore = rest;
+    }
+    counts->n_prefetch = n_pf;
+    counts->n_requests = n_req;
+    counts->hbm_free_after = int32_t(hbm_pos);
+    counts->n_restore_total = with_tables ? rest : *n_restore + n_pf;
+    counts->link_ns_left = link_start;
+    return status;
+}
+
 uint32_t orc_kv_restore(uint8_t *hbm_pool, int64_t hbm_blocks, int32_t n_chunks, int64_t chunk_bytes,
                         int64_t chunk_stride, int64_t block_stride, const uint8_t *host_pool, int64_t host_blocks,
                         const int32_t *src_ids, const int32_t *dst_ids, int n_copies) {

@@ -122,6 +122,24 @@ uint32_t orc_tier_plan(const orc_params *p, int n,
                        int32_t *evict_src, int32_t *evict_dst, int32_t evict_cap,
                        orc_plan_counts *counts);
 
+/* counts written by orc_prefetch_plan */
+typedef struct orc_prefetch_counts {
+    int32_t n_prefetch;      /* blocks appended to the restore list                   */
+    int32_t n_requests;      /* queued requests that got at least one block           */
+    int32_t hbm_free_after;  /* HBM free-list length afterwards                       */
+    int32_t n_restore_total; /* restore-list length afterwards (plan + prefetch)      */
+    int64_t link_ns_left;    /* link time left after the admitted set's own restores  */
+} orc_prefetch_counts;
+
+/* Budget-bounded prefetch for queued requests (see the .cpp).  Tables NULL = plan-only. */
+uint32_t orc_prefetch_plan(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
+                           const int32_t *n2, const int64_t *budget, const uint32_t *order, const int32_t *grant,
+                           const uint8_t *action, const int32_t *x1, int32_t D_act, int64_t K_act,
+                           int64_t link_budget_ns, int32_t hbm_reserve, int32_t *hbm_tbl, const int32_t *host_tbl,
+                           int32_t maxb, int32_t *hbm_free, int32_t *hbm_free_count, int32_t hbm_free_cap,
+                           int32_t *restore_src, int32_t *restore_dst, int32_t restore_cap, int32_t *n_restore,
+                           int32_t *pf_out, orc_prefetch_counts *counts);
+
 /* Step K2: paged copies.  HBM pool: chunk c of block b starts at
  * c*chunk_stride + b*block_stride.  Host pool: record h starts at h*n_chunks*chunk_bytes,
  * its chunks stored back to back.  Ids outside a pool are skipped and flagged. */

@@ -150,7 +150,7 @@ def place_blocks(rng, reqs, n_hbm, n_host, maxb, occupancy, hbm_free_target, pri
     return hbm_tbl, host_tbl, hbm_free, hbm_free_count, host_free, host_free_count
 
 
-def config_tiny(seed: int = 0) -> Workload:
+def config_tiny(seed: int = 0, hbm_free_target: int = 32) -> Workload:
     """64 requests, two SLO classes, 16 KiB blocks, 512+512 block pools, one iteration."""
     rng = np.random.default_rng(seed)
     ttft = [S // 2, 5 * S]
@@ -163,7 +163,7 @@ def config_tiny(seed: int = 0) -> Workload:
     reqs = draw_requests(rng, 64, [0.5, 0.5], ttft, 256, (16, 2048), [128, 128], (1, 4096), now, None,
                          lambda g, n: g.uniform(0, 1, n), 0.5, params["bt"])
     maxb = 128
-    tbl = place_blocks(rng, reqs, 512, 512, maxb, 1.0, 32, 0.5)
+    tbl = place_blocks(rng, reqs, 512, 512, maxb, 1.0, hbm_free_target, 0.5)
     return Workload("tiny", params, reqs, now, 8, 8 * 512, kv_layout(512, n_chunks, chunk_bytes), 512, maxb, *tbl)
 
 

@@ -267,6 +267,39 @@ int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *bu
                       int32_t *grant, int n, int32_t D_act, int64_t K_act, const cascade_pools *pools,
                       const cascade_plan *plan_out, void *stream);
 
+/* written to device memory by cascade_prefetch_plan */
+typedef struct cascade_prefetch_counts {
+    int32_t n_prefetch;      /* blocks appended to the restore list                  */
+    int32_t n_requests;      /* queued requests that got at least one block          */
+    int32_t hbm_free_after;  /* HBM free-list length afterwards                      */
+    int32_t n_restore_total; /* restore-list length afterwards (plan + prefetch)     */
+    int64_t link_ns_left;    /* link time left after the admitted set's own restores */
+} cascade_prefetch_counts;
+
+/*
+ * Budget-bounded prefetch for requests that stay queued: the paper's prefix prefetcher "prefetching
+ * required prefix KV states within their budget bounds" (overview of the system; Eq. 6, Eq. 7) applied
+ * ahead of admission.  Call it after cascade_tier_plan and before cascade_kv_restore.
+ *   Link time left this iteration = link_budget_ns - sum of T_1(x1) over the admitted requests.
+ *   Walking `order`, every request that is valid, not admitted (grant <= 0), not preempted by this
+ *   iteration's plan (action EVICT / DROP) and holds host blocks (n1 > 0) gets
+ *       m = min(n1, Eq. 7 bound from its budget), or 0 if restoring m blocks is predicted slower than
+ *           recomputing them,
+ *       b = min(m, blocks that still fit the link time left, free HBM blocks above hbm_reserve),
+ *   and uses up T_1(b) of link time and b HBM blocks.
+ * Outputs: pf_out[n] (blocks prefetched per slot); for each such block an HBM id is popped from
+ * hbm_free, written to hbm_tbl[r][n0 + j] and the pair (host_tbl[r][n0 + j], id) is appended to the
+ * plan's restore list; plan->counts->n_restore and *hbm_free_count are updated so that the following
+ * cascade_kv_restore moves the prefetched blocks together with the admitted set's.  The caller folds
+ * pf_out into next iteration's hit profile (n0 += pf, n1 -= pf).  With pools->hbm_tbl == NULL only
+ * pf_out and the counts are produced.  0 <= link_budget_ns <= 2^50, hbm_reserve >= 0.
+ */
+int cascade_prefetch_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *budget, const uint32_t *order,
+                          const int32_t *grant, const uint8_t *action, int n, int32_t D_act, int64_t K_act,
+                          int64_t link_budget_ns, int32_t hbm_reserve, const cascade_pools *pools,
+                          const cascade_plan *plan, int32_t *pf_out, cascade_prefetch_counts *counts_dev,
+                          void *stream);
+
 /*
  * Restore: for i < count, copy host record src_ids[i] into HBM block dst_ids[i]
  * (n_chunks pieces of chunk_bytes scattered into the paged layout).

@@ -231,7 +231,7 @@ class OrcPrefetchCounts(C.Structure):
 
 def prefetch_plan(p: OrcParams, reqs: dict, budget_: np.ndarray, order: np.ndarray, grant: np.ndarray,
                   action: np.ndarray, x1: np.ndarray, D_act: int, K_act: int, link_budget_ns: int, hbm_reserve: int,
-                  pools: Pools, restore_src: np.ndarray, restore_dst: np.ndarray):
+                  pools: Pools, restore_src: np.ndarray, restore_dst: np.ndarray, n_restore: int | None = None):
     """Budget-bounded prefetch for queued requests.  ``pools`` (HBM table, HBM free list and its count) is
     updated in place; the restore list passed in is extended.  Returns a dict with pf (blocks per request),
     the extended restore_src/dst, counts and status bits."""
@@ -244,7 +244,7 @@ def prefetch_plan(p: OrcParams, reqs: dict, budget_: np.ndarray, order: np.ndarr
     rd = np.full(cap, -1, np.int32)
     rs[: len(restore_src)] = restore_src
     rd[: len(restore_dst)] = restore_dst
-    nrest = C.c_int32(len(restore_src))
+    nrest = C.c_int32(len(restore_src) if n_restore is None else n_restore)
     hc = C.c_int32(pools.hbm_free_count)
     pf = np.empty(n, np.int32)
     cnt = OrcPrefetchCounts()

@@ -23,7 +23,7 @@ ACT_NONE, ACT_RETAIN, ACT_EVICT, ACT_DROP = 0, 1, 2, 3
 
 EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_budget", "cascade_schedule",
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
-           "cascade_tier_plan_noalloc", "cascade_latency_regimes")
+           "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan")
 
 
 class Params(C.Structure):
@@ -90,6 +90,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_set_params.argtypes = [vp, C.POINTER(Params)]
     lib.cascade_budget.argtypes = [vp, C.POINTER(Reqs), C.c_int, i64, i32, i64, vp, vp, vp]
     lib.cascade_latency_regimes.argtypes = [vp, C.POINTER(Reqs), C.c_int, i32, i64, vp, vp]
+    lib.cascade_prefetch_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, vp, C.c_int, i32, i64, i64, i32,
+                                          C.POINTER(Pools), C.POINTER(Plan), vp, vp, vp]
     lib.cascade_schedule.argtypes = [vp, C.POINTER(Reqs), vp, C.c_int, i32, vp, vp, vp, vp]
     lib.cascade_tier_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64, C.POINTER(Pools),
                                       C.POINTER(Plan), vp]
@@ -201,6 +203,12 @@ class Context:
         _check(_lib.cascade_tier_plan(self._h, C.byref(reqs), _p(budget), _p(order), _p(grant), n, D_act, K_act,
                                       C.byref(pools), C.byref(plan), _stream(stream)), "cascade_tier_plan")
 
+    def prefetch_plan(self, reqs: Reqs, budget, order, grant, action, n, D_act, K_act, link_budget_ns, hbm_reserve,
+                      pools: Pools, plan: Plan, pf_out, counts_dev, stream=None):
+        _check(_lib.cascade_prefetch_plan(self._h, C.byref(reqs), _p(budget), _p(order), _p(grant), _p(action), n,
+                                          D_act, K_act, link_budget_ns, hbm_reserve, C.byref(pools), C.byref(plan),
+                                          _p(pf_out), _p(counts_dev), _stream(stream)), "cascade_prefetch_plan")
+
     def kv_restore(self, layout: KvLayout, hbm_pool, src_pool, src_blocks, src_is_device, src_ids, dst_ids,
                    n_copies_dev, n_copies_max, stream=None):
         _check(_lib.cascade_kv_restore(self._h, C.byref(layout), _p(hbm_pool), _p(src_pool), src_blocks,
@@ -227,7 +235,7 @@ def tier_plan_noalloc(params: Params, reqs: Reqs, budget, order, grant, n, D_act
     when ``n`` exceeds NOALLOC_MAX_REQUESTS."""
     _check(_lib.cascade_tier_plan_noalloc(C.byref(params), C.byref(reqs), _p(budget), _p(order), _p(grant), n,
                                           D_act, K_act, C.byref(pools), C.byref(plan), _p(status_dev),
-                                          _stream(stream)), "cascade_tier_plan_noalloc", "cascade_latency_regimes")
+                                          _stream(stream)), "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan")
 
 
 def raw():

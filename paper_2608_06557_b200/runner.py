@@ -124,6 +124,22 @@ class Instance:
         c.tier_plan(self.reqs_struct, self.budget, self.order, self.grant, self.n, self.D_act, self.K_act,
                     self.pools_struct, self.plan_struct, stream)
 
+    def run_prefetch(self, link_budget_ns: int, hbm_reserve: int = 0, stream=None):
+        """Budget-bounded prefetch for the requests that stay queued (after run_schedule, before run_copies)."""
+        if not hasattr(self, "pf"):
+            self.pf = torch.empty(self.cap, dtype=torch.int32, device=self.device)
+            self.prefetch_counts = torch.zeros(6, dtype=torch.int32, device=self.device)   # 24-byte struct
+        self.ctx.prefetch_plan(self.reqs_struct, self.budget, self.order, self.grant, self.action, self.n, self.D_act,
+                               self.K_act, link_budget_ns, hbm_reserve, self.pools_struct, self.plan_struct, self.pf,
+                               self.prefetch_counts, stream)
+
+    def fetch_prefetch(self) -> dict:
+        torch.cuda.synchronize(self.device)
+        c = self.prefetch_counts.cpu().numpy()
+        return dict(pf=self.pf[: self.n].cpu().numpy(),
+                    counts=dict(n_prefetch=int(c[0]), n_requests=int(c[1]), hbm_free_after=int(c[2]),
+                                n_restore_total=int(c[3]), link_ns_left=int(c[4:6].view(np.int64)[0])))
+
     def run_copies(self, stream=None, record_pool=None, record_is_device: bool = False):
         """evict then restore, with the counts the plan left in device memory."""
         c = self.ctx

@@ -30,6 +30,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "restored KV GB/s vs host-link/HBM roofline; per-iteration schedule latency us"
+# dram__bytes_read.sum + dram__bytes_write.sum per 2 MiB block of the host-link copy kernel, from the
+# 128-block ncu captures summarised in profiles/kv_copy_bulk_kernel_pinned_host_128_blocks.md; the traffic
+# grows in proportion to the blocks moved, so a launch's traffic is this figure times its block count
+# (the restore figure is low because part of the written lines is still in L2 when the kernel ends)
+NCU_DRAM_BYTES_PER_BLOCK = {"evict": (268_630_272 + 3_547_648) / 128, "restore": (99_840 + 209_025_792) / 128}
 GB = 1e9
 
 
@@ -416,7 +421,9 @@ def ours_main(args):
     dom_launch_bytes = (ev_bytes if dominant.endswith("<evict>") else rs_bytes) / K
     roofline = dict(bound="host_link", kernel=dominant, achieved=round(dom_ach, 2), peak=round(dom_peak, 2),
                     unit="GB/s", frac=round(dom_ach / dom_peak, 4) if dom_peak else None,
-                    traffic=None,
+                    traffic=int(NCU_DRAM_BYTES_PER_BLOCK["evict" if dominant.endswith("<evict>") else "restore"]
+                                * dom_launch_bytes / bb),
+                    traffic_source="ncu capture of 128 blocks, scaled by the blocks per launch",
                     algorithmic_bytes_per_launch=int(dom_launch_bytes),
                     peak_source="pinned cudaMemcpyAsync of one contiguous 1 GiB buffer measured by this run "
                                 "(MEASURED_PEAKS.json holds no host-link figure)",

@@ -14,9 +14,11 @@ from dataclasses import dataclass, field
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "cascade_oracle.cpp")
 _HDR = os.path.join(_HERE, "cascade_oracle.h")
-_LIB = os.path.join(_HERE, "liboracle.so")
+# CASCADE_ORACLE_SRC points the tests at an altered copy of the source (the mutation check of the pins);
+# its library is built next to that copy, never over the real one
+_SRC = os.environ.get("CASCADE_ORACLE_SRC") or os.path.join(_HERE, "cascade_oracle.cpp")
+_LIB = (os.path.splitext(_SRC)[0] + ".so") if os.environ.get("CASCADE_ORACLE_SRC") else os.path.join(_HERE, "liboracle.so")
 
 MAX_CLASSES = 8
 FLAG_HBM_PRIVATE, FLAG_RUNNING = 1, 2
@@ -55,7 +57,8 @@ def build(force: bool = False) -> str:
     newest = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".{os.getpid()}.tmp"
-        subprocess.check_call(["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-Wall", "-Wextra", "-o", tmp, _SRC])
+        subprocess.check_call(["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-Wall", "-Wextra", "-I", _HERE, "-o", tmp,
+                               _SRC])
         os.replace(tmp, _LIB)
     return _LIB
 

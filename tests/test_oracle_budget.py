@@ -184,3 +184,14 @@ def test_precondition_flag():
         b, k, st = oracle.budget(p, bad, 10 * S, 0, 0)
         assert st == oracle.ST_EPRECOND
         assert int(k[0]) >> 63 == 1
+
+
+def test_zero_budget_goes_to_tier_two():
+    """Eq. 4 with B exactly 0: only a strictly positive budget enters the Tier-1 queue."""
+    d = wl.default_params(gamma_q16=65536, c_attn_q20=0, c_dseq_q20=0, c_dkv_q20=0, c_tok_q20=30_000 * wl.Q20,
+                          c_iter_q20=512 * 1000 * wl.Q20, ttft_ns=[1000 * 31_000, 1000 * 31_000 + 1], tpot_ns=[0, 0])
+    p = oracle.make_params(d)
+    b, k, _ = oracle.budget(p, one_request(1000, 1, (0, 0, 0), 0, cls=0), 10 * S, 0, 0)
+    assert int(b[0]) == 0 and int(k[0]) >> 63 == 1
+    b, k, _ = oracle.budget(p, one_request(1000, 1, (0, 0, 0), 0, cls=1), 10 * S, 0, 0)
+    assert int(b[0]) == 1 and int(k[0]) >> 63 == 0

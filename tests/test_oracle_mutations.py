@@ -1,0 +1,87 @@
+"""The pins must be able to fail: each plausible slip, planted in a copy of the oracle's source, has to
+break at least one of them.  (The real oracle is untouched: the altered copy is compiled elsewhere.)"""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "cascade_oracle.cpp")
+PINS = ["test_oracle_budget.py", "test_oracle_schedule.py", "test_oracle_plan.py", "test_oracle_copy.py",
+        "test_oracle_prefetch.py", "test_oracle_policies.py"]
+
+MUTATIONS = [
+    ("eq3 drops the one half", "const int64_t L = ((L_act + L_max) * p->gamma_q16) >> 17;",
+     "const int64_t L = ((L_act + L_max) * p->gamma_q16) >> 16;"),
+    ("eq4 sign", "const int64_t B = p->ttft_ns[cls[r]] - L;", "const int64_t B = p->ttft_ns[cls[r]] + L;"),
+    ("eq5 sign", "const int64_t B_rem = B - elapsed;", "const int64_t B_rem = B + elapsed;"),
+    ("tier test", "const int tier = (B > 0) ? 1 : 2;", "const int tier = (B >= 0) ? 1 : 2;"),
+    ("attention term sign", "p->c_attn_q20 * (P * P - s * s)", "p->c_attn_q20 * (P * P + s * s)"),
+    ("eq6 overhead charged for nothing", "return x == 0 ? 0 : p->delta_ns[k] + x * p->blk_ns[k];",
+     "return p->delta_ns[k] + x * p->blk_ns[k];"),
+    ("eq7 rounds up", "return std::min<int64_t>(nk, head / p->blk_ns[k]);",
+     "return std::min<int64_t>(nk, (head + p->blk_ns[k] - 1) / p->blk_ns[k]);"),
+    ("key shift", "(uint64_t(u) << 23)", "(uint64_t(u) << 24)"),
+    ("maximum-load regime off by one", "std::max<int64_t>(D_act, p->max_batch - 1)",
+     "std::max<int64_t>(D_act, p->max_batch)"),
+    ("decode step without the request itself", "const Load act1{act.D + 1, act.K + P};",
+     "const Load act1{act.D, act.K + P};"),
+    ("penalty ignores the class target", "pen = O * std::max<int64_t>(0, tdec - tpot);",
+     "pen = O * std::max<int64_t>(0, tdec);"),
+    ("reserve not limited by tier-2 demand",
+     "const int64_t R2 = std::min<int64_t>(std::min<int64_t>(p->tier2_reserve, W2), TB);",
+     "const int64_t R2 = std::min<int64_t>(p->tier2_reserve, TB);"),
+    ("decodes do not take tokens", "std::max<int64_t>(0, int64_t(p->token_budget) - D_act)",
+     "std::max<int64_t>(0, int64_t(p->token_budget))"),
+    ("batch cap off by one", "if (rank >= seq_cap) grant_out[r] = 0;", "if (rank > seq_cap) grant_out[r] = 0;"),
+    ("tie goes to recompute", "if (F <= bF) { bF = F; bx1 = x1max; bx2 = 0; }",
+     "if (F < bF) { bF = F; bx1 = x1max; bx2 = 0; }"),
+    ("deep fetch still runs tokens", "const int64_t run = (bx2 > 0) ? 0 : std::min<int64_t>(grant[r], P - have);",
+     "const int64_t run = std::min<int64_t>(grant[r], P - have);"),
+    ("capacity cut off by one", "if (c > cap) {", "if (c >= cap) {"),
+    ("victims walked from the front", "for (int i = n - 1; i >= 0; --i) {", "for (int i = 0; i < n; ++i) {"),
+    ("shared holders preempted",
+     "const bool eligible = valid[r] && grant[r] <= 0 && (flags[r] & ORC_FLAG_HBM_PRIVATE) && n0[r] > 0;",
+     "const bool eligible = valid[r] && grant[r] <= 0 && n0[r] > 0;"),
+    ("host room test off by one", "if (fits && h + n0[r] <= host_cnt)", "if (fits && h + n0[r] < host_cnt)"),
+    ("evict list swapped", "evict_src[n_evict] = g; evict_dst[n_evict] = hslot;",
+     "evict_src[n_evict] = hslot; evict_dst[n_evict] = g;"),
+    ("restore reads the wrong table column", "restore_src[n_restore] = host_tbl[int64_t(r) * maxb + j];",
+     "restore_src[n_restore] = host_tbl[int64_t(r) * maxb + j - n0[r]];"),
+    ("record chunks strided like the pool", "host_pool + s * bb + c * chunk_bytes", "host_pool + s * bb + c * chunk_stride"),
+    ("evict copies the wrong way", "std::memcpy(host_pool + d * bb + c * chunk_bytes, hbm_pool + c * chunk_stride + s * block_stride,",
+     "std::memcpy(const_cast<uint8_t *>(hbm_pool) + c * chunk_stride + s * block_stride, host_pool + d * bb + c * chunk_bytes,"),
+    ("prefetch ignores the admitted set's link time", "if (ok && grant[r] > 0) link_left -= restore_time(p, 1, x1[r]);",
+     "if (ok && grant[r] > 0) link_left -= 0;"),
+    ("prefetch serves preempted requests", "if (action[r] == ORC_ACT_EVICT || action[r] == ORC_ACT_DROP) continue;", ""),
+    ("edf uses the wrong sign", "v = p->ttft_ns[cls[r]] - elapsed; tier2 = false;", "v = p->ttft_ns[cls[r]] + elapsed; tier2 = false;"),
+    ("regime 1 reuses the prefix", "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, 0) >> 20;",
+     "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, s_hit) >> 20;"),
+]
+
+
+def run_pins(env):
+    cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider"] + [os.path.join(ROOT, "tests", f) for f in PINS]
+    return subprocess.run(cmd, env=env, cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+
+
+def test_every_planted_slip_is_caught(tmp_path):
+    text = open(SRC).read()
+    survivors = []
+    for i, (name, old, new) in enumerate(MUTATIONS):
+        assert text.count(old) == 1, f"mutation '{name}' no longer matches the source exactly once"
+        path = tmp_path / f"mutant_{i}.cpp"
+        path.write_text(text.replace(old, new))
+        env = dict(os.environ, CASCADE_ORACLE_SRC=str(path))
+        res = run_pins(env)
+        if res.returncode == 0:
+            survivors.append(name)
+    assert not survivors, f"pins did not notice: {survivors}"
+
+
+def test_the_unaltered_copy_passes(tmp_path):
+    path = tmp_path / "copy.cpp"
+    path.write_text(open(SRC).read())
+    res = run_pins(dict(os.environ, CASCADE_ORACLE_SRC=str(path)))
+    assert res.returncode == 0, res.stdout[-2000:]

@@ -268,3 +268,81 @@ def test_transfer_beyond_budget_falls_back_to_recompute():
     out = oracle.tier_plan(p, reqs, np.array([30_000], np.int64), np.array([0], np.uint32),
                            np.array([512], np.int32), 0, 0, oracle.Pools(None, None, None, 1 << 30, None, 1 << 30))
     assert out["x1"][0] == 0 and out["tokens_run"][0] == 512
+
+
+def _plan_only():
+    return oracle.Pools(None, None, None, 1 << 30, None, 1 << 30)
+
+
+def test_equal_cost_restores():
+    """Transfer time exactly equal to the compute it saves: the tie goes to the restore."""
+    d = wl.default_params(c_attn_q20=0, c_dseq_q20=0, c_dkv_q20=0, c_tok_q20=30_000 * wl.Q20,
+                          c_iter_q20=512 * 1000 * wl.Q20, delta_ns=[0, 0, 0], blk_ns=[0, 16 * 31_000, 10**6])
+    p = oracle.make_params(d)
+    reqs = dict(prompt=[1000], n0=[2], n1=[7], n2=[0], flags=[0])
+    assert oracle.plan_cost_q20(p, 0, 0, 1000, 2, 7, 0) == oracle.plan_cost_q20(p, 0, 0, 1000, 2, 0, 0)
+    out = oracle.tier_plan(p, reqs, np.array([10**9], np.int64), np.array([0], np.uint32), np.array([64], np.int32),
+                           0, 0, _plan_only())
+    assert out["x1"][0] == 7
+    d["blk_ns"][1] += 1                        # one nanosecond dearer per block: recompute
+    out = oracle.tier_plan(oracle.make_params(d), reqs, np.array([10**9], np.int64), np.array([0], np.uint32),
+                           np.array([64], np.int32), 0, 0, _plan_only())
+    assert out["x1"][0] == 0
+
+
+def three_requests(hbm_free, host_free, victim_n0=10, victim_n1=0, victim_budget=10**9):
+    """Slot 0 is admitted and needs 2 restored + 4 new blocks; slot 1 holds `victim_n0` private HBM blocks
+    and sits at the end of the order; slot 2 is queued without HBM blocks."""
+    maxb = 32
+    reqs = dict(prompt=[160, 400, 100], n0=[0, victim_n0, 0], n1=[2, victim_n1, 3], n2=[0, 0, 0],
+                flags=[0, PRIV, 0])
+    hbm_tbl = np.full((3, maxb), -1, np.int32)
+    host_tbl = np.full((3, maxb), -1, np.int32)
+    hbm_tbl[1, :victim_n0] = 100 + np.arange(victim_n0)
+    host_tbl[0, :2] = [50, 51]
+    host_tbl[1, victim_n0:victim_n0 + victim_n1] = 60 + np.arange(victim_n1)
+    host_tbl[2, :3] = [70, 71, 72]
+    hf = np.full(256, -1, np.int32)
+    hf[:hbm_free] = 200 + np.arange(hbm_free)
+    of = np.full(256, -1, np.int32)
+    of[:host_free] = 300 + np.arange(host_free)
+    pools = oracle.Pools(hbm_tbl, host_tbl, hf, hbm_free, of, host_free, 256, 256)
+    budget = np.array([10**9, victim_budget, 5 * 10**8], np.int64)
+    order = np.array([0, 2, 1], np.uint32)
+    grant = np.array([64, 0, 0], np.int32)
+    return reqs, budget, order, grant, pools
+
+
+def test_capacity_and_host_room_exactly_met():
+    p = oracle.make_params(wl.default_params())
+    # need = 2 restored + 4 computed = 6; free 1 + preemptable 5 = 6: still admitted, the victim is taken
+    reqs, budget, order, grant, pools = three_requests(hbm_free=1, host_free=5, victim_n0=5)
+    out = oracle.tier_plan(p, reqs, budget, order, grant, 0, 0, pools)
+    assert out["counts"]["n_unadmitted"] == 0 and out["counts"]["hbm_need"] == 6 and grant[0] == 64
+    # the victim's 5 blocks fit the 5 free host records exactly: spilled, not dropped
+    assert out["action"][1] == oracle.ACT_EVICT and out["counts"]["n_evict"] == 5
+    # spilled blocks: sources are the victim's HBM ids in table order, destinations come off the top of the host stack
+    assert out["evict_src"].tolist() == [100, 101, 102, 103, 104]
+    assert out["evict_dst"].tolist() == [304, 303, 302, 301, 300]
+    assert pools.host_tbl[1, :5].tolist() == [304, 303, 302, 301, 300] and np.all(pools.hbm_tbl[1, :5] == -1)
+    # freed ids are pushed, then popped from the top for the restored and the computed blocks
+    assert out["restore_src"].tolist() == [50, 51] and out["restore_dst"].tolist() == [104, 103]
+    assert pools.hbm_tbl[0, :6].tolist() == [104, 103, 102, 101, 100, 200]
+    assert pools.hbm_free_count == 0 and pools.host_free_count == 0
+    # one block less of room on either side flips the decisions
+    reqs, budget, order, grant, pools = three_requests(hbm_free=0, host_free=5, victim_n0=5)
+    out = oracle.tier_plan(p, reqs, budget, order, grant, 0, 0, pools)
+    assert out["counts"]["n_unadmitted"] == 1 and grant[0] == 0
+    reqs, budget, order, grant, pools = three_requests(hbm_free=1, host_free=4, victim_n0=5)
+    out = oracle.tier_plan(p, reqs, budget, order, grant, 0, 0, pools)
+    assert out["action"][1] == oracle.ACT_DROP and out["counts"]["n_evict"] == 0
+
+
+def test_iteration_invariants_with_restores():
+    """Looser class targets leave the admitted set budget to restore with: the restore list is exercised."""
+    restored = 0
+    for seed in range(6):
+        w = wl.config_tiny(seed, hbm_free_target=120)
+        w.params["ttft_ns"] = [20 * t for t in w.params["ttft_ns"]]
+        restored += check_iteration(w)["plan"]["counts"]["n_restore"]
+    assert restored > 20

@@ -106,3 +106,17 @@ def test_prefetch_serves_the_tightest_budget_first_and_stops_at_the_link_budget(
         i += 1
     assert 0 < i < len(served)
     assert all(v == 0 for v in served[i + 1:])
+
+
+def test_preempted_requests_are_not_prefetched():
+    """A request spilled by this iteration's plan keeps host blocks but must not get them back at once."""
+    from test_oracle_plan import three_requests
+    p = oracle.make_params(wl.default_params())
+    reqs, budget, order, grant, pools = three_requests(hbm_free=1, host_free=20, victim_n0=10, victim_n1=5)
+    plan = oracle.tier_plan(p, reqs, budget, order, grant, 0, 0, pools)
+    assert plan["action"][1] == oracle.ACT_EVICT and pools.hbm_free_count == 5
+    r = dict(reqs, arrival_ns=[0, 0, 0], pred_out=[1, 1, 1], id=[0, 1, 2], cls=[0, 0, 0])
+    out = oracle.prefetch_plan(p, r, budget, order, grant, plan["action"], plan["x1"], 0, 0, 10**9, 0, pools,
+                               plan["restore_src"], plan["restore_dst"])
+    assert out["pf"].tolist() == [0, 0, 3]          # only the queued request that was left alone
+    assert out["counts"]["n_prefetch"] == 3 and pools.hbm_free_count == 2

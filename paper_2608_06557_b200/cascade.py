@@ -235,7 +235,7 @@ def tier_plan_noalloc(params: Params, reqs: Reqs, budget, order, grant, n, D_act
     when ``n`` exceeds NOALLOC_MAX_REQUESTS."""
     _check(_lib.cascade_tier_plan_noalloc(C.byref(params), C.byref(reqs), _p(budget), _p(order), _p(grant), n,
                                           D_act, K_act, C.byref(pools), C.byref(plan), _p(status_dev),
-                                          _stream(stream)), "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan")
+                                          _stream(stream)), "cascade_tier_plan_noalloc")
 
 
 def raw():

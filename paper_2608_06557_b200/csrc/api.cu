@@ -51,6 +51,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->sort_match = e ? atoi(e) : 0;
     e = getenv("CASCADE_SORT_STAGE");
     ctx->sort_stage = e ? atoi(e) : -1;  // -1: staged scatter only when a thread holds four or more keys
+    e = getenv("CASCADE_SORT_ASYNC");
+    ctx->sort_async = e ? atoi(e) : 1;
     e = getenv("CASCADE_COPY_CTAS_HOST");
     ctx->copy_ctas_host = e && atoi(e) > 0 ? atoi(e) : 4;
     e = getenv("CASCADE_COPY_CTAS_DEV");

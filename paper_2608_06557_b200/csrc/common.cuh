@@ -24,6 +24,7 @@ struct cascade_ctx {
     int sort_threads;            // threads per CTA override (0 = automatic)
     int sort_match;              // 1: rank digits with match.any, 0: with eight ballots
     int sort_stage;              // 1: group elements by digit locally before the remote scatter
+    int sort_async;              // 1: per-pass exchanges complete on mbarriers instead of cluster barriers
     int copy_ctas_host;          // copy CTAs per SM when the record pool is pinned host memory
     int copy_ctas_dev;           // copy CTAs per SM when the record pool is device memory
     int copy_bulk_host;          // >0: TMA bulk-copy ring (that many CTAs per SM) for the pinned-host path
@@ -90,9 +91,9 @@ static inline bool cascade_pick_geometry(const cascade_ctx *ctx, int n, int *T, 
     int t, c, k;
     if (n <= 1024) { t = 256; c = 4; k = 1; }
     else if (n <= 2048) { t = 256; c = 8; k = 1; }
-    else if (n <= 4096) { t = 256; c = 8; k = 2; }
+    else if (n <= 4096) { t = 256; c = 16; k = 1; }
     else if (n <= 8192) { t = 256; c = 16; k = 2; }
-    else if (n <= 16384) { t = 512; c = 16; k = 2; }
+    else if (n <= 16384) { t = 256; c = 16; k = 4; }
     else if (n <= 32768) { t = 512; c = 16; k = 4; }
     else { t = 512; c = 16; k = 8; }
     if (ctx->sort_threads == 256 || ctx->sort_threads == 512 || ctx->sort_threads == 1024) t = ctx->sort_threads;

@@ -12,11 +12,18 @@
 //   (d) scatters every element straight into the destination CTA's shared memory (16-byte
 //       remote store), so keys never visit global memory between passes.
 // Passes whose digit is the same in every key are skipped.  The admission scans run on the sorted
-// elements while they are still on chip.  Two cluster barriers per pass are the only inter-CTA
-// waits; they are hardware barriers (no spin loops).
+// elements while they are still on chip.
+// The two exchanges of a pass are data driven: histograms and elements travel as 16-byte
+// asynchronous stores (st.async) that report their bytes to an mbarrier of the receiving CTA, so a
+// CTA goes on as soon as ITS inputs have landed instead of waiting at a cluster-wide barrier.  The
+// histogram exchange doubles as the guard for buffer reuse: nobody scatters into a CTA before that
+// CTA has published the histogram of the elements it already holds in registers.  The mbarrier waits
+// are clock-bounded (CASCADE_ST_ETIMEOUT, results then undefined but every CTA still walks the same
+// cluster barriers and exits).  CASCADE_SORT_ASYNC=0 selects plain cluster barriers instead.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "mbarrier.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -26,6 +33,7 @@ constexpr int kBins = 256;
 constexpr int kWhistStride = kBins + 2;  // in uint16 units: column reads by 32 lanes hit 32 banks
 constexpr int kMaxCluster = 16;
 constexpr unsigned kFull = 0xffffffffu;
+constexpr long long kWaitLimit = 2000000000LL;  // clocks a CTA waits for its peers' data before giving up
 
 struct __align__(16) SortElem {
     uint64_t key;
@@ -53,6 +61,8 @@ struct ScheduleArgs {
     int n;
     int bt;
     int stage;          // 1: group by digit locally before the remote copy
+    int async_sync;     // 1: per-pass exchanges complete on mbarriers (data driven), 0: cluster barriers
+    uint32_t *status;
 };
 
 #ifdef CASCADE_PHASE_TIMING
@@ -84,11 +94,13 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     SortElem *elems = reinterpret_cast<SortElem *>(smem);
     SortElem *stage = elems + per;
     uint16_t *whist = reinterpret_cast<uint16_t *>(smem + 2 * size_t(per) * sizeof(SortElem));
-    uint16_t *allhist = whist + W * kWhistStride;                      // [kMaxCluster][kBins]
-    uint32_t *base = reinterpret_cast<uint32_t *>(allhist + kMaxCluster * kBins);
+    uint16_t *allhist = whist + W * kWhistStride;                      // [2][kMaxCluster][kBins]
+    uint32_t *base = reinterpret_cast<uint32_t *>(allhist + 2 * kMaxCluster * kBins);
     uint32_t *lbase = base + kBins;
     long long *wtmp = reinterpret_cast<long long *>(lbase + kBins);    // 3 * 32 entries
     Exch *exall = reinterpret_cast<Exch *>(wtmp + 3 * 32);             // [kMaxCluster]
+    uint16_t *minehist = reinterpret_cast<uint16_t *>(exall + kMaxCluster);   // [kBins], 16-byte aligned
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(minehist + kBins);  // hist[2], elem[2]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned lt_mask = (1u << lane) - 1u;
@@ -96,6 +108,10 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     if (crank == 0 && tid == 0) {
         a.counts->n_admitted = 0;
         a.counts->tokens_granted = 0;
+    }
+    if (tid == 0) {
+        for (int i = 0; i < 4; ++i) mbarrier_init(cta_smem_addr(&bars[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
     TICK(66);
@@ -141,9 +157,21 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         if (c < csize) alld |= exall[c].diff;
 
     // ---- LSD radix sort, 8 bits per pass --------------------------------------------------------
+    int ep = 0;          // passes executed so far: selects the mbarrier pair and its phase
+    bool dead = false;   // a bounded wait expired: stop exchanging, keep walking the barriers
     for (int pass = 0; pass < 8; ++pass) {
         const int shift = pass * 8;
         if (((alld >> shift) & 0xffull) == 0) continue;  // same digit in every key: nothing moves
+        if (dead) continue;
+        const int q = ep & 1;
+        const unsigned phase = (unsigned)(ep >> 1) & 1u;
+        uint16_t *hist_in = allhist + q * kMaxCluster * kBins;
+        const unsigned hist_bar = cta_smem_addr(&bars[q]), elem_bar = cta_smem_addr(&bars[2 + q]);
+        if (a.async_sync && tid == 0) {
+            mbarrier_arrive_expect(hist_bar, csize * kBins * (unsigned)sizeof(uint16_t));
+            mbarrier_arrive_expect(elem_bar, (unsigned)(per * sizeof(SortElem)));
+        }
+        ++ep;
 
         TICK(pass * 8 + 0);
         // (a) stable rank of each element among equal digits of its warp's chunk
@@ -187,13 +215,32 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                 whist[w * kWhistStride + tid] = (uint16_t)mine;
                 mine += v[w];
             }
+            if (a.async_sync) {
+                minehist[tid] = (uint16_t)mine;
+            } else {
 #pragma unroll
-            for (int c = 0; c < kMaxCluster; ++c)
-                if (c < csize) cluster.map_shared_rank(allhist, c)[crank * kBins + tid] = (uint16_t)mine;
+                for (int c = 0; c < kMaxCluster; ++c)
+                    if (c < csize) cluster.map_shared_rank(hist_in, c)[crank * kBins + tid] = (uint16_t)mine;
+            }
         }
         TICK(pass * 8 + 2);
-        cluster.sync();  // histograms delivered; every CTA holds its elements in registers
+        if (a.async_sync) {
+            // 16-byte pieces of this CTA's histogram go to every CTA and count on its histogram barrier;
+            // a CTA goes on as soon as the sixteen histograms it needs have landed
+            __syncthreads();
+            for (unsigned op = tid; op < csize * (kBins / 8); op += T) {
+                const unsigned dst = op / (kBins / 8), piece = op % (kBins / 8);
+                const uint4 v = *reinterpret_cast<const uint4 *>(minehist + piece * 8);
+                st_async_16(cluster_addr(cta_smem_addr(hist_in + crank * kBins + piece * 8), dst), v,
+                            cluster_addr(hist_bar, dst));
+            }
+            const bool ok = mbarrier_wait_bounded(hist_bar, phase, kWaitLimit);
+            if (__syncthreads_or(!ok)) dead = true;
+        } else {
+            cluster.sync();  // histograms delivered; every CTA holds its elements in registers
+        }
         TICK(pass * 8 + 3);
+        if (dead) continue;
 
         // (c) per digit: global base of this CTA (high bits) and local base inside this CTA (low 14
         //     bits), both from one packed exclusive scan over the 256 digits
@@ -203,7 +250,7 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
 #pragma unroll
             for (int c = 0; c < kMaxCluster; ++c) {
                 if (c < csize) {
-                    const unsigned h = allhist[c * kBins + tid];
+                    const unsigned h = hist_in[c * kBins + tid];
                     total += h;
                     if (c < crank) before += h;
                 }
@@ -244,8 +291,13 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                 const unsigned long long key = ((unsigned long long)v.y << 32) | v.x;
                 const unsigned d = (unsigned)(key >> shift) & 0xffu;
                 const unsigned pos = base[d] + (i - lbase[d]);
-                SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
-                *reinterpret_cast<uint4 *>(dst) = v;
+                if (a.async_sync) {
+                    st_async_16(cluster_addr(cta_smem_addr(elems + (pos % per)), pos / per), v,
+                                cluster_addr(elem_bar, pos / per));
+                } else {
+                    SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
+                    *reinterpret_cast<uint4 *>(dst) = v;
+                }
             }
         } else {
             // (d) scatter every element straight to its owner
@@ -253,18 +305,31 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
             for (int k = 0; k < K; ++k) {
                 const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
                 const unsigned pos = base[d] + whist[warp * kWhistStride + d] + off[k];
-                SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
-                *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(&e[k]);
+                if (a.async_sync) {
+                    st_async_16(cluster_addr(cta_smem_addr(elems + (pos % per)), pos / per),
+                                *reinterpret_cast<const uint4 *>(&e[k]), cluster_addr(elem_bar, pos / per));
+                } else {
+                    SortElem *dst = cluster.map_shared_rank(elems, pos / per) + (pos % per);
+                    *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(&e[k]);
+                }
             }
         }
         TICK(pass * 8 + 5);
-        cluster.sync();  // all remote stores have landed
+        if (a.async_sync) {
+            // this CTA's slice is complete when all of its T*K elements have arrived
+            const bool ok = mbarrier_wait_bounded(elem_bar, phase, kWaitLimit);
+            if (__syncthreads_or(!ok)) dead = true;
+            if (dead) continue;
+        } else {
+            cluster.sync();  // all remote stores have landed
+        }
         TICK(pass * 8 + 6);
 #pragma unroll
         for (int k = 0; k < K; ++k) e[k] = elems[(warp * K + k) * 32 + lane];
         TICK(pass * 8 + 7);
     }
     TICK(64);
+    if (dead && tid == 0) atomicOr(a.status, CASCADE_ST_ETIMEOUT);
 
     // ---- admission: clamped prefix sums over the sorted elements ---------------------------------
     long long ex[K];
@@ -398,8 +463,8 @@ __global__ void zero_counts_kernel(cascade_sched_counts *c) {
 
 size_t smem_bytes(int T, int K) {
     return 2 * size_t(T) * K * sizeof(SortElem) + size_t(T / 32) * kWhistStride * sizeof(uint16_t) +
-           size_t(kMaxCluster) * kBins * sizeof(uint16_t) + 2 * kBins * sizeof(uint32_t) + 3 * 32 * sizeof(long long) +
-           kMaxCluster * sizeof(Exch) + 16;
+           2 * size_t(kMaxCluster) * kBins * sizeof(uint16_t) + 2 * kBins * sizeof(uint32_t) +
+           3 * 32 * sizeof(long long) + kMaxCluster * sizeof(Exch) + kBins * sizeof(uint16_t) + 4 * 8 + 16;
 }
 
 template <int T, int K, bool kMatch>
@@ -492,6 +557,8 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.n = n;
     a.bt = p.bt;
     a.stage = ctx->sort_stage >= 0 ? ctx->sort_stage : (K >= 4);
+    a.async_sync = ctx->sort_async;
+    a.status = ctx->status_dev;
     cudaError_t e = ctx->sort_match ? launch_t<true>(T, K, a, C, ctx->device, s)
                                     : launch_t<false>(T, K, a, C, ctx->device, s);
     CASCADE_CUDA_TRY(ctx, e);

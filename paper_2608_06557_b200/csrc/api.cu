@@ -47,8 +47,6 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->sort_items = e ? atoi(e) : 0;
     e = getenv("CASCADE_SORT_THREADS");
     ctx->sort_threads = e ? atoi(e) : 0;
-    e = getenv("CASCADE_SORT_MATCH");
-    ctx->sort_match = e ? atoi(e) : 0;
     e = getenv("CASCADE_SORT_STAGE");
     ctx->sort_stage = e ? atoi(e) : -1;  // -1: staged scatter only when a thread holds four or more keys
     e = getenv("CASCADE_SORT_ASYNC");

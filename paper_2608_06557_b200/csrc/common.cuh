@@ -22,7 +22,6 @@ struct cascade_ctx {
     int sort_cluster;            // cluster size override for the ordering kernel (0 = automatic)
     int sort_items;              // keys per thread override (0 = automatic)
     int sort_threads;            // threads per CTA override (0 = automatic)
-    int sort_match;              // 1: rank digits with match.any, 0: with eight ballots
     int sort_stage;              // 1: group elements by digit locally before the remote scatter
     int sort_async;              // 1: per-pass exchanges complete on mbarriers instead of cluster barriers
     int copy_ctas_host;          // copy CTAs per SM when the record pool is pinned host memory
@@ -96,7 +95,7 @@ static inline bool cascade_pick_geometry(const cascade_ctx *ctx, int n, int *T, 
     else if (n <= 16384) { t = 256; c = 16; k = 4; }
     else if (n <= 32768) { t = 512; c = 16; k = 4; }
     else { t = 512; c = 16; k = 8; }
-    if (ctx->sort_threads == 256 || ctx->sort_threads == 512 || ctx->sort_threads == 1024) t = ctx->sort_threads;
+    if (ctx->sort_threads == 256 || ctx->sort_threads == 512) t = ctx->sort_threads;
     if (ctx->sort_items == 1 || ctx->sort_items == 2 || ctx->sort_items == 4 || ctx->sort_items == 8)
         k = ctx->sort_items;
     if (ctx->sort_cluster == 1 || ctx->sort_cluster == 2 || ctx->sort_cluster == 4 || ctx->sort_cluster == 8 ||

@@ -456,9 +456,7 @@ cudaError_t launch_plan_k(int K, const cascade_params &p, const PlanArgs &a, int
         case 1: return launch_plan<T, 1>(p, a, C, s);
         case 2: return launch_plan<T, 2>(p, a, C, s);
         case 4: return launch_plan<T, 4>(p, a, C, s);
-        default:
-            if constexpr (T <= 512) return launch_plan<T, 8>(p, a, C, s);
-            else return cudaErrorInvalidConfiguration;
+        default: return launch_plan<T, 8>(p, a, C, s);
     }
 }
 
@@ -503,9 +501,7 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     a.with_tables = with_tables ? 1 : 0;
     int T, C, K;
     if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, s)
-                  : T == 512 ? launch_plan_k<512>(K, ctx->params, a, C, s)
-                             : launch_plan_k<1024>(K, ctx->params, a, C, s);
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, s) : launch_plan_k<512>(K, ctx->params, a, C, s);
     CASCADE_CUDA_TRY(ctx, e);
     if (with_tables && n > 0) {
         const int grid = ctx->num_sms * 2;
@@ -625,9 +621,7 @@ extern "C" int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_
     cascade_ctx geo = {};
     int T, C, K;
     if (!cascade_pick_geometry(&geo, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_plan_k<256>(K, *p, a, C, s)
-                  : T == 512 ? launch_plan_k<512>(K, *p, a, C, s)
-                             : launch_plan_k<1024>(K, *p, a, C, s);
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, *p, a, C, s) : launch_plan_k<512>(K, *p, a, C, s);
     if (e != cudaSuccess) return CASCADE_ECUDA;
     if (with_tables && n > 0) {
         const int grid = dev->num_sms * 2;

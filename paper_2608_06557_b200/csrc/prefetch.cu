@@ -275,9 +275,7 @@ cudaError_t launch_pf_k(int K, const cascade_params &p, const PrefetchArgs &a, i
         case 1: return launch_pf<T, 1>(p, a, C, s);
         case 2: return launch_pf<T, 2>(p, a, C, s);
         case 4: return launch_pf<T, 4>(p, a, C, s);
-        default:
-            if constexpr (T <= 512) return launch_pf<T, 8>(p, a, C, s);
-            else return cudaErrorInvalidConfiguration;
+        default: return launch_pf<T, 8>(p, a, C, s);
     }
 }
 
@@ -325,9 +323,7 @@ extern "C" int cascade_prefetch_plan(cascade_ctx *ctx, const cascade_reqs *r, co
     a.with_tables = with_tables ? 1 : 0;
     int T, C, K;
     if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_pf_k<256>(K, ctx->params, a, C, s)
-                  : T == 512 ? launch_pf_k<512>(K, ctx->params, a, C, s)
-                             : launch_pf_k<1024>(K, ctx->params, a, C, s);
+    cudaError_t e = T == 256 ? launch_pf_k<256>(K, ctx->params, a, C, s) : launch_pf_k<512>(K, ctx->params, a, C, s);
     CASCADE_CUDA_TRY(ctx, e);
     if (with_tables && n > 0) {
         apply_prefetch_kernel<<<ctx->num_sms * 2, 256, 0, s>>>(a);

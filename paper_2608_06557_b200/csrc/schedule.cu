@@ -82,7 +82,7 @@ __device__ __forceinline__ T seg_incl_scan(T v, int pos, int width) {
     return v;
 }
 
-template <int T, int K, bool kMatch>
+template <int T, int K>
 __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ ScheduleArgs a) {
     constexpr int W = T / 32;          // warps per CTA
     constexpr int per = T * K;         // elements per CTA
@@ -182,16 +182,13 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
 #pragma unroll
         for (int k = 0; k < K; ++k) {
             const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
-            unsigned peers;
-            if (kMatch) {
-                peers = __match_any_sync(kFull, d);
-            } else {
-                peers = kFull;
+            // lanes holding the same digit: eight ballots, one per bit (cheaper than match.any on
+            // high-entropy digits, and its cost does not depend on the data)
+            unsigned peers = kFull;
 #pragma unroll
-                for (int b = 0; b < 8; ++b) {
-                    const unsigned bal = __ballot_sync(kFull, (d >> b) & 1u);
-                    peers &= ((d >> b) & 1u) ? bal : ~bal;
-                }
+            for (int b = 0; b < 8; ++b) {
+                const unsigned bal = __ballot_sync(kFull, (d >> b) & 1u);
+                peers &= ((d >> b) & 1u) ? bal : ~bal;
             }
             const unsigned lower = peers & lt_mask;
             const unsigned pre = myhist[d];
@@ -467,17 +464,17 @@ size_t smem_bytes(int T, int K) {
            3 * 32 * sizeof(long long) + kMaxCluster * sizeof(Exch) + kBins * sizeof(uint16_t) + 4 * 8 + 16;
 }
 
-template <int T, int K, bool kMatch>
+template <int T, int K>
 cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, cudaStream_t stream) {
     static bool configured_dev[64] = {};
     bool unknown = false;
     bool &configured = (device >= 0 && device < 64) ? configured_dev[device] : unknown;
     const size_t smem = smem_bytes(T, K);
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(schedule_kernel<T, K, kMatch>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(schedule_kernel<T, K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(schedule_kernel<T, K, kMatch>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        e = cudaFuncSetAttribute(schedule_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -493,27 +490,16 @@ cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, cudaStre
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, schedule_kernel<T, K, kMatch>, a);
+    return cudaLaunchKernelEx(&cfg, schedule_kernel<T, K>, a);
 }
 
-template <int T, bool kMatch>
+template <int T>
 cudaError_t launch_k(int K, const ScheduleArgs &a, int C, int device, cudaStream_t s) {
     switch (K) {
-        case 1: return launch<T, 1, kMatch>(a, C, device, s);
-        case 2: return launch<T, 2, kMatch>(a, C, device, s);
-        case 4: return launch<T, 4, kMatch>(a, C, device, s);
-        default:
-            if constexpr (T <= 512) return launch<T, 8, kMatch>(a, C, device, s);
-            else return cudaErrorInvalidConfiguration;
-    }
-}
-
-template <bool kMatch>
-cudaError_t launch_t(int T, int K, const ScheduleArgs &a, int C, int device, cudaStream_t s) {
-    switch (T) {
-        case 256: return launch_k<256, kMatch>(K, a, C, device, s);
-        case 512: return launch_k<512, kMatch>(K, a, C, device, s);
-        default: return launch_k<1024, kMatch>(K, a, C, device, s);
+        case 1: return launch<T, 1>(a, C, device, s);
+        case 2: return launch<T, 2>(a, C, device, s);
+        case 4: return launch<T, 4>(a, C, device, s);
+        default: return launch<T, 8>(a, C, device, s);
     }
 }
 
@@ -559,8 +545,7 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.stage = ctx->sort_stage >= 0 ? ctx->sort_stage : (K >= 4);
     a.async_sync = ctx->sort_async;
     a.status = ctx->status_dev;
-    cudaError_t e = ctx->sort_match ? launch_t<true>(T, K, a, C, ctx->device, s)
-                                    : launch_t<false>(T, K, a, C, ctx->device, s);
+    cudaError_t e = T == 256 ? launch_k<256>(K, a, C, ctx->device, s) : launch_k<512>(K, a, C, ctx->device, s);
     CASCADE_CUDA_TRY(ctx, e);
     return CASCADE_OK;
 }

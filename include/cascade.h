@@ -319,6 +319,23 @@ int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, const void 
                      int64_t dst_blocks, int dst_is_device, const int32_t *src_ids, const int32_t *dst_ids,
                      const int32_t *n_copies_dev, int n_copies_max, void *stream);
 
+/*
+ * Evict and restore in one call, with the host link used in both directions at once.  Same result as
+ * cascade_kv_evict on the evict list followed by cascade_kv_restore on the restore list (the order the
+ * tier plan requires): a restore whose HBM block is also evicted by this call waits, block by block,
+ * until that block has been read out.  Both lists as in the two calls above; the host pool must be
+ * pinned, mapped host memory (or device memory).
+ *   scratch   caller-owned device array of n_evict_max + n_restore_max int32 (contents irrelevant)
+ * The grid is one CTA per SM; the per-block waits assume those CTAs become resident (true unless
+ * the GPU is saturated by other long-running kernels) and are clock-bounded: on expiry
+ * CASCADE_ST_ETIMEOUT is set and that block is not written.
+ */
+int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, void *host_pool,
+                    int64_t host_blocks, const int32_t *evict_src, const int32_t *evict_dst,
+                    const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,
+                    const int32_t *restore_dst, const int32_t *n_restore_dev, int n_restore_max, int32_t *scratch,
+                    void *stream);
+
 /* Waits for `stream`, copies the status word to *host_out and, if clear != 0, resets it. */
 int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream);
 

@@ -23,7 +23,7 @@ ACT_NONE, ACT_RETAIN, ACT_EVICT, ACT_DROP = 0, 1, 2, 3
 
 EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_budget", "cascade_schedule",
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
-           "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan")
+           "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan", "cascade_kv_move")
 
 
 class Params(C.Structure):
@@ -98,6 +98,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_kv_restore.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, C.c_int, vp, vp, vp, C.c_int, vp]
     lib.cascade_kv_evict.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, C.c_int, vp, vp, vp, C.c_int, vp]
     lib.cascade_status.argtypes = [vp, C.POINTER(Status), C.c_int, vp]
+    lib.cascade_kv_move.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int,
+                                    vp, vp]
     lib.cascade_tier_plan_noalloc.argtypes = [C.POINTER(Params), C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64,
                                               C.POINTER(Pools), C.POINTER(Plan), vp, vp]
     for name in EXPORTS:
@@ -220,6 +222,13 @@ class Context:
         _check(_lib.cascade_kv_evict(self._h, C.byref(layout), _p(hbm_pool), _p(dst_pool), dst_blocks,
                                      int(dst_is_device), _p(src_ids), _p(dst_ids), _p(n_copies_dev), n_copies_max,
                                      _stream(stream)), "cascade_kv_evict")
+
+    def kv_move(self, layout: KvLayout, hbm_pool, host_pool, host_blocks, evict_src, evict_dst, n_evict_dev,
+                n_evict_max, restore_src, restore_dst, n_restore_dev, n_restore_max, scratch, stream=None):
+        _check(_lib.cascade_kv_move(self._h, C.byref(layout), _p(hbm_pool), _p(host_pool), host_blocks,
+                                    _p(evict_src), _p(evict_dst), _p(n_evict_dev), n_evict_max, _p(restore_src),
+                                    _p(restore_dst), _p(n_restore_dev), n_restore_max, _p(scratch),
+                                    _stream(stream)), "cascade_kv_move")
 
     def status(self, clear: bool = True, stream=None) -> tuple[int, int]:
         st = Status()

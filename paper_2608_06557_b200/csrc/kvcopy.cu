@@ -204,6 +204,152 @@ __global__ void __launch_bounds__(32) kv_copy_bulk_kernel(const __grid_constant_
     if (st) atomicOr(a.status, st);
 }
 
+// ---- fused evict + restore ("move"): both directions of the host link at once ----------------------
+// The evict list and the restore list of one iteration in ONE ring kernel.  Evicted blocks travel
+// device -> host while restored blocks travel host -> device, so the link is used in both directions
+// at the same time.  A restore may target an HBM block that the same call evicts (the tier plan hands
+// freed blocks out again at once): its store into HBM waits until every piece of that block has been
+// read by the evict side.  Even CTAs work on the evict list (walking it backwards, because the blocks
+// freed last are handed out first), odd CTAs on the restore list; only restore CTAs ever wait, and
+// only for evict CTAs, which never wait for anybody, so with all CTAs resident (one per SM at most)
+// the waits cannot deadlock.  They are clock-bounded all the same (CASCADE_ST_ETIMEOUT, that store
+// is skipped).
+struct MoveArgs {
+    char *paged;
+    char *record;
+    const int32_t *evict_src, *evict_dst, *restore_src, *restore_dst;
+    const int32_t *n_evict_dev, *n_restore_dev;
+    int32_t *dep;    // per restore: index into the evict list of the entry that frees its HBM block, or -1
+    int32_t *done;   // per evict entry: pieces of the block already read out of HBM
+    uint32_t *status;
+    long long paged_blocks, record_blocks;
+    long long chunk_bytes, chunk_stride, block_stride;
+    int n_chunks;
+    int n_evict_max, n_restore_max;
+    int pieces_per_chunk;
+};
+
+__device__ __forceinline__ int clamp_count(const int32_t *dev, int maxv) {
+    if (!dev) return maxv;
+    const int c = *dev;
+    return c < 0 ? 0 : (c < maxv ? c : maxv);
+}
+
+__global__ void __launch_bounds__(256) kv_move_prepare_kernel(const __grid_constant__ MoveArgs a) {
+    const int ne = clamp_count(a.n_evict_dev, a.n_evict_max), nr = clamp_count(a.n_restore_dev, a.n_restore_max);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int stride = gridDim.x * blockDim.x;
+    for (int j = i; j < ne; j += stride) a.done[j] = 0;
+    for (int r = i; r < nr; r += stride) {
+        const int32_t g = a.restore_dst[r];
+        int dep = -1;
+        for (int j = 0; j < ne; ++j)
+            if (a.evict_src[j] == g) dep = j;
+        a.dep[r] = dep;
+    }
+}
+
+__global__ void __launch_bounds__(32) kv_move_kernel(const __grid_constant__ MoveArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long bars[kStages];
+    if (threadIdx.x != 0) return;
+    for (int s = 0; s < kStages; ++s) mbar_init(smem_addr(&bars[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+    const int ne = clamp_count(a.n_evict_dev, a.n_evict_max), nr = clamp_count(a.n_restore_dev, a.n_restore_max);
+    const int ppc = a.pieces_per_chunk;
+    const long long per_block = (long long)a.n_chunks * ppc;
+    const long long bb = (long long)a.n_chunks * a.chunk_bytes;
+    uint32_t st = 0;
+    // even CTAs evict, odd CTAs restore; a single-CTA grid does the evict list first, then the restores
+    const bool split = gridDim.x > 1;
+    const bool evict_role = !split || (blockIdx.x & 1) == 0;
+    const long long evict_items = (split && !evict_role) ? 0 : (long long)ne * per_block;
+    const long long items = evict_items + ((split && evict_role) ? 0 : (long long)nr * per_block);
+    const long long step = split ? (evict_role ? (gridDim.x + 1) / 2 : gridDim.x / 2) : 1;
+
+    long long next = split ? blockIdx.x / 2 : 0;
+    char *dst_of[kStages];
+    unsigned bytes_of[kStages];
+    int evict_of[kStages];  // evict-list index to signal after the load (evict piece), -1 otherwise
+    int wait_of[kStages];   // evict-list index to wait for before the store (restore piece), -1 if none
+    long long issued = 0, stored = 0;
+    auto issue_next = [&]() -> bool {
+        while (next < items) {
+            const long long it = next;
+            next += step;
+            const bool is_evict = it < evict_items;
+            const long long local = is_evict ? it : it - evict_items;
+            long long i = local / per_block;
+            const int rem = (int)(local - i * per_block);
+            if (is_evict) i = ne - 1 - i;  // blocks freed last are reused first: read them out first
+            const int c = rem / ppc, pc = rem - c * ppc;
+            const long long rec_id = is_evict ? a.evict_dst[i] : a.restore_src[i];
+            const long long pg_id = is_evict ? a.evict_src[i] : a.restore_dst[i];
+            if (rec_id < 0 || rec_id >= a.record_blocks || pg_id < 0 || pg_id >= a.paged_blocks) {
+                st |= CASCADE_ST_EBOUNDS;
+                // a skipped evict piece still counts as read, or a restore into that block would wait for nothing
+                if (is_evict) atomicAdd(&a.done[i], 1);
+                continue;
+            }
+            const long long off = (long long)pc * kBulkPiece;
+            const long long left = a.chunk_bytes - off;
+            const unsigned bytes = (unsigned)(left < kBulkPiece ? left : kBulkPiece);
+            char *rec = a.record + rec_id * bb + (long long)c * a.chunk_bytes + off;
+            char *pg = a.paged + (long long)c * a.chunk_stride + pg_id * a.block_stride + off;
+            const int slot = (int)(issued % kStages);
+            const unsigned bar = smem_addr(&bars[slot]);
+            mbar_expect_tx(bar, bytes);
+            bulk_load(smem_addr(ring + (size_t)slot * kBulkPiece), is_evict ? pg : rec, bytes, bar);
+            dst_of[slot] = is_evict ? rec : pg;
+            bytes_of[slot] = bytes;
+            evict_of[slot] = is_evict ? (int)i : -1;
+            wait_of[slot] = is_evict ? -1 : a.dep[i];
+            ++issued;
+            return true;
+        }
+        return false;
+    };
+    for (int k = 0; k < kAhead; ++k)
+        if (!issue_next()) break;
+    while (stored < issued) {
+        const int slot = (int)(stored % kStages);
+        const unsigned parity = (unsigned)((stored / kStages) & 1);
+        const unsigned bar = smem_addr(&bars[slot]);
+        long long t0 = clock64();
+        bool arrived = mbar_try_wait(bar, parity);
+        while (!arrived && clock64() - t0 < kWaitCycles) arrived = mbar_try_wait(bar, parity);
+        if (!arrived) {
+            st |= CASCADE_ST_ETIMEOUT;
+            break;
+        }
+        bool skip = false;
+        if (evict_of[slot] >= 0) {
+            atomicAdd(&a.done[evict_of[slot]], 1);  // this piece of the block has left HBM
+        } else if (wait_of[slot] >= 0) {
+            // the HBM block is being evicted by this same call: write only after it has been read out
+            const volatile int32_t *flag = a.done + wait_of[slot];
+            t0 = clock64();
+            if (st & CASCADE_ST_ETIMEOUT) skip = true;  // one expired wait is enough: do not queue up more
+            while (!skip && *flag < (int)per_block) {
+                if (clock64() - t0 > kWaitCycles) {
+                    st |= CASCADE_ST_ETIMEOUT;
+                    skip = true;
+                    break;
+                }
+            }
+            __threadfence();
+        }
+        if (!skip) bulk_store(dst_of[slot], smem_addr(ring + (size_t)slot * kBulkPiece), bytes_of[slot]);
+        ++stored;
+        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        issue_next();
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (st) atomicOr(a.status, st);
+}
+
 int check_layout(const cascade_kv_layout *l, const void *paged, const void *record, long long record_blocks) {
     if (!l || !paged || !record) return CASCADE_EINVAL;
     if (l->n_blocks < 0 || record_blocks < 0 || l->n_chunks < 1 || l->chunk_bytes < 16) return CASCADE_EINVAL;
@@ -283,4 +429,58 @@ extern "C" int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, 
                                 const int32_t *n_copies_dev, int n_copies_max, void *stream) {
     return launch_copy<false>(ctx, hbm, (char *)const_cast<void *>(hbm_pool), (char *)dst_pool, dst_blocks,
                               dst_is_device, src_ids, dst_ids, n_copies_dev, n_copies_max, (cudaStream_t)stream);
+}
+
+extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, void *host_pool,
+                               int64_t host_blocks, const int32_t *evict_src, const int32_t *evict_dst,
+                               const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,
+                               const int32_t *restore_dst, const int32_t *n_restore_dev, int n_restore_max,
+                               int32_t *scratch, void *stream) {
+    if (!ctx || n_evict_max < 0 || n_restore_max < 0) return CASCADE_EINVAL;
+    if (n_evict_max == 0 && n_restore_max == 0) return CASCADE_OK;
+    int rc = check_layout(hbm, hbm_pool, host_pool, host_blocks);
+    if (rc != CASCADE_OK) return rc;
+    if (!scratch || (n_evict_max > 0 && (!evict_src || !evict_dst)) || (n_restore_max > 0 && (!restore_src || !restore_dst)))
+        return CASCADE_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    MoveArgs a;
+    a.paged = (char *)hbm_pool;
+    a.record = (char *)host_pool;
+    a.evict_src = evict_src;
+    a.evict_dst = evict_dst;
+    a.restore_src = restore_src;
+    a.restore_dst = restore_dst;
+    a.n_evict_dev = n_evict_dev;
+    a.n_restore_dev = n_restore_dev;
+    a.dep = scratch;
+    a.done = scratch + n_restore_max;
+    a.status = ctx->status_dev;
+    a.paged_blocks = hbm->n_blocks;
+    a.record_blocks = host_blocks;
+    a.chunk_bytes = hbm->chunk_bytes;
+    a.chunk_stride = hbm->chunk_stride;
+    a.block_stride = hbm->block_stride;
+    a.n_chunks = hbm->n_chunks;
+    a.n_evict_max = n_evict_max;
+    a.n_restore_max = n_restore_max;
+    a.pieces_per_chunk = (int)((hbm->chunk_bytes + kBulkPiece - 1) / kBulkPiece);
+    const int most = n_evict_max > n_restore_max ? n_evict_max : n_restore_max;
+    int pgrid = (most + 255) / 256;
+    if (pgrid > ctx->num_sms * 4) pgrid = ctx->num_sms * 4;
+    kv_move_prepare_kernel<<<pgrid, 256, 0, s>>>(a);
+    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    const long long items = ((long long)n_evict_max + n_restore_max) * hbm->n_chunks * a.pieces_per_chunk;
+    long long grid = ctx->num_sms;  // one resident CTA per SM: every CTA that can be waited for is running
+    if (grid > items) grid = items;
+    const size_t smem = (size_t)kStages * kBulkPiece;
+    static bool configured_dev[64] = {};
+    bool unknown = false;
+    bool &configured = (ctx->device >= 0 && ctx->device < 64) ? configured_dev[ctx->device] : unknown;
+    if (!configured) {
+        CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured = true;
+    }
+    kv_move_kernel<<<(unsigned)grid, 32, smem, s>>>(a);
+    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    return CASCADE_OK;
 }

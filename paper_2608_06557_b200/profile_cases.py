@@ -2,6 +2,7 @@
 
     python -m paper_2608_06557_b200.profile_cases copy-hbm   [blocks]   # staging buffer <-> paged pool (HBM bound)
     python -m paper_2608_06557_b200.profile_cases copy-host  [blocks]   # pinned host pool <-> paged pool (host link)
+    python -m paper_2608_06557_b200.profile_cases move       [blocks]   # fused evict + restore, both link directions
     python -m paper_2608_06557_b200.profile_cases schedule   [requests] # budget + schedule + tier plan, plan-only
 
 Each case holds at most a few GB on the device, moves more than the 126 MB L2 per launch and
@@ -55,6 +56,30 @@ def copy_case(record_on_device: bool, n: int):
     print("status", ctx.status())
 
 
+def move_case(n: int):
+    """n blocks evicted and n restored by one cascade_kv_move; half of the restores reuse evicted blocks."""
+    import numpy as np
+    n_chunks, chunk_bytes = 64, 32 * 1024
+    bb = n_chunks * chunk_bytes
+    n_hbm, n_rec = 3 * n + 64, 3 * n + 64
+    lay = wl.kv_layout(n_hbm, n_chunks, chunk_bytes)
+    hbm = torch.empty(n_hbm * bb, dtype=torch.uint8, device="cuda").fill_(1)
+    rec = torch.empty(n_rec * bb, dtype=torch.uint8, pin_memory=True).fill_(2)
+    ctx = cs.Context(wl.default_params(), 16, 0)
+    layout = cs.make_layout(lay)
+    rng = np.random.default_rng(3)
+    hp, op = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_rec).astype(np.int32)
+    es, ed, rs = hp[:n], op[:n], op[n:2 * n]
+    rd = np.concatenate([es[::-1][: n // 2], hp[n:2 * n - n // 2]]).astype(np.int32)
+    t = [torch.from_numpy(np.ascontiguousarray(x)).cuda() for x in (es, ed, rs, rd)]
+    scratch = torch.empty(2 * n, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    ts = _timed(lambda: ctx.kv_move(layout, hbm, rec, n_rec, t[0], t[1], None, n, t[2], t[3], None, n, scratch))
+    print(f"move: {n} evicted + {n} restored blocks x {bb} B, us per call {[round(x, 1) for x in ts]}, "
+          f"best {2 * n * bb / min(ts) / 1e3:.1f} GB/s over the link (both directions)")
+    print("status", ctx.status())
+
+
 def schedule_case(n: int):
     sw = wl.SchedulerSweep(n, seed=0)
     inst = Instance(sw.workload(), alloc_pools=False)
@@ -70,6 +95,8 @@ def main(argv):
         copy_case(True, int(argv[2]) if len(argv) > 2 else 256)
     elif case == "copy-host":
         copy_case(False, int(argv[2]) if len(argv) > 2 else 256)
+    elif case == "move":
+        move_case(int(argv[2]) if len(argv) > 2 else 128)
     elif case == "schedule":
         schedule_case(int(argv[2]) if len(argv) > 2 else 16384)
     else:

@@ -151,10 +151,21 @@ class Instance:
         c.kv_restore(self.layout, self.hbm_pool, rec, self.host_blocks, record_is_device, self.restore_src,
                      self.restore_dst, n_restore, self.restore_cap, stream)
 
-    def run_iteration(self, stream=None):
+    def run_move(self, stream=None):
+        """evict + restore as one call that uses both directions of the host link at once."""
+        if not hasattr(self, "move_scratch"):
+            self.move_scratch = torch.empty(self.evict_cap + self.restore_cap, dtype=torch.int32, device=self.device)
+        self.ctx.kv_move(self.layout, self.hbm_pool, self.host_pool, self.host_blocks, self.evict_src, self.evict_dst,
+                         self.plan_counts[1:2], self.evict_cap, self.restore_src, self.restore_dst,
+                         self.plan_counts[0:1], self.restore_cap, self.move_scratch, stream)
+
+    def run_iteration(self, stream=None, fused_move: bool = False):
         self.run_schedule(stream)
         if self.with_tables and self.hbm_pool is not None:
-            self.run_copies(stream)
+            if fused_move:
+                self.run_move(stream)
+            else:
+                self.run_copies(stream)
 
     # -- outputs --------------------------------------------------------------------------------
     def fetch(self) -> dict:

@@ -160,3 +160,67 @@ def test_full_iteration_tiny_with_copies(seed, ttft_scale):
     assert np.array_equal(inst.host_pool.cpu().numpy(), host_np)
     if ttft_scale > 1:
         assert plan["counts"]["n_restore"] > 0
+
+
+@pytest.mark.parametrize("shape", [(64, 48, 4, 4096), (40, 40, 3, 208), (48, 48, 64, 32768), (30, 30, 2, 32 * 1024 + 64)])
+def test_fused_move_equals_evict_then_restore(shape):
+    """One call, both directions at once; half of the restores land in blocks the same call evicts."""
+    n_hbm, n_host, n_chunks, cb = shape
+    rig = CopyRig(n_hbm, n_host, n_chunks, cb)
+    torch = rig.torch
+    rng = np.random.default_rng(n_hbm)
+    ne, nr = n_hbm // 3, n_host // 3
+    hperm, operm = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_host).astype(np.int32)
+    evict_src, evict_dst = hperm[:ne], operm[:ne]
+    restore_src = operm[ne:ne + nr]
+    # restore destinations: the blocks evicted LAST (as the plan's stack hands them out), then untouched blocks
+    reuse = evict_src[::-1][: nr // 2]
+    restore_dst = np.concatenate([reuse, hperm[ne:ne + nr - len(reuse)]]).astype(np.int32)
+    ref_hbm, ref_host = rig.hbm_np.copy(), rig.host_np.copy()
+    assert oracle.kv_evict(ref_hbm, rig.lay, ref_host, n_host, evict_src, evict_dst) == 0
+    assert oracle.kv_restore(ref_hbm, rig.lay, ref_host, n_host, restore_src, restore_dst) == 0
+    cap_e, cap_r = ne + 3, nr + 2
+    pad = lambda a, cap: rig.ids(np.concatenate([a, np.full(cap - len(a), 10**6, np.int32)]))
+    counts = torch.tensor([nr, ne], dtype=torch.int32, device="cuda")
+    scratch = torch.empty(cap_e + cap_r, dtype=torch.int32, device="cuda")
+    for rep in range(2):                              # twice: the scratch is reused as it was left
+        rig.hbm.copy_(torch.from_numpy(rig.hbm_np))
+        rig.host.copy_(torch.from_numpy(rig.host_np))
+        rig.ctx.kv_move(rig.layout, rig.hbm, rig.host, n_host, pad(evict_src, cap_e), pad(evict_dst, cap_e),
+                        counts[1:2], cap_e, pad(restore_src, cap_r), pad(restore_dst, cap_r), counts[0:1], cap_r,
+                        scratch)
+        torch.cuda.synchronize()
+        assert np.array_equal(rig.hbm.cpu().numpy(), ref_hbm), rep
+        assert np.array_equal(rig.host.cpu().numpy(), ref_host), rep
+    assert rig.guards_intact() and rig.ctx.status()[0] == 0
+    # one list empty, and a bad id on each side
+    rig.ctx.kv_move(rig.layout, rig.hbm, rig.host, n_host, None, None, None, 0, pad(restore_src, cap_r),
+                    pad(restore_dst, cap_r), counts[0:1], cap_r, scratch)
+    bad_e = evict_src.copy()
+    bad_e[0] = -5
+    rig.ctx.kv_move(rig.layout, rig.hbm, rig.host, n_host, pad(bad_e, cap_e), pad(evict_dst, cap_e), counts[1:2],
+                    cap_e, None, None, None, 0, scratch)
+    torch.cuda.synchronize()
+    assert rig.ctx.status()[0] == 1 and rig.guards_intact()
+
+
+@pytest.mark.parametrize("seed", [0, 3, 5])
+def test_full_iteration_with_fused_move(seed):
+    torch, cs, Instance = _gpu()
+    w = wl.config_tiny(seed, hbm_free_target=60)
+    w.params["ttft_ns"] = [20 * t for t in w.params["ttft_ns"]]
+    ref = oracle_iteration(w)
+    bb = w.block_bytes
+    hbm_np = wl.pool_bytes(3, w.layout["n_blocks"] * bb).copy()
+    host_np = wl.pool_bytes(4, w.host_blocks * bb).copy()
+    inst = Instance(w)
+    inst.hbm_pool.copy_(torch.from_numpy(hbm_np))
+    inst.host_pool.copy_(torch.from_numpy(host_np))
+    inst.run_iteration(fused_move=True)
+    got = inst.fetch()
+    plan = ref["plan"]
+    assert oracle.kv_evict(hbm_np, w.layout, host_np, w.host_blocks, plan["evict_src"], plan["evict_dst"]) == 0
+    assert oracle.kv_restore(hbm_np, w.layout, host_np, w.host_blocks, plan["restore_src"], plan["restore_dst"]) == 0
+    assert got["plan_counts"] == plan["counts"] and got["status"] == ref["status"]
+    assert np.array_equal(inst.hbm_pool.cpu().numpy(), hbm_np)
+    assert np.array_equal(inst.host_pool.cpu().numpy(), host_np)

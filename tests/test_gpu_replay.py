@@ -49,13 +49,14 @@ def verify_by_content(torch, hbm, host, lay, n_host, hbm_content, host_content):
         assert torch.equal(got, oc[base:base + len(got), None] * P1 + j[None, :] * P2), base
 
 
-@pytest.mark.parametrize("variant", ["pressure", "restore_heavy"])
+@pytest.mark.parametrize("variant", ["pressure", "restore_heavy", "pressure_fused_move"])
 def test_replay_iterations_match_oracle_and_bytes_end_up_where_they_should(variant):
     import torch
     from paper_2608_06557_b200 import cascade as cs
     from paper_2608_06557_b200.runner import Instance
 
-    if variant == "pressure":
+    fused = variant.endswith("fused_move")
+    if variant.startswith("pressure"):
         tr = wl.config_llama70b_trace(1, n=1024, hbm_bytes=12 * 10**9, host_bytes=8 * 10**9, hbm_occupancy=0.7,
                                       rate_per_s=60.0)
         iters = 200
@@ -81,7 +82,7 @@ def test_replay_iterations_match_oracle_and_bytes_end_up_where_they_should(varia
         ref = oracle_iteration(w)
         plan, pools = ref["plan"], ref["pools"]
         inst = Instance(w, ctx=ctx, hbm_pool=hbm, host_pool=host, alloc_pools=False)
-        inst.run_iteration()
+        inst.run_iteration(fused_move=fused)
         got = inst.fetch()
         for k in ("budget", "key", "order", "grant"):
             assert np.array_equal(got[k], ref[k]), (it, k)
@@ -104,6 +105,6 @@ def test_replay_iterations_match_oracle_and_bytes_end_up_where_they_should(varia
                            host_free_count=pools.host_free_count))
         del inst
     assert tot["n_restore"] > 200
-    if variant == "pressure":
+    if variant.startswith("pressure"):
         assert tot["n_evict"] > 0 and tot["n_drop_blocks"] > 0 and tot["n_unadmitted"] > 0
     verify_by_content(torch, hbm, host, lay, tr.host_blocks, hbm_content, host_content)

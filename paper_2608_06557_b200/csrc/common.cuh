@@ -28,6 +28,7 @@ struct cascade_ctx {
     int copy_ctas_dev;           // copy CTAs per SM when the record pool is device memory
     int copy_bulk_host;          // >0: TMA bulk-copy ring (that many CTAs per SM) for the pinned-host path
     int copy_bulk_dev;           // >0: TMA bulk-copy ring for the device-staging path
+    int move_ctas;               // >0: CTAs of the fused evict+restore kernel (at most one per SM)
 };
 
 // plan_scalars layout

@@ -471,6 +471,7 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     CASCADE_CUDA_TRY(ctx, cudaGetLastError());
     const long long items = ((long long)n_evict_max + n_restore_max) * hbm->n_chunks * a.pieces_per_chunk;
     long long grid = ctx->num_sms;  // one resident CTA per SM: every CTA that can be waited for is running
+    if (ctx->move_ctas > 0 && ctx->move_ctas < grid) grid = ctx->move_ctas;
     if (grid > items) grid = items;
     const size_t smem = (size_t)kStages * kBulkPiece;
     static bool configured_dev[64] = {};

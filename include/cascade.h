@@ -90,13 +90,19 @@ typedef struct cascade_params {
     int64_t ttft_ns[CASCADE_MAX_CLASSES]; /* class TTFT targets                                */
     int64_t tpot_ns[CASCADE_MAX_CLASSES]; /* class TPOT targets; 0 disables the decode term    */
     int32_t policy;        /* CASCADE_POLICY_*: what the queue is ordered by (0 = the paper's method)     */
-    int32_t reserved;      /* must be 0                                                                   */
+    int32_t plan_first;    /* 0 | 1: plan-first admission, see below                                       */
 } cascade_params;
 
 /* Ordering policies.  BUDGET is the method: least remaining budget first with the Tier-1 / Tier-2 split.
  * The others are the comparison policies of the paper's evaluation, one queue, same key packing:
  * FCFS orders by arrival time, EDF by the TTFT deadline arrival + ttft_ns[cls], SJF by the tokens left
  * to prefill.  budget_out is the latency budget under every policy (the tier plan needs it). */
+/* plan_first = 1: every request's own restore choice (the Eq. 7 bounds and the restore-vs-recompute
+ * comparison of cascade_tier_plan, taken from its budget alone) is made before admission, and admission
+ * offers it exactly the tokens that choice leaves to compute, prompt - (n0 + x1)*bt, instead of assuming
+ * the whole matched prefix is reused; a request that chooses a deep-tier fetch asks for nothing this
+ * iteration.  Every admitted request then runs exactly its grant.  cascade_budget stores the offers in the
+ * context, so cascade_schedule must follow cascade_budget on the same context and request arrays. */
 #define CASCADE_POLICY_BUDGET 0
 #define CASCADE_POLICY_FCFS 1
 #define CASCADE_POLICY_EDF 2

@@ -35,7 +35,7 @@ class OrcParams(C.Structure):
         ("c_dseq_q20", C.c_int64), ("c_dkv_q20", C.c_int64),
         ("delta_ns", C.c_int64 * 3), ("blk_ns", C.c_int64 * 3),
         ("ttft_ns", C.c_int64 * MAX_CLASSES), ("tpot_ns", C.c_int64 * MAX_CLASSES),
-        ("policy", C.c_int32), ("reserved", C.c_int32),
+        ("policy", C.c_int32), ("plan_first", C.c_int32),
     ]
 
 
@@ -97,6 +97,7 @@ def make_params(d: dict) -> OrcParams:
     for i, v in enumerate(d["tpot_ns"]):
         p.tpot_ns[i] = int(v)
     p.policy = int(d.get("policy", 0))
+    p.plan_first = int(d.get("plan_first", 0))
     return p
 
 
@@ -152,8 +153,9 @@ def latency_regimes(p: OrcParams, reqs: dict, D_act: int, K_act: int):
     return out, int(st)
 
 
-def schedule(p: OrcParams, reqs: dict, key: np.ndarray, D_act: int):
-    """Steps S1-S3.  Returns (order uint32[n], grant int32[n], counts dict, status bits)."""
+def schedule(p: OrcParams, reqs: dict, key: np.ndarray, D_act: int, budget_: np.ndarray | None = None, K_act: int = 0):
+    """Steps S1-S3.  Returns (order uint32[n], grant int32[n], counts dict, status bits).
+    ``budget_`` and ``K_act`` are needed only when the parameters select plan-first admission."""
     n = len(reqs["prompt"])
     order = np.empty(n, np.uint32)
     grant = np.empty(n, np.int32)
@@ -162,7 +164,8 @@ def schedule(p: OrcParams, reqs: dict, key: np.ndarray, D_act: int):
     key = _arr(key, np.uint64)
     st = lib().orc_schedule(C.byref(p), C.c_int(n), _ptr(key, C.c_uint64), _ptr(a["prompt"], C.c_int32),
                             _ptr(a["n0"], C.c_int32), _ptr(a["n1"], C.c_int32), _ptr(a["n2"], C.c_int32),
-                            C.c_int32(D_act), _ptr(order, C.c_uint32), _ptr(grant, C.c_int32), C.byref(cnt))
+                            C.c_int32(D_act), _ptr(order, C.c_uint32), _ptr(grant, C.c_int32), C.byref(cnt),
+                            _ptr(None if budget_ is None else _arr(budget_, np.int64), C.c_int64), C.c_int64(K_act))
     counts = {k: int(getattr(cnt, k)) for k, _ in OrcSchedCounts._fields_}
     return order, grant, counts, int(st)
 

@@ -88,6 +88,31 @@ int64_t plan_cost_q20(const orc_params *p, Load act, int64_t P, int64_t n0, int6
     return (transfer << 20) + comp_q(p, tok_q(p, act), P, (n0 + x1 + x2) * p->bt);
 }
 
+/* P1 + P2: the Eq. 7 bounds (host first, deep tier from what is left and only behind a fully restored
+ * host segment), then the endpoint candidate with the smallest predicted completion time; ties restore more. */
+void choose_restore(const orc_params *p, Load act, int64_t P, int64_t n0, int64_t n1, int64_t n2, int64_t budget,
+                    int64_t *x1, int64_t *x2) {
+    const int64_t rem = std::max<int64_t>(0, budget);
+    const int64_t x1max = max_restorable(p, 1, rem, n1);
+    int64_t x2max = 0;
+    if (x1max == n1 && n2 > 0) {
+        const int64_t rem2 = rem - restore_time(p, 1, n1);
+        x2max = max_restorable(p, 2, rem2, n2);
+    }
+    int64_t bx1 = 0, bx2 = 0;
+    int64_t bF = plan_cost_q20(p, act, P, n0, 0, 0);
+    if (x1max > 0) {
+        const int64_t F = plan_cost_q20(p, act, P, n0, x1max, 0);
+        if (F <= bF) { bF = F; bx1 = x1max; bx2 = 0; }
+    }
+    if (x2max > 0) {
+        const int64_t F = plan_cost_q20(p, act, P, n0, n1, x2max);
+        if (F <= bF) { bF = F; bx1 = n1; bx2 = x2max; }
+    }
+    *x1 = bx1;
+    *x2 = bx2;
+}
+
 }  // namespace
 
 extern "C" {
@@ -189,7 +214,7 @@ uint32_t orc_latency_regimes(const orc_params *p, int n, const int32_t *prompt, 
 
 uint32_t orc_schedule(const orc_params *p, int n, const uint64_t *key, const int32_t *prompt, const int32_t *n0,
                       const int32_t *n1, const int32_t *n2, int32_t D_act, uint32_t *order_out, int32_t *grant_out,
-                      orc_sched_counts *counts) {
+                      orc_sched_counts *counts, const int64_t *budget, int64_t K_act) {
     /* S1: ascending by key; equal keys keep slot order */
     std::vector<uint32_t> order(n);
     std::iota(order.begin(), order.end(), 0u);
@@ -198,10 +223,17 @@ uint32_t orc_schedule(const orc_params *p, int n, const uint64_t *key, const int
     /* S2: tokens each request would compute if its whole matched prefix is reused */
     std::vector<int64_t> want(n);
     for (int r = 0; r < n; ++r) {
-        if (request_valid(p, prompt[r], n0[r], n1[r], n2[r]))
-            want[r] = int64_t(prompt[r]) - int64_t(n0[r] + n1[r] + n2[r]) * p->bt;
-        else
+        if (!request_valid(p, prompt[r], n0[r], n1[r], n2[r])) {
             want[r] = 0;
+        } else if (p->plan_first) {
+            /* the request's own restore choice decides what is left to compute; a deep fetch is staged
+             * first, so such a request asks for nothing this iteration */
+            int64_t x1, x2;
+            choose_restore(p, load_act(D_act, K_act), prompt[r], n0[r], n1[r], n2[r], budget[r], &x1, &x2);
+            want[r] = x2 > 0 ? 0 : int64_t(prompt[r]) - (n0[r] + x1) * p->bt;
+        } else {
+            want[r] = int64_t(prompt[r]) - int64_t(n0[r] + n1[r] + n2[r]) * p->bt;
+        }
     }
     /* every in-flight decode sequence takes one token of the iteration */
     const int64_t TB = std::max<int64_t>(0, int64_t(p->token_budget) - D_act);
@@ -302,25 +334,8 @@ uint32_t orc_tier_plan(const orc_params *p, int n, const int32_t *prompt, const 
         action_out[r] = ORC_ACT_NONE;
         if (!valid[r] || grant[r] <= 0) continue;
         const int64_t P = prompt[r];
-        /* P1 (Eq. 7): host first, deep tier from what is left and only behind a fully restored host segment */
-        const int64_t rem = std::max<int64_t>(0, budget[r]);
-        const int64_t x1max = max_restorable(p, 1, rem, n1[r]);
-        int64_t x2max = 0;
-        if (x1max == n1[r] && n2[r] > 0) {
-            const int64_t rem2 = rem - restore_time(p, 1, n1[r]);
-            x2max = max_restorable(p, 2, rem2, n2[r]);
-        }
-        /* P2: smallest predicted completion time over the endpoint candidates; ties restore more */
-        int64_t bx1 = 0, bx2 = 0;
-        int64_t bF = plan_cost_q20(p, act, P, n0[r], 0, 0);
-        if (x1max > 0) {
-            const int64_t F = plan_cost_q20(p, act, P, n0[r], x1max, 0);
-            if (F <= bF) { bF = F; bx1 = x1max; bx2 = 0; }
-        }
-        if (x2max > 0) {
-            const int64_t F = plan_cost_q20(p, act, P, n0[r], n1[r], x2max);
-            if (F <= bF) { bF = F; bx1 = n1[r]; bx2 = x2max; }
-        }
+        int64_t bx1, bx2;
+        choose_restore(p, act, P, n0[r], n1[r], n2[r], budget[r], &bx1, &bx2);
         x1_out[r] = int32_t(bx1);
         x2_out[r] = int32_t(bx2);
         /* a deep fetch is staged first: nothing runs this iteration, HBM is taken only at the last hop */

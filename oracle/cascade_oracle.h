@@ -58,7 +58,7 @@ typedef struct orc_params {
     int64_t ttft_ns[ORC_MAX_CLASSES]; /* class TTFT targets                                  */
     int64_t tpot_ns[ORC_MAX_CLASSES]; /* class TPOT targets; 0 disables the decode term      */
     int32_t policy;        /* ordering: 0 least remaining budget, 1 FCFS, 2 EDF, 3 SJF (comparison policies) */
-    int32_t reserved;
+    int32_t plan_first;    /* 1: admission offers each request the tokens its own restore choice leaves to compute */
 } orc_params;
 
 #define ORC_POLICY_BUDGET 0
@@ -103,7 +103,8 @@ uint32_t orc_schedule(const orc_params *p, int n,
                       const uint64_t *key, const int32_t *prompt,
                       const int32_t *n0, const int32_t *n1, const int32_t *n2,
                       int32_t D_act,
-                      uint32_t *order_out, int32_t *grant_out, orc_sched_counts *counts);
+                      uint32_t *order_out, int32_t *grant_out, orc_sched_counts *counts,
+                      const int64_t *budget /* plan_first only */, int64_t K_act /* plan_first only */);
 
 /* Steps P1-P6 and K1: restore bound (Eq. 7), restore-vs-recompute choice, HBM
  * capacity, preemption victims and their disposition, block-id allocation.

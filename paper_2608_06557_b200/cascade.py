@@ -35,7 +35,7 @@ class Params(C.Structure):
         ("c_dseq_q20", C.c_int64), ("c_dkv_q20", C.c_int64),
         ("delta_ns", C.c_int64 * 3), ("blk_ns", C.c_int64 * 3),
         ("ttft_ns", C.c_int64 * MAX_CLASSES), ("tpot_ns", C.c_int64 * MAX_CLASSES),
-        ("policy", C.c_int32), ("reserved", C.c_int32),
+        ("policy", C.c_int32), ("plan_first", C.c_int32),
     ]
 
 
@@ -126,6 +126,7 @@ def make_params(d: dict) -> Params:
     for i, v in enumerate(d["tpot_ns"]):
         p.tpot_ns[i] = int(v)
     p.policy = int(d.get("policy", 0))
+    p.plan_first = int(d.get("plan_first", 0))
     return p
 
 

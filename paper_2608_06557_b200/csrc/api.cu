@@ -16,7 +16,7 @@ int cascade_validate_params(const cascade_params *p) {
               in_range(p->c_iter_q20, 0, one << 50) && in_range(p->c_dseq_q20, 0, one << 40) &&
               in_range(p->c_dkv_q20, 0, one << 28);
     if (ok) ok = (int64_t)(p->max_batch - 1) * p->max_ctx_avg <= (one << 32);
-    if (ok) ok = in_range(p->policy, CASCADE_POLICY_BUDGET, CASCADE_POLICY_SJF) && p->reserved == 0;
+    if (ok) ok = in_range(p->policy, CASCADE_POLICY_BUDGET, CASCADE_POLICY_SJF) && in_range(p->plan_first, 0, 1);
     for (int k = 1; ok && k <= 2; ++k)
         ok = in_range(p->delta_ns[k], 0, one << 30) && in_range(p->blk_ns[k], 1, one << 27);
     for (int c = 0; ok && c < p->n_classes; ++c)
@@ -64,6 +64,7 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     size_t n = (size_t)max_requests;
     bool ok = cudaMalloc(&ctx->status_dev, sizeof(uint32_t)) == cudaSuccess &&
               cudaMallocHost(&ctx->status_host, sizeof(uint32_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->want_by_slot, n * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&ctx->work_admit, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->work_victim, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->plan_scalars, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
@@ -83,6 +84,7 @@ extern "C" void cascade_destroy(cascade_ctx *ctx) {
     cudaSetDevice(ctx->device);
     cudaFree(ctx->status_dev);
     cudaFreeHost(ctx->status_host);
+    cudaFree(ctx->want_by_slot);
     cudaFree(ctx->work_admit);
     cudaFree(ctx->work_victim);
     cudaFree(ctx->plan_scalars);

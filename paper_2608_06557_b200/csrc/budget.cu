@@ -11,7 +11,7 @@ constexpr int kThreads = 256;
 __global__ void __launch_bounds__(kThreads)
 budget_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ LoadConsts lc,
               const __grid_constant__ cascade_reqs r, int n, int64_t now_ns, int64_t *__restrict__ budget_out,
-              uint64_t *__restrict__ key_out, uint32_t *__restrict__ status) {
+              uint64_t *__restrict__ key_out, int32_t *__restrict__ want_out, uint32_t *__restrict__ status) {
     const int i = blockIdx.x * kThreads + threadIdx.x;
     if (i >= n) return;
     const int64_t P = r.prompt[i];
@@ -28,6 +28,7 @@ budget_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ 
         atomicOr(status, CASCADE_ST_EPRECOND);
         budget_out[i] = -(int64_t(1) << 62);
         key_out[i] = (uint64_t(1) << 63) | id;
+        if (p.plan_first) want_out[i] = 0;
         return;
     }
     const int64_t s_hit = (n0 + n1 + n2) * p.bt;
@@ -61,6 +62,12 @@ budget_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ 
     u += clampv;
     budget_out[i] = budget;
     key_out[i] = (uint64_t(tier2) << 63) | (uint64_t(u) << 23) | id;
+    if (p.plan_first) {
+        // plan-first admission: the request's own restore choice fixes what it is offered
+        int64_t x1, x2;
+        dev_choose_restore(p, lc.A_act, P, n0, n1, n2, budget, &x1, &x2);
+        want_out[i] = x2 > 0 ? 0 : (int32_t)(P - (n0 + x1) * p.bt);
+    }
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -100,7 +107,7 @@ extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, in
     const LoadConsts lc = make_load_consts(ctx->params, D_act, K_act);
     const int grid = (n + kThreads - 1) / kThreads;
     budget_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(ctx->params, lc, *r, n, now_ns, budget_out, key_out,
-                                                              ctx->status_dev);
+                                                              ctx->want_by_slot, ctx->status_dev);
     CASCADE_CUDA_TRY(ctx, cudaGetLastError());
     return CASCADE_OK;
 }

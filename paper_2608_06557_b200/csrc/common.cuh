@@ -16,6 +16,7 @@ struct cascade_ctx {
     uint32_t *status_host;       // pinned mirror used by cascade_status
     int cuda_error;              // last failing cudaError_t
     // tier-plan scratch
+    int32_t *want_by_slot;       // plan-first admission: tokens each request is offered (budget -> schedule)
     int4 *work_admit;            // per admitted request: slot, pop offset, restore offset, counts
     int4 *work_victim;           // per preempted request: slot, freed offset, evict offset, action
     int32_t *plan_scalars;       // device scalars handed from the plan kernel to the apply kernels
@@ -104,6 +105,41 @@ static inline bool cascade_pick_geometry(const cascade_ctx *ctx, int n, int *T, 
         c = ctx->sort_cluster;
     *T = t; *C = c; *K = k;
     return (long long)c * t * k >= n && t * k <= 4096;
+}
+
+// The Eq. 7 bounds (host first, deep tier from what is left and only behind a fully restored host
+// segment) and the endpoint candidate with the smallest predicted completion time; ties restore more.
+__device__ __forceinline__ void dev_choose_restore(const cascade_params &p, int64_t A_act, int64_t P, int64_t n0,
+                                                   int64_t n1, int64_t n2, int64_t budget, int64_t *x1, int64_t *x2) {
+    const int64_t rem = budget > 0 ? budget : 0;
+    const int64_t bt = p.bt;
+    int64_t x1max = 0;
+    if (n1 > 0) {
+        int64_t head = rem - p.delta_ns[1];
+        if (head < 0) head = 0;
+        x1max = head / p.blk_ns[1];
+        if (x1max > n1) x1max = n1;
+    }
+    int64_t x2max = 0;
+    if (x1max == n1 && n2 > 0) {
+        int64_t head = rem - dev_restore_time(p, 1, n1) - p.delta_ns[2];
+        if (head < 0) head = 0;
+        x2max = head / p.blk_ns[2];
+        if (x2max > n2) x2max = n2;
+    }
+    int64_t bx1 = 0, bx2 = 0;
+    int64_t bF = dev_comp_q(A_act, p.c_attn_q20, P, n0 * bt);
+    if (x1max > 0) {
+        const int64_t F = (dev_restore_time(p, 1, x1max) << 20) + dev_comp_q(A_act, p.c_attn_q20, P, (n0 + x1max) * bt);
+        if (F <= bF) { bF = F; bx1 = x1max; }
+    }
+    if (x2max > 0) {
+        const int64_t F = ((dev_restore_time(p, 1, n1) + dev_restore_time(p, 2, x2max)) << 20) +
+                          dev_comp_q(A_act, p.c_attn_q20, P, (n0 + n1 + x2max) * bt);
+        if (F <= bF) { bF = F; bx1 = n1; bx2 = x2max; }
+    }
+    *x1 = bx1;
+    *x2 = bx2;
 }
 
 // entry points implemented in the other translation units

@@ -52,6 +52,7 @@ struct __align__(16) Exch {
 struct ScheduleArgs {
     const uint64_t *key;
     const int32_t *prompt, *n0, *n1, *n2;
+    const int32_t *want_in;   // plan-first admission: the offers cascade_budget left in the context, else NULL
     uint32_t *order_out;
     int32_t *grant_out;
     cascade_sched_counts *counts;
@@ -127,7 +128,7 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
             const unsigned long long key = a.key[g];
             const long long P = a.prompt[g], h0 = a.n0[g], h1 = a.n1[g], h2 = a.n2[g];
             long long want = 0;
-            if (dev_request_valid(a.bt, P, h0, h1, h2)) want = P - (h0 + h1 + h2) * a.bt;
+            if (dev_request_valid(a.bt, P, h0, h1, h2)) want = a.want_in ? a.want_in[g] : P - (h0 + h1 + h2) * a.bt;
             e[k].key = key;
             e[k].idx = (uint32_t)g;
             e[k].want = (int32_t)want;
@@ -532,6 +533,7 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.n0 = r->n0;
     a.n1 = r->n1;
     a.n2 = r->n2;
+    a.want_in = p.plan_first ? ctx->want_by_slot : nullptr;
     a.order_out = order_out;
     a.grant_out = grant_out;
     a.counts = counts_dev;

@@ -11,7 +11,7 @@ def oracle_iteration(w, with_tables=True, restore_cap=None, evict_cap=None):
     workload's tables and free lists are copied first, so ``w`` itself is left untouched."""
     p = oracle.make_params(w.params)
     budget, key, st_b = oracle.budget(p, w.reqs, w.now_ns, w.D_act, w.K_act)
-    order, grant, sc, st_s = oracle.schedule(p, w.reqs, key, w.D_act)
+    order, grant, sc, st_s = oracle.schedule(p, w.reqs, key, w.D_act, budget, w.K_act)
     grant_sched = grant.copy()
     if with_tables and w.hbm_tbl is not None:
         pools = oracle.Pools(hbm_tbl=w.hbm_tbl.copy(), host_tbl=w.host_tbl.copy(), hbm_free=w.hbm_free.copy(),

@@ -196,3 +196,20 @@ def test_latency_regimes_match():
         ref, st = oracle.latency_regimes(oracle.make_params(w.params), w.reqs, w.D_act, w.K_act)
         assert np.array_equal(lat.cpu().numpy(), ref)
         assert inst.ctx.status()[0] == st == 8
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_plan_first_admission(seed):
+    w = wl.config_tiny(seed, hbm_free_target=200)
+    w.params = dict(w.params, plan_first=1)
+    if seed % 2:
+        w.params["ttft_ns"] = [20 * t for t in w.params["ttft_ns"]]
+    compare_iteration(w, f"plan-first{seed}")
+    w = wl.config_llama8b(seed=30 + seed, n=7000, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9, elapsed_scale=0.3)
+    w.hbm_tbl = w.host_tbl = w.hbm_free = w.host_free = None
+    w.hbm_free_count, w.host_free_count = 1 << 30, 1 << 30
+    w.reqs["n2"][::5] = 3                                  # some deep-tier hits (the prompt bound still holds)
+    w.reqs["prompt"][::5] += 48
+    w.params = dict(w.params, plan_first=1, token_budget=200_000, max_batch=2048)
+    got, ref = compare_iteration(w, f"plan-first-7000-{seed}")
+    assert got["sched_counts"]["n_admitted"] > 50

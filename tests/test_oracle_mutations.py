@@ -8,7 +8,7 @@ import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SRC = os.path.join(ROOT, "oracle", "cascade_oracle.cpp")
-PINS = ["test_oracle_budget.py", "test_oracle_schedule.py", "test_oracle_plan.py", "test_oracle_copy.py",
+PINS = ["test_oracle_plan_first.py", "test_oracle_budget.py", "test_oracle_schedule.py", "test_oracle_plan.py", "test_oracle_copy.py",
         "test_oracle_prefetch.py", "test_oracle_policies.py"]
 
 MUTATIONS = [
@@ -56,6 +56,10 @@ MUTATIONS = [
      "if (ok && grant[r] > 0) link_left -= 0;"),
     ("prefetch serves preempted requests", "if (action[r] == ORC_ACT_EVICT || action[r] == ORC_ACT_DROP) continue;", ""),
     ("edf uses the wrong sign", "v = p->ttft_ns[cls[r]] - elapsed; tier2 = false;", "v = p->ttft_ns[cls[r]] + elapsed; tier2 = false;"),
+    ("plan-first offer ignores the restore choice", "want[r] = x2 > 0 ? 0 : int64_t(prompt[r]) - (n0[r] + x1) * p->bt;",
+     "want[r] = x2 > 0 ? 0 : int64_t(prompt[r]) - (n0[r] + n1[r]) * p->bt;"),
+    ("plan-first offer for a staged deep fetch", "want[r] = x2 > 0 ? 0 : int64_t(prompt[r]) - (n0[r] + x1) * p->bt;",
+     "want[r] = int64_t(prompt[r]) - (n0[r] + x1) * p->bt;"),
     ("regime 1 reuses the prefix", "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, 0) >> 20;",
      "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, s_hit) >> 20;"),
 ]

@@ -57,8 +57,9 @@ def build(force: bool = False) -> str:
     newest = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".{os.getpid()}.tmp"
-        subprocess.check_call(["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-Wall", "-Wextra", "-I", _HERE, "-o", tmp,
-                               _SRC])
+        extra = os.environ.get("CASCADE_ORACLE_CXXFLAGS", "").split()   # e.g. -fsanitize=undefined for the UB check
+        subprocess.check_call(["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-Wall", "-Wextra", "-I", _HERE] + extra +
+                              ["-o", tmp, _SRC])
         os.replace(tmp, _LIB)
     return _LIB
 

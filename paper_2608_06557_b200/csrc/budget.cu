@@ -98,6 +98,7 @@ regimes_kernel(const __grid_constant__ cascade_params p, const __grid_constant__
 
 extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, int64_t now_ns, int32_t D_act,
                               int64_t K_act, int64_t *budget_out, uint64_t *key_out, void *stream) {
+    CascadeRange nvtx_range("cascade_budget");
     if (!ctx || !r || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
     if (n == 0) return CASCADE_OK;
     if (!budget_out || !key_out || !r->arrival_ns || !r->prompt || !r->pred_out || !r->n0 || !r->n1 || !r->n2 ||
@@ -114,6 +115,7 @@ extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, in
 
 extern "C" int cascade_latency_regimes(cascade_ctx *ctx, const cascade_reqs *r, int n, int32_t D_act, int64_t K_act,
                                        int64_t *lat4_out, void *stream) {
+    CascadeRange nvtx_range("cascade_latency_regimes");
     if (!ctx || !r || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
     if (n == 0) return CASCADE_OK;
     if (!lat4_out || !r->prompt || !r->n0 || !r->n1 || !r->n2) return CASCADE_EINVAL;

@@ -6,6 +6,8 @@
 
 #include "cascade.h"
 
+#include <nvtx3/nvToolsExt.h>
+
 // Context: parameters, scratch sized at creation, the sticky device status word.
 struct cascade_ctx {
     cascade_params params;
@@ -34,6 +36,12 @@ struct cascade_ctx {
 
 // plan_scalars layout
 enum { PS_N_ADMIT = 0, PS_N_VICTIM, PS_HBM_CNT0, PS_HOST_CNT0, PS_TOTAL_FREED, PS_COUNT };
+
+// NVTX range around the launches of one entry point (visible in Nsight timelines; a no-op without a tool)
+struct CascadeRange {
+    explicit CascadeRange(const char *name) { nvtxRangePushA(name); }
+    ~CascadeRange() { nvtxRangePop(); }
+};
 
 #define CASCADE_CUDA_TRY(ctx, expr)                         \
     do {                                                    \

@@ -420,6 +420,7 @@ extern "C" int cascade_kv_restore(cascade_ctx *ctx, const cascade_kv_layout *hbm
                                   int64_t src_blocks, int src_is_device, const int32_t *src_ids,
                                   const int32_t *dst_ids, const int32_t *n_copies_dev, int n_copies_max,
                                   void *stream) {
+    CascadeRange nvtx_range("cascade_kv_restore");
     return launch_copy<true>(ctx, hbm, (char *)hbm_pool, (char *)const_cast<void *>(src_pool), src_blocks,
                              src_is_device, src_ids, dst_ids, n_copies_dev, n_copies_max, (cudaStream_t)stream);
 }
@@ -427,6 +428,7 @@ extern "C" int cascade_kv_restore(cascade_ctx *ctx, const cascade_kv_layout *hbm
 extern "C" int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, const void *hbm_pool, void *dst_pool,
                                 int64_t dst_blocks, int dst_is_device, const int32_t *src_ids, const int32_t *dst_ids,
                                 const int32_t *n_copies_dev, int n_copies_max, void *stream) {
+    CascadeRange nvtx_range("cascade_kv_evict");
     return launch_copy<false>(ctx, hbm, (char *)const_cast<void *>(hbm_pool), (char *)dst_pool, dst_blocks,
                               dst_is_device, src_ids, dst_ids, n_copies_dev, n_copies_max, (cudaStream_t)stream);
 }
@@ -436,6 +438,7 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
                                const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,
                                const int32_t *restore_dst, const int32_t *n_restore_dev, int n_restore_max,
                                int32_t *scratch, void *stream) {
+    CascadeRange nvtx_range("cascade_kv_move");
     if (!ctx || n_evict_max < 0 || n_restore_max < 0) return CASCADE_EINVAL;
     if (n_evict_max == 0 && n_restore_max == 0) return CASCADE_OK;
     int rc = check_layout(hbm, hbm_pool, host_pool, host_blocks);

@@ -28,6 +28,13 @@ namespace {
 
 constexpr int kMaxCluster = 16;
 
+#ifdef CASCADE_PHASE_TIMING
+__device__ long long g_plan_ticks[16];
+#define PTICK(i) do { if (threadIdx.x == 0 && crank == 0) g_plan_ticks[(i)] = clock64(); } while (0)
+#else
+#define PTICK(i) do { } while (0)
+#endif
+
 // element flags
 constexpr unsigned kAdm = 1u, kPriv = 2u, kFits = 4u, kValid = 8u, kReal = 16u;
 
@@ -92,6 +99,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         }
     }
 
+    PTICK(0);
     // ---- phase 1: gather through the order, Eq. 7 bounds, restore-vs-recompute choice -----------
     uint32_t slot[K];
     unsigned fl[K];
@@ -169,6 +177,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         a.plan.x2[r] = x2;   // rewritten below if the request is un-admitted
     }
 
+    PTICK(1);
     // ---- phase 2: forward scan over the admitted set, capacity cut --------------------------------
     int s_need[K], s_x1[K], s_cnt[K];
     long long evictable = 0;
@@ -184,6 +193,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     cta_scan3<T, K>(s_need, s_x1, s_cnt, tot, ws3);
     long long red1[1] = {evictable};
     cta_sum<T, 1>(red1, ws8);
+    PTICK(2);
     if (tid < csize) {
         Exch1 x;
         x.need = tot[0];
@@ -193,6 +203,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         cluster.map_shared_rank(ex1, tid)[crank] = x;
     }
     cluster.sync();
+    PTICK(3);
     long long off_need = 0, cap = hbm_cnt;
     int off_x1 = 0, off_cnt = 0;
 #pragma unroll
@@ -228,6 +239,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         }
     }
 
+    PTICK(4);
     // ---- phase 3: preemptable holders, walked backwards ---------------------------------------------
     int s_v[K], s_h[K], s_c[K];
 #pragma unroll
@@ -240,6 +252,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     cta_scan3<T, K>(s_v, s_h, s_c, tot, ws3);
     long long red5[5] = {k_need, k_cnt, k_x1, k_unadm, k_tok};
     cta_sum<T, 5>(red5, ws8);
+    PTICK(5);
     if (tid < csize) {
         Exch2 x;
         x.v = tot[0];
@@ -255,6 +268,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         cluster.map_shared_rank(ex2, tid)[crank] = x;
     }
     cluster.sync();
+    PTICK(6);
     long long need_total = 0, V = 0, H = 0, tokens = 0;
     int Cn = 0, off_v = 0, off_h = 0, off_c = 0, n_adm = 0, n_rest = 0, n_unadm = 0;
 #pragma unroll
@@ -302,8 +316,10 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         a.plan.x1[slot[k]] = x1v[k];
         a.plan.tokens_run[slot[k]] = runv[k];
     }
+    PTICK(7);
     long long red3[3] = {s_nv, s_freed, s_nev};
     cta_sum<T, 3>(red3, ws8);
+    PTICK(8);
     if (tid == 0) {
         Exch3 x;
         x.nv = (int)red3[0];
@@ -315,6 +331,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     st = __reduce_or_sync(kFull, st);
     if (lane == 0 && st) atomicOr(a.status, st);
     cluster.sync();
+    PTICK(9);
     if (crank == 0 && tid == 0) {
         long long nv = 0, freed = 0, nev = 0;
         for (unsigned c = 0; c < csize; ++c) {
@@ -462,9 +479,16 @@ cudaError_t launch_plan_k(int K, const cascade_params &p, const PlanArgs &a, int
 
 }  // namespace
 
+#ifdef CASCADE_PHASE_TIMING
+extern "C" int cascade_debug_plan_ticks(long long *host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_plan_ticks, sizeof(g_plan_ticks));
+}
+#endif
+
 extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *budget,
                                  const uint32_t *order, int32_t *grant, int n, int32_t D_act, int64_t K_act,
                                  const cascade_pools *pools, const cascade_plan *plan_out, void *stream) {
+    CascadeRange nvtx_range("cascade_tier_plan");
     if (!ctx || !r || !pools || !plan_out || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
     if (!plan_out->counts || !pools->hbm_free_count || !pools->host_free_count) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
@@ -570,6 +594,7 @@ extern "C" int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_
                                          const uint32_t *order, int32_t *grant, int n, int32_t D_act, int64_t K_act,
                                          const cascade_pools *pools, const cascade_plan *plan_out,
                                          uint32_t *status_dev, void *stream) {
+    CascadeRange nvtx_range("cascade_tier_plan_noalloc");
     if (!p || !r || !pools || !plan_out || !status_dev || n < 0) return CASCADE_EINVAL;
     if (n > CASCADE_NOALLOC_MAX_REQUESTS) return CASCADE_ETOOBIG;  // beyond the fixed scratch
     int rc = cascade_validate_params(p);

@@ -286,6 +286,7 @@ extern "C" int cascade_prefetch_plan(cascade_ctx *ctx, const cascade_reqs *r, co
                                      int32_t D_act, int64_t K_act, int64_t link_budget_ns, int32_t hbm_reserve,
                                      const cascade_pools *pools, const cascade_plan *plan, int32_t *pf_out,
                                      cascade_prefetch_counts *counts_dev, void *stream) {
+    CascadeRange nvtx_range("cascade_prefetch_plan");
     if (!ctx || !r || !pools || !plan || !counts_dev || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
     if (!plan->counts || !pools->hbm_free_count) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;

@@ -515,6 +515,7 @@ extern "C" int cascade_debug_ticks(long long *host_out) {
 extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const uint64_t *key, int n, int32_t D_act,
                                 uint32_t *order_out, int32_t *grant_out, cascade_sched_counts *counts_dev,
                                 void *stream) {
+    CascadeRange nvtx_range("cascade_schedule");
     if (!ctx || !r || n < 0 || n > ctx->max_requests || !counts_dev) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16)) return CASCADE_ERANGE;
     cudaStream_t s = (cudaStream_t)stream;

@@ -89,3 +89,14 @@ def test_the_unaltered_copy_passes(tmp_path):
     path.write_text(open(SRC).read())
     res = run_pins(dict(os.environ, CASCADE_ORACLE_SRC=str(path)))
     assert res.returncode == 0, res.stdout[-2000:]
+
+
+def test_pins_pass_under_the_undefined_behaviour_sanitizer(tmp_path):
+    """Signed overflow, bad shifts and out-of-range indexing in the oracle would make its outputs meaningless:
+    the whole pin suite is run once more on a copy built with -fsanitize=undefined (any report aborts)."""
+    path = tmp_path / "ubsan.cpp"
+    path.write_text(open(SRC).read())
+    env = dict(os.environ, CASCADE_ORACLE_SRC=str(path),
+               CASCADE_ORACLE_CXXFLAGS="-fsanitize=undefined -fno-sanitize-recover=all -g")
+    res = run_pins(env)
+    assert res.returncode == 0, res.stdout[-3000:]

@@ -362,12 +362,13 @@ def ours_main(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     torch.cuda.set_device(local_rank)
-    if world > 1:
+    use_dist = "RANK" in os.environ and "MASTER_ADDR" in os.environ     # launched by torchrun, at any world size
+    if use_dist:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     import __graft_entry__ as ge
     if rank == 0:
         ge.build()
-    if world > 1:
+    if use_dist:
         dist.barrier()
     from paper_2608_06557_b200 import cascade as cs
     from paper_2608_06557_b200.runner import Instance, alloc_pinned_pool, fill_pools
@@ -393,7 +394,7 @@ def ours_main(args):
     peaks = measure_link_peaks(torch, host_pool, hbm_pool)
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -435,7 +436,7 @@ def ours_main(args):
     t_sched = np.array([ev[i][0].elapsed_time(ev[i][1]) for i in range(K)])
     t_evict = np.array([ev[i][1].elapsed_time(ev[i][2]) for i in range(K)])
     t_rest = np.array([ev[i][2].elapsed_time(ev[i][3]) for i in range(K)])
-    if world > 1:
+    if use_dist:
         ms_total, moved = aggregate_over_ranks(dist, ms_total, moved, dev)
     value = moved / (ms_total * 1e-3) / GB
 
@@ -512,7 +513,7 @@ def ours_main(args):
         line["cpu_baseline"] = {k: v for k, v in run_oracle_arm(args, args.cpu_seconds, first_seed=W).items()
                                 if k in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(line))
-    if world > 1:
+    if use_dist:
         dist.barrier()
         dist.destroy_process_group()
 

@@ -210,7 +210,7 @@ typedef struct cascade_status_t {
 typedef struct cascade_ctx cascade_ctx;
 
 /* Creates a context on `device` for queues of up to max_requests (<= CASCADE_MAX_REQUESTS).
- * Validates the parameters against the bounds above.  Allocates scratch (about 32 bytes per request).
+ * Validates the parameters against the bounds above.  Allocates scratch (about 44 bytes per request).
  * `p` and `out` are host pointers. */
 int cascade_create(cascade_ctx **out, const cascade_params *p, int max_requests, int device);
 void cascade_destroy(cascade_ctx *ctx);
@@ -351,7 +351,7 @@ int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void
  *
  * Same computation, same arguments and same results as cascade_tier_plan, but no context: the
  * per-request offsets that the first plan kernel hands to the two table-rewrite kernels live in a
- * fixed scratch area compiled into the library (about 256 KiB of device memory on every GPU that
+ * fixed scratch area compiled into the library (about 320 KiB of device memory on every GPU that
  * loads the library, held from load to exit) instead of memory obtained in cascade_create.  It is
  * meant for callers that cannot call cudaMalloc: an engine that has already handed all free HBM to
  * its KV block pool, code running under a host framework that owns the allocator, or a loop that

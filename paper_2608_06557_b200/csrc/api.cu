@@ -64,6 +64,7 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     size_t n = (size_t)max_requests;
     bool ok = cudaMalloc(&ctx->status_dev, sizeof(uint32_t)) == cudaSuccess &&
               cudaMallocHost(&ctx->status_host, sizeof(uint32_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->pack_by_slot, n * sizeof(unsigned long long)) == cudaSuccess &&
               cudaMalloc(&ctx->want_by_slot, n * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&ctx->work_admit, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->work_victim, n * sizeof(int4)) == cudaSuccess &&
@@ -84,6 +85,7 @@ extern "C" void cascade_destroy(cascade_ctx *ctx) {
     cudaSetDevice(ctx->device);
     cudaFree(ctx->status_dev);
     cudaFreeHost(ctx->status_host);
+    cudaFree(ctx->pack_by_slot);
     cudaFree(ctx->want_by_slot);
     cudaFree(ctx->work_admit);
     cudaFree(ctx->work_victim);

@@ -18,6 +18,7 @@ struct cascade_ctx {
     uint32_t *status_host;       // pinned mirror used by cascade_status
     int cuda_error;              // last failing cudaError_t
     // tier-plan scratch
+    unsigned long long *pack_by_slot;  // tier plan: one decision word per request, slot order
     int32_t *want_by_slot;       // plan-first admission: tokens each request is offered (budget -> schedule)
     int4 *work_admit;            // per admitted request: slot, pop offset, restore offset, counts
     int4 *work_victim;           // per preempted request: slot, freed offset, evict offset, action

@@ -3,8 +3,10 @@
 //
 // Kernel 1 (one thread-block cluster, the queue spread over its CTAs in schedule order, K
 // elements per thread held in registers):
-//   phase 1  gather each request's fields through `order`, evaluate Eq. 7 and the candidate plans
-//            (the only int64 divisions of the path, at most two per admitted request);
+//   phase 1  in slot order (coalesced loads): Eq. 7 and the candidate plans (the only int64 divisions
+//            of the path, at most two per admitted request), default per-request outputs, and one
+//            packed decision word per request; after a cluster barrier the schedule-order phases
+//            gather just that word through `order`;
 //   phase 2  forward prefix sums over the admitted set (cumulative HBM need, restore-list offsets)
 //            and the sum of preemptable blocks; one exchange of per-CTA totals through distributed
 //            shared memory; the admitted set is cut where the cumulative need exceeds the capacity;
@@ -13,7 +15,7 @@
 //            sequential "pop one request / preempt the largest budget" loops of Algorithm 1 become
 //            two scans because admitted requests and victims are prefixes of the two walks;
 //   phase 4  per-request outputs are scattered by slot; CTA 0 writes the counts.
-// Three hardware cluster barriers are the only inter-CTA waits (no spin loops).
+// Four hardware cluster barriers are the only inter-CTA waits (no spin loops).
 // Kernels 2 and 3 (many CTAs, one warp per request): rewrite block tables, free lists and the two
 // copy lists from the offsets kernel 1 left in scratch; pushes of freed ids (kernel 2) finish
 // before any pop (kernel 3).  In plan-only mode (no tables) only kernel 1 runs.
@@ -46,6 +48,7 @@ struct PlanArgs {
     int32_t *grant;
     cascade_pools pools;
     cascade_plan plan;
+    unsigned long long *pack;          // one decision word per request, slot order (scratch)
     int4 *work_admit, *work_victim;
     int32_t *scalars;
     uint32_t *status;
@@ -100,11 +103,54 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     }
 
     PTICK(0);
-    // ---- phase 1: gather through the order, Eq. 7 bounds, restore-vs-recompute choice -----------
+    // ---- phase 1a, slot order (coalesced): Eq. 7 bounds and the restore-vs-recompute choice; the
+    //      per-request outputs get their default values here and one packed word per request
+    //      (n0 | x1 << 14 | tokens_run << 28 | flags << 46) is left for the schedule-order phases
+    const long long pos0 = (long long)crank * per + (warp * K) * 32 + lane;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const long long r = pos0 + k * 32;
+        if (r >= n) continue;
+        const long long P = a.prompt[r], n0 = a.n0[r], n1 = a.n1[r], n2 = a.n2[r];
+        const long long b = a.budget[r];
+        const int g = a.grant[r];
+        const unsigned rf = a.flags[r];
+        bool valid = dev_request_valid(bt, P, n0, n1, n2);
+        if (valid && a.with_tables) valid = (P + bt - 1) / bt <= a.pools.maxb;
+        unsigned long long w = (unsigned long long)kReal << 46;
+        int x1 = 0, x2 = 0, run = 0;
+        if (!valid) {
+            st |= CASCADE_ST_EPRECOND;
+            if (g != 0) a.grant[r] = 0;
+        } else {
+            unsigned f = kReal | kValid;
+            if (rf & CASCADE_FLAG_HBM_PRIVATE) f |= kPriv;
+            if (dev_restore_time(p, 1, n0) <= b) f |= kFits;
+            if (g > 0) {
+                int64_t bx1, bx2;
+                dev_choose_restore(p, a.A_act, P, n0, n1, n2, b, &bx1, &bx2);
+                // a deep fetch is staged first: nothing runs now, HBM is taken at the last hop only
+                const long long left = P - (n0 + bx1) * bt;
+                x1 = (int)bx1;
+                x2 = (int)bx2;
+                run = bx2 > 0 ? 0 : (int)(g < left ? g : left);
+                f |= kAdm;
+            }
+            w = (unsigned long long)n0 | ((unsigned long long)x1 << 14) | ((unsigned long long)run << 28) |
+                ((unsigned long long)f << 46);
+        }
+        a.pack[r] = w;
+        a.plan.x1[r] = x1;
+        a.plan.x2[r] = x2;
+        a.plan.tokens_run[r] = run;
+        a.plan.action[r] = (valid && n0 > 0) ? CASCADE_ACT_RETAIN : CASCADE_ACT_NONE;
+    }
+    cluster.sync();  // the packed words are visible to every CTA of the cluster
+
+    // ---- phase 1b, schedule order: one 8-byte gather per element --------------------------------
     uint32_t slot[K];
     unsigned fl[K];
     int n0v[K], x1v[K], runv[K];
-    long long pos0 = (long long)crank * per + (warp * K) * 32 + lane;
 #pragma unroll
     for (int k = 0; k < K; ++k) {
         const long long q = pos0 + k * 32;
@@ -113,68 +159,11 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
 #pragma unroll
     for (int k = 0; k < K; ++k) {
         const long long q = pos0 + k * 32;
-        fl[k] = 0;
-        n0v[k] = 0;
-        x1v[k] = 0;
-        runv[k] = 0;
-        if (q >= n) continue;
-        const uint32_t r = slot[k];
-        const long long P = a.prompt[r], n0 = a.n0[r], n1 = a.n1[r], n2 = a.n2[r];
-        const long long b = a.budget[r];
-        const int g = a.grant[r];
-        const unsigned rf = a.flags[r];
-        bool valid = dev_request_valid(bt, P, n0, n1, n2);
-        if (valid && a.with_tables) valid = (P + bt - 1) / bt <= a.pools.maxb;
-        int x2 = 0;
-        if (!valid) {
-            st |= CASCADE_ST_EPRECOND;
-            if (g != 0) a.grant[r] = 0;
-            fl[k] = kReal;
-        } else {
-            fl[k] = kReal | kValid;
-            n0v[k] = (int)n0;
-            if (rf & CASCADE_FLAG_HBM_PRIVATE) fl[k] |= kPriv;
-            if (dev_restore_time(p, 1, n0) <= b) fl[k] |= kFits;
-            if (g > 0) {
-                const long long rem = b > 0 ? b : 0;
-                // Eq. 7, host tier first
-                long long x1max = 0;
-                if (n1 > 0) {
-                    long long head = rem - p.delta_ns[1];
-                    if (head < 0) head = 0;
-                    x1max = head / p.blk_ns[1];
-                    if (x1max > n1) x1max = n1;
-                }
-                // deep tier from what is left, only behind a fully restored host segment
-                long long x2max = 0;
-                if (x1max == n1 && n2 > 0) {
-                    long long head = rem - dev_restore_time(p, 1, n1) - p.delta_ns[2];
-                    if (head < 0) head = 0;
-                    x2max = head / p.blk_ns[2];
-                    if (x2max > n2) x2max = n2;
-                }
-                // smallest predicted completion time; ties restore more
-                long long bx1 = 0, bx2 = 0;
-                long long bF = dev_comp_q(a.A_act, p.c_attn_q20, P, n0 * bt);
-                if (x1max > 0) {
-                    const long long F = (dev_restore_time(p, 1, x1max) << 20) +
-                                        dev_comp_q(a.A_act, p.c_attn_q20, P, (n0 + x1max) * bt);
-                    if (F <= bF) { bF = F; bx1 = x1max; }
-                }
-                if (x2max > 0) {
-                    const long long F = ((dev_restore_time(p, 1, n1) + dev_restore_time(p, 2, x2max)) << 20) +
-                                        dev_comp_q(a.A_act, p.c_attn_q20, P, (n0 + n1 + x2max) * bt);
-                    if (F <= bF) { bF = F; bx1 = n1; bx2 = x2max; }
-                }
-                // a deep fetch is staged first: nothing runs now, HBM is taken at the last hop only
-                const long long left = P - (n0 + bx1) * bt;
-                x1v[k] = (int)bx1;
-                x2 = (int)bx2;
-                runv[k] = bx2 > 0 ? 0 : (int)(g < left ? g : left);
-                fl[k] |= kAdm;
-            }
-        }
-        a.plan.x2[r] = x2;   // rewritten below if the request is un-admitted
+        const unsigned long long w = q < n ? a.pack[slot[k]] : 0ull;
+        fl[k] = (unsigned)(w >> 46);
+        n0v[k] = (int)(w & 0x3fff);
+        x1v[k] = (int)((w >> 14) & 0x3fff);
+        runv[k] = (int)((w >> 28) & 0x3ffff);
     }
 
     PTICK(1);
@@ -226,7 +215,9 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
             x1v[k] = 0;
             runv[k] = 0;
             a.grant[slot[k]] = 0;
+            a.plan.x1[slot[k]] = 0;
             a.plan.x2[slot[k]] = 0;
+            a.plan.tokens_run[slot[k]] = 0;
             ++k_unadm;
             st |= CASCADE_ST_ENOSPC;
         } else {
@@ -311,10 +302,8 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
                 act = CASCADE_ACT_RETAIN;
             }
         }
-        // ---- phase 4: per-request outputs, scattered by slot ---------------------------------------
-        a.plan.action[slot[k]] = act;
-        a.plan.x1[slot[k]] = x1v[k];
-        a.plan.tokens_run[slot[k]] = runv[k];
+        // ---- phase 4: only preempted requests change the action written in phase 1a -----------------
+        if (act == CASCADE_ACT_EVICT || act == CASCADE_ACT_DROP) a.plan.action[slot[k]] = act;
     }
     PTICK(7);
     long long red3[3] = {s_nv, s_freed, s_nev};
@@ -516,6 +505,7 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     a.grant = grant;
     a.pools = *pools;
     a.plan = *plan_out;
+    a.pack = ctx->pack_by_slot;
     a.work_admit = ctx->work_admit;
     a.work_victim = ctx->work_victim;
     a.scalars = ctx->plan_scalars;
@@ -557,12 +547,13 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
 namespace {
 
 struct NoAllocScratch {
+    unsigned long long pack[CASCADE_NOALLOC_MAX_REQUESTS];
     int4 work_admit[CASCADE_NOALLOC_MAX_REQUESTS];
     int4 work_victim[CASCADE_NOALLOC_MAX_REQUESTS];
     int32_t scalars[PS_COUNT];
 };
 
-// ~256 KiB + a few scalars per GPU; shared by every call on that GPU
+// ~320 KiB + a few scalars per GPU; shared by every call on that GPU
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
 
 struct NoAllocDevice {
@@ -631,6 +622,7 @@ extern "C" int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_
     a.grant = grant;
     a.pools = *pools;
     a.plan = *plan_out;
+    a.pack = dev->scratch->pack;
     a.work_admit = dev->scratch->work_admit;
     a.work_victim = dev->scratch->work_victim;
     a.scalars = dev->scratch->scalars;

@@ -209,7 +209,8 @@ typedef struct cascade_status_t {
 
 typedef struct cascade_ctx cascade_ctx;
 
-/* Creates a context on `device` for queues of up to max_requests (<= CASCADE_MAX_REQUESTS).
+/* Creates a context on `device` for queues of up to max_requests (<= CASCADE_MAX_REQUESTS, and
+ * <= 4096 times the largest thread-block cluster the device co-schedules: 16 on a full B200).
  * Validates the parameters against the bounds above.  Allocates scratch (about 44 bytes per request).
  * `p` and `out` are host pointers. */
 int cascade_create(cascade_ctx **out, const cascade_params *p, int max_requests, int device);

@@ -41,7 +41,14 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->device = device;
     ctx->max_requests = max_requests;
     cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
-    const char *e = getenv("CASCADE_SORT_CLUSTER");
+    ctx->max_cluster = cascade_probe_max_cluster();
+    const char *e = getenv("CASCADE_MAX_CLUSTER");   // lower it to exercise the fallback geometry
+    if (e && atoi(e) > 0 && atoi(e) < ctx->max_cluster) ctx->max_cluster = atoi(e);
+    if ((long long)max_requests > (long long)ctx->max_cluster * 4096) {  // the cluster kernels could not hold the queue
+        free(ctx);
+        return CASCADE_EINVAL;
+    }
+    e = getenv("CASCADE_SORT_CLUSTER");
     ctx->sort_cluster = e ? atoi(e) : 0;
     e = getenv("CASCADE_SORT_ITEMS");
     ctx->sort_items = e ? atoi(e) : 0;

@@ -23,6 +23,7 @@ struct cascade_ctx {
     int4 *work_admit;            // per admitted request: slot, pop offset, restore offset, counts
     int4 *work_victim;           // per preempted request: slot, freed offset, evict offset, action
     int32_t *plan_scalars;       // device scalars handed from the plan kernel to the apply kernels
+    int max_cluster;             // largest cluster the device co-schedules for the cluster kernels
     int sort_cluster;            // cluster size override for the ordering kernel (0 = automatic)
     int sort_items;              // keys per thread override (0 = automatic)
     int sort_threads;            // threads per CTA override (0 = automatic)
@@ -112,6 +113,12 @@ static inline bool cascade_pick_geometry(const cascade_ctx *ctx, int n, int *T, 
     if (ctx->sort_cluster == 1 || ctx->sort_cluster == 2 || ctx->sort_cluster == 4 || ctx->sort_cluster == 8 ||
         ctx->sort_cluster == 16)
         c = ctx->sort_cluster;
+    // a device that cannot co-schedule the preferred cluster gets a smaller one with more keys per CTA
+    const int cmax = ctx->max_cluster > 0 ? ctx->max_cluster : 16;
+    while (c > cmax && c > 1) {
+        c /= 2;
+        if (k < 8) k *= 2; else if (t < 512) t = 512;
+    }
     *T = t; *C = c; *K = k;
     return (long long)c * t * k >= n && t * k <= 4096;
 }
@@ -153,3 +160,4 @@ __device__ __forceinline__ void dev_choose_restore(const cascade_params &p, int6
 
 // entry points implemented in the other translation units
 int cascade_validate_params(const cascade_params *p);
+int cascade_probe_max_cluster();

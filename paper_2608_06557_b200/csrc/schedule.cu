@@ -506,6 +506,25 @@ cudaError_t launch_k(int K, const ScheduleArgs &a, int C, int device, cudaStream
 
 }  // namespace
 
+// Largest cluster the device will co-schedule for the ordering kernel (its shared-memory footprint is
+// the largest of the cluster kernels); 16 on a full B200, less on partitioned or smaller parts.
+int cascade_probe_max_cluster() {
+    cudaFuncSetAttribute(schedule_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(256, 8));
+    cudaFuncSetAttribute(schedule_kernel<256, 1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(16, 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes(256, 8);
+    int size = 0;
+    if (cudaOccupancyMaxPotentialClusterSize(&size, schedule_kernel<256, 1>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 8;  // the portable maximum
+    }
+    // restore the kernel's own footprint for later launches
+    cudaFuncSetAttribute(schedule_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(256, 1));
+    return size < 1 ? 1 : (size > 16 ? 16 : size);
+}
+
 #ifdef CASCADE_PHASE_TIMING
 extern "C" int cascade_debug_ticks(long long *host_out) {
     return (int)cudaMemcpyFromSymbol(host_out, g_phase_ticks, sizeof(g_phase_ticks));

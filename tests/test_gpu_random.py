@@ -1,0 +1,78 @@
+"""Randomised GPU parity: many small seeded cases of the ordering kernel and of the fused evict+restore
+kernel, with sizes and shapes drawn at random (ragged tails, tiny chunks, overlapping block reuse)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_06557_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def test_ordering_of_random_keys_and_sizes():
+    import torch
+    from paper_2608_06557_b200.runner import Instance
+    rng = np.random.default_rng(123)
+    w = wl.config_llama8b(seed=1, n=65536, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9)
+    w.hbm_tbl = w.host_tbl = w.hbm_free = w.host_free = None
+    w.hbm_free_count, w.host_free_count = 1 << 30, 1 << 30
+    inst = Instance(w, alloc_pools=False)
+    sizes = [1, 2, 33, 255, 256, 257, 1000, 1024, 1025, 2048, 3000, 4096, 4097, 8192, 10000, 16384, 16385, 30000,
+             32768, 50000, 65536]
+    for trial in range(300):
+        n = int(rng.choice(sizes))
+        mode = trial % 4
+        if mode == 0:
+            key = rng.integers(0, 1 << 63, n, dtype=np.int64).astype(np.uint64) * np.uint64(2) \
+                + rng.integers(0, 2, n).astype(np.uint64)
+        elif mode == 1:     # few distinct values in one digit: most passes are skipped, ties keep slot order
+            key = rng.integers(0, 16, n).astype(np.uint64) << np.uint64(int(rng.integers(0, 60)))
+        elif mode == 2:     # reverse sorted
+            key = np.sort(rng.integers(0, 1 << 62, n, dtype=np.int64)).astype(np.uint64)[::-1].copy()
+        else:               # the library's own key shape: 40-bit value, 23-bit id
+            key = (rng.integers(0, 1 << 40, n, dtype=np.int64).astype(np.uint64) << np.uint64(23)) \
+                | np.arange(n, dtype=np.uint64)
+        inst.n = n
+        inst.key.view(torch.int64)[:n].copy_(torch.from_numpy(key.view(np.int64)))
+        inst.ctx.schedule(inst.reqs_struct, inst.key, n, w.D_act, inst.order, inst.grant, inst.sched_counts)
+        torch.cuda.synchronize()
+        assert np.array_equal(inst.order[:n].cpu().numpy(), np.argsort(key, kind="stable")), (trial, n, mode)
+    assert inst.ctx.status()[0] == 0
+
+
+def test_fused_move_on_random_shapes():
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    rng = np.random.default_rng(7)
+    ctx = cs.Context(wl.default_params(), 16, 0)
+    done = 0
+    while done < 120:
+        n_hbm, n_host = int(rng.integers(8, 300)), int(rng.integers(8, 300))
+        n_chunks = int(rng.choice([1, 3, 8, 64]))
+        cb = int(rng.choice([16, 48, 4096, 32768, 32768 + 16]))
+        if n_chunks * cb * (n_hbm + n_host) > 300e6:
+            continue
+        lay = wl.kv_layout(n_hbm, n_chunks, cb)
+        bb = n_chunks * cb
+        hbm_np = rng.integers(0, 256, n_hbm * bb, dtype=np.uint8)
+        host_np = rng.integers(0, 256, n_host * bb, dtype=np.uint8)
+        ne = int(rng.integers(0, min(n_hbm, n_host) // 2 + 1))
+        nr = int(rng.integers(0, min(n_hbm, n_host) // 2 + 1))
+        hp, op = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_host).astype(np.int32)
+        es, ed, rs = hp[:ne], op[:ne], op[ne:ne + nr]
+        k = int(rng.integers(0, min(ne, nr) + 1))          # restores that land in blocks evicted by the same call
+        rd = rng.permutation(np.concatenate([rng.permutation(es)[:k], hp[ne:ne + nr - k]])).astype(np.int32)
+        ref_h, ref_o = hbm_np.copy(), host_np.copy()
+        assert oracle.kv_evict(ref_h, lay, ref_o, n_host, es, ed) == 0
+        assert oracle.kv_restore(ref_h, lay, ref_o, n_host, rs, rd) == 0
+        hbm = torch.from_numpy(hbm_np).cuda()
+        host = torch.from_numpy(host_np).pin_memory()
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda() if len(a) else \
+            torch.zeros(1, dtype=torch.int32, device="cuda")
+        scratch = torch.empty(ne + nr + 1, dtype=torch.int32, device="cuda")
+        ctx.kv_move(cs.make_layout(lay), hbm, host, n_host, t(es), t(ed), None, ne, t(rs), t(rd), None, nr, scratch)
+        torch.cuda.synchronize()
+        assert np.array_equal(hbm.cpu().numpy(), ref_h), (n_hbm, n_host, n_chunks, cb, ne, nr, k)
+        assert np.array_equal(host.numpy(), ref_o), (n_hbm, n_host, n_chunks, cb, ne, nr, k)
+        done += 1
+    assert ctx.status()[0] == 0

@@ -297,3 +297,82 @@ def kv_evict(hbm_pool: np.ndarray, layout: dict, host_pool: np.ndarray, host_blo
     return int(lib().orc_kv_evict(_ptr(hbm_pool, C.c_uint8), *_layout_args(layout), _ptr(host_pool, C.c_uint8),
                                   C.c_int64(host_blocks), _ptr(src, C.c_int32), _ptr(dst, C.c_int32),
                                   C.c_int(len(src))))
+
+
+class OrcStageCounts(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("n_stage", "n_requests", "n_short", "host_free_after")] + \
+               [("link_ns_left", C.c_int64)]
+
+
+def stage_plan(p: OrcParams, reqs: dict, budget_: np.ndarray, order: np.ndarray, action: np.ndarray, D_act: int,
+               K_act: int, link_budget_ns: int, host_reserve: int, pools: Pools, deep_tbl: np.ndarray | None,
+               stage_cap: int):
+    """First hop of the deep-tier path.  ``pools.host_tbl`` and the host free count are updated in place.
+    Returns a dict with staged (blocks per slot), stage_src/dst (trimmed), counts and status bits."""
+    n = len(reqs["prompt"])
+    a = {k: _arr(reqs[k], np.int32) for k in ("prompt", "n0", "n1", "n2")}
+    with_tables = pools.host_tbl is not None
+    maxb = pools.host_tbl.shape[1] if with_tables else 0
+    ss = np.full(max(stage_cap, 1), -1, np.int32)
+    sd = np.full(max(stage_cap, 1), -1, np.int32)
+    staged = np.empty(n, np.int32)
+    oc = C.c_int32(pools.host_free_count)
+    cnt = OrcStageCounts()
+    lib().orc_stage_plan.restype = C.c_uint32
+    st = lib().orc_stage_plan(
+        C.byref(p), C.c_int(n), _ptr(a["prompt"], C.c_int32), _ptr(a["n0"], C.c_int32), _ptr(a["n1"], C.c_int32),
+        _ptr(a["n2"], C.c_int32), _ptr(_arr(budget_, np.int64), C.c_int64), _ptr(_arr(order, np.uint32), C.c_uint32),
+        _ptr(_arr(action, np.uint8), C.c_uint8), C.c_int32(D_act), C.c_int64(K_act), C.c_int64(link_budget_ns),
+        C.c_int32(host_reserve), _ptr(pools.host_tbl, C.c_int32), _ptr(deep_tbl, C.c_int32), C.c_int32(maxb),
+        _ptr(pools.host_free, C.c_int32), C.byref(oc),
+        C.c_int32(0 if pools.host_free is None else len(pools.host_free)), _ptr(ss, C.c_int32), _ptr(sd, C.c_int32),
+        C.c_int32(stage_cap), _ptr(staged, C.c_int32), C.byref(cnt))
+    pools.host_free_count = int(oc.value)
+    counts = {k: int(getattr(cnt, k)) for k, _ in OrcStageCounts._fields_}
+    ns = min(counts["n_stage"], stage_cap)
+    return dict(staged=staged, stage_src=ss[:ns], stage_dst=sd[:ns], counts=counts, status=int(st))
+
+
+class OrcDedupCounts(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("n_in", "n_unique", "n_surplus", "n_shared_requests", "max_share",
+                                         "free_after")]
+
+
+def dedup(lo_a, lo_b, len_a, len_b, src_tbl: np.ndarray, dst_tbl: np.ndarray, list_src, list_dst, list_count: int,
+          n_src_ids: int, n_dst_ids: int, free_list: np.ndarray, free_count: int, ref: np.ndarray):
+    """One copy per distinct source block.  ``dst_tbl``, ``free_list`` and ``ref`` are updated in place.
+    Returns a dict with out_src/out_dst (trimmed), shared (per slot), free_count, counts and status bits."""
+    n, maxb = src_tbl.shape
+    assert dst_tbl.shape == src_tbl.shape and dst_tbl.dtype == np.int32 and dst_tbl.flags["C_CONTIGUOUS"]
+    assert free_list.dtype == np.int32 and ref.dtype == np.int32
+    ls, ld = _arr(list_src, np.int32), _arr(list_dst, np.int32)
+    cap = len(ls)
+    os_ = np.full(max(cap, 1), -1, np.int32)
+    od = np.full(max(cap, 1), -1, np.int32)
+    shared = np.empty(n, np.uint8)
+    fc = C.c_int32(free_count)
+    cnt = OrcDedupCounts()
+    lib().orc_dedup.restype = C.c_uint32
+    st = lib().orc_dedup(
+        C.c_int(n), _ptr(_arr(lo_a, np.int32), C.c_int32), _ptr(None if lo_b is None else _arr(lo_b, np.int32), C.c_int32),
+        _ptr(_arr(len_a, np.int32), C.c_int32), _ptr(None if len_b is None else _arr(len_b, np.int32), C.c_int32),
+        _ptr(_arr(src_tbl, np.int32), C.c_int32), _ptr(dst_tbl, C.c_int32), C.c_int32(maxb), _ptr(ls, C.c_int32),
+        _ptr(ld, C.c_int32), C.c_int32(list_count), C.c_int32(cap), _ptr(os_, C.c_int32), _ptr(od, C.c_int32),
+        C.c_int32(n_src_ids), C.c_int32(n_dst_ids), _ptr(free_list, C.c_int32), C.byref(fc),
+        C.c_int32(len(free_list)), _ptr(ref, C.c_int32), _ptr(shared, C.c_uint8), C.byref(cnt))
+    counts = {k: int(getattr(cnt, k)) for k, _ in OrcDedupCounts._fields_}
+    nu = counts["n_unique"]
+    return dict(out_src=os_[:nu], out_dst=od[:nu], shared=shared, free_count=int(fc.value), counts=counts,
+                status=int(st))
+
+
+def kv_stage(deep_pool: np.ndarray, deep_blocks: int, host_pool: np.ndarray, host_blocks: int, block_bytes: int,
+             src_ids: np.ndarray, dst_ids: np.ndarray) -> int:
+    """Deep-tier record -> host record (both pools record-major)."""
+    src = _arr(src_ids, np.int32)
+    dst = _arr(dst_ids, np.int32)
+    assert deep_pool.dtype == np.uint8 and host_pool.dtype == np.uint8
+    lib().orc_kv_stage.restype = C.c_uint32
+    return int(lib().orc_kv_stage(_ptr(deep_pool, C.c_uint8), C.c_int64(deep_blocks), _ptr(host_pool, C.c_uint8),
+                                  C.c_int64(host_blocks), C.c_int64(block_bytes), _ptr(src, C.c_int32),
+                                  _ptr(dst, C.c_int32), C.c_int(len(src))))

@@ -541,6 +541,161 @@ uint32_t orc_prefetch_plan(const orc_params *p, int n, const int32_t *prompt, co
     return status;
 }
 
+/* First hop of P(2): deep tier -> host DRAM.  Walking the order, every valid request that this
+ * iteration's plan did not preempt and whose own restore choice (Eq. 7 bounds, then the cheapest
+ * candidate, from its budget) contains a deep fetch x2 > 0 gets host records for its first x2 deep
+ * blocks while the deep link's time budget and the host pool (above a reserve) last.  One hop costs
+ * what P(2) adds to P(1) in Eq. 6.  HBM is not touched ("allocated only at the final hop"): the
+ * staged blocks become host blocks of the request and a later iteration restores them. */
+uint32_t orc_stage_plan(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
+                        const int32_t *n2, const int64_t *budget, const uint32_t *order, const uint8_t *action,
+                        int32_t D_act, int64_t K_act, int64_t link_budget_ns, int32_t host_reserve,
+                        int32_t *host_tbl, const int32_t *deep_tbl, int32_t maxb, const int32_t *host_free,
+                        int32_t *host_free_count, int32_t host_free_cap, int32_t *stage_src, int32_t *stage_dst,
+                        int32_t stage_cap, int32_t *staged_out, orc_stage_counts *counts) {
+    uint32_t status = 0;
+    const bool with_tables = host_tbl != nullptr;
+    const Load act = load_act(D_act, K_act);
+    int64_t host_pos = *host_free_count;
+    if (with_tables && (host_pos < 0 || host_pos > host_free_cap)) {
+        status |= ORC_ST_EBOUNDS;
+        host_pos = std::min<int64_t>(std::max<int64_t>(host_pos, 0), host_free_cap);
+    }
+    const int64_t hop_delta = std::max<int64_t>(0, p->delta_ns[2] - p->delta_ns[1]);
+    const int64_t hop_blk = std::max<int64_t>(1, p->blk_ns[2] - p->blk_ns[1]);
+    int64_t room = host_pos - host_reserve;
+    int64_t link_left = link_budget_ns;
+    int32_t n_stage = 0, n_req = 0, n_short = 0;
+    for (int r = 0; r < n; ++r) staged_out[r] = 0;
+    for (int i = 0; i < n; ++i) {
+        const uint32_t r = order[i];
+        bool ok = request_valid(p, prompt[r], n0[r], n1[r], n2[r]);
+        if (ok && with_tables) ok = ceil_div(prompt[r], p->bt) <= maxb;
+        if (!ok || n2[r] <= 0) continue;
+        const bool preempted = action[r] == ORC_ACT_EVICT || action[r] == ORC_ACT_DROP;
+        if (preempted) continue;
+        int64_t bx1, bx2;
+        choose_restore(p, act, prompt[r], n0[r], n1[r], n2[r], budget[r], &bx1, &bx2);
+        if (bx2 <= 0) continue;
+        const int64_t by_link = link_left > hop_delta ? (link_left - hop_delta) / hop_blk : 0;
+        const int64_t b = std::min(bx2, std::min(by_link, std::max<int64_t>(room, 0)));
+        if (b < bx2) ++n_short;
+        if (b <= 0) continue;
+        link_left -= hop_delta + b * hop_blk;
+        room -= b;
+        staged_out[r] = int32_t(b);
+        ++n_req;
+        for (int64_t j = 0; j < b; ++j) {
+            --host_pos;
+            if (with_tables) {
+                const int64_t t = int64_t(r) * maxb + n0[r] + n1[r] + j;
+                const int32_t rec = host_pos < host_free_cap ? host_free[host_pos] : -1;
+                if (n_stage < stage_cap) { stage_src[n_stage] = deep_tbl[t]; stage_dst[n_stage] = rec; }
+                else status |= ORC_ST_ELISTCAP;
+                host_tbl[t] = rec;
+            }
+            ++n_stage;
+        }
+    }
+    if (with_tables) *host_free_count = int32_t(host_pos);
+    counts->n_stage = n_stage;
+    counts->n_requests = n_req;
+    counts->n_short = n_short;
+    counts->host_free_after = int32_t(host_pos);
+    counts->link_ns_left = link_left;
+    return status;
+}
+
+/* One copy per distinct source block of a copy list (shared prefixes restored or staged by several
+ * requests in one iteration). */
+uint32_t orc_dedup(int n, const int32_t *lo_a, const int32_t *lo_b, const int32_t *len_a, const int32_t *len_b,
+                   const int32_t *src_tbl, int32_t *dst_tbl, int32_t maxb, const int32_t *list_src,
+                   const int32_t *list_dst, int32_t list_count, int32_t list_cap, int32_t *out_src, int32_t *out_dst,
+                   int32_t n_src_ids, int32_t n_dst_ids, int32_t *free_list, int32_t *free_count, int32_t free_cap,
+                   int32_t *ref, uint8_t *shared_out, orc_dedup_counts *counts) {
+    uint32_t status = 0;
+    int64_t m = list_count;
+    if (m < 0 || m > list_cap) {
+        if (m < 0) status |= ORC_ST_EBOUNDS;   /* a count above the capacity is a list the producer already cut */
+        m = std::min<int64_t>(std::max<int64_t>(m, 0), list_cap);
+    }
+    int64_t fpos = *free_count;
+    if (fpos < 0 || fpos > free_cap) {
+        status |= ORC_ST_EBOUNDS;
+        fpos = std::min<int64_t>(std::max<int64_t>(fpos, 0), free_cap);
+    }
+    /* kept[s] = destination of the first entry with source s; merged[s] = entries with source s */
+    std::vector<int32_t> kept(size_t(std::max(n_src_ids, 0)), -1), merged(size_t(std::max(n_src_ids, 0)), 0);
+    int32_t n_unique = 0, n_surplus = 0, max_share = 0;
+    for (int64_t i = 0; i < m; ++i) {
+        const int32_t s = list_src[i], d = list_dst[i];
+        if (s < 0 || s >= n_src_ids || d < 0 || d >= n_dst_ids) {
+            status |= ORC_ST_EBOUNDS;
+            out_src[n_unique] = s;
+            out_dst[n_unique] = d;
+            ++n_unique;
+            continue;
+        }
+        if (merged[s] == 0) {
+            kept[s] = d;
+            out_src[n_unique] = s;
+            out_dst[n_unique] = d;
+            ++n_unique;
+        } else {
+            if (fpos < free_cap) free_list[fpos] = d; else status |= ORC_ST_EBOUNDS;
+            ++fpos;
+            ++n_surplus;
+        }
+        ++merged[s];
+    }
+    for (int64_t i = 0; i < m; ++i) {
+        const int32_t s = list_src[i];
+        if (s < 0 || s >= n_src_ids || kept[s] < 0) continue;
+        ref[kept[s]] = merged[s];
+        max_share = std::max(max_share, merged[s]);
+    }
+    int32_t n_shared = 0;
+    for (int r = 0; r < n; ++r) {
+        const int64_t lo = int64_t(lo_a[r]) + (lo_b ? lo_b[r] : 0);
+        const int64_t len = int64_t(len_a[r]) + (len_b ? len_b[r] : 0);
+        uint8_t shared = 0;
+        if (lo >= 0 && len > 0 && lo + len <= maxb) {
+            for (int64_t j = lo; j < lo + len; ++j) {
+                const int32_t s = src_tbl[int64_t(r) * maxb + j];
+                if (s < 0 || s >= n_src_ids || merged[s] == 0) continue;
+                dst_tbl[int64_t(r) * maxb + j] = kept[s];
+                if (merged[s] > 1) shared = 1;
+            }
+        } else if (len > 0) {
+            status |= ORC_ST_EPRECOND;
+        }
+        shared_out[r] = shared;
+        n_shared += shared;
+    }
+    *free_count = int32_t(fpos);
+    counts->n_in = int32_t(m);
+    counts->n_unique = n_unique;
+    counts->n_surplus = n_surplus;
+    counts->n_shared_requests = n_shared;
+    counts->max_share = max_share;
+    counts->free_after = int32_t(fpos);
+    return status;
+}
+
+uint32_t orc_kv_stage(const uint8_t *deep_pool, int64_t deep_blocks, uint8_t *host_pool, int64_t host_blocks,
+                      int64_t block_bytes, const int32_t *src_ids, const int32_t *dst_ids, int n_copies) {
+    uint32_t status = 0;
+    for (int i = 0; i < n_copies; ++i) {
+        const int64_t s = src_ids[i], d = dst_ids[i];
+        if (s < 0 || s >= deep_blocks || d < 0 || d >= host_blocks) {
+            status |= ORC_ST_EBOUNDS;
+            continue;
+        }
+        std::memcpy(host_pool + d * block_bytes, deep_pool + s * block_bytes, size_t(block_bytes));
+    }
+    return status;
+}
+
 uint32_t orc_kv_restore(uint8_t *hbm_pool, int64_t hbm_blocks, int32_t n_chunks, int64_t chunk_bytes,
                         int64_t chunk_stride, int64_t block_stride, const uint8_t *host_pool, int64_t host_blocks,
                         const int32_t *src_ids, const int32_t *dst_ids, int n_copies) {

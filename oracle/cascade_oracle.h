@@ -141,6 +141,50 @@ uint32_t orc_prefetch_plan(const orc_params *p, int n, const int32_t *prompt, co
                            int32_t *restore_src, int32_t *restore_dst, int32_t restore_cap, int32_t *n_restore,
                            int32_t *pf_out, orc_prefetch_counts *counts);
 
+/* counts written by orc_stage_plan */
+typedef struct orc_stage_counts {
+    int32_t n_stage;         /* entries of the stage list (blocks)                          */
+    int32_t n_requests;      /* requests that staged at least one block                     */
+    int32_t n_short;         /* requests that got fewer blocks than their choice asked for  */
+    int32_t host_free_after; /* host free-list length afterwards                            */
+    int64_t link_ns_left;    /* deep-link time left                                         */
+} orc_stage_counts;
+
+/* First hop of the two-hop path P(2) (deep tier -> host DRAM -> HBM), see the .cpp.
+ * Tables NULL = counts and staged_out only. */
+uint32_t orc_stage_plan(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
+                        const int32_t *n2, const int64_t *budget, const uint32_t *order, const uint8_t *action,
+                        int32_t D_act, int64_t K_act, int64_t link_budget_ns, int32_t host_reserve,
+                        int32_t *host_tbl, const int32_t *deep_tbl, int32_t maxb, const int32_t *host_free,
+                        int32_t *host_free_count, int32_t host_free_cap, int32_t *stage_src, int32_t *stage_dst,
+                        int32_t stage_cap, int32_t *staged_out, orc_stage_counts *counts);
+
+/* counts written by orc_dedup */
+typedef struct orc_dedup_counts {
+    int32_t n_in;              /* list entries read                                         */
+    int32_t n_unique;          /* entries of the output list                                */
+    int32_t n_surplus;         /* destination ids handed back to the free list              */
+    int32_t n_shared_requests; /* slots with at least one block shared with another entry   */
+    int32_t max_share;         /* largest number of entries merged into one copy            */
+    int32_t free_after;        /* free-list length afterwards                               */
+} orc_dedup_counts;
+
+/* One copy per distinct source block.  The list (src[i], dst[i]) is read in order; the first entry
+ * of every source id is kept (output list, same relative order), each later entry gives its
+ * destination id back to the free list (pushed in list order) and every table cell in the ranges
+ * [lo[r], lo[r] + len[r]) whose source id has a kept entry is pointed at that entry's destination.
+ * ref[d] = number of entries merged into destination d, shared_out[r] = 1 if any cell of r's range
+ * is merged with another entry.  Entries with an id outside its pool are kept untouched (EBOUNDS). */
+uint32_t orc_dedup(int n, const int32_t *lo_a, const int32_t *lo_b, const int32_t *len_a, const int32_t *len_b,
+                   const int32_t *src_tbl, int32_t *dst_tbl, int32_t maxb, const int32_t *list_src,
+                   const int32_t *list_dst, int32_t list_count, int32_t list_cap, int32_t *out_src, int32_t *out_dst,
+                   int32_t n_src_ids, int32_t n_dst_ids, int32_t *free_list, int32_t *free_count, int32_t free_cap,
+                   int32_t *ref, uint8_t *shared_out, orc_dedup_counts *counts);
+
+/* Record-major pool to record-major pool (deep tier -> host DRAM), one record per list entry. */
+uint32_t orc_kv_stage(const uint8_t *deep_pool, int64_t deep_blocks, uint8_t *host_pool, int64_t host_blocks,
+                      int64_t block_bytes, const int32_t *src_ids, const int32_t *dst_ids, int n_copies);
+
 /* Step K2: paged copies.  HBM pool: chunk c of block b starts at
  * c*chunk_stride + b*block_stride.  Host pool: record h starts at h*n_chunks*chunk_bytes,
  * its chunks stored back to back.  Ids outside a pool are skipped and flagged. */

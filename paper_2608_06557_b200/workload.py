@@ -75,6 +75,8 @@ class Workload:
     host_free: np.ndarray | None = None
     host_free_count: int = 0
     notes: dict = field(default_factory=dict)
+    deep_tbl: np.ndarray | None = None   # int32 [n, maxb]: deep-tier record of table positions n0+n1 .. n0+n1+n2
+    deep_blocks: int = 0
 
     @property
     def n(self) -> int:
@@ -165,6 +167,92 @@ def config_tiny(seed: int = 0, hbm_free_target: int = 32) -> Workload:
     maxb = 128
     tbl = place_blocks(rng, reqs, 512, 512, maxb, 1.0, hbm_free_target, 0.5)
     return Workload("tiny", params, reqs, now, 8, 8 * 512, kv_layout(512, n_chunks, chunk_bytes), 512, maxb, *tbl)
+
+
+def config_deep_shared(seed: int = 0, n: int = 256, n_hbm: int = 4096, n_host: int = 4096, n_deep: int = 8192,
+                       group_frac: float = 0.4, hbm_free_target: int = 2048, host_free_target: int = 1 << 30,
+                       n_chunks: int = 4, chunk_bytes: int = 4096) -> Workload:
+    """Matched prefixes that reach into the deep tier, with shared prefixes.
+
+    Every request reuses a uniform fraction of its prompt, split 30 % HBM / 35 % host / 35 % deep tier (head
+    to tail).  ``group_frac`` of the requests form prefix groups of 2 to 6: a group's members hold nothing in
+    HBM, and their host and deep table cells hold the SAME record ids as the group leader's over the length
+    they share with it (a member's match may stop anywhere inside the leader's)."""
+    rng = np.random.default_rng(seed)
+    ttft = [2 * S, 20 * S]
+    params = default_params(ttft_ns=ttft, tpot_ns=[50 * MS, 50 * MS], token_budget=4096, tier2_reserve=512,
+                            max_batch=128)
+    bb = n_chunks * chunk_bytes
+    host_blk = -(-bb * 1_000_000_000 // 50_000_000_000)
+    params["blk_ns"] = [0, host_blk, host_blk + 20_000]
+    params["delta_ns"] = [0, 10_000, 110_000]
+    bt = params["bt"]
+    now = 50 * S
+    reqs = draw_requests(rng, n, [0.5, 0.5], ttft, 512, (32, 4096), [128, 128], (1, 4096), now, 0.5,
+                         lambda g, m: g.uniform(0, 1, m), 0.3, bt)
+    hit = reqs["n0"] + reqs["n1"]
+    n0 = np.ceil(hit * 0.3).astype(np.int32)
+    n1 = np.ceil((hit - n0) * 0.5).astype(np.int32)
+    n2 = (hit - n0 - n1).astype(np.int32)
+    prompt = reqs["prompt"]
+    maxb = 4096 // bt + 8
+    hbm_ids = rng.permutation(n_hbm).astype(np.int32)
+    host_ids = rng.permutation(n_host).astype(np.int32)
+    deep_ids = rng.permutation(n_deep).astype(np.int32)
+    hbm_tbl = np.full((n, maxb), -1, np.int32)
+    host_tbl = np.full((n, maxb), -1, np.int32)
+    deep_tbl = np.full((n, maxb), -1, np.int32)
+    # prefix groups: consecutive runs of a random permutation
+    perm = rng.permutation(n)
+    grouped = perm[: int(n * group_frac)]
+    leader = np.full(n, -1, np.int64)
+    i = 0
+    while i < len(grouped):
+        size = int(rng.integers(2, 7))
+        members = grouped[i:i + size]
+        i += size
+        if len(members) < 2:
+            break
+        lead = members[np.argmax(prompt[members])]      # the longest prompt leads: its match covers the others'
+        leader[members] = lead
+    hbm_used = host_used = deep_used = 0
+    order = np.argsort(np.where(leader == np.arange(n), 0, 1), kind="stable")   # leaders first
+    for r in order:
+        ld = leader[r]
+        if ld >= 0:
+            n0[r] = 0
+        if ld >= 0 and ld != r:
+            # match a prefix of the leader's blocks: m blocks, first its host part, then its deep part
+            m = int(min(rng.integers(1, n1[ld] + n2[ld] + 1) if n1[ld] + n2[ld] > 0 else 0, (prompt[r] - 1) // bt))
+            n1[r] = min(m, n1[ld])
+            n2[r] = m - n1[r]
+            if n2[r] > 0 and n1[r] < n1[ld]:
+                n2[r] = 0
+            host_tbl[r, : n1[r]] = host_tbl[ld, : n1[r]]
+            deep_tbl[r, n1[r]: n1[r] + n2[r]] = deep_tbl[ld, n1[ld]: n1[ld] + n2[r]]
+            continue
+        a, b, c = int(n0[r]), int(n1[r]), int(n2[r])
+        if hbm_used + a > n_hbm or host_used + b > n_host or deep_used + c > n_deep:
+            n0[r] = n1[r] = n2[r] = 0
+            continue
+        hbm_tbl[r, :a] = hbm_ids[hbm_used:hbm_used + a]
+        host_tbl[r, a:a + b] = host_ids[host_used:host_used + b]
+        deep_tbl[r, a + b:a + b + c] = deep_ids[deep_used:deep_used + c]
+        hbm_used, host_used, deep_used = hbm_used + a, host_used + b, deep_used + c
+    reqs["n0"], reqs["n1"], reqs["n2"] = n0, n1, n2
+    private = (n0 > 0) & (rng.uniform(0, 1, n) < 0.5)
+    reqs["flags"][private] |= FLAG_HBM_PRIVATE | FLAG_RUNNING
+    hbm_free_count = min(n_hbm - hbm_used, hbm_free_target)
+    hbm_free = np.full(n_hbm, -1, np.int32)
+    hbm_free[:hbm_free_count] = hbm_ids[n_hbm - hbm_free_count:]
+    host_free_count = min(n_host - host_used, host_free_target)
+    host_free = np.full(n_host, -1, np.int32)
+    host_free[:host_free_count] = host_ids[n_host - host_free_count:]
+    w = Workload("deep_shared", params, reqs, now, 8, 8 * 512, kv_layout(n_hbm, n_chunks, chunk_bytes), n_host, maxb,
+                 hbm_tbl, host_tbl, hbm_free, hbm_free_count, host_free, host_free_count)
+    w.deep_tbl, w.deep_blocks = deep_tbl, n_deep
+    w.notes["leader"] = leader
+    return w
 
 
 LLAMA8B_CLASSES = dict(mix=[0.6, 0.3, 0.1], ttft=[1 * S, 3 * S, 30 * S], out_median=[256, 256, 4096])

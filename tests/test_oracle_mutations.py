@@ -11,6 +11,8 @@ SRC = os.path.join(ROOT, "oracle", "cascade_oracle.cpp")
 PINS = ["test_oracle_plan_first.py", "test_oracle_budget.py", "test_oracle_schedule.py", "test_oracle_plan.py", "test_oracle_copy.py",
         "test_oracle_prefetch.py", "test_oracle_policies.py"]
 
+DEEP_PINS = ["test_oracle_deep.py"]
+
 MUTATIONS = [
     ("eq3 drops the one half", "const int64_t L = ((L_act + L_max) * p->gamma_q16) >> 17;",
      "const int64_t L = ((L_act + L_max) * p->gamma_q16) >> 16;"),
@@ -62,32 +64,57 @@ MUTATIONS = [
      "want[r] = int64_t(prompt[r]) - (n0[r] + x1) * p->bt;"),
     ("regime 1 reuses the prefix", "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, 0) >> 20;",
      "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, s_hit) >> 20;"),
+    # the deep-tier stage, the one-copy-per-source pass and the record copy have pins of their own
+    ("stage hop charged the whole path", "std::max<int64_t>(0, p->delta_ns[2] - p->delta_ns[1]);",
+     "std::max<int64_t>(0, p->delta_ns[2]);", DEEP_PINS),
+    ("stage hop per block charged the whole path", "std::max<int64_t>(1, p->blk_ns[2] - p->blk_ns[1]);",
+     "std::max<int64_t>(1, p->blk_ns[2]);", DEEP_PINS),
+    ("stage ignores the host reserve", "int64_t room = host_pos - host_reserve;", "int64_t room = host_pos;", DEEP_PINS),
+    ("stage writes the host segment's cells", "const int64_t t = int64_t(r) * maxb + n0[r] + n1[r] + j;",
+     "const int64_t t = int64_t(r) * maxb + n0[r] + j;", DEEP_PINS),
+    ("stage list swapped", "stage_src[n_stage] = deep_tbl[t]; stage_dst[n_stage] = rec;",
+     "stage_src[n_stage] = rec; stage_dst[n_stage] = deep_tbl[t];", DEEP_PINS),
+    ("stage serves preempted requests", "if (preempted) continue;", "", DEEP_PINS),
+    ("stage forgets the per-transfer overhead", "link_left -= hop_delta + b * hop_blk;", "link_left -= b * hop_blk;",
+     DEEP_PINS),
+    ("stage takes the deep fetch although the host segment is cut", "if (bx2 <= 0) continue;",
+     "bx2 = std::max<int64_t>(bx2, bx1 < n1[r] ? 1 : bx2); if (bx2 <= 0) continue;", DEEP_PINS),
+    ("merged copy frees the kept block", "if (fpos < free_cap) free_list[fpos] = d; else status |= ORC_ST_EBOUNDS;",
+     "if (fpos < free_cap) free_list[fpos] = kept[s]; else status |= ORC_ST_EBOUNDS;", DEEP_PINS),
+    ("share count off by one", "ref[kept[s]] = merged[s];", "ref[kept[s]] = merged[s] - 1;", DEEP_PINS),
+    ("every merged cell counts as shared", "if (merged[s] > 1) shared = 1;", "if (merged[s] >= 1) shared = 1;", DEEP_PINS),
+    ("merged cells keep their own block", "dst_tbl[int64_t(r) * maxb + j] = kept[s];", "", DEEP_PINS),
+    ("record copy the wrong way", "std::memcpy(host_pool + d * block_bytes, deep_pool + s * block_bytes, size_t(block_bytes));",
+     "std::memcpy(host_pool + s * block_bytes, deep_pool + d * block_bytes, size_t(block_bytes));", DEEP_PINS),
 ]
 
 
-def run_pins(env):
-    cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider"] + [os.path.join(ROOT, "tests", f) for f in PINS]
+def run_pins(env, pins=None):
+    cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider"] + [os.path.join(ROOT, "tests", f) for f in pins or PINS]
     return subprocess.run(cmd, env=env, cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
 
 
 def test_every_planted_slip_is_caught(tmp_path):
+    from concurrent.futures import ThreadPoolExecutor
     text = open(SRC).read()
-    survivors = []
-    for i, (name, old, new) in enumerate(MUTATIONS):
+
+    def survives(item):
+        i, (name, old, new, *pins) = item
         assert text.count(old) == 1, f"mutation '{name}' no longer matches the source exactly once"
         path = tmp_path / f"mutant_{i}.cpp"
         path.write_text(text.replace(old, new))
         env = dict(os.environ, CASCADE_ORACLE_SRC=str(path))
-        res = run_pins(env)
-        if res.returncode == 0:
-            survivors.append(name)
+        return name if run_pins(env, pins[0] if pins else None).returncode == 0 else None
+
+    with ThreadPoolExecutor(max_workers=max(1, min(8, (os.cpu_count() or 2) // 2))) as pool:
+        survivors = [s for s in pool.map(survives, enumerate(MUTATIONS)) if s]
     assert not survivors, f"pins did not notice: {survivors}"
 
 
 def test_the_unaltered_copy_passes(tmp_path):
     path = tmp_path / "copy.cpp"
     path.write_text(open(SRC).read())
-    res = run_pins(dict(os.environ, CASCADE_ORACLE_SRC=str(path)))
+    res = run_pins(dict(os.environ, CASCADE_ORACLE_SRC=str(path)), PINS + DEEP_PINS)
     assert res.returncode == 0, res.stdout[-2000:]
 
 
@@ -98,5 +125,5 @@ def test_pins_pass_under_the_undefined_behaviour_sanitizer(tmp_path):
     path.write_text(open(SRC).read())
     env = dict(os.environ, CASCADE_ORACLE_SRC=str(path),
                CASCADE_ORACLE_CXXFLAGS="-fsanitize=undefined -fno-sanitize-recover=all -g")
-    res = run_pins(env)
+    res = run_pins(env, PINS + DEEP_PINS)
     assert res.returncode == 0, res.stdout[-3000:]

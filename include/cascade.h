@@ -343,6 +343,118 @@ int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_po
                     const int32_t *restore_dst, const int32_t *n_restore_dev, int n_restore_max, int32_t *scratch,
                     void *stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * Deep tier as a real stage, and one copy per shared block.
+ *
+ * Section "Memory management and HBM allocation": a deep-tier hit travels deep tier -> host DRAM -> HBM
+ * (path P(2) of Eq. 6) and HBM is taken only at the last hop.  Here the first hop is a plan step of its
+ * own (cascade_stage_plan) with a copy (cascade_kv_stage); the staged blocks become host blocks of the
+ * request and the ordinary restore path of a later iteration is the last hop.  Section "Prefix hit
+ * detection": several requests can match the same cached blocks; cascade_dedup makes a copy list carry
+ * each such block once and counts the sharers.
+ * ------------------------------------------------------------------------------------------------- */
+
+/* written to device memory by cascade_stage_plan */
+typedef struct cascade_stage_counts {
+    int32_t n_stage;         /* entries of the stage list (blocks)                         */
+    int32_t n_requests;      /* requests that staged at least one block                    */
+    int32_t n_short;         /* requests that got fewer blocks than their choice asked for */
+    int32_t host_free_after; /* host free-list length afterwards                           */
+    int64_t link_ns_left;    /* deep-link time left                                        */
+} cascade_stage_counts;
+
+/* Inputs and outputs of cascade_stage_plan (host struct of device pointers). */
+typedef struct cascade_stage {
+    const int32_t *deep_tbl; /* [n][maxb]: deep_tbl[r][j] = deep-tier record of table position j, for
+                                j in [n0+n1, n0+n1+n2); NULL = counts and `staged` only              */
+    int32_t *stage_src;      /* deep-tier record ids, in schedule order                              */
+    int32_t *stage_dst;      /* host record ids                                                      */
+    int32_t stage_cap;
+    int32_t *staged;         /* [n]: blocks staged per slot                                          */
+    cascade_stage_counts *counts; /* device */
+} cascade_stage;
+
+/*
+ * First hop of the two-hop path P(2).  Call it after cascade_tier_plan (it reads `action`; the host free
+ * list must already reflect this iteration's evictions).  Walking `order`, every request that is valid,
+ * holds deep blocks (n2 > 0), was not preempted by this iteration's plan and whose own restore choice
+ * (the Eq. 7 bounds and the restore-vs-recompute comparison of cascade_tier_plan, from its budget alone)
+ * contains a deep fetch of x2 > 0 blocks gets
+ *     b = min(x2, blocks that still fit the deep link's time, host records free above host_reserve)
+ * where one hop of x blocks costs what P(2) adds to P(1) in Eq. 6:
+ *     max(0, delta_ns[2]-delta_ns[1]) + x * max(1, blk_ns[2]-blk_ns[1]),
+ * and uses up that time and b host records.  For each such block a host record is popped from
+ * pools->host_free, written to pools->host_tbl[r][n0+n1+j], and the pair (deep_tbl[r][n0+n1+j], record)
+ * is appended to the stage list; *pools->host_free_count is updated.  No HBM block, table or list is
+ * touched.  The caller folds `staged` into the next iteration's hit profile (n1 += staged, n2 -= staged).
+ * Admission does not matter: with plan_first = 1 a request that chooses a deep fetch asks for no tokens
+ * and stays queued while its blocks are staged.  0 <= link_budget_ns <= 2^50, host_reserve >= 0.
+ * Only pools->host_tbl, maxb, host_free, host_free_count and host_free_cap are used.
+ */
+int cascade_stage_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *budget, const uint32_t *order,
+                       const uint8_t *action, int n, int32_t D_act, int64_t K_act, int64_t link_budget_ns,
+                       int32_t host_reserve, const cascade_pools *pools, const cascade_stage *stage, void *stream);
+
+/*
+ * Stage copy: for i < count, copy deep-tier record src_ids[i] into host record dst_ids[i].  Both pools are
+ * record-major with records of block_bytes (a multiple of 16) and device-accessible: the deep pool is
+ * pinned, mapped host memory standing in for the storage tier, or device memory.  Count arguments as in
+ * cascade_kv_restore.  Ids outside a pool are skipped (CASCADE_ST_EBOUNDS).
+ */
+int cascade_kv_stage(cascade_ctx *ctx, const void *deep_pool, int64_t deep_blocks, void *host_pool,
+                     int64_t host_blocks, int64_t block_bytes, const int32_t *src_ids, const int32_t *dst_ids,
+                     const int32_t *n_copies_dev, int n_copies_max, void *stream);
+
+/* written to device memory by cascade_dedup */
+typedef struct cascade_dedup_counts {
+    int32_t n_in;              /* list entries read                                        */
+    int32_t n_unique;          /* entries of the output list                               */
+    int32_t n_surplus;         /* destination ids handed back to the free list             */
+    int32_t n_shared_requests; /* slots with at least one block shared with another entry  */
+    int32_t max_share;         /* largest number of entries merged into one copy           */
+    int32_t free_after;        /* free-list length afterwards                              */
+} cascade_dedup_counts;
+
+/* Arguments of cascade_dedup (host struct of device pointers). */
+typedef struct cascade_dedup_args {
+    const int32_t *lo_a, *lo_b;   /* [n] each, lo_b may be NULL: first table cell of slot r = lo_a[r] + lo_b[r] */
+    const int32_t *len_a, *len_b; /* [n] each, len_b may be NULL: number of cells = len_a[r] + len_b[r]          */
+    const int32_t *src_tbl;       /* [n][maxb] table holding the source ids of those cells                       */
+    int32_t *dst_tbl;             /* [n][maxb] table holding their destination ids (rewritten)                   */
+    int32_t maxb;
+    const int32_t *list_src, *list_dst; /* the copy list                                                         */
+    const int32_t *list_count;    /* device scalar: its length (a value above list_cap means list_cap)           */
+    int32_t list_cap;
+    int32_t *out_src, *out_dst;   /* the merged list, list_cap entries each; must not alias the input list       */
+    int32_t n_src_ids, n_dst_ids; /* sizes of the source and destination pools (ids are 0 .. size-1)             */
+    int32_t *free_list;           /* stack of free destination ids; surplus ids are pushed                       */
+    int32_t *free_count;          /* device scalar, updated                                                      */
+    int32_t free_cap;
+    int32_t *ref;                 /* [n_dst_ids]: ref[d] = entries merged into kept destination d (written)      */
+    uint8_t *shared;              /* [n]: 1 if a cell of the slot's range is shared with another entry           */
+    int32_t *scratch;             /* caller-owned, scratch_len int32; contents irrelevant before and after       */
+    int64_t scratch_len;          /* >= 2*n_src_ids + (list_cap + 1023)/1024 + 8                                 */
+    cascade_dedup_counts *counts; /* device */
+} cascade_dedup_args;
+
+/*
+ * One copy per distinct source block of a copy list: for shared prefixes that several requests restore
+ * (list = the tier plan's restore list, source table = host_tbl, destination table = hbm_tbl, free list =
+ * the HBM free list, cells [n0, n0 + x1 + prefetched)) or stage (list = the stage list, source table =
+ * deep_tbl, destination table = host_tbl, free list = the host free list, cells [n0+n1, n0+n1+staged)) in
+ * the same iteration.  Call it between the plan that wrote the list and the copy.
+ *   - The first entry of every source id is kept; out_src/out_dst hold the kept entries in their
+ *     original order and counts->n_unique their number (a device scalar usable as a copy count).
+ *   - Every later entry of that source hands its destination id back: pushed on free_list in list order.
+ *   - Every table cell in the slots' ranges whose source id has a kept entry is pointed at that entry's
+ *     destination; ref[destination] = number of entries merged; shared[r] says whether slot r now shares
+ *     a block (the caller then clears CASCADE_FLAG_HBM_PRIVATE for it: a shared block is never a victim).
+ *   - An entry with an id outside its pool is passed through unchanged (CASCADE_ST_EBOUNDS); a slot whose
+ *     range leaves its table row is skipped (CASCADE_ST_EPRECOND).
+ * Source ids index a direct-address table in `scratch` (no sort): the cost is linear in the list length.
+ */
+int cascade_dedup(cascade_ctx *ctx, const cascade_dedup_args *a, int n, void *stream);
+
 /* Waits for `stream`, copies the status word to *host_out and, if clear != 0, resets it. */
 int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream);
 

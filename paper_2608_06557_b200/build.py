@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcascade.so")
-SOURCES = ["api.cu", "budget.cu", "schedule.cu", "plan.cu", "prefetch.cu", "kvcopy.cu"]
+SOURCES = ["api.cu", "budget.cu", "schedule.cu", "plan.cu", "prefetch.cu", "deep.cu", "kvcopy.cu"]
 
 
 def sources():
@@ -20,7 +20,7 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "cluster_scan.cuh"),
+    deps = sources() + [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "cluster_scan.cuh"), os.path.join(CSRC, "mbarrier.cuh"),
                         os.path.join(ROOT, "include", "cascade.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 

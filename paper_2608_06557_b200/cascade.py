@@ -23,7 +23,8 @@ ACT_NONE, ACT_RETAIN, ACT_EVICT, ACT_DROP = 0, 1, 2, 3
 
 EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_budget", "cascade_schedule",
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
-           "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan", "cascade_kv_move")
+           "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan", "cascade_kv_move",
+           "cascade_stage_plan", "cascade_kv_stage", "cascade_dedup")
 
 
 class Params(C.Structure):
@@ -69,6 +70,45 @@ class Plan(C.Structure):
                 ("counts", C.c_void_p)]
 
 
+class StageCounts(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("n_stage", "n_requests", "n_short", "host_free_after")] + \
+               [("link_ns_left", C.c_int64)]
+
+
+class Stage(C.Structure):
+    _fields_ = [("deep_tbl", C.c_void_p), ("stage_src", C.c_void_p), ("stage_dst", C.c_void_p),
+                ("stage_cap", C.c_int32), ("staged", C.c_void_p), ("counts", C.c_void_p)]
+
+
+class DedupCounts(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("n_in", "n_unique", "n_surplus", "n_shared_requests", "max_share",
+                                         "free_after")]
+
+
+class DedupArgs(C.Structure):
+    _fields_ = [("lo_a", C.c_void_p), ("lo_b", C.c_void_p), ("len_a", C.c_void_p), ("len_b", C.c_void_p),
+                ("src_tbl", C.c_void_p), ("dst_tbl", C.c_void_p), ("maxb", C.c_int32),
+                ("list_src", C.c_void_p), ("list_dst", C.c_void_p), ("list_count", C.c_void_p),
+                ("list_cap", C.c_int32), ("out_src", C.c_void_p), ("out_dst", C.c_void_p),
+                ("n_src_ids", C.c_int32), ("n_dst_ids", C.c_int32), ("free_list", C.c_void_p),
+                ("free_count", C.c_void_p), ("free_cap", C.c_int32), ("ref", C.c_void_p), ("shared", C.c_void_p),
+                ("scratch", C.c_void_p), ("scratch_len", C.c_int64), ("counts", C.c_void_p)]
+
+
+def dedup_scratch_len(n_src_ids: int, list_cap: int) -> int:
+    """int32 entries cascade_dedup needs in its caller-owned scratch."""
+    return 2 * n_src_ids + (list_cap + 1023) // 1024 + 8
+
+
+def make_dedup_args(**kw) -> DedupArgs:
+    """DedupArgs from keyword arguments: tensors become device addresses, integers stay integers."""
+    a = DedupArgs()
+    for k, ctype in DedupArgs._fields_:
+        v = kw.get(k)
+        setattr(a, k, _p(v) if ctype is C.c_void_p else int(v))
+    return a
+
+
 class KvLayout(C.Structure):
     _fields_ = [("n_blocks", C.c_int64), ("n_chunks", C.c_int32), ("reserved", C.c_int32),
                 ("chunk_bytes", C.c_int64), ("chunk_stride", C.c_int64), ("block_stride", C.c_int64)]
@@ -100,6 +140,10 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_status.argtypes = [vp, C.POINTER(Status), C.c_int, vp]
     lib.cascade_kv_move.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int,
                                     vp, vp]
+    lib.cascade_stage_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64, i64, i32, C.POINTER(Pools),
+                                       C.POINTER(Stage), vp]
+    lib.cascade_kv_stage.argtypes = [vp, vp, i64, vp, i64, i64, vp, vp, vp, C.c_int, vp]
+    lib.cascade_dedup.argtypes = [vp, C.POINTER(DedupArgs), C.c_int, vp]
     lib.cascade_tier_plan_noalloc.argtypes = [C.POINTER(Params), C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64,
                                               C.POINTER(Pools), C.POINTER(Plan), vp, vp]
     for name in EXPORTS:
@@ -230,6 +274,21 @@ class Context:
                                     _p(evict_src), _p(evict_dst), _p(n_evict_dev), n_evict_max, _p(restore_src),
                                     _p(restore_dst), _p(n_restore_dev), n_restore_max, _p(scratch),
                                     _stream(stream)), "cascade_kv_move")
+
+    def stage_plan(self, reqs: Reqs, budget, order, action, n, D_act, K_act, link_budget_ns, host_reserve,
+                   pools: Pools, stage: Stage, stream=None):
+        _check(_lib.cascade_stage_plan(self._h, C.byref(reqs), _p(budget), _p(order), _p(action), n, D_act, K_act,
+                                       link_budget_ns, host_reserve, C.byref(pools), C.byref(stage),
+                                       _stream(stream)), "cascade_stage_plan")
+
+    def kv_stage(self, deep_pool, deep_blocks, host_pool, host_blocks, block_bytes, src_ids, dst_ids, n_copies_dev,
+                 n_copies_max, stream=None):
+        _check(_lib.cascade_kv_stage(self._h, _p(deep_pool), deep_blocks, _p(host_pool), host_blocks, block_bytes,
+                                     _p(src_ids), _p(dst_ids), _p(n_copies_dev), n_copies_max, _stream(stream)),
+               "cascade_kv_stage")
+
+    def dedup(self, args: DedupArgs, n, stream=None):
+        _check(_lib.cascade_dedup(self._h, C.byref(args), n, _stream(stream)), "cascade_dedup")
 
     def status(self, clear: bool = True, stream=None) -> tuple[int, int]:
         st = Status()

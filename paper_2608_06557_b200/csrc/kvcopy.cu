@@ -433,6 +433,24 @@ extern "C" int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, 
                               dst_is_device, src_ids, dst_ids, n_copies_dev, n_copies_max, (cudaStream_t)stream);
 }
 
+// Deep-tier record -> host record: the bulk-copy ring with a "paged" side that is itself record-major
+// (one chunk per record).
+extern "C" int cascade_kv_stage(cascade_ctx *ctx, const void *deep_pool, int64_t deep_blocks, void *host_pool,
+                                int64_t host_blocks, int64_t block_bytes, const int32_t *src_ids,
+                                const int32_t *dst_ids, const int32_t *n_copies_dev, int n_copies_max, void *stream) {
+    CascadeRange nvtx_range("cascade_kv_stage");
+    if (block_bytes < 16 || (block_bytes & 15) || host_blocks < 0) return CASCADE_EINVAL;
+    cascade_kv_layout rec;
+    rec.n_blocks = host_blocks;
+    rec.n_chunks = 1;
+    rec.reserved = 0;
+    rec.chunk_bytes = block_bytes;
+    rec.chunk_stride = block_bytes;
+    rec.block_stride = block_bytes;
+    return launch_copy<true>(ctx, &rec, (char *)host_pool, (char *)const_cast<void *>(deep_pool), deep_blocks, 0,
+                             src_ids, dst_ids, n_copies_dev, n_copies_max, (cudaStream_t)stream);
+}
+
 extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, void *host_pool,
                                int64_t host_blocks, const int32_t *evict_src, const int32_t *evict_dst,
                                const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,

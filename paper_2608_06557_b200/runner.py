@@ -159,6 +159,113 @@ class Instance:
                          self.plan_counts[1:2], self.evict_cap, self.restore_src, self.restore_dst,
                          self.plan_counts[0:1], self.restore_cap, self.move_scratch, stream)
 
+    # -- deep tier and shared blocks -------------------------------------------------------------
+    def enable_deep(self, w, deep_pool=None, alloc_pool: bool = True):
+        """Upload the deep-tier table of ``w`` and allocate what the stage plan and the one-copy-per-source
+        pass need: the stage list, the merged lists, share counts and the pass's scratch."""
+        d = self.device
+        self.deep_blocks = w.deep_blocks
+        self.deep_tbl = _to_dev(w.deep_tbl, d)
+        self.stage_cap = self.evict_cap
+        self.stage_src = torch.full((self.stage_cap,), -1, dtype=torch.int32, device=d)
+        self.stage_dst = torch.full((self.stage_cap,), -1, dtype=torch.int32, device=d)
+        self.staged = torch.zeros(self.cap, dtype=torch.int32, device=d)
+        self.stage_counts = torch.zeros(6, dtype=torch.int32, device=d)           # cascade_stage_counts (24 B)
+        self.stage_struct = cs.Stage(cs._p(self.deep_tbl), cs._p(self.stage_src), cs._p(self.stage_dst),
+                                     self.stage_cap, cs._p(self.staged), cs._p(self.stage_counts))
+        self.restore_src_m = torch.full((self.restore_cap,), -1, dtype=torch.int32, device=d)
+        self.restore_dst_m = torch.full((self.restore_cap,), -1, dtype=torch.int32, device=d)
+        self.stage_src_m = torch.full((self.stage_cap,), -1, dtype=torch.int32, device=d)
+        self.stage_dst_m = torch.full((self.stage_cap,), -1, dtype=torch.int32, device=d)
+        n_hbm = self.layout_dict["n_blocks"]
+        self.hbm_ref = torch.zeros(n_hbm, dtype=torch.int32, device=d)
+        self.host_ref = torch.zeros(self.host_blocks, dtype=torch.int32, device=d)
+        self.shared_restore = torch.zeros(self.cap, dtype=torch.uint8, device=d)
+        self.shared_stage = torch.zeros(self.cap, dtype=torch.uint8, device=d)
+        self.dedup_counts_restore = torch.zeros(6, dtype=torch.int32, device=d)
+        self.dedup_counts_stage = torch.zeros(6, dtype=torch.int32, device=d)
+        len_r = cs.dedup_scratch_len(self.host_blocks, self.restore_cap)
+        len_s = cs.dedup_scratch_len(self.deep_blocks, self.stage_cap)
+        self.dedup_scratch = torch.empty(max(len_r, len_s), dtype=torch.int32, device=d)
+        self.dedup_restore_args = lambda: cs.make_dedup_args(
+            lo_a=self.reqs["n0"], lo_b=None, len_a=self.x1, len_b=getattr(self, "pf", None), src_tbl=self.host_tbl,
+            dst_tbl=self.hbm_tbl, maxb=self.maxb, list_src=self.restore_src, list_dst=self.restore_dst,
+            list_count=self.plan_counts[0:1], list_cap=self.restore_cap, out_src=self.restore_src_m,
+            out_dst=self.restore_dst_m, n_src_ids=self.host_blocks, n_dst_ids=n_hbm, free_list=self.hbm_free,
+            free_count=self.hbm_free_count, free_cap=len(self.hbm_free), ref=self.hbm_ref, shared=self.shared_restore,
+            scratch=self.dedup_scratch, scratch_len=self.dedup_scratch.numel(), counts=self.dedup_counts_restore)
+        self.dedup_stage_args = lambda: cs.make_dedup_args(
+            lo_a=self.reqs["n0"], lo_b=self.reqs["n1"], len_a=self.staged, len_b=None, src_tbl=self.deep_tbl,
+            dst_tbl=self.host_tbl, maxb=self.maxb, list_src=self.stage_src, list_dst=self.stage_dst,
+            list_count=self.stage_counts[0:1], list_cap=self.stage_cap, out_src=self.stage_src_m,
+            out_dst=self.stage_dst_m, n_src_ids=self.deep_blocks, n_dst_ids=self.host_blocks,
+            free_list=self.host_free, free_count=self.host_free_count, free_cap=len(self.host_free),
+            ref=self.host_ref, shared=self.shared_stage, scratch=self.dedup_scratch,
+            scratch_len=self.dedup_scratch.numel(), counts=self.dedup_counts_stage)
+        self.deep_pool = deep_pool
+        if deep_pool is None and alloc_pool:
+            self.deep_pool = torch.empty(w.deep_blocks * self.block_bytes, dtype=torch.uint8, pin_memory=True)
+
+    def run_stage_plan(self, link_budget_ns: int, host_reserve: int = 0, stream=None):
+        """First hop of the deep-tier path for this iteration (after run_schedule)."""
+        self.ctx.stage_plan(self.reqs_struct, self.budget, self.order, self.action, self.n, self.D_act, self.K_act,
+                            link_budget_ns, host_reserve, self.pools_struct, self.stage_struct, stream)
+
+    def run_dedup_restore(self, stream=None):
+        """One copy per shared host block of the restore list (after the plan and the prefetch plan)."""
+        self.ctx.dedup(self.dedup_restore_args(), self.n, stream)
+
+    def run_dedup_stage(self, stream=None):
+        """One copy per shared deep-tier block of the stage list (after run_stage_plan)."""
+        self.ctx.dedup(self.dedup_stage_args(), self.n, stream)
+
+    def run_move_merged(self, stream=None):
+        """evict + restore over the merged restore list."""
+        if not hasattr(self, "move_scratch"):
+            self.move_scratch = torch.empty(self.evict_cap + self.restore_cap, dtype=torch.int32, device=self.device)
+        self.ctx.kv_move(self.layout, self.hbm_pool, self.host_pool, self.host_blocks, self.evict_src, self.evict_dst,
+                         self.plan_counts[1:2], self.evict_cap, self.restore_src_m, self.restore_dst_m,
+                         self.dedup_counts_restore[1:2], self.restore_cap, self.move_scratch, stream)
+
+    def run_stage_copy(self, merged: bool = True, stream=None):
+        """deep-tier records -> host records over the (merged) stage list."""
+        src, dst = (self.stage_src_m, self.stage_dst_m) if merged else (self.stage_src, self.stage_dst)
+        cnt = self.dedup_counts_stage[1:2] if merged else self.stage_counts[0:1]
+        self.ctx.kv_stage(self.deep_pool, self.deep_blocks, self.host_pool, self.host_blocks, self.block_bytes, src, dst,
+                          cnt, self.stage_cap, stream)
+
+    def run_iteration_deep(self, link_budget_ns: int, host_reserve: int = 0, stream=None):
+        """budget -> schedule -> tier plan -> merge the restore list -> stage plan -> merge the stage list ->
+        evict + restore -> stage copy.  (The stage copy writes host records that this iteration's restore list
+        never reads and its evict list never writes: both came off the free list after them.)"""
+        self.run_schedule(stream)
+        self.run_dedup_restore(stream)
+        self.run_stage_plan(link_budget_ns, host_reserve, stream)
+        self.run_dedup_stage(stream)
+        self.run_move_merged(stream)
+        self.run_stage_copy(True, stream)
+
+    def fetch_deep(self) -> dict:
+        torch.cuda.synchronize(self.device)
+        n = self.n
+        sc = self.stage_counts.cpu().numpy()
+        names = ("n_in", "n_unique", "n_surplus", "n_shared_requests", "max_share", "free_after")
+        dr = {k: int(v) for k, v in zip(names, self.dedup_counts_restore.cpu().numpy())}
+        ds = {k: int(v) for k, v in zip(names, self.dedup_counts_stage.cpu().numpy())}
+        ns = min(int(sc[0]), self.stage_cap)
+        return dict(staged=self.staged[:n].cpu().numpy(), stage_src=self.stage_src[:ns].cpu().numpy(),
+                    stage_dst=self.stage_dst[:ns].cpu().numpy(),
+                    stage_counts=dict(n_stage=int(sc[0]), n_requests=int(sc[1]), n_short=int(sc[2]),
+                                      host_free_after=int(sc[3]), link_ns_left=int(sc[4:6].view(np.int64)[0])),
+                    dedup_restore=dr, dedup_stage=ds,
+                    restore_src_m=self.restore_src_m[: dr["n_unique"]].cpu().numpy(),
+                    restore_dst_m=self.restore_dst_m[: dr["n_unique"]].cpu().numpy(),
+                    stage_src_m=self.stage_src_m[: ds["n_unique"]].cpu().numpy(),
+                    stage_dst_m=self.stage_dst_m[: ds["n_unique"]].cpu().numpy(),
+                    hbm_ref=self.hbm_ref.cpu().numpy(), host_ref=self.host_ref.cpu().numpy(),
+                    shared_restore=self.shared_restore[:n].cpu().numpy(),
+                    shared_stage=self.shared_stage[:n].cpu().numpy())
+
     def run_iteration(self, stream=None, fused_move: bool = False):
         self.run_schedule(stream)
         if self.with_tables and self.hbm_pool is not None:

@@ -309,6 +309,83 @@ def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, st
             if it >= 2:
                 best = min(best, a.elapsed_time(b))
         out[f"move_host_{n}+{n}"] = round(2 * m * bb / best / 1e6, 1)
+    # first hop of the deep-tier path: pinned "deep" records -> pinned host records (the bytes cross the host
+    # link twice, once in each direction)
+    m = min(256, host_blocks)
+    deep = torch.empty(m * bb, dtype=torch.uint8, pin_memory=True)
+    src, dst = wl.copy_lists(77, m, m, host_blocks)
+    s, d = torch.from_numpy(src).cuda(), torch.from_numpy(dst).cuda()
+    best = 1e30
+    for it in range(6):
+        a, b = event_pair(torch)
+        a.record()
+        ctx.kv_stage(deep, m, host_pool, host_blocks, bb, s, d, None, m)
+        b.record()
+        torch.cuda.synchronize()
+        if it >= 2:
+            best = min(best, a.elapsed_time(b))
+    out[f"stage_host_{m}"] = round(m * bb / best / 1e6, 1)
+    del deep
+    return out
+
+
+def deep_sweep(torch, cs):
+    """Latency of the deep-tier plan steps on the shared-prefix workload (tables on the device, no pools):
+    the tier plan alone, then each added step, captured in CUDA graphs of 20 iterations (each iteration also
+    restores the two free-list counts with 4-byte copies so that every replay sees the same state)."""
+    from paper_2608_06557_b200 import workload as wl
+    from paper_2608_06557_b200.runner import Instance
+    out = {}
+    for n in (1024, 8192):
+        w = wl.config_deep_shared(0, n=n, n_hbm=16 * n, n_host=16 * n, n_deep=32 * n, hbm_free_target=8 * n)
+        w.params["plan_first"] = 1
+        inst = Instance(w, alloc_pools=False)
+        inst.enable_deep(w, alloc_pool=False)
+        st = torch.cuda.Stream()
+        saved = (inst.hbm_free_count.clone(), inst.host_free_count.clone(), inst.plan_counts.clone())
+        with torch.cuda.stream(st):
+            inst.run_schedule(st)
+            inst.run_dedup_restore(st)
+            inst.run_stage_plan(10**9, 0, st)
+            inst.run_dedup_stage(st)
+        torch.cuda.synchronize()
+        after_plan = inst.plan_counts.clone()
+        info = inst.fetch_deep()
+
+        def reset(full):
+            inst.hbm_free_count.copy_(saved[0], non_blocking=True)
+            inst.host_free_count.copy_(saved[1], non_blocking=True)
+
+        steps = dict(
+            budget_schedule_plan=lambda: inst.run_schedule(st),
+            merge_restore_list=lambda: inst.run_dedup_restore(st),
+            stage_plan=lambda: inst.run_stage_plan(10**9, 0, st),
+            merge_stage_list=lambda: inst.run_dedup_stage(st),
+        )
+        res = {}
+        for name, fn in steps.items():
+            g = torch.cuda.CUDAGraph()
+            reps = 20
+            with torch.cuda.graph(g, stream=st):
+                for _ in range(reps):
+                    reset(True)
+                    fn()
+            ts = []
+            for it in range(8):
+                a, b = event_pair(torch)
+                a.record()
+                g.replay()
+                b.record()
+                torch.cuda.synchronize()
+                if it >= 3:
+                    ts.append(a.elapsed_time(b) / reps * 1e3)
+            res[name + "_us"] = round(statistics.median(ts), 1)
+            inst.plan_counts.copy_(after_plan)
+        res.update(restore_list=info["dedup_restore"]["n_in"], restore_unique=info["dedup_restore"]["n_unique"],
+                   stage_list=info["dedup_stage"]["n_in"], stage_unique=info["dedup_stage"]["n_unique"])
+        inst.ctx.status(clear=True)
+        out[str(n)] = res
+        del inst
     return out
 
 
@@ -514,6 +591,7 @@ def ours_main(args):
                                         algorithmic_bytes_per_launch=int(2 * 4096 * bb), peak_source=hbm_peak[1])
             del insts
             line["schedule_latency_us"] = schedule_sweep(torch, cs)
+            line["deep_tier_us"] = deep_sweep(torch, cs)
         line["cpu_baseline"] = {k: v for k, v in run_oracle_arm(args, args.cpu_seconds, first_seed=W).items()
                                 if k in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(line))

@@ -10,6 +10,10 @@
  *   cascade_kv_evict   paged HBM blocks  -> contiguous host records            (preemption under HBM pressure)
  *   cascade_kv_restore contiguous host records -> paged HBM blocks             (TriggerPrefetch of Algorithm 1)
  *
+ * Optional steps on the same stream: cascade_prefetch_plan (prefetch for queued requests), cascade_stage_plan +
+ * cascade_kv_stage (first hop of a deep-tier fetch), cascade_dedup (one copy per shared block), cascade_kv_move
+ * (evict and restore in one call).
+ *
  * Conventions
  *   - Every time is an int64 number of nanoseconds, every token / block count an int32, every
  *     cost coefficient a Q20 fixed-point int64 (value * 2^20).  All results are exact integers.

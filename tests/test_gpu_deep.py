@@ -302,3 +302,77 @@ def test_entry_points_reject_bad_arguments():
     with pytest.raises(cs.CascadeError):
         ctx.stage_plan(reqs, z, z, z, 17, 0, 0, 0, 0, pools, stage)          # more requests than the context holds
     assert ctx.status()[0] == 0
+
+
+def test_two_iterations_staged_blocks_reach_hbm_through_the_ordinary_restore():
+    """Iteration 1 stages deep blocks (plan-first admission keeps those requests queued); the caller folds
+    `staged` into the hit profile; iteration 2, over the requests that stayed queued, restores them.  Both
+    iterations run on the GPU and on the oracle; plans and pools must agree, and the HBM block of every
+    staged cell that iteration 2 restored must hold the bytes of the deep record the cell named at the start."""
+    import torch
+    from paper_2608_06557_b200.runner import Instance
+    w = wl.config_deep_shared(11, n=256, hbm_free_target=1500)
+    w.params["plan_first"] = 1
+    bb = w.block_bytes
+    rng = np.random.default_rng(4)
+    hbm = rng.integers(0, 256, w.layout["n_blocks"] * bb, dtype=np.uint8)
+    host = rng.integers(0, 256, w.host_blocks * bb, dtype=np.uint8)
+    deep = rng.integers(0, 256, w.deep_blocks * bb, dtype=np.uint8)
+
+    def oracle_side(w, ref_hbm, ref_host):
+        res, dr, st, ds, _, _ = oracle_deep(w, 10**9, 0)
+        plan = res["plan"]
+        assert oracle.kv_evict(ref_hbm, w.layout, ref_host, w.host_blocks, plan["evict_src"], plan["evict_dst"]) == 0
+        assert oracle.kv_restore(ref_hbm, w.layout, ref_host, w.host_blocks, dr["out_src"], dr["out_dst"]) == 0
+        assert oracle.kv_stage(deep, w.deep_blocks, ref_host, w.host_blocks, bb, ds["out_src"], ds["out_dst"]) == 0
+        return res, dr, st, ds
+
+    def gpu_side(w, pools):
+        inst = Instance(w, hbm_pool=pools[0], host_pool=pools[1])
+        inst.enable_deep(w, deep_pool=pools[2])
+        inst.run_iteration_deep(10**9, 0)
+        return inst, inst.fetch(), inst.fetch_deep()
+
+    ref_hbm, ref_host = hbm.copy(), host.copy()
+    pools = (torch.from_numpy(hbm).cuda(), torch.from_numpy(host).pin_memory(), torch.from_numpy(deep).pin_memory())
+    res1, dr1, st1, ds1 = oracle_side(w, ref_hbm, ref_host)
+    inst1, got1, deep1 = gpu_side(w, pools)
+    assert got1["status"] == 0 and np.array_equal(deep1["staged"], st1["staged"]) and st1["counts"]["n_stage"] > 50
+    assert np.array_equal(pools[0].cpu().numpy(), ref_hbm) and np.array_equal(pools[1].numpy(), ref_host)
+
+    # fold: the requests that stayed queued and were not preempted go on, with their staged blocks now on host
+    p1 = res1["pools"]
+    keep = np.nonzero((res1["grant"] <= 0) & (res1["plan"]["action"] <= oracle.ACT_RETAIN))[0]
+    staged = st1["staged"][keep]
+    reqs2 = {k: np.ascontiguousarray(v[keep]) for k, v in w.reqs.items()}
+    reqs2["n1"] = (reqs2["n1"] + staged).astype(np.int32)
+    reqs2["n2"] = (reqs2["n2"] - staged).astype(np.int32)
+    shared = (dr1["shared"][keep] | ds1["shared"][keep]).astype(bool)
+    reqs2["flags"] = np.where(shared, reqs2["flags"] & ~np.uint8(wl.FLAG_HBM_PRIVATE), reqs2["flags"]).astype(np.uint8)
+    params2 = dict(w.params, ttft_ns=[500 * wl.S, 500 * wl.S], token_budget=1 << 20, max_batch=4096)
+    w2 = wl.Workload("second", params2, reqs2, w.now_ns + 10 * wl.MS, w.D_act, w.K_act, w.layout, w.host_blocks, w.maxb,
+                     p1.hbm_tbl[keep].copy(), p1.host_tbl[keep].copy(), p1.hbm_free.copy(), p1.hbm_free_count,
+                     p1.host_free.copy(), p1.host_free_count)
+    w2.deep_tbl, w2.deep_blocks = w.deep_tbl[keep].copy(), w.deep_blocks
+    res2, dr2, st2, ds2 = oracle_side(w2, ref_hbm, ref_host)
+    inst2, got2, deep2 = gpu_side(w2, pools)
+    assert got2["status"] == res2["status"] | dr2["status"] | st2["status"] | ds2["status"]
+    assert np.array_equal(got2["grant"], res2["grant"]) and np.array_equal(got2["x1"], res2["plan"]["x1"])
+    assert np.array_equal(deep2["restore_src_m"], dr2["out_src"]) and np.array_equal(deep2["restore_dst_m"], dr2["out_dst"])
+    assert np.array_equal(got2["hbm_tbl"], res2["pools"].hbm_tbl)
+    assert np.array_equal(pools[0].cpu().numpy(), ref_hbm) and np.array_equal(pools[1].numpy(), ref_host)
+    # content: staged cells that iteration 2 restored hold the deep record's bytes
+    lay, out_hbm, checked = w.layout, pools[0].cpu().numpy(), 0
+    for s in range(len(keep)):
+        if res2["grant"][s] <= 0 or staged[s] == 0:
+            continue
+        lo = int(w.reqs["n0"][keep[s]] + w.reqs["n1"][keep[s]])
+        upto = int(reqs2["n0"][s] + res2["plan"]["x1"][s])
+        for j in range(lo, min(lo + int(staged[s]), upto)):
+            g, dr = int(got2["hbm_tbl"][s, j]), int(w2.deep_tbl[s, j])
+            for c in range(lay["n_chunks"]):
+                a = c * lay["chunk_stride"] + g * lay["block_stride"]
+                b = dr * bb + c * lay["chunk_bytes"]
+                assert np.array_equal(out_hbm[a:a + lay["chunk_bytes"]], deep[b:b + lay["chunk_bytes"]]), (s, j, c)
+            checked += 1
+    assert checked > 50

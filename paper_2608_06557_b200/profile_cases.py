@@ -4,6 +4,8 @@
     python -m paper_2608_06557_b200.profile_cases copy-host  [blocks]   # pinned host pool <-> paged pool (host link)
     python -m paper_2608_06557_b200.profile_cases move       [blocks]   # fused evict + restore, both link directions
     python -m paper_2608_06557_b200.profile_cases schedule   [requests] # budget + schedule + tier plan, plan-only
+    python -m paper_2608_06557_b200.profile_cases deep       [requests] # whole iteration with the deep-tier stage and
+                                                                        # the shared-block merge (16 KiB blocks)
 
 Each case holds at most a few GB on the device, moves more than the 126 MB L2 per launch and
 launches its kernel five times, printing the CUDA-event time of every launch.
@@ -89,6 +91,26 @@ def schedule_case(n: int):
     print("status", inst.ctx.status())
 
 
+def deep_case(n: int):
+    """Three independent iterations (seeds 0..2) of the shared-prefix workload: plan, merge of the restore
+    list, stage plan, merge of the stage list, evict + restore, stage copy."""
+    for seed in range(3):
+        w = wl.config_deep_shared(seed, n=n, n_hbm=16 * n, n_host=16 * n, n_deep=32 * n, hbm_free_target=8 * n)
+        w.params["plan_first"] = 1
+        inst = Instance(w)
+        inst.enable_deep(w)
+        inst.hbm_pool.fill_(1)
+        inst.host_pool.fill_(2)
+        inst.deep_pool.fill_(3)
+        torch.cuda.synchronize()
+        ts = _timed(lambda: inst.run_iteration_deep(10**9, 0), reps=1)
+        d = inst.fetch_deep()
+        print(f"seed {seed}: {n} requests, iteration {ts[0]:.1f} us; restore list {d['dedup_restore']['n_in']} -> "
+              f"{d['dedup_restore']['n_unique']}, stage list {d['dedup_stage']['n_in']} -> {d['dedup_stage']['n_unique']}, "
+              f"status {inst.ctx.status()}")
+        del inst
+
+
 def main(argv):
     case = argv[1] if len(argv) > 1 else "copy-hbm"
     if case == "copy-hbm":
@@ -99,6 +121,8 @@ def main(argv):
         move_case(int(argv[2]) if len(argv) > 2 else 128)
     elif case == "schedule":
         schedule_case(int(argv[2]) if len(argv) > 2 else 16384)
+    elif case == "deep":
+        deep_case(int(argv[2]) if len(argv) > 2 else 1024)
     else:
         raise SystemExit(__doc__)
 

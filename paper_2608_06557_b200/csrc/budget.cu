@@ -12,6 +12,8 @@ __global__ void __launch_bounds__(kThreads)
 budget_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ LoadConsts lc,
               const __grid_constant__ cascade_reqs r, int n, int64_t now_ns, int64_t *__restrict__ budget_out,
               uint64_t *__restrict__ key_out, int32_t *__restrict__ want_out, uint32_t *__restrict__ status) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int i = blockIdx.x * kThreads + threadIdx.x;
     if (i >= n) return;
     const int64_t P = r.prompt[i];
@@ -107,9 +109,9 @@ extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, in
     if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
     const LoadConsts lc = make_load_consts(ctx->params, D_act, K_act);
     const int grid = (n + kThreads - 1) / kThreads;
-    budget_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(ctx->params, lc, *r, n, now_ns, budget_out, key_out,
-                                                              ctx->want_by_slot, ctx->status_dev);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(grid), dim3(kThreads), 0, (cudaStream_t)stream, budget_kernel,
+                                         ctx->params, lc, *r, n, (int64_t)now_ns, budget_out, key_out,
+                                         ctx->want_by_slot, ctx->status_dev));
     return CASCADE_OK;
 }
 

@@ -34,6 +34,7 @@ struct cascade_ctx {
     int copy_bulk_host;          // >0: TMA bulk-copy ring (that many CTAs per SM) for the pinned-host path
     int copy_bulk_dev;           // >0: TMA bulk-copy ring for the device-staging path
     int move_ctas;               // >0: CTAs of the fused evict+restore kernel (at most one per SM)
+    int pdl;                     // 1: programmatic dependent launch between the calls' kernels
 };
 
 // plan_scalars layout
@@ -156,6 +157,45 @@ __device__ __forceinline__ void dev_choose_restore(const cascade_params &p, int6
     }
     *x1 = bx1;
     *x2 = bx2;
+}
+
+// ---- programmatic dependent launch -----------------------------------------------------------
+// Every kernel of the path starts with cascade_grid_wait(): launched with the programmatic
+// stream-serialization attribute it may be scheduled while its predecessor in the stream is still
+// running and blocks here until that grid has completed and its writes are visible; launched
+// without the attribute the instruction does nothing.  The short plan kernels then call
+// cascade_grid_trigger() at once, so that the launch latency of the next kernel overlaps their own
+// run time; the long copy kernels never trigger early (their successor starts when they exit).
+// No kernel touches global memory before the wait, and every thread executes it (also threads that
+// return right after), so completion of a grid implies completion of everything before it.
+__device__ __forceinline__ void cascade_grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void cascade_grid_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t cascade_launch(bool pdl, int cluster, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                         void (*kernel)(KArgs...), Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    unsigned na = 0;
+    if (cluster > 0) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = cluster;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args &&>(args)...);
 }
 
 // entry points implemented in the other translation units

@@ -66,6 +66,8 @@ __device__ __forceinline__ long long hop_time(const StageArgs &a, long long x) {
 template <int T, int K>
 __global__ void __launch_bounds__(T, 1)
 stage_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ StageArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     constexpr int per = T * K;
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned crank = cluster.block_rank();
@@ -218,6 +220,8 @@ stage_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ S
 }
 
 __global__ void __launch_bounds__(256) apply_stage_kernel(const __grid_constant__ StageArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int n_warps = (gridDim.x * blockDim.x) >> 5;
@@ -250,7 +254,7 @@ __global__ void __launch_bounds__(256) apply_stage_kernel(const __grid_constant_
 }
 
 template <int T, int K>
-cudaError_t launch_stage(const cascade_params &p, const StageArgs &a, int cluster_size, cudaStream_t stream) {
+cudaError_t launch_stage(const cascade_params &p, const StageArgs &a, int cluster_size, bool pdl, cudaStream_t stream) {
     static bool configured_dev[64] = {};
     int device = 0;
     cudaGetDevice(&device);
@@ -259,28 +263,16 @@ cudaError_t launch_stage(const cascade_params &p, const StageArgs &a, int cluste
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) configured_dev[device] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cluster_size, 1, 1);
-    cfg.blockDim = dim3(T, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cluster_size;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, stage_kernel<T, K>, p, a);
+    return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), 0, stream, stage_kernel<T, K>, p, a);
 }
 
 template <int T>
-cudaError_t launch_stage_k(int K, const cascade_params &p, const StageArgs &a, int C, cudaStream_t s) {
+cudaError_t launch_stage_k(int K, const cascade_params &p, const StageArgs &a, int C, bool pdl, cudaStream_t s) {
     switch (K) {
-        case 1: return launch_stage<T, 1>(p, a, C, s);
-        case 2: return launch_stage<T, 2>(p, a, C, s);
-        case 4: return launch_stage<T, 4>(p, a, C, s);
-        default: return launch_stage<T, 8>(p, a, C, s);
+        case 1: return launch_stage<T, 1>(p, a, C, pdl, s);
+        case 2: return launch_stage<T, 2>(p, a, C, pdl, s);
+        case 4: return launch_stage<T, 4>(p, a, C, pdl, s);
+        default: return launch_stage<T, 8>(p, a, C, pdl, s);
     }
 }
 
@@ -315,6 +307,8 @@ __device__ __forceinline__ bool dd_entry_valid(const DedupArgs &a, int s, int d)
 }
 
 __global__ void __launch_bounds__(kDdThreads) dedup_init_kernel(const __grid_constant__ DedupArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int m = dd_list_len(a);
     uint32_t st = 0;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -342,6 +336,8 @@ __global__ void __launch_bounds__(kDdThreads) dedup_init_kernel(const __grid_con
 }
 
 __global__ void __launch_bounds__(kDdThreads) dedup_mark_kernel(const __grid_constant__ DedupArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int m = a.sc[0];
     for (long long i = (long long)blockIdx.x * kDdThreads + threadIdx.x; i < m; i += (long long)gridDim.x * kDdThreads) {
         const int s = a.u.list_src[i], d = a.u.list_dst[i];
@@ -354,6 +350,8 @@ __global__ void __launch_bounds__(kDdThreads) dedup_mark_kernel(const __grid_con
 
 // blocks [0, n_tiles): kept entries per tile; the remaining blocks: one warp per slot rewrites its cells
 __global__ void __launch_bounds__(kDdThreads) dedup_tables_kernel(const __grid_constant__ DedupArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int m = a.sc[0];
     if ((int)blockIdx.x < a.n_tiles) {
         const long long base = (long long)blockIdx.x * kDdTile;
@@ -409,6 +407,8 @@ __global__ void __launch_bounds__(kDdThreads) dedup_tables_kernel(const __grid_c
 }
 
 __global__ void __launch_bounds__(kDdThreads) dedup_compact_kernel(const __grid_constant__ DedupArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     __shared__ int red[kDdThreads / 32];
     __shared__ int wsum[kDdThreads / 32];
     const int m = a.sc[0];
@@ -529,11 +529,10 @@ extern "C" int cascade_stage_plan(cascade_ctx *ctx, const cascade_reqs *r, const
     a.with_tables = with_tables ? 1 : 0;
     int T, C, K;
     if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_stage_k<256>(K, p, a, C, s) : launch_stage_k<512>(K, p, a, C, s);
+    cudaError_t e = T == 256 ? launch_stage_k<256>(K, p, a, C, ctx->pdl, s) : launch_stage_k<512>(K, p, a, C, ctx->pdl, s);
     CASCADE_CUDA_TRY(ctx, e);
     if (with_tables && n > 0) {
-        apply_stage_kernel<<<ctx->num_sms * 2, 256, 0, s>>>(a);
-        CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(ctx->num_sms * 2), dim3(256), 0, s, apply_stage_kernel, a));
     }
     return CASCADE_OK;
 }
@@ -565,15 +564,12 @@ extern "C" int cascade_dedup(cascade_ctx *ctx, const cascade_dedup_args *u, int 
     a.n_tiles = n_tiles;
     int grid = n_tiles * kDdRounds;
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
-    dedup_init_kernel<<<grid, kDdThreads, 0, s>>>(a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
-    dedup_mark_kernel<<<grid, kDdThreads, 0, s>>>(a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(grid), dim3(kDdThreads), 0, s, dedup_init_kernel, a));
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(grid), dim3(kDdThreads), 0, s, dedup_mark_kernel, a));
     int slot_blocks = (n + kDdThreads / 32 - 1) / (kDdThreads / 32);
     if (slot_blocks > ctx->num_sms * 4) slot_blocks = ctx->num_sms * 4;
-    dedup_tables_kernel<<<n_tiles + slot_blocks, kDdThreads, 0, s>>>(a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
-    dedup_compact_kernel<<<n_tiles, kDdThreads, 0, s>>>(a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(n_tiles + slot_blocks), dim3(kDdThreads), 0, s,
+                                         dedup_tables_kernel, a));
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(n_tiles), dim3(kDdThreads), 0, s, dedup_compact_kernel, a));
     return CASCADE_OK;
 }

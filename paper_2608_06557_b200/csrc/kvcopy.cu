@@ -34,6 +34,7 @@ struct CopyArgs {
 
 template <bool kRestore>
 __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant__ CopyArgs a) {
+    cascade_grid_wait();
     int count = a.n_max;
     if (a.n_dev) {
         const int c = *a.n_dev;
@@ -120,6 +121,7 @@ __device__ __forceinline__ void bulk_store(void *dst, unsigned src_smem, unsigne
 
 template <bool kRestore>
 __global__ void __launch_bounds__(32) kv_copy_bulk_kernel(const __grid_constant__ CopyArgs a) {
+    cascade_grid_wait();
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ __align__(8) unsigned long long bars[kStages];
     if (threadIdx.x != 0) return;
@@ -209,8 +211,9 @@ __global__ void __launch_bounds__(32) kv_copy_bulk_kernel(const __grid_constant_
 // device -> host while restored blocks travel host -> device, so the link is used in both directions
 // at the same time.  A restore may target an HBM block that the same call evicts (the tier plan hands
 // freed blocks out again at once): its store into HBM waits until every piece of that block has been
-// read by the evict side.  Even CTAs work on the evict list (walking it backwards, because the blocks
-// freed last are handed out first), odd CTAs on the restore list; only restore CTAs ever wait, and
+// read by the evict side.  Each CTA works on one list: the CTAs are shared out in proportion to the
+// lists' lengths; evict CTAs walk their list backwards, because the blocks freed last are handed out
+// first.  Only restore CTAs ever wait, and
 // only for evict CTAs, which never wait for anybody, so with all CTAs resident (one per SM at most)
 // the waits cannot deadlock.  They are clock-bounded all the same (CASCADE_ST_ETIMEOUT, that store
 // is skipped).
@@ -236,6 +239,8 @@ __device__ __forceinline__ int clamp_count(const int32_t *dev, int maxv) {
 }
 
 __global__ void __launch_bounds__(256) kv_move_prepare_kernel(const __grid_constant__ MoveArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int ne = clamp_count(a.n_evict_dev, a.n_evict_max), nr = clamp_count(a.n_restore_dev, a.n_restore_max);
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int stride = gridDim.x * blockDim.x;
@@ -250,6 +255,7 @@ __global__ void __launch_bounds__(256) kv_move_prepare_kernel(const __grid_const
 }
 
 __global__ void __launch_bounds__(32) kv_move_kernel(const __grid_constant__ MoveArgs a) {
+    cascade_grid_wait();
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ __align__(8) unsigned long long bars[kStages];
     if (threadIdx.x != 0) return;
@@ -262,14 +268,25 @@ __global__ void __launch_bounds__(32) kv_move_kernel(const __grid_constant__ Mov
     const long long per_block = (long long)a.n_chunks * ppc;
     const long long bb = (long long)a.n_chunks * a.chunk_bytes;
     uint32_t st = 0;
-    // even CTAs evict, odd CTAs restore; a single-CTA grid does the evict list first, then the restores
-    const bool split = gridDim.x > 1;
-    const bool evict_role = !split || (blockIdx.x & 1) == 0;
-    const long long evict_items = (split && !evict_role) ? 0 : (long long)ne * per_block;
-    const long long items = evict_items + ((split && evict_role) ? 0 : (long long)nr * per_block);
-    const long long step = split ? (evict_role ? (gridDim.x + 1) / 2 : gridDim.x / 2) : 1;
+    // Each CTA serves one direction, so that both directions of the link are busy at once; the CTAs are shared
+    // out in proportion to the bytes of the two lists (interleaved over the grid), at least one per non-empty
+    // list.  A single-CTA grid does the evict list first, then the restores.
+    const long long G = gridDim.x, b = blockIdx.x;
+    const bool both = G == 1;                          // one CTA walks both lists
+    long long ge = G;                                  // CTAs that evict
+    if (ne > 0 && nr > 0) {
+        ge = (G * ne + (ne + (long long)nr) / 2) / (ne + (long long)nr);
+        ge = ge < 1 ? 1 : (ge > G - 1 ? G - 1 : ge);
+    } else if (ne == 0) {
+        ge = 0;
+    }
+    const long long e_before = b * ge / G;             // evict CTAs among the blocks before this one
+    const bool evict_role = (b + 1) * ge / G > e_before;
+    const long long evict_items = (both || evict_role) ? (long long)ne * per_block : 0;
+    const long long items = evict_items + ((both || !evict_role) ? (long long)nr * per_block : 0);
+    const long long step = both ? 1 : (evict_role ? ge : G - ge);
 
-    long long next = split ? blockIdx.x / 2 : 0;
+    long long next = both ? 0 : (evict_role ? e_before : b - e_before);
     char *dst_of[kStages];
     unsigned bytes_of[kStages];
     int evict_of[kStages];  // evict-list index to signal after the load (evict piece), -1 otherwise
@@ -400,8 +417,8 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
                                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             configured = true;
         }
-        kv_copy_bulk_kernel<kRestore><<<(unsigned)grid, 32, smem, s>>>(a);
-        CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(32), smem, s,
+                                             kv_copy_bulk_kernel<kRestore>, a));
         return CASCADE_OK;
     }
     a.pieces_per_chunk = (int)((l->chunk_bytes + kPiece - 1) / kPiece);
@@ -409,8 +426,7 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
     const int per_sm = record_is_device ? ctx->copy_ctas_dev : ctx->copy_ctas_host;
     long long grid = (long long)ctx->num_sms * per_sm;
     if (grid > items) grid = items;
-    kv_copy_kernel<kRestore><<<(unsigned)grid, kThreads, 0, s>>>(a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(kThreads), 0, s, kv_copy_kernel<kRestore>, a));
     return CASCADE_OK;
 }
 
@@ -488,8 +504,7 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     const int most = n_evict_max > n_restore_max ? n_evict_max : n_restore_max;
     int pgrid = (most + 255) / 256;
     if (pgrid > ctx->num_sms * 4) pgrid = ctx->num_sms * 4;
-    kv_move_prepare_kernel<<<pgrid, 256, 0, s>>>(a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(pgrid), dim3(256), 0, s, kv_move_prepare_kernel, a));
     const long long items = ((long long)n_evict_max + n_restore_max) * hbm->n_chunks * a.pieces_per_chunk;
     long long grid = ctx->num_sms;  // one resident CTA per SM: every CTA that can be waited for is running
     if (ctx->move_ctas > 0 && ctx->move_ctas < grid) grid = ctx->move_ctas;
@@ -502,7 +517,6 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
         CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured = true;
     }
-    kv_move_kernel<<<(unsigned)grid, 32, smem, s>>>(a);
-    CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(32), smem, s, kv_move_kernel, a));
     return CASCADE_OK;
 }

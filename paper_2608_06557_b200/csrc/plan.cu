@@ -75,6 +75,8 @@ struct __align__(16) Exch3 {
 template <int T, int K>
 __global__ void __launch_bounds__(T, 1)
 plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ PlanArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     constexpr int per = T * K;
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned crank = cluster.block_rank();
@@ -356,6 +358,8 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
 // records, fill the evict list and the host table.
 __global__ void __launch_bounds__(256)
 apply_victims_kernel(const __grid_constant__ PlanArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int n_warps = (gridDim.x * blockDim.x) >> 5;
@@ -394,6 +398,8 @@ apply_victims_kernel(const __grid_constant__ PlanArgs a) {
 // restore list and the HBM table.
 __global__ void __launch_bounds__(256)
 apply_admitted_kernel(const __grid_constant__ PlanArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int n_warps = (gridDim.x * blockDim.x) >> 5;
@@ -431,7 +437,7 @@ apply_admitted_kernel(const __grid_constant__ PlanArgs a) {
 
 
 template <int T, int K>
-cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_size, cudaStream_t stream) {
+cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_size, bool pdl, cudaStream_t stream) {
     // clusters of 16 CTAs need the non-portable size opt-in, once per device
     static bool configured_dev[64] = {};
     int device = 0;
@@ -441,28 +447,16 @@ cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) configured_dev[device] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cluster_size, 1, 1);
-    cfg.blockDim = dim3(T, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cluster_size;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, plan_kernel<T, K>, p, a);
+    return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), 0, stream, plan_kernel<T, K>, p, a);
 }
 
 template <int T>
-cudaError_t launch_plan_k(int K, const cascade_params &p, const PlanArgs &a, int C, cudaStream_t s) {
+cudaError_t launch_plan_k(int K, const cascade_params &p, const PlanArgs &a, int C, bool pdl, cudaStream_t s) {
     switch (K) {
-        case 1: return launch_plan<T, 1>(p, a, C, s);
-        case 2: return launch_plan<T, 2>(p, a, C, s);
-        case 4: return launch_plan<T, 4>(p, a, C, s);
-        default: return launch_plan<T, 8>(p, a, C, s);
+        case 1: return launch_plan<T, 1>(p, a, C, pdl, s);
+        case 2: return launch_plan<T, 2>(p, a, C, pdl, s);
+        case 4: return launch_plan<T, 4>(p, a, C, pdl, s);
+        default: return launch_plan<T, 8>(p, a, C, pdl, s);
     }
 }
 
@@ -515,14 +509,12 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     a.with_tables = with_tables ? 1 : 0;
     int T, C, K;
     if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, s) : launch_plan_k<512>(K, ctx->params, a, C, s);
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, ctx->pdl, s) : launch_plan_k<512>(K, ctx->params, a, C, ctx->pdl, s);
     CASCADE_CUDA_TRY(ctx, e);
     if (with_tables && n > 0) {
         const int grid = ctx->num_sms * 2;
-        apply_victims_kernel<<<grid, 256, 0, s>>>(a);
-        CASCADE_CUDA_TRY(ctx, cudaGetLastError());
-        apply_admitted_kernel<<<grid, 256, 0, s>>>(a);
-        CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(grid), dim3(256), 0, s, apply_victims_kernel, a));
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(grid), dim3(256), 0, s, apply_admitted_kernel, a));
     }
     return CASCADE_OK;
 }
@@ -638,7 +630,7 @@ extern "C" int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_
     cascade_ctx geo = {};
     int T, C, K;
     if (!cascade_pick_geometry(&geo, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_plan_k<256>(K, *p, a, C, s) : launch_plan_k<512>(K, *p, a, C, s);
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, *p, a, C, false, s) : launch_plan_k<512>(K, *p, a, C, false, s);
     if (e != cudaSuccess) return CASCADE_ECUDA;
     if (with_tables && n > 0) {
         const int grid = dev->num_sms * 2;

@@ -53,6 +53,8 @@ struct __align__(16) PfExch2 {
 template <int T, int K>
 __global__ void __launch_bounds__(T, 1)
 prefetch_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ PrefetchArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     constexpr int per = T * K;
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned crank = cluster.block_rank();
@@ -213,6 +215,8 @@ prefetch_kernel(const __grid_constant__ cascade_params p, const __grid_constant_
 }
 
 __global__ void __launch_bounds__(256) apply_prefetch_kernel(const __grid_constant__ PrefetchArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int n_warps = (gridDim.x * blockDim.x) >> 5;
@@ -245,7 +249,7 @@ __global__ void __launch_bounds__(256) apply_prefetch_kernel(const __grid_consta
 }
 
 template <int T, int K>
-cudaError_t launch_pf(const cascade_params &p, const PrefetchArgs &a, int cluster_size, cudaStream_t stream) {
+cudaError_t launch_pf(const cascade_params &p, const PrefetchArgs &a, int cluster_size, bool pdl, cudaStream_t stream) {
     static bool configured_dev[64] = {};
     int device = 0;
     cudaGetDevice(&device);
@@ -254,28 +258,16 @@ cudaError_t launch_pf(const cascade_params &p, const PrefetchArgs &a, int cluste
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) configured_dev[device] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cluster_size, 1, 1);
-    cfg.blockDim = dim3(T, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cluster_size;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefetch_kernel<T, K>, p, a);
+    return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), 0, stream, prefetch_kernel<T, K>, p, a);
 }
 
 template <int T>
-cudaError_t launch_pf_k(int K, const cascade_params &p, const PrefetchArgs &a, int C, cudaStream_t s) {
+cudaError_t launch_pf_k(int K, const cascade_params &p, const PrefetchArgs &a, int C, bool pdl, cudaStream_t s) {
     switch (K) {
-        case 1: return launch_pf<T, 1>(p, a, C, s);
-        case 2: return launch_pf<T, 2>(p, a, C, s);
-        case 4: return launch_pf<T, 4>(p, a, C, s);
-        default: return launch_pf<T, 8>(p, a, C, s);
+        case 1: return launch_pf<T, 1>(p, a, C, pdl, s);
+        case 2: return launch_pf<T, 2>(p, a, C, pdl, s);
+        case 4: return launch_pf<T, 4>(p, a, C, pdl, s);
+        default: return launch_pf<T, 8>(p, a, C, pdl, s);
     }
 }
 
@@ -324,11 +316,10 @@ extern "C" int cascade_prefetch_plan(cascade_ctx *ctx, const cascade_reqs *r, co
     a.with_tables = with_tables ? 1 : 0;
     int T, C, K;
     if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_pf_k<256>(K, ctx->params, a, C, s) : launch_pf_k<512>(K, ctx->params, a, C, s);
+    cudaError_t e = T == 256 ? launch_pf_k<256>(K, ctx->params, a, C, ctx->pdl, s) : launch_pf_k<512>(K, ctx->params, a, C, ctx->pdl, s);
     CASCADE_CUDA_TRY(ctx, e);
     if (with_tables && n > 0) {
-        apply_prefetch_kernel<<<ctx->num_sms * 2, 256, 0, s>>>(a);
-        CASCADE_CUDA_TRY(ctx, cudaGetLastError());
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(ctx->num_sms * 2), dim3(256), 0, s, apply_prefetch_kernel, a));
     }
     return CASCADE_OK;
 }

@@ -85,6 +85,8 @@ __device__ __forceinline__ T seg_incl_scan(T v, int pos, int width) {
 
 template <int T, int K>
 __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ ScheduleArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
     constexpr int W = T / 32;          // warps per CTA
     constexpr int per = T * K;         // elements per CTA
     cg::cluster_group cluster = cg::this_cluster();
@@ -466,7 +468,7 @@ size_t smem_bytes(int T, int K) {
 }
 
 template <int T, int K>
-cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, cudaStream_t stream) {
+cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, bool pdl, cudaStream_t stream) {
     static bool configured_dev[64] = {};
     bool unknown = false;
     bool &configured = (device >= 0 && device < 64) ? configured_dev[device] : unknown;
@@ -479,28 +481,16 @@ cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, cudaStre
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cluster_size, 1, 1);
-    cfg.blockDim = dim3(T, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cluster_size;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, schedule_kernel<T, K>, a);
+    return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), smem, stream, schedule_kernel<T, K>, a);
 }
 
 template <int T>
-cudaError_t launch_k(int K, const ScheduleArgs &a, int C, int device, cudaStream_t s) {
+cudaError_t launch_k(int K, const ScheduleArgs &a, int C, int device, bool pdl, cudaStream_t s) {
     switch (K) {
-        case 1: return launch<T, 1>(a, C, device, s);
-        case 2: return launch<T, 2>(a, C, device, s);
-        case 4: return launch<T, 4>(a, C, device, s);
-        default: return launch<T, 8>(a, C, device, s);
+        case 1: return launch<T, 1>(a, C, device, pdl, s);
+        case 2: return launch<T, 2>(a, C, device, pdl, s);
+        case 4: return launch<T, 4>(a, C, device, pdl, s);
+        default: return launch<T, 8>(a, C, device, pdl, s);
     }
 }
 
@@ -567,7 +557,7 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.stage = ctx->sort_stage >= 0 ? ctx->sort_stage : (K >= 4);
     a.async_sync = ctx->sort_async;
     a.status = ctx->status_dev;
-    cudaError_t e = T == 256 ? launch_k<256>(K, a, C, ctx->device, s) : launch_k<512>(K, a, C, ctx->device, s);
+    cudaError_t e = T == 256 ? launch_k<256>(K, a, C, ctx->device, ctx->pdl, s) : launch_k<512>(K, a, C, ctx->device, ctx->pdl, s);
     CASCADE_CUDA_TRY(ctx, e);
     return CASCADE_OK;
 }

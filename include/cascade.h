@@ -249,6 +249,19 @@ int cascade_latency_regimes(cascade_ctx *ctx, const cascade_reqs *r, int n, int3
                             int64_t *lat4_out, void *stream);
 
 /*
+ * Queue maintenance (the paper has no counterpart; "the only per-iteration write is the priority key" there
+ * because its queue lives in host memory): overwrite m slots of the device-resident request arrays.
+ *   dst     the queue's arrays (device), cap entries each
+ *   src     the new values, m entries each, compact; device-accessible: pinned mapped host memory is read in
+ *           place over the host link, which for a few hundred slots is cheaper than staging copies
+ *   slots   m destination indices (device-accessible), each < cap; others are skipped (CASCADE_ST_EBOUNDS);
+ *           indices must be distinct
+ * Stream-ordered like every other call; m = 0 is a no-op.
+ */
+int cascade_reqs_update(cascade_ctx *ctx, const cascade_reqs *dst, int cap, const cascade_reqs *src,
+                        const int32_t *slots, int m, void *stream);
+
+/*
  * Least-remaining-budget-first order and admission (Algorithm 1, phase 2).
  *   order_out[n]  slot indices sorted ascending by key (stable: equal keys keep slot order)
  *   grant_out[n]  tokens granted to each slot this iteration (0 = not admitted): the Tier-1 queue

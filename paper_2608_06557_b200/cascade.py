@@ -24,7 +24,7 @@ ACT_NONE, ACT_RETAIN, ACT_EVICT, ACT_DROP = 0, 1, 2, 3
 EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_budget", "cascade_schedule",
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
            "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan", "cascade_kv_move",
-           "cascade_stage_plan", "cascade_kv_stage", "cascade_dedup")
+           "cascade_stage_plan", "cascade_kv_stage", "cascade_dedup", "cascade_reqs_update")
 
 
 class Params(C.Structure):
@@ -140,6 +140,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_status.argtypes = [vp, C.POINTER(Status), C.c_int, vp]
     lib.cascade_kv_move.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int,
                                     vp, vp]
+    lib.cascade_reqs_update.argtypes = [vp, C.POINTER(Reqs), C.c_int, C.POINTER(Reqs), vp, C.c_int, vp]
     lib.cascade_stage_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64, i64, i32, C.POINTER(Pools),
                                        C.POINTER(Stage), vp]
     lib.cascade_kv_stage.argtypes = [vp, vp, i64, vp, i64, i64, vp, vp, vp, C.c_int, vp]
@@ -233,6 +234,10 @@ class Context:
     def set_params(self, params: dict | Params):
         self.params = params if isinstance(params, Params) else make_params(params)
         _check(_lib.cascade_set_params(self._h, C.byref(self.params)), "cascade_set_params")
+
+    def reqs_update(self, dst: Reqs, cap, src: Reqs, slots, m, stream=None):
+        _check(_lib.cascade_reqs_update(self._h, C.byref(dst), cap, C.byref(src), _p(slots), m, _stream(stream)),
+               "cascade_reqs_update")
 
     def budget(self, reqs: Reqs, n, now_ns, D_act, K_act, budget_out, key_out, stream=None):
         _check(_lib.cascade_budget(self._h, C.byref(reqs), n, now_ns, D_act, K_act, _p(budget_out), _p(key_out),

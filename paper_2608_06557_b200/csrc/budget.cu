@@ -96,7 +96,51 @@ regimes_kernel(const __grid_constant__ cascade_params p, const __grid_constant__
     lat4[4 * (size_t)i + 3] = out.w;
 }
 
+__global__ void __launch_bounds__(kThreads)
+reqs_update_kernel(const __grid_constant__ cascade_reqs dst, int cap, const __grid_constant__ cascade_reqs src,
+                   const int32_t *__restrict__ slots, int m, uint32_t *__restrict__ status) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i >= m) return;
+    const int s = slots[i];
+    // all loads first (they may cross the host link: one round trip, not nine), then the stores
+    const int64_t v_arr = src.arrival_ns[i];
+    const int32_t v_prompt = src.prompt[i], v_out = src.pred_out[i], v_n0 = src.n0[i], v_n1 = src.n1[i], v_n2 = src.n2[i];
+    const uint32_t v_id = src.id[i];
+    const uint8_t v_cls = src.cls[i], v_flags = src.flags[i];
+    if (s < 0 || s >= cap) {
+        atomicOr(status, CASCADE_ST_EBOUNDS);
+        return;
+    }
+    const_cast<int64_t *>(dst.arrival_ns)[s] = v_arr;
+    const_cast<int32_t *>(dst.prompt)[s] = v_prompt;
+    const_cast<int32_t *>(dst.pred_out)[s] = v_out;
+    const_cast<int32_t *>(dst.n0)[s] = v_n0;
+    const_cast<int32_t *>(dst.n1)[s] = v_n1;
+    const_cast<int32_t *>(dst.n2)[s] = v_n2;
+    const_cast<uint32_t *>(dst.id)[s] = v_id;
+    const_cast<uint8_t *>(dst.cls)[s] = v_cls;
+    const_cast<uint8_t *>(dst.flags)[s] = v_flags;
+}
+
 }  // namespace
+
+extern "C" int cascade_reqs_update(cascade_ctx *ctx, const cascade_reqs *dst, int cap, const cascade_reqs *src,
+                                   const int32_t *slots, int m, void *stream) {
+    CascadeRange nvtx_range("cascade_reqs_update");
+    if (!ctx || !dst || !src || cap < 0 || m < 0) return CASCADE_EINVAL;
+    if (m == 0) return CASCADE_OK;
+    const cascade_reqs *both[2] = {dst, src};
+    for (const cascade_reqs *q : both)
+        if (!q->arrival_ns || !q->prompt || !q->pred_out || !q->n0 || !q->n1 || !q->n2 || !q->id || !q->cls || !q->flags)
+            return CASCADE_EINVAL;
+    if (!slots) return CASCADE_EINVAL;
+    const int grid = (m + kThreads - 1) / kThreads;
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(grid), dim3(kThreads), 0, (cudaStream_t)stream,
+                                         reqs_update_kernel, *dst, cap, *src, slots, m, ctx->status_dev));
+    return CASCADE_OK;
+}
 
 extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, int64_t now_ns, int32_t D_act,
                               int64_t K_act, int64_t *budget_out, uint64_t *key_out, void *stream) {

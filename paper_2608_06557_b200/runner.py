@@ -109,6 +109,24 @@ class Instance:
             self.reqs_host[k][:n].numpy()[...] = src if dt != np.uint32 else src
             self.reqs[k][:n].copy_(self.reqs_host[k][:n], non_blocking=True)
 
+    def stage_slot_update(self, reqs: dict, slots: np.ndarray) -> int:
+        """Write the new values of ``slots`` (taken from the full arrays ``reqs``) into the pinned staging
+        arrays; host work only.  Returns the number of bytes the device will read."""
+        m = len(slots)
+        if not hasattr(self, "upd_host"):
+            self.upd_host = {k: torch.empty(self.cap, dtype=dt, pin_memory=True) for k, dt in _REQ_DTYPES.items()}
+            self.upd_slots = torch.empty(self.cap, dtype=torch.int32, pin_memory=True)
+            self.upd_struct = cs.make_reqs(self.upd_host)
+        for k, dt in _NP_DTYPES.items():
+            self.upd_host[k][:m].numpy()[...] = np.ascontiguousarray(reqs[k], dtype=dt)[slots]
+        self.upd_slots[:m].numpy()[...] = slots
+        self.upd_m = m
+        return m * (sum(self.reqs[k].element_size() for k in self.reqs) + 4)
+
+    def run_slot_update(self, stream=None):
+        """Scatter the staged slots into the device queue (the kernel reads the pinned staging arrays in place)."""
+        self.ctx.reqs_update(self.reqs_struct, self.cap, self.upd_struct, self.upd_slots, self.upd_m, stream)
+
     def request_bytes(self) -> int:
         return sum(self.reqs[k].element_size() for k in self.reqs) * self.n
 

@@ -115,19 +115,50 @@ def test_scheduler_sweep_iterations_with_churn(n, iters):
     torch, cs, Instance = _gpu()
     sw = wl.SchedulerSweep(n, seed=1)
     inst = Instance(sw.workload(), alloc_pools=False)
+    slots = None
     for it in range(iters):
         w = sw.workload()
         ref = oracle_iteration(w, with_tables=False)
-        inst.upload_requests(w.reqs)
+        if slots is None:
+            inst.upload_requests(w.reqs)
+        else:                                   # only the replaced slots travel, scattered by the library
+            inst.stage_slot_update(w.reqs, slots)
+            inst.run_slot_update()
         inst.set_clock(w.now_ns, w.D_act, w.K_act)
         inst.run_schedule()
         got = inst.fetch()
+        assert got["status"] == 0
         for k in ("budget", "key", "order", "grant"):
             assert np.array_equal(got[k], ref[k]), (it, k)
         for k in ("x1", "x2", "tokens_run", "action"):
             assert np.array_equal(got[k], ref["plan"][k]), (it, k)
         assert got["plan_counts"] == ref["plan"]["counts"]
-        sw.step()
+        if it + 1 < iters:
+            slots = sw.step()
+    for k, v in w.reqs.items():                 # the device queue is the host queue of the last iteration
+        assert np.array_equal(inst.reqs[k][:n].cpu().numpy().view(v.dtype), v), k
+
+
+def test_slot_update_edges():
+    torch, cs, Instance = _gpu()
+    w = wl.config_tiny(0)
+    inst = Instance(w, alloc_pools=False)
+    before = {k: inst.reqs[k].clone() for k in inst.reqs}
+    inst.stage_slot_update(w.reqs, np.zeros(0, np.int64))
+    inst.run_slot_update()                      # m = 0: nothing happens
+    new = {k: (v.copy() if k != "prompt" else v + 1) for k, v in w.reqs.items()}
+    inst.stage_slot_update(new, np.array([5, 9], np.int64))
+    inst.upd_slots[1] = w.n + 100               # outside the queue: skipped and flagged
+    inst.run_slot_update()
+    torch.cuda.synchronize()
+    assert inst.ctx.status()[0] == cs.ST_EBOUNDS
+    got = inst.reqs["prompt"].cpu().numpy()
+    want = before["prompt"].cpu().numpy().copy()
+    want[5] += 1
+    assert np.array_equal(got, want)
+    for k in inst.reqs:
+        if k != "prompt":
+            assert torch.equal(inst.reqs[k], before[k]), k
 
 
 def test_precondition_flag_and_parking():

@@ -265,10 +265,11 @@ def measure_link_peaks(torch, host_pool, hbm_pool):
 
 def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, stage):
     """Evict / restore bandwidth for 1, 16, 256 and 4096 scattered blocks per call, through the pinned
-    host pool (host link) and through a device staging buffer (HBM), best of 5 after 2 warm-ups."""
+    host pool (host link) and through a device staging buffer (HBM): 3 warm-ups, then 20 timed calls (10 for
+    4096 blocks over the host link); best and median."""
     from paper_2608_06557_b200 import workload as wl
     bb = lay["n_chunks"] * lay["chunk_bytes"]
-    out = {}
+    out, median = {}, {}
     stage_blocks = stage.numel() // bb
     for n in (1, 16, 256, 4096):
         for name, rec, nrec, isdev in (("host", host_pool, host_blocks, False), ("hbm", stage, stage_blocks, True)):
@@ -276,8 +277,8 @@ def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, st
             src, dst = wl.copy_lists(100 + n, m, nrec, lay["n_blocks"])
             s, d = torch.from_numpy(src).cuda(), torch.from_numpy(dst).cuda()
             for kind in ("evict", "restore"):
-                best = 1e30
-                for it in range(7):
+                ts = []
+                for it in range(3 + (20 if n <= 256 or isdev else 10)):
                     a, b = event_pair(torch)
                     a.record()
                     if kind == "evict":
@@ -286,9 +287,11 @@ def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, st
                         ctx.kv_restore(layout, hbm_pool, rec, nrec, isdev, s, d, None, m)
                     b.record()
                     torch.cuda.synchronize()
-                    if it >= 2:
-                        best = min(best, a.elapsed_time(b))
-                out[f"{kind}_{name}_{n}"] = round((2 if isdev else 1) * m * bb / best / 1e6, 1)
+                    if it >= 3:
+                        ts.append(a.elapsed_time(b))
+                scale = (2 if isdev else 1) * m * bb / 1e6
+                out[f"{kind}_{name}_{n}"] = round(scale / min(ts), 1)
+                median[f"{kind}_{name}_{n}"] = round(scale / statistics.median(ts), 1)
     # both directions at once: n blocks evicted and n restored by one cascade_kv_move, half of the restores
     # into blocks the same call evicts
     for n in (16, 256, 2048):
@@ -326,7 +329,7 @@ def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, st
             best = min(best, a.elapsed_time(b))
     out[f"stage_host_{m}"] = round(m * bb / best / 1e6, 1)
     del deep
-    return out
+    return out, median
 
 
 def deep_sweep(torch, cs):
@@ -617,9 +620,10 @@ def ours_main(args):
             lay = dict(w0.layout)
             lay_small = dict(lay, n_blocks=(hbm_pool.numel() - stage_bytes) // bb // 2)
             lay_small["chunk_stride"] = lay_small["n_blocks"] * lay["chunk_bytes"]
-            sweep = copy_sweep(torch, cs, ctx, cs.make_layout(lay_small), lay_small, hbm_pool, host_pool,
-                               w0.host_blocks, stage)
+            sweep, sweep_median = copy_sweep(torch, cs, ctx, cs.make_layout(lay_small), lay_small, hbm_pool, host_pool,
+                                             w0.host_blocks, stage)
             line["copy_sweep_GBps"] = sweep
+            line["copy_sweep_median_GBps"] = sweep_median
             hbm_peak = load_hbm_peak()
             big = sweep.get("restore_hbm_4096", 0.0)
             line["roofline_hbm"] = dict(bound="hbm", kernel="kv_copy_bulk_kernel<restore>, device staging buffer, "

@@ -51,3 +51,37 @@ def test_host_validation_without_a_device():
         assert lib.cascade_create(ctypes.byref(h), ctypes.byref(q), 16, 0) == cs.ERANGE, bad
     assert lib.cascade_budget(None, None, 0, 0, 0, 0, None, None, None) == cs.EINVAL
     assert lib.cascade_status(None, None, 0, None) == cs.EINVAL
+
+
+def test_header_is_plain_c_and_the_binding_mirrors_its_struct_layouts(tmp_path):
+    """The header must compile as C99 on its own, and every ctypes mirror must have the size and the field
+    offsets the C compiler gives the struct (a silent mismatch would shift every pointer behind it)."""
+    import subprocess
+    from paper_2608_06557_b200 import cascade as cs
+    pairs = [("cascade_params", cs.Params), ("cascade_reqs", cs.Reqs), ("cascade_sched_counts", cs.SchedCounts),
+             ("cascade_plan_counts", cs.PlanCounts), ("cascade_pools", cs.Pools), ("cascade_plan", cs.Plan),
+             ("cascade_kv_layout", cs.KvLayout), ("cascade_status_t", cs.Status),
+             ("cascade_stage_counts", cs.StageCounts), ("cascade_stage", cs.Stage),
+             ("cascade_dedup_counts", cs.DedupCounts), ("cascade_dedup_args", cs.DedupArgs)]
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "cascade.h"', 'int main(void) {']
+    for cname, ct in pairs:
+        lines.append(f'  printf("{cname} %zu", sizeof({cname}));')
+        for fname, _ in ct._fields_:
+            lines.append(f'  printf(" %zu", offsetof({cname}, {fname}));')
+        lines.append('  printf("\\n");')
+    lines += ['  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                           "-o", str(exe), str(src)])
+    out = subprocess.check_output([str(exe)], text=True).splitlines()
+    for (cname, ct), line in zip(pairs, out):
+        got = [int(x) for x in line.split()[1:]]
+        want = [ctypes.sizeof(ct)] + [getattr(ct, f).offset for f, _ in ct._fields_]
+        assert got == want, (cname, got, want)
+    # prefetch counts have no ctypes mirror (the runner reads them as six int32): pin their size here
+    src2 = tmp_path / "pf.c"
+    src2.write_text('#include <stdio.h>\n#include "cascade.h"\nint main(void){printf("%zu", sizeof(cascade_prefetch_counts));return 0;}')
+    subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), "-o", str(tmp_path / "pf"), str(src2)])
+    assert subprocess.check_output([str(tmp_path / "pf")], text=True) == "24"

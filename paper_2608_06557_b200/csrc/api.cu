@@ -34,7 +34,14 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     if (rc != CASCADE_OK) return rc;
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return CASCADE_ECUDA;
+    int prev_device = 0;
+    if (cudaGetDevice(&prev_device) != cudaSuccess) return CASCADE_ECUDA;
     if (cudaSetDevice(device) != cudaSuccess) return CASCADE_ECUDA;
+    // the calling thread's current device is put back before returning, whatever the outcome
+    struct Restore {
+        int d;
+        ~Restore() { cudaSetDevice(d); }
+    } restore{prev_device};
     cascade_ctx *ctx = (cascade_ctx *)calloc(1, sizeof(cascade_ctx));
     if (!ctx) return CASCADE_ENOMEM;
     ctx->params = *p;
@@ -91,6 +98,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
 
 extern "C" void cascade_destroy(cascade_ctx *ctx) {
     if (!ctx) return;
+    int prev_device = -1;
+    cudaGetDevice(&prev_device);
     cudaSetDevice(ctx->device);
     cudaFree(ctx->status_dev);
     cudaFreeHost(ctx->status_host);
@@ -99,6 +108,7 @@ extern "C" void cascade_destroy(cascade_ctx *ctx) {
     cudaFree(ctx->work_admit);
     cudaFree(ctx->work_victim);
     cudaFree(ctx->plan_scalars);
+    if (prev_device >= 0) cudaSetDevice(prev_device);
     free(ctx);
 }
 

@@ -376,3 +376,36 @@ def test_two_iterations_staged_blocks_reach_hbm_through_the_ordinary_restore():
                 assert np.array_equal(out_hbm[a:a + lay["chunk_bytes"]], deep[b:b + lay["chunk_bytes"]]), (s, j, c)
             checked += 1
     assert checked > 50
+
+
+@pytest.mark.parametrize("seed,plan_first", [(0, 1), (3, 0), (6, 1)])
+def test_merge_after_the_prefetch_plan(seed, plan_first):
+    """Restore list = the admitted set's blocks followed by the prefetched ones; the merge pass then covers the
+    cells [n0, n0 + x1 + prefetched) of every slot (two length arrays)."""
+    w = wl.config_deep_shared(seed, n=256)
+    w.params["plan_first"] = plan_first
+    res = oracle_iteration(w)
+    plan, pools, r = res["plan"], res["pools"], w.reqs
+    p = oracle.make_params(w.params)
+    pf = oracle.prefetch_plan(p, r, res["budget"], res["order"], res["grant"], plan["action"], plan["x1"], w.D_act,
+                              w.K_act, 10**9, 4, pools, plan["restore_src"], plan["restore_dst"])
+    assert pf["counts"]["n_prefetch"] > 0
+    ref = np.zeros(w.layout["n_blocks"], np.int32)
+    x1 = np.where(res["grant"] > 0, plan["x1"], 0).astype(np.int32)
+    dr = oracle.dedup(r["n0"], None, x1, pf["pf"], pools.host_tbl, pools.hbm_tbl, pf["restore_src"], pf["restore_dst"],
+                      len(pf["restore_src"]), w.host_blocks, w.layout["n_blocks"], pools.hbm_free, pools.hbm_free_count,
+                      ref)
+    assert dr["counts"]["n_surplus"] > 0
+    inst = make_instance(w, pools=False)
+    inst.run_schedule()
+    inst.run_prefetch(10**9, 4)
+    inst.run_dedup_restore()
+    got, gp, deep = inst.fetch(), inst.fetch_prefetch(), inst.fetch_deep()
+    assert np.array_equal(gp["pf"], pf["pf"]) and gp["counts"] == pf["counts"]
+    assert deep["dedup_restore"] == dr["counts"]
+    assert np.array_equal(deep["restore_src_m"], dr["out_src"]) and np.array_equal(deep["restore_dst_m"], dr["out_dst"])
+    assert np.array_equal(deep["hbm_ref"], ref) and np.array_equal(deep["shared_restore"], dr["shared"])
+    assert np.array_equal(got["hbm_tbl"], pools.hbm_tbl)
+    assert got["hbm_free_count"] == dr["free_count"]
+    assert np.array_equal(got["hbm_free"][: dr["free_count"]], pools.hbm_free[: dr["free_count"]])
+    assert got["status"] == res["status"] | pf["status"] | dr["status"]

@@ -409,3 +409,31 @@ def test_merge_after_the_prefetch_plan(seed, plan_first):
     assert got["hbm_free_count"] == dr["free_count"]
     assert np.array_equal(got["hbm_free"][: dr["free_count"]], pools.hbm_free[: dr["free_count"]])
     assert got["status"] == res["status"] | pf["status"] | dr["status"]
+
+
+@pytest.mark.parametrize("n", [3000, 20000])
+def test_plan_steps_on_large_queues(n):
+    """Several keys per thread and the full cluster: the same comparison as above on 3 000 and 20 000 requests."""
+    import torch
+    w = wl.config_deep_shared(1, n=n, n_hbm=16 * n, n_host=16 * n, n_deep=32 * n, hbm_free_target=8 * n)
+    w.params["plan_first"] = 1
+    res, dr, st, ds, hbm_ref, host_ref = oracle_deep(w, 10**9, 100)
+    assert st["counts"]["n_stage"] > n and ds["counts"]["n_surplus"] > 0
+    inst = make_instance(w, pools=False)
+    inst.run_schedule()
+    inst.run_dedup_restore()
+    inst.run_stage_plan(10**9, 100)
+    inst.run_dedup_stage()
+    got, deep = inst.fetch(), inst.fetch_deep()
+    pools = res["pools"]
+    assert np.array_equal(deep["staged"], st["staged"]) and deep["stage_counts"] == st["counts"]
+    assert np.array_equal(deep["stage_src"], st["stage_src"]) and np.array_equal(deep["stage_dst"], st["stage_dst"])
+    assert deep["dedup_restore"] == dr["counts"] and deep["dedup_stage"] == ds["counts"]
+    assert np.array_equal(deep["stage_src_m"], ds["out_src"]) and np.array_equal(deep["stage_dst_m"], ds["out_dst"])
+    assert np.array_equal(deep["host_ref"], host_ref) and np.array_equal(deep["shared_stage"], ds["shared"])
+    assert np.array_equal(got["host_tbl"], pools.host_tbl) and np.array_equal(got["hbm_tbl"], pools.hbm_tbl)
+    assert got["host_free_count"] == pools.host_free_count
+    assert np.array_equal(got["host_free"][: pools.host_free_count], pools.host_free[: pools.host_free_count])
+    assert got["status"] == (res["status"] | dr["status"] | st["status"] | ds["status"])
+    del inst
+    torch.cuda.empty_cache()

@@ -30,7 +30,9 @@ budget_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ 
         atomicOr(status, CASCADE_ST_EPRECOND);
         budget_out[i] = -(int64_t(1) << 62);
         key_out[i] = (uint64_t(1) << 63) | id;
-        if (p.plan_first) want_out[i] = 0;
+        // parked, but still a request: with a usable shape it is offered tokens like any other (its budget
+        // allows no restore, so the offer is everything behind its HBM blocks), in both admission modes
+        if (p.plan_first) want_out[i] = dev_request_valid(p.bt, P, n0, n1, n2) ? (int32_t)(P - n0 * p.bt) : 0;
         return;
     }
     const int64_t s_hit = (n0 + n1 + n2) * p.bt;

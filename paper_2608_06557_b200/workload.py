@@ -441,3 +441,90 @@ def config_llama70b_trace(seed: int = 0, n: int = 4096, rate_per_s: float = 20.0
     return Trace(params, arrival, prompt, pred_out, cls, n0, n1, agentic_hit, hbm_tbl, host_tbl, hbm_free,
                  hbm_free_count, host_free, host_free_count, kv_layout(n_hbm, n_chunks, chunk_bytes), n_host, maxb,
                  shared_ids)
+
+
+def fuzz_params(rng) -> dict:
+    """Random parameters anywhere inside the library's validated bounds, extremes included."""
+    nc = int(rng.integers(1, 5))
+    bt = int(rng.choice([1, 4, 16, 16, 16, 32, 128]))
+    d = dict(bt=bt, chunk_shift=int(rng.integers(0, 13)), max_batch=int(rng.choice([1, 4, 64, 128, 512, 4096])),
+             max_ctx_avg=int(rng.choice([0, 512, 2048, 1 << 15])), gamma_q16=int(rng.choice([0, 65536, 81920, 1 << 17])),
+             token_budget=int(rng.choice([0, 64, 2048, 8192, 1 << 20])), tier2_reserve=int(rng.choice([0, 64, 1024, 1 << 21])),
+             c_tok_q20=int(rng.choice([0, 1000, 50_000, 1 << 19])) * Q20, c_attn_q20=int(rng.choice([0, 1, Q20 // 2, Q20])),
+             c_iter_q20=int(rng.choice([0, 2_000_000, 1 << 29])) * Q20, c_dseq_q20=int(rng.choice([0, 10_000, 1 << 19])) * Q20,
+             c_dkv_q20=int(rng.choice([0, 20, 255])) * Q20,
+             delta_ns=[0, int(rng.choice([0, 10_000, 1 << 30])), int(rng.choice([0, 110_000, 5000]))],
+             blk_ns=[0, int(rng.choice([1, 328, 40_000, 1 << 27])), int(rng.choice([1, 20_000, 340_000]))],
+             ttft_ns=[int(rng.choice([0, 10**8, 10**9, 3 * 10**10, 1 << 40])) for _ in range(nc)],
+             tpot_ns=[int(rng.choice([0, 10**6, 5 * 10**7])) for _ in range(nc)],
+             policy=int(rng.choice([0, 0, 0, 1, 2, 3])), plan_first=int(rng.integers(0, 2)))
+    if (d["max_batch"] - 1) * d["max_ctx_avg"] > (1 << 32):
+        d["max_ctx_avg"] = 512
+    return d
+
+
+def fuzz_workload(rng, d: dict) -> Workload:
+    """A random queue with tables, free lists and a deep tier for the parameters ``d``: sizes from 1 to 3000,
+    hit profiles of every shape, a few requests outside the input bounds, rows too short for their prompt,
+    shared host / deep record ids, free lists from empty to ample, loads from idle to the maximum."""
+    n = int(rng.choice([1, 2, 33, 200, 1000, 1025, 3000]))
+    bt = d["bt"]
+    nc = len(d["ttft_ns"])
+    maxb = int(rng.choice([8, 64, 200]))
+    prompt = rng.integers(1, maxb * bt + 1, n).astype(np.int32)
+    if rng.uniform() < 0.3:
+        prompt[rng.integers(0, n, max(1, n // 50))] = maxb * bt + int(rng.integers(1, 100))   # row too short: invalid with tables
+    hit = np.floor(rng.uniform(0, 1, n) * ((prompt - 1) // bt)).astype(np.int64)
+    a = rng.uniform(0, 1, n); b = rng.uniform(0, 1, n)
+    n0 = np.floor(hit * a).astype(np.int32)
+    n1 = np.floor((hit - n0) * b).astype(np.int32)
+    n2 = (hit - n0 - n1).astype(np.int32)
+    z = rng.uniform(0, 1, n)
+    n1[z < 0.2] += n2[z < 0.2]; n2[z < 0.2] = 0
+    now = int(rng.choice([0, 10**10, 1 << 45]))
+    elapsed = rng.integers(0, 4 * 10**10, n) if rng.uniform() < 0.8 else rng.integers(-10**6, 1 << 49, n)
+    reqs = dict(arrival_ns=(now - elapsed).astype(np.int64), prompt=prompt,
+                pred_out=rng.integers(0, 1 << 16, n).astype(np.int32), n0=n0, n1=n1, n2=n2,
+                id=rng.permutation(1 << 23)[:n].astype(np.uint32) if rng.uniform() < 0.7 else rng.integers(0, 1 << 32, n, dtype=np.uint64).astype(np.uint32),
+                cls=rng.integers(0, nc, n).astype(np.uint8), flags=rng.integers(0, 4, n).astype(np.uint8))
+    # some broken requests
+    if rng.uniform() < 0.3 and n > 3:
+        k = rng.integers(0, n, 3)
+        reqs["prompt"][k[0]] = 0; reqs["n0"][k[1]] = -1; reqs["cls"][k[2]] = 7
+    tot0, tot1, tot2 = int(np.maximum(n0, 0).sum()), int(n1.sum()), int(n2.sum())
+    n_hbm = tot0 + int(rng.choice([0, 5, 200, 5000])) + 1
+    n_host = tot1 + int(rng.choice([0, 5, 200, 5000])) + 1
+    n_deep = tot2 + 8
+    hbm_ids, host_ids, deep_ids = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_host).astype(np.int32), rng.permutation(n_deep).astype(np.int32)
+    hbm_tbl = np.full((n, maxb + 1), -1, np.int32); host_tbl = hbm_tbl.copy(); deep_tbl = hbm_tbl.copy()
+    u0 = u1 = u2 = 0
+    share = rng.uniform() < 0.5
+    filled = np.zeros(n, bool)
+    for r in range(n):
+        a0, a1, a2 = max(int(n0[r]), 0), int(n1[r]), int(n2[r])
+        if a0 + a1 + a2 > maxb + 1:
+            continue
+        filled[r] = True
+        hbm_tbl[r, :a0] = hbm_ids[u0:u0 + a0]; u0 += a0
+        m1 = m2 = 0
+        q = int(rng.integers(0, r)) if (share and r > 0 and rng.uniform() < 0.3) else -1
+        if q >= 0 and filled[q]:
+            q0, q1, q2 = max(int(n0[q]), 0), int(n1[q]), int(n2[q])
+            m1 = min(a1, q1)
+            host_tbl[r, a0:a0 + m1] = host_tbl[q, q0:q0 + m1]
+            m2 = min(a2, q2)
+            deep_tbl[r, a0 + a1:a0 + a1 + m2] = deep_tbl[q, q0 + q1:q0 + q1 + m2]
+        host_tbl[r, a0 + m1:a0 + a1] = host_ids[u1:u1 + a1 - m1]; u1 += a1 - m1
+        deep_tbl[r, a0 + a1 + m2:a0 + a1 + a2] = deep_ids[u2:u2 + a2 - m2]; u2 += a2 - m2
+    # -1 cells inside ranges (from sharing with shorter rows) are replaced by fresh ids where possible
+    hbm_free = np.full(n_hbm, -1, np.int32); hf = n_hbm - u0
+    hbm_free[:hf] = hbm_ids[u0:]
+    host_free = np.full(n_host, -1, np.int32); of = n_host - u1
+    host_free[:of] = host_ids[u1:]
+    hfc = int(rng.choice([hf, hf, min(hf, 3), 0]))
+    ofc = int(rng.choice([of, of, min(of, 3), 0]))
+    D = int(rng.choice([0, 8, 64, 1 << 16])); K = int(rng.choice([0, 4096, 1 << 20, 1 << 32]))
+    lay = kv_layout(n_hbm, 1, 16)
+    w = Workload("fuzz", d, reqs, now, D, K, lay, n_host, maxb + 1, hbm_tbl, host_tbl, hbm_free, hfc, host_free, ofc)
+    w.deep_tbl, w.deep_blocks = deep_tbl, n_deep
+    return w

@@ -75,6 +75,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->copy_bulk_dev = e ? atoi(e) : 2;
     e = getenv("CASCADE_MOVE_CTAS");
     ctx->move_ctas = e ? atoi(e) : 0;
+    e = getenv("CASCADE_RANK_SORT_MAX");
+    ctx->rank_sort_max = e ? atoi(e) : 2048;
     e = getenv("CASCADE_PDL");
     ctx->pdl = e ? (atoi(e) != 0) : 1;
     size_t n = (size_t)max_requests;

@@ -35,6 +35,7 @@ struct cascade_ctx {
     int copy_bulk_dev;           // >0: TMA bulk-copy ring for the device-staging path
     int move_ctas;               // >0: CTAs of the fused evict+restore kernel (at most one per SM)
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels
+    int rank_sort_max;           // queues up to this size are ordered by counting instead of radix passes
 };
 
 // plan_scalars layout

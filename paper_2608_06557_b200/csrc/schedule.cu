@@ -20,6 +20,11 @@
 // CTA has published the histogram of the elements it already holds in registers.  The mbarrier waits
 // are clock-bounded (CASCADE_ST_ETIMEOUT, results then undefined but every CTA still walks the same
 // cluster barriers and exits).  CASCADE_SORT_ASYNC=0 selects plain cluster barriers instead.
+//
+// Small queues (up to 2048 requests by default) skip the radix passes: with every key in each CTA's
+// shared memory, the final position of an element is simply the number of (key, slot) pairs below
+// it, counted by a few threads per element, and ONE exchange places every element.  The work is
+// quadratic but perfectly parallel, and at these sizes the eight passes' sixteen exchanges cost more.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -34,6 +39,8 @@ constexpr int kWhistStride = kBins + 2;  // in uint16 units: column reads by 32 
 constexpr int kMaxCluster = 16;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr long long kWaitLimit = 2000000000LL;  // clocks a CTA waits for its peers' data before giving up
+constexpr int kRankMaxKeys = 4096;              // keys the counting path can hold per CTA
+constexpr size_t kRankExtra = kRankMaxKeys * sizeof(uint64_t) + 256 * sizeof(int);
 
 struct __align__(16) SortElem {
     uint64_t key;
@@ -63,6 +70,7 @@ struct ScheduleArgs {
     int bt;
     int stage;          // 1: group by digit locally before the remote copy
     int async_sync;     // 1: per-pass exchanges complete on mbarriers (data driven), 0: cluster barriers
+    int rank_per;       // >0: small queue, order by counting (see rank_order below) with this many elements per CTA
     uint32_t *status;
 };
 
@@ -104,6 +112,11 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     Exch *exall = reinterpret_cast<Exch *>(wtmp + 3 * 32);             // [kMaxCluster]
     uint16_t *minehist = reinterpret_cast<uint16_t *>(exall + kMaxCluster);   // [kBins], 16-byte aligned
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(minehist + kBins);  // hist[2], elem[2]
+    // counting path only (the <256, 1> instance): every key of the queue, then per-thread partial counts
+    uint64_t *keys_all = reinterpret_cast<uint64_t *>(bars + 4);
+    int *partial = reinterpret_cast<int *>(keys_all + kRankMaxKeys);
+    const bool by_rank = (K == 1) && a.rank_per > 0;
+    const int per_rt = by_rank ? a.rank_per : per;   // elements this CTA holds
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned lt_mask = (1u << lane) - 1u;
@@ -125,8 +138,8 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
 #pragma unroll
     for (int k = 0; k < K; ++k) {
         const int li = (warp * K + k) * 32 + lane;
-        const long long g = (long long)crank * per + li;
-        if (g < a.n) {
+        const long long g = (long long)crank * per_rt + li;
+        if (li < per_rt && g < a.n) {
             const unsigned long long key = a.key[g];
             const long long P = a.prompt[g], h0 = a.n0[g], h1 = a.n1[g], h2 = a.n2[g];
             long long want = 0;
@@ -141,6 +154,51 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
             e[k].want = 0;
         }
     }
+    if (by_rank) {
+        if constexpr (K == 1) {
+            // ---- order by counting ----------------------------------------------------------------
+            // all keys of the queue into shared memory (coalesced, read once per CTA)
+            const int n = a.n;
+            for (int j = tid; j < n; j += T) keys_all[j] = a.key[j];
+            __syncthreads();
+            // S = T / per_rt threads share one element: thread t counts, for element t % per_rt, the pairs
+            // (key, slot) below it among the slots of segment t / per_rt
+            const int S = T / per_rt;
+            const int el = tid % per_rt, seg = tid / per_rt;
+            const long long gi = (long long)crank * per_rt + el;
+            int cnt = 0;
+            if (seg < S && gi < n) {
+                const unsigned long long ki = keys_all[gi];
+                const int seg_len = (n + S - 1) / S;
+                const int lo = seg * seg_len, hi = min(n, lo + seg_len);
+                const int mid = (int)min((long long)hi, max((long long)lo, gi));   // slots below gi: ties count
+                int j = lo;
+                for (; j + 4 <= mid; j += 4) {
+                    cnt += (keys_all[j] <= ki) + (keys_all[j + 1] <= ki) + (keys_all[j + 2] <= ki) + (keys_all[j + 3] <= ki);
+                }
+                for (; j < mid; ++j) cnt += keys_all[j] <= ki;
+                j = (int)max((long long)mid, min((long long)hi, gi + 1));            // slots above gi: ties do not
+                for (; j + 4 <= hi; j += 4) {
+                    cnt += (keys_all[j] < ki) + (keys_all[j + 1] < ki) + (keys_all[j + 2] < ki) + (keys_all[j + 3] < ki);
+                }
+                for (; j < hi; ++j) cnt += keys_all[j] < ki;
+            }
+            partial[tid] = cnt;
+            __syncthreads();
+            // the element's owner adds the partial counts and sends the element to its final place
+            if (tid < per_rt && e[0].idx != 0xffffffffu) {
+                int pos = 0;
+                for (int q = 0; q < S; ++q) pos += partial[q * per_rt + tid];
+                SortElem *dst = cluster.map_shared_rank(elems, pos / per_rt) + (pos % per_rt);
+                *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(&e[0]);
+            }
+            cluster.sync();
+            // slots n .. C*per_rt-1 of the sorted layout received nothing: they are padding
+            const long long g = (long long)crank * per_rt + tid;
+            if (tid < per_rt && g < n) e[0] = elems[tid];
+            else { e[0].key = ~0ull; e[0].idx = 0xffffffffu; e[0].want = 0; }
+        }
+    } else {
     {
         unsigned lo = __reduce_or_sync(kFull, (unsigned)diff);
         unsigned hi = __reduce_or_sync(kFull, (unsigned)(diff >> 32));
@@ -330,6 +388,7 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     }
     TICK(64);
     if (dead && tid == 0) atomicOr(a.status, CASCADE_ST_ETIMEOUT);
+    }  // radix path
 
     // ---- admission: clamped prefix sums over the sorted elements ---------------------------------
     long long ex[K];
@@ -433,7 +492,7 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     for (int k = 0; k < K; ++k) {
         if (grant[k] > 0 && (long long)(cnt_off + exf[k]) >= (long long)a.seq_cap) grant[k] = 0;
         if (e[k].idx != 0xffffffffu) {
-            const long long g = (long long)crank * per + (warp * K + k) * 32 + lane;
+            const long long g = (long long)crank * per_rt + (warp * K + k) * 32 + lane;
             a.order_out[g] = e[k].idx;
             a.grant_out[e[k].idx] = grant[k];
             tok += grant[k];
@@ -462,7 +521,7 @@ __global__ void zero_counts_kernel(cascade_sched_counts *c) {
 }
 
 size_t smem_bytes(int T, int K) {
-    return 2 * size_t(T) * K * sizeof(SortElem) + size_t(T / 32) * kWhistStride * sizeof(uint16_t) +
+    return (T == 256 && K == 1 ? kRankExtra : 0) + 2 * size_t(T) * K * sizeof(SortElem) + size_t(T / 32) * kWhistStride * sizeof(uint16_t) +
            2 * size_t(kMaxCluster) * kBins * sizeof(uint16_t) + 2 * kBins * sizeof(uint32_t) +
            3 * 32 * sizeof(long long) + kMaxCluster * sizeof(Exch) + kBins * sizeof(uint16_t) + 4 * 8 + 16;
 }
@@ -556,6 +615,20 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.bt = p.bt;
     a.stage = ctx->sort_stage >= 0 ? ctx->sort_stage : (K >= 4);
     a.async_sync = ctx->sort_async;
+    a.rank_per = 0;
+    if (n <= ctx->rank_sort_max && n <= kRankMaxKeys) {
+        // counting path: the widest cluster the device schedules, 256 threads, 32..256 elements per CTA
+        const int c = ctx->max_cluster > 0 ? (ctx->max_cluster < 16 ? ctx->max_cluster : 16) : 16;
+        int per_rank = (n + c - 1) / c;
+        per_rank = per_rank <= 32 ? 32 : (per_rank <= 64 ? 64 : (per_rank <= 128 ? 128 : 256));
+        if ((long long)per_rank * c >= n && per_rank <= 256) {
+            T = 256;
+            K = 1;
+            C = 1;
+            while (C * per_rank < n) C *= 2;      // cluster sizes stay powers of two; CTAs past the data hold padding
+            a.rank_per = per_rank;
+        }
+    }
     a.status = ctx->status_dev;
     cudaError_t e = T == 256 ? launch_k<256>(K, a, C, ctx->device, ctx->pdl, s) : launch_k<512>(K, a, C, ctx->device, ctx->pdl, s);
     CASCADE_CUDA_TRY(ctx, e);

@@ -64,7 +64,8 @@ def test_tiny_schedule_counts_match():
     assert int(sc[1]) == ref["sched_counts"]["tokens_granted"]
 
 
-@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 1023, 1024, 1025, 3000, 8192, 8193, 16384, 40000, 65536])
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 64, 65, 500, 513, 1023, 1024, 1025, 2047, 2048, 2049, 3000, 8192, 8193, 16384,
+                               40000, 65536])
 def test_llama8b_shaped_queue_sizes(n):
     """Spans every cluster / keys-per-thread configuration of the ordering kernel and ragged tails."""
     w = wl.config_llama8b(seed=n, n=n, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9, hbm_free_target=64)

@@ -76,3 +76,26 @@ def test_fused_move_on_random_shapes():
         assert np.array_equal(host.numpy(), ref_o), (n_hbm, n_host, n_chunks, cb, ne, nr, k)
         done += 1
     assert ctx.status()[0] == 0
+
+
+@pytest.mark.parametrize("n,reps", [(1024, 400), (2048, 200), (16384, 200), (65536, 40)])
+def test_repeated_runs_give_identical_results(n, reps):
+    """The cluster kernels exchange data through shared memory of other CTAs; an ordering bug there would show
+    as results that change from run to run.  Same inputs, many runs, every output compared with the first."""
+    import torch
+    from paper_2608_06557_b200.runner import Instance
+    sw = wl.SchedulerSweep(n, seed=5)
+    inst = Instance(sw.workload(), alloc_pools=False)
+    ref = None
+    for _ in range(reps):
+        for t in (inst.order, inst.grant, inst.x1, inst.tokens_run, inst.action):
+            t.fill_(0)
+        inst.run_schedule()
+        cur = [t[:n].clone() for t in (inst.budget, inst.key.view(torch.int64), inst.order.view(torch.int32), inst.grant,
+                                       inst.x1, inst.x2, inst.tokens_run, inst.action)] + [inst.plan_counts.clone(),
+                                                                                         inst.sched_counts.clone()]
+        if ref is None:
+            ref = cur
+        else:
+            assert all(torch.equal(a, b) for a, b in zip(ref, cur))
+    assert inst.ctx.status()[0] == 0

@@ -9,7 +9,7 @@ import pytest
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SRC = os.path.join(ROOT, "oracle", "cascade_oracle.cpp")
 PINS = ["test_oracle_plan_first.py", "test_oracle_budget.py", "test_oracle_schedule.py", "test_oracle_plan.py", "test_oracle_copy.py",
-        "test_oracle_prefetch.py", "test_oracle_policies.py"]
+        "test_oracle_prefetch.py", "test_oracle_policies.py", "test_oracle_more_pins.py"]
 
 DEEP_PINS = ["test_oracle_deep.py"]
 
@@ -64,6 +64,43 @@ MUTATIONS = [
      "want[r] = int64_t(prompt[r]) - (n0[r] + x1) * p->bt;"),
     ("regime 1 reuses the prefix", "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, 0) >> 20;",
      "lat4_out[4 * r + 1] = comp_q(p, tok_q(p, act), P, s_hit) >> 20;"),
+    # second batch: boundaries and terms the first batch did not touch
+    ("class index test off by one", "ok = ok && cls[r] < p->n_classes;", "ok = ok && cls[r] <= p->n_classes;"),
+    ("predicted output bound ignored", "ok = ok && O >= 0 && O <= (int64_t(1) << 20);", "ok = ok && O >= 0;"),
+    ("transfer of the deep part left out of the estimate",
+     "const int64_t tp = restore_time(p, 1, n1[r]) + restore_time(p, 2, n2[r]);\n        const int64_t L_act",
+     "const int64_t tp = restore_time(p, 1, n1[r]);\n        const int64_t L_act"),
+    ("maximum-load estimate uses the actual load",
+     "const int64_t L_max = tp + (comp_q(p, tok_q(p, mx), P, s_hit) >> 20);\n        /* B3",
+     "const int64_t L_max = tp + (comp_q(p, tok_q(p, act), P, s_hit) >> 20);\n        /* B3"),
+    ("decode step leaves out the prefill chunk", "const int64_t tdec_act = (iter_q(p, act1) + chunk_q) >> 20;",
+     "const int64_t tdec_act = (iter_q(p, act1)) >> 20;"),
+    ("clamp one too wide", "std::min(std::max(v, -kBudgetClamp), kBudgetClamp - 1) + kBudgetClamp;",
+     "std::min(std::max(v, -kBudgetClamp), kBudgetClamp) + kBudgetClamp;"),
+    ("fcfs newest first", "if (p->policy == ORC_POLICY_FCFS) { v = -elapsed; tier2 = false; }",
+     "if (p->policy == ORC_POLICY_FCFS) { v = elapsed; tier2 = false; }"),
+    ("sjf by whole prompt", "if (p->policy == ORC_POLICY_SJF) { v = P - s_hit; tier2 = false; }",
+     "if (p->policy == ORC_POLICY_SJF) { v = P; tier2 = false; }"),
+    ("sort not stable", "std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return key[a] < key[b]; });",
+     "std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return key[a] < key[b] || (key[a] == key[b] && a > b); });"),
+    ("offer ignores the deep part", "want[r] = int64_t(prompt[r]) - int64_t(n0[r] + n1[r] + n2[r]) * p->bt;",
+     "want[r] = int64_t(prompt[r]) - int64_t(n0[r] + n1[r]) * p->bt;"),
+    ("tier-2 queue does not get what tier-1 left", "left = TB - used1;", "left = R2;"),
+    ("regime 0 under the actual load", "lat4_out[4 * r + 0] = comp_q(p, tok_q(p, idle), P, 0) >> 20;",
+     "lat4_out[4 * r + 0] = comp_q(p, tok_q(p, act), P, 0) >> 20;"),
+    ("deep bound forgets the host transfer", "const int64_t rem2 = rem - restore_time(p, 1, n1);", "const int64_t rem2 = rem;"),
+    ("need forgets the partly filled block", "need[r] = int32_t(bx1 + (ceil_div(have + run, p->bt) - (n0[r] + bx1)));",
+     "need[r] = int32_t(bx1 + ((have + run) / p->bt - (n0[r] + bx1)));"),
+    ("spill test ignores the victim's budget", "const bool fits = restore_time(p, 1, n0[r]) <= budget[r];",
+     "const bool fits = true;"),
+    ("deficit off by one", "const int64_t deficit = std::max<int64_t>(0, need_total - hbm_cnt);",
+     "const int64_t deficit = std::max<int64_t>(0, need_total - hbm_cnt + 1);"),
+    ("prefetch bound ignores the reserve", "int64_t avail = hbm_pos - hbm_reserve;", "int64_t avail = hbm_pos;"),
+    ("prefetch restores although recomputing is cheaper",
+     "if (m > 0 && plan_cost_q20(p, act, prompt[r], n0[r], m, 0) > plan_cost_q20(p, act, prompt[r], n0[r], 0, 0)) m = 0;", ""),
+    ("prefetch link test forgets the overhead",
+     "const int64_t by_link = link_left > p->delta_ns[1] ? (link_left - p->delta_ns[1]) / p->blk_ns[1] : 0;",
+     "const int64_t by_link = link_left / p->blk_ns[1];"),
     # the deep-tier stage, the one-copy-per-source pass and the record copy have pins of their own
     ("stage hop charged the whole path", "std::max<int64_t>(0, p->delta_ns[2] - p->delta_ns[1]);",
      "std::max<int64_t>(0, p->delta_ns[2]);", DEEP_PINS),

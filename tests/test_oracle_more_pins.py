@@ -107,3 +107,29 @@ def test_prefetch_leaves_blocks_that_are_cheaper_to_recompute():
     fast = wl.default_params(blk_ns=[0, 40_000, 340_000])
     out = _queued_request(fast, n1=10, budget_ns=10 * S, link_budget=10 * S)
     assert out["pf"].tolist() == [10]
+
+
+def test_a_dropped_victim_takes_no_host_room_from_the_next_one():
+    """Two victims are needed.  The first one walked (last in the order) cannot be brought back within its own
+    budget and is dropped; the second fits and finds the host pool's 4 free records all its own."""
+    PRIV = oracle.FLAG_HBM_PRIVATE
+    p = oracle.make_params(wl.default_params())
+    maxb = 32
+    reqs = dict(prompt=[16 * 10, 400, 400], n0=[0, 4, 3], n1=[0, 0, 0], n2=[0, 0, 0], flags=[0, PRIV, PRIV])
+    hbm_tbl = np.full((3, maxb), -1, np.int32)
+    host_tbl = np.full((3, maxb), -1, np.int32)
+    hbm_tbl[1, :4] = [10, 11, 12, 13]
+    hbm_tbl[2, :3] = [20, 21, 22]
+    hf = np.full(64, -1, np.int32)
+    hf[:4] = [1, 2, 3, 4]
+    of = np.full(8, -1, np.int32)
+    of[:4] = [30, 31, 32, 33]
+    pools = oracle.Pools(hbm_tbl, host_tbl, hf, 4, of, 4, 64, 8)
+    budget = np.array([10**9, 10**9, 1000], np.int64)        # slot 2: T_1(3) = 10 us + 3 * 40 us > 1 us
+    order = np.array([0, 1, 2], np.uint32)
+    grant = np.array([160, 0, 0], np.int32)                  # slot 0 computes 10 blocks: 4 free, 6 short
+    out = oracle.tier_plan(p, reqs, budget, order, grant, 0, 0, pools)
+    assert out["counts"]["deficit"] == 6 and out["counts"]["n_victims"] == 2
+    assert out["action"].tolist() == [oracle.ACT_NONE, oracle.ACT_EVICT, oracle.ACT_DROP]
+    assert out["evict_src"].tolist() == [10, 11, 12, 13] and out["evict_dst"].tolist() == [33, 32, 31, 30]
+    assert out["counts"]["n_drop_blocks"] == 3 and pools.host_free_count == 0

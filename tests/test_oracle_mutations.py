@@ -101,6 +101,25 @@ MUTATIONS = [
     ("prefetch link test forgets the overhead",
      "const int64_t by_link = link_left > p->delta_ns[1] ? (link_left - p->delta_ns[1]) / p->blk_ns[1] : 0;",
      "const int64_t by_link = link_left / p->blk_ns[1];"),
+    # third batch
+    ("host room counted for victims that are dropped anyway", "if (fits) h += n0[r];", "h += n0[r];"),
+    ("one victim too many", "if (v < deficit) {", "if (v <= deficit) {"),
+    ("evicted block recorded one cell off", "host_tbl[int64_t(r) * maxb + j] = hslot;", "host_tbl[int64_t(r) * maxb + j + 1] = hslot;"),
+    ("admitted holders counted as preemptable",
+     "if (valid[r] && grant[r] <= 0 && (flags[r] & ORC_FLAG_HBM_PRIVATE)) evictable += n0[r];",
+     "if (valid[r] && (flags[r] & ORC_FLAG_HBM_PRIVATE)) evictable += n0[r];"),
+    ("restored blocks not counted as held", "const int64_t have = (n0[r] + bx1) * int64_t(p->bt);",
+     "const int64_t have = (n0[r]) * int64_t(p->bt);"),
+    ("runs one token past the prompt", "const int64_t run = (bx2 > 0) ? 0 : std::min<int64_t>(grant[r], P - have);",
+     "const int64_t run = (bx2 > 0) ? 0 : std::min<int64_t>(grant[r], P - have + 1);"),
+    ("tier-1 count from the wrong bit", "if (key[r] >> 63)\n            W2 += want[r];", "if (key[r] >> 62)\n            W2 += want[r];"),
+    ("unadmitted request keeps its restore", "x1_out[r] = x2_out[r] = tokens_run_out[r] = 0;\n            need[r] = 0;",
+     "x2_out[r] = tokens_run_out[r] = 0;\n            need[r] = 0;"),
+    ("victim keeps its table row", "if (with_tables) hbm_tbl[int64_t(r) * maxb + j] = -1;", ""),
+    ("retain mark for requests without blocks", "if (valid[r] && action_out[r] == ORC_ACT_NONE && n0[r] > 0) action_out[r] = ORC_ACT_RETAIN;",
+     "if (valid[r] && action_out[r] == ORC_ACT_NONE) action_out[r] = ORC_ACT_RETAIN;"),
+    ("copy skips the last chunk", "for (int c = 0; c < n_chunks; ++c)\n            std::memcpy(hbm_pool + c * chunk_stride + d * block_stride,",
+     "for (int c = 0; c + 1 < n_chunks; ++c)\n            std::memcpy(hbm_pool + c * chunk_stride + d * block_stride,"),
     # the deep-tier stage, the one-copy-per-source pass and the record copy have pins of their own
     ("stage hop charged the whole path", "std::max<int64_t>(0, p->delta_ns[2] - p->delta_ns[1]);",
      "std::max<int64_t>(0, p->delta_ns[2]);", DEEP_PINS),

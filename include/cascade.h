@@ -232,7 +232,11 @@ int cascade_set_params(cascade_ctx *ctx, const cascade_params *p);
  *   B_rem  = B - (now_ns - arrival_ns)                          Eq. 5
  *   budget = B_rem - pred_out * max(0, t_dec - tpot_ns[cls])    decode-overrun penalty, 0 if tpot_ns == 0
  *   key    = tier2 << 63 | (clamp(budget, -2^39, 2^39-1) + 2^39) << 23 | (id & 0x7FFFFF)
- * budget_out[n] and key_out[n] are written.
+ * budget_out[n] and key_out[n] are written (caller-owned device arrays).
+ * Errors: CASCADE_EINVAL (NULL pointer, n < 0, n > max_requests), CASCADE_ERANGE (D_act or K_act outside the
+ * bounds above), CASCADE_ECUDA (launch failed).  On the device: a request outside the input bounds, with a class
+ * index >= n_classes or with |now - arrival| > 2^50 gets budget -2^62 and the key (1 << 63 | id), i.e. the very
+ * end of the Tier-2 queue, and sets CASCADE_ST_EPRECOND.
  */
 int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, int64_t now_ns, int32_t D_act, int64_t K_act,
                    int64_t *budget_out, uint64_t *key_out, void *stream);
@@ -270,6 +274,9 @@ int cascade_reqs_update(cascade_ctx *ctx, const cascade_reqs *dst, int cap, cons
  *                 queue from the reserve plus what Tier-1 left; each request is offered
  *                 prompt - (n0+n1+n2)*bt tokens; at most max_batch - D_act requests are admitted.
  *   counts_dev    device struct, written.
+ * n = 0 writes zero counts.  A request outside the input bounds is offered nothing.
+ * Errors: CASCADE_EINVAL (NULL pointer, n out of range), CASCADE_ERANGE (D_act), CASCADE_ECUDA.  On the device:
+ * CASCADE_ST_ETIMEOUT if a bounded wait between the CTAs of the cluster expires (results then undefined).
  */
 int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const uint64_t *key, int n, int32_t D_act,
                      uint32_t *order_out, int32_t *grant_out, cascade_sched_counts *counts_dev, void *stream);
@@ -287,6 +294,12 @@ int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const uint64_t *ke
  *     computed blocks; tables, free lists, counts and the two copy lists are updated.
  * `grant` is read and updated.  `pools` and `plan_out` are host structs (copied during the call).
  * The evict list must be executed before the restore list (a freed block may be reused at once).
+ * Errors: CASCADE_EINVAL (NULL pointer, n out of range, tables without free lists, negative capacities),
+ * CASCADE_ERANGE (D_act, K_act), CASCADE_ECUDA.  On the device: CASCADE_ST_ENOSPC (admitted set cut),
+ * CASCADE_ST_EPRECOND (a request outside the input bounds, or whose prompt needs more than maxb table cells:
+ * its grant is zeroed and it is never a victim), CASCADE_ST_ELISTCAP (a copy list shorter than the plan:
+ * the counts still say how many entries there should have been), CASCADE_ST_EBOUNDS (a free-list count
+ * outside [0, capacity]: clamped).
  */
 int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *budget, const uint32_t *order,
                       int32_t *grant, int n, int32_t D_act, int64_t K_act, const cascade_pools *pools,
@@ -334,6 +347,9 @@ int cascade_prefetch_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t
  *   n_copies_dev   device scalar holding the count, or NULL to use n_copies_max itself
  *   n_copies_max   upper bound of the count (list capacity)
  * Destination ids must be distinct within a call.
+ * Errors: CASCADE_EINVAL (NULL pointer, negative count, chunk_bytes < 16, a size, stride or pool address that is
+ * not a multiple of 16), CASCADE_ECUDA.  On the device: CASCADE_ST_EBOUNDS (that pair is skipped),
+ * CASCADE_ST_ETIMEOUT (a bounded wait on a copy in flight expired: the CTA stops issuing work and returns).
  */
 int cascade_kv_restore(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, const void *src_pool,
                        int64_t src_blocks, int src_is_device, const int32_t *src_ids, const int32_t *dst_ids,

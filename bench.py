@@ -145,6 +145,30 @@ def run_oracle_arm(args, seconds, first_seed=0, max_steps=None, warmup=1):
                 ms_per_step=total_t / steps * 1e3, steps=steps)
 
 
+def oracle_schedule_latency():
+    """The oracle's budget + schedule + plan on the scheduler-scale sweep (plan-only), one core: median
+    microseconds over a few iterations with churn, per queue size."""
+    import oracle
+    from paper_2608_06557_b200 import workload as wl
+    out = {}
+    for n, iters in ((1024, 20), (4096, 10), (16384, 6), (65536, 4)):
+        sw = wl.SchedulerSweep(n, seed=0)
+        p = oracle.make_params(sw.params)
+        ts = []
+        for it in range(iters):
+            w = sw.workload()
+            pools = oracle.Pools(None, None, None, w.hbm_free_count, None, w.host_free_count, 0, 0)
+            t0 = time.perf_counter()
+            budget, key, _ = oracle.budget(p, w.reqs, w.now_ns, w.D_act, w.K_act)
+            order, grant, _, _ = oracle.schedule(p, w.reqs, key, w.D_act)
+            oracle.tier_plan(p, w.reqs, budget, order, grant, w.D_act, w.K_act, pools)
+            if it:                                   # the first iteration warms the caches
+                ts.append((time.perf_counter() - t0) * 1e6)
+            sw.step()
+        out[str(n)] = round(statistics.median(ts), 1)
+    return out
+
+
 def reference_main(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -647,6 +671,8 @@ def ours_main(args):
                 parity="bit-exact against the CPU oracle: see tests/ (-m gpu)")
         line["cpu_baseline"] = {k: v for k, v in run_oracle_arm(args, args.cpu_seconds, first_seed=W).items()
                                 if k in ("value", "unit", "cores", "kind", "sample")}
+        if not args.no_sweeps:
+            line["cpu_baseline"]["schedule_latency_us"] = oracle_schedule_latency()
         print(json.dumps(line))
     if use_dist:
         dist.barrier()

@@ -172,16 +172,27 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                 const int seg_len = (n + S - 1) / S;
                 const int lo = seg * seg_len, hi = min(n, lo + seg_len);
                 const int mid = (int)min((long long)hi, max((long long)lo, gi));   // slots below gi: ties count
-                int j = lo;
-                for (; j + 4 <= mid; j += 4) {
-                    cnt += (keys_all[j] <= ki) + (keys_all[j + 1] <= ki) + (keys_all[j + 2] <= ki) + (keys_all[j + 3] <= ki);
-                }
-                for (; j < mid; ++j) cnt += keys_all[j] <= ki;
-                j = (int)max((long long)mid, min((long long)hi, gi + 1));            // slots above gi: ties do not
-                for (; j + 4 <= hi; j += 4) {
-                    cnt += (keys_all[j] < ki) + (keys_all[j + 1] < ki) + (keys_all[j + 2] < ki) + (keys_all[j + 3] < ki);
-                }
-                for (; j < hi; ++j) cnt += keys_all[j] < ki;
+                // two keys per 16-byte shared-memory load, eight keys per round: the loads of a round are
+                // independent, so their latency overlaps
+                auto count_range = [&](int from, int to, bool ties) {
+                    int j = from;
+                    int c = 0;
+                    for (; j < to && (j & 1); ++j) c += ties ? keys_all[j] <= ki : keys_all[j] < ki;
+                    const ulonglong2 *pairs = reinterpret_cast<const ulonglong2 *>(keys_all);
+                    for (; j + 8 <= to; j += 8) {
+                        ulonglong2 v[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) v[u] = pairs[(j >> 1) + u];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            c += ties ? (v[u].x <= ki) + (v[u].y <= ki) : (v[u].x < ki) + (v[u].y < ki);
+                        }
+                    }
+                    for (; j < to; ++j) c += ties ? keys_all[j] <= ki : keys_all[j] < ki;
+                    return c;
+                };
+                cnt = count_range(lo, mid, true);
+                cnt += count_range((int)max((long long)mid, min((long long)hi, gi + 1)), hi, false);   // above gi: ties do not count
             }
             partial[tid] = cnt;
             __syncthreads();

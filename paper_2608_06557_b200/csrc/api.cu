@@ -77,6 +77,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->move_ctas = e ? atoi(e) : 0;
     e = getenv("CASCADE_RANK_SORT_MAX");
     ctx->rank_sort_max = e ? atoi(e) : 2048;
+    e = getenv("CASCADE_TEST_MOVE_STALL");
+    ctx->test_move_stall = e ? (atoi(e) != 0) : 0;
     e = getenv("CASCADE_PDL");
     ctx->pdl = e ? (atoi(e) != 0) : 1;
     size_t n = (size_t)max_requests;

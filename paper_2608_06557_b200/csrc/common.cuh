@@ -36,6 +36,7 @@ struct cascade_ctx {
     int move_ctas;               // >0: CTAs of the fused evict+restore kernel (at most one per SM)
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels
     int rank_sort_max;           // queues up to this size are ordered by counting instead of radix passes
+    int test_move_stall;         // test hook (CASCADE_TEST_MOVE_STALL=1): see MoveArgs::stall
 };
 
 // plan_scalars layout

@@ -230,6 +230,7 @@ struct MoveArgs {
     int n_chunks;
     int n_evict_max, n_restore_max;
     int pieces_per_chunk;
+    int stall;       // test hook: the evict side never reports a block as read out (exercises the bounded wait)
 };
 
 __device__ __forceinline__ int clamp_count(const int32_t *dev, int maxv) {
@@ -343,14 +344,15 @@ __global__ void __launch_bounds__(32) kv_move_kernel(const __grid_constant__ Mov
         }
         bool skip = false;
         if (evict_of[slot] >= 0) {
-            atomicAdd(&a.done[evict_of[slot]], 1);  // this piece of the block has left HBM
+            if (!a.stall) atomicAdd(&a.done[evict_of[slot]], 1);  // this piece of the block has left HBM
         } else if (wait_of[slot] >= 0) {
             // the HBM block is being evicted by this same call: write only after it has been read out
             const volatile int32_t *flag = a.done + wait_of[slot];
             t0 = clock64();
             if (st & CASCADE_ST_ETIMEOUT) skip = true;  // one expired wait is enough: do not queue up more
+            const long long limit = a.stall ? kWaitCycles / 20 : kWaitCycles;
             while (!skip && *flag < (int)per_block) {
-                if (clock64() - t0 > kWaitCycles) {
+                if (clock64() - t0 > limit) {
                     st |= CASCADE_ST_ETIMEOUT;
                     skip = true;
                     break;
@@ -501,6 +503,7 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     a.n_evict_max = n_evict_max;
     a.n_restore_max = n_restore_max;
     a.pieces_per_chunk = (int)((hbm->chunk_bytes + kBulkPiece - 1) / kBulkPiece);
+    a.stall = ctx->test_move_stall;
     const int most = n_evict_max > n_restore_max ? n_evict_max : n_restore_max;
     int pgrid = (most + 255) / 256;
     if (pgrid > ctx->num_sms * 4) pgrid = ctx->num_sms * 4;

@@ -224,3 +224,44 @@ def test_full_iteration_with_fused_move(seed):
     assert got["plan_counts"] == plan["counts"] and got["status"] == ref["status"]
     assert np.array_equal(inst.hbm_pool.cpu().numpy(), hbm_np)
     assert np.array_equal(inst.host_pool.cpu().numpy(), host_np)
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable(monkeypatch):
+    """The fused move makes a restore wait until the block it lands in has been read out by the evict side.
+    With the library's test hook the evict side never reports that, so the wait runs into its clock limit
+    (a tenth of a second here): the call returns, CASCADE_ST_ETIMEOUT is set, the evicted bytes are on the
+    host, the blocks whose restores gave up are untouched, and the same GPU context goes on working."""
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    n_chunks, cb = 2, 4096
+    bb = n_chunks * cb
+    n_hbm, n_host = 16, 16
+    lay = wl.kv_layout(n_hbm, n_chunks, cb)
+    rng = np.random.default_rng(0)
+    hbm_np = rng.integers(0, 256, n_hbm * bb, dtype=np.uint8)
+    host_np = rng.integers(0, 256, n_host * bb, dtype=np.uint8)
+    es, ed = np.array([1, 2], np.int32), np.array([5, 6], np.int32)
+    rs, rd = np.array([8, 9], np.int32), np.array([2, 12], np.int32)      # the first restore lands in an evicted block
+    t = lambda a: torch.from_numpy(a).cuda()
+    monkeypatch.setenv("CASCADE_TEST_MOVE_STALL", "1")
+    stalled = cs.Context(wl.default_params(), 16, 0)
+    monkeypatch.delenv("CASCADE_TEST_MOVE_STALL")
+    hbm, host = torch.from_numpy(hbm_np.copy()).cuda(), torch.from_numpy(host_np.copy()).pin_memory()
+    scratch = torch.empty(8, dtype=torch.int32, device="cuda")
+    stalled.kv_move(cs.make_layout(lay), hbm, host, n_host, t(es), t(ed), None, 2, t(rs), t(rd), None, 2, scratch)
+    torch.cuda.synchronize()
+    assert stalled.status()[0] == cs.ST_ETIMEOUT
+    want_host = host_np.copy()
+    assert oracle.kv_evict(hbm_np.copy(), lay, want_host, n_host, es, ed) == 0
+    assert np.array_equal(host.numpy(), want_host)                        # the evictions happened
+    want_hbm = hbm_np.copy()
+    assert oracle.kv_restore(want_hbm, lay, host_np, n_host, rs[1:], rd[1:]) == 0
+    assert np.array_equal(hbm.cpu().numpy(), want_hbm)                    # the independent restore too; block 2 untouched
+    # same process, same GPU, ordinary context: the full result
+    ctx = cs.Context(wl.default_params(), 16, 0)
+    hbm, host = torch.from_numpy(hbm_np.copy()).cuda(), torch.from_numpy(host_np.copy()).pin_memory()
+    ctx.kv_move(cs.make_layout(lay), hbm, host, n_host, t(es), t(ed), None, 2, t(rs), t(rd), None, 2, scratch)
+    torch.cuda.synchronize()
+    ref_h, ref_o = hbm_np.copy(), host_np.copy()
+    assert oracle.kv_evict(ref_h, lay, ref_o, n_host, es, ed) == 0 and oracle.kv_restore(ref_h, lay, ref_o, n_host, rs, rd) == 0
+    assert ctx.status()[0] == 0 and np.array_equal(hbm.cpu().numpy(), ref_h) and np.array_equal(host.numpy(), ref_o)

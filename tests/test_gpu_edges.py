@@ -102,3 +102,70 @@ def test_degenerate_policies_and_pools(case):
         assert got["sched_counts"]["n_tier1"] == 0 and got["sched_counts"]["n_admitted"] > 0
     if case == "no_hbm":
         assert got["plan_counts"]["n_admitted"] == 0 and got["status"] & 2
+
+
+def test_empty_queue_and_empty_lists_through_the_added_calls():
+    """n = 0 and zero-length lists for the stage plan, the merge pass, the stage copy and the queue update."""
+    import torch
+    from paper_2608_06557_b200.runner import Instance
+    w = wl.config_deep_shared(0, n=64, n_hbm=512, n_host=512, n_deep=512, n_chunks=2, chunk_bytes=64)
+    inst = Instance(w)
+    inst.enable_deep(w)
+    pools = [inst.hbm_pool.fill_(1).clone(), inst.host_pool.fill_(2).clone(), inst.deep_pool.fill_(3).clone()]
+    inst.n = 0
+    host_before, hbm_before = inst.host_free_count.item(), inst.hbm_free_count.item()
+    tbl_before = (inst.hbm_tbl.clone(), inst.host_tbl.clone())
+    inst.stage_counts.fill_(7)
+    inst.dedup_counts_restore.fill_(7)
+    inst.dedup_counts_stage.fill_(7)
+    inst.run_iteration_deep(10**9, 0)
+    inst.stage_slot_update(w.reqs, np.zeros(0, np.int64))
+    inst.run_slot_update()
+    got, deep = inst.fetch(), inst.fetch_deep()
+    assert got["status"] == 0
+    assert deep["stage_counts"] == dict(n_stage=0, n_requests=0, n_short=0, host_free_after=host_before,
+                                        link_ns_left=10**9)
+    for k in ("dedup_restore", "dedup_stage"):
+        c = deep[k]
+        assert (c["n_in"], c["n_unique"], c["n_surplus"], c["n_shared_requests"], c["max_share"]) == (0, 0, 0, 0, 0)
+    assert deep["dedup_restore"]["free_after"] == hbm_before and deep["dedup_stage"]["free_after"] == host_before
+    assert got["hbm_free_count"] == hbm_before and got["host_free_count"] == host_before
+    assert torch.equal(inst.hbm_tbl, tbl_before[0]) and torch.equal(inst.host_tbl, tbl_before[1])
+    assert torch.equal(inst.hbm_pool, pools[0]) and torch.equal(inst.host_pool, pools[1]) and torch.equal(inst.deep_pool, pools[2])
+
+
+def test_parameters_replaced_between_iterations():
+    """cascade_set_params takes effect for the calls made afterwards; a rejected block leaves the old one in place."""
+    from paper_2608_06557_b200 import cascade as cs
+    from paper_2608_06557_b200.runner import Instance
+    w = wl.config_tiny(2)
+    inst = Instance(w, alloc_pools=False)
+    inst.run_schedule()
+    first = inst.fetch()
+    ref = oracle_iteration(w)
+    assert np.array_equal(first["budget"], ref["budget"]) and np.array_equal(first["grant"], ref["grant"])
+    w2 = wl.config_tiny(2)
+    w2.params = dict(w2.params, ttft_ns=[4 * S, 9 * S], gamma_q16=70000, token_budget=999, plan_first=1, c_tok_q20=30_000 << 20)
+    inst2 = Instance(w2, alloc_pools=False, ctx=inst.ctx)          # same context, new parameters
+    inst2.run_schedule()
+    second = inst2.fetch()
+    ref2 = oracle_iteration(w2)
+    for k in ("budget", "key", "order", "grant"):
+        assert np.array_equal(second[k], ref2[k]), k
+    assert second["plan_counts"] == ref2["plan"]["counts"] and not np.array_equal(second["budget"], first["budget"])
+    with pytest.raises(cs.CascadeError):
+        inst.ctx.set_params(dict(w2.params, bt=0))
+    inst3 = Instance(w2, alloc_pools=False, ctx=None)               # reference run with a fresh context
+    inst3.run_schedule()
+    third = inst3.fetch()
+    inst2.ctx.params = cs.make_params(w2.params)
+    inst2.hbm_free_count.fill_(w2.hbm_free_count)
+    inst2.host_free_count.fill_(w2.host_free_count)
+    inst2.hbm_tbl.copy_(inst3.hbm_tbl.new_tensor(w2.hbm_tbl))
+    inst2.host_tbl.copy_(inst3.host_tbl.new_tensor(w2.host_tbl))
+    inst2.hbm_free.copy_(inst3.hbm_free.new_tensor(w2.hbm_free))
+    inst2.host_free.copy_(inst3.host_free.new_tensor(w2.host_free))
+    inst2.run_schedule()                                            # the rejected call changed nothing
+    again = inst2.fetch()
+    for k in ("budget", "key", "order", "grant", "x1", "action"):
+        assert np.array_equal(again[k], third[k]), k

@@ -232,8 +232,9 @@ class Context:
     __del__ = close
 
     def set_params(self, params: dict | Params):
-        self.params = params if isinstance(params, Params) else make_params(params)
-        _check(_lib.cascade_set_params(self._h, C.byref(self.params)), "cascade_set_params")
+        new = params if isinstance(params, Params) else make_params(params)
+        _check(_lib.cascade_set_params(self._h, C.byref(new)), "cascade_set_params")
+        self.params = new
 
     def reqs_update(self, dst: Reqs, cap, src: Reqs, slots, m, stream=None):
         _check(_lib.cascade_reqs_update(self._h, C.byref(dst), cap, C.byref(src), _p(slots), m, _stream(stream)),

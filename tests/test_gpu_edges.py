@@ -158,7 +158,6 @@ def test_parameters_replaced_between_iterations():
     inst3 = Instance(w2, alloc_pools=False, ctx=None)               # reference run with a fresh context
     inst3.run_schedule()
     third = inst3.fetch()
-    inst2.ctx.params = cs.make_params(w2.params)
     inst2.hbm_free_count.fill_(w2.hbm_free_count)
     inst2.host_free_count.fill_(w2.host_free_count)
     inst2.hbm_tbl.copy_(inst3.hbm_tbl.new_tensor(w2.hbm_tbl))

@@ -325,7 +325,7 @@ def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, st
         es, ed, rs = hp[:m], op[:m], op[m:2 * m]
         rd = np.concatenate([es[::-1][: m // 2], hp[m:2 * m - m // 2]]).astype(np.int32)
         t = [torch.from_numpy(np.ascontiguousarray(x)).cuda() for x in (es, ed, rs, rd)]
-        scratch = torch.empty(2 * m, dtype=torch.int32, device="cuda")
+        scratch = torch.empty(cs.kv_move_scratch_len(m, m), dtype=torch.int32, device="cuda")
         best = 1e30
         for it in range(6):
             a, b = event_pair(torch)

@@ -217,7 +217,8 @@ typedef struct cascade_ctx cascade_ctx;
  * <= 4096 times the largest thread-block cluster the device co-schedules: 16 on a full B200).
  * Validates the parameters against the bounds above.  Allocates scratch (about 44 bytes per request).
  * `p` and `out` are host pointers.  The calling thread's current device is left as it was; the hot calls
- * launch on the current device, so make `device` current (and pass one of its streams) when calling them. */
+ * launch on the current device, so make `device` current (and pass one of its streams) when calling them:
+ * a call made while another device is current returns CASCADE_EINVAL and launches nothing. */
 int cascade_create(cascade_ctx **out, const cascade_params *p, int max_requests, int device);
 void cascade_destroy(cascade_ctx *ctx);
 /* Replaces the parameters (same validation); takes effect for calls made afterwards. */
@@ -349,7 +350,8 @@ int cascade_prefetch_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t
  * Destination ids must be distinct within a call.
  * Errors: CASCADE_EINVAL (NULL pointer, negative count, chunk_bytes < 16, a size, stride or pool address that is
  * not a multiple of 16), CASCADE_ECUDA.  On the device: CASCADE_ST_EBOUNDS (that pair is skipped),
- * CASCADE_ST_ETIMEOUT (a bounded wait on a copy in flight expired: the CTA stops issuing work and returns).
+ * CASCADE_ST_ETIMEOUT (a bounded wait on a copy in flight expired: the CTA stops issuing work, waits, bounded
+ * again, for the loads it already issued, and returns).
  */
 int cascade_kv_restore(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, const void *src_pool,
                        int64_t src_blocks, int src_is_device, const int32_t *src_ids, const int32_t *dst_ids,
@@ -361,16 +363,25 @@ int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, const void 
                      const int32_t *n_copies_dev, int n_copies_max, void *stream);
 
 /*
- * Evict and restore in one call, with the host link used in both directions at once.  Same result as
- * cascade_kv_evict on the evict list followed by cascade_kv_restore on the restore list (the order the
- * tier plan requires): a restore whose HBM block is also evicted by this call waits, block by block,
- * until that block has been read out.  Both lists as in the two calls above; the host pool must be
+ * Evict and restore in one call, with the host link used in both directions at once ("Budget-aware
+ * preemption": a victim's KV is spilled and its freed HBM blocks are handed out again in the same iteration).
+ * Same result as cascade_kv_evict on the evict list followed by cascade_kv_restore on the restore list (the
+ * order the tier plan requires): a restore whose HBM block is also evicted by this call waits, block by
+ * block, until that block has been read out.  Both lists as in the two calls above; the host pool must be
  * pinned, mapped host memory (or device memory).
- *   scratch   caller-owned device array of n_evict_max + n_restore_max int32 (contents irrelevant)
- * The grid is one CTA per SM; the per-block waits assume those CTAs become resident (true unless
- * the GPU is saturated by other long-running kernels) and are clock-bounded: on expiry
- * CASCADE_ST_ETIMEOUT is set and that block is not written.
+ *   scratch   caller-owned device array of cascade_kv_move_scratch_len(n_evict_max, n_restore_max) int32;
+ *             contents irrelevant before the call.  After the call scratch[i], i < restore count, is the
+ *             number of pieces of restore i that were NOT written: 0 = that block is complete, > 0 = a
+ *             bounded wait ran out or an id was outside its pool (the matching status bit is set as well).
+ * Residency rule: the evict side and the restore side are two grids of at most half the SMs each.  The
+ * restore grid is a programmatic dependent of the evict grid, so the hardware starts it only when every
+ * CTA of the evict grid is running or done; a waiting restore CTA therefore only ever waits for CTAs that
+ * already hold an SM and that never wait themselves.  The call is safe beside other long-running kernels
+ * (it only gets slower).  With programmatic launch off (CASCADE_PDL=0) the two grids run one after the other.
+ * The per-block waits are clock-bounded all the same: on expiry CASCADE_ST_ETIMEOUT is set and that piece
+ * is not written.
  */
+int64_t cascade_kv_move_scratch_len(int n_evict_max, int n_restore_max);
 int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, void *host_pool,
                     int64_t host_blocks, const int32_t *evict_src, const int32_t *evict_dst,
                     const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,

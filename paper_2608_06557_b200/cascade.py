@@ -24,7 +24,8 @@ ACT_NONE, ACT_RETAIN, ACT_EVICT, ACT_DROP = 0, 1, 2, 3
 EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_budget", "cascade_schedule",
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
            "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan", "cascade_kv_move",
-           "cascade_stage_plan", "cascade_kv_stage", "cascade_dedup", "cascade_reqs_update")
+           "cascade_stage_plan", "cascade_kv_stage", "cascade_dedup", "cascade_reqs_update",
+           "cascade_kv_move_scratch_len")
 
 
 class Params(C.Structure):
@@ -140,6 +141,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_status.argtypes = [vp, C.POINTER(Status), C.c_int, vp]
     lib.cascade_kv_move.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int,
                                     vp, vp]
+    lib.cascade_kv_move_scratch_len.argtypes = [C.c_int, C.c_int]
     lib.cascade_reqs_update.argtypes = [vp, C.POINTER(Reqs), C.c_int, C.POINTER(Reqs), vp, C.c_int, vp]
     lib.cascade_stage_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64, i64, i32, C.POINTER(Pools),
                                        C.POINTER(Stage), vp]
@@ -150,6 +152,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     for name in EXPORTS:
         if name != "cascade_destroy":
             getattr(lib, name).restype = C.c_int
+    lib.cascade_kv_move_scratch_len.restype = C.c_int64
     return lib
 
 
@@ -207,6 +210,11 @@ def _check(rc: int, what: str):
         names = {EINVAL: "CASCADE_EINVAL", ERANGE: "CASCADE_ERANGE", ECUDA: "CASCADE_ECUDA", ENOMEM: "CASCADE_ENOMEM",
                  ETOOBIG: "CASCADE_ETOOBIG"}
         raise CascadeError(f"{what} failed: {names.get(rc, rc)}")
+
+
+def kv_move_scratch_len(n_evict_max: int, n_restore_max: int) -> int:
+    """int32 entries cascade_kv_move needs in its caller-owned scratch."""
+    return int(_lib.cascade_kv_move_scratch_len(n_evict_max, n_restore_max))
 
 
 def make_reqs(t: dict) -> Reqs:

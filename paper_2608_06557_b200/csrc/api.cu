@@ -75,10 +75,17 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->copy_bulk_dev = e ? atoi(e) : 2;
     e = getenv("CASCADE_MOVE_CTAS");
     ctx->move_ctas = e ? atoi(e) : 0;
+    e = getenv("CASCADE_COPY_PIECE");
+    ctx->copy_piece = e ? atoi(e) : 0;
+    if (ctx->copy_piece != 8192 && ctx->copy_piece != 16384 && ctx->copy_piece != 32768) ctx->copy_piece = 0;
+    e = getenv("CASCADE_COPY_RING_KB");
+    ctx->copy_ring_kb = e ? atoi(e) : 0;
+    if (ctx->copy_ring_kb < 64 || ctx->copy_ring_kb > 128) ctx->copy_ring_kb = 0;
     e = getenv("CASCADE_RANK_SORT_MAX");
     ctx->rank_sort_max = e ? atoi(e) : 2048;
     e = getenv("CASCADE_TEST_MOVE_STALL");
-    ctx->test_move_stall = e ? (atoi(e) != 0) : 0;
+    ctx->test_move_stall = e ? atoi(e) : 0;
+    if (ctx->test_move_stall < 0 || ctx->test_move_stall > 3) ctx->test_move_stall = 0;
     e = getenv("CASCADE_PDL");
     ctx->pdl = e ? (atoi(e) != 0) : 1;
     size_t n = (size_t)max_requests;
@@ -126,6 +133,7 @@ extern "C" int cascade_set_params(cascade_ctx *ctx, const cascade_params *p) {
 
 extern "C" int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream) {
     if (!ctx || !host_out) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     cudaStream_t s = (cudaStream_t)stream;
     CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(uint32_t),
                                           cudaMemcpyDeviceToHost, s));

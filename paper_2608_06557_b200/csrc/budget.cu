@@ -132,6 +132,7 @@ extern "C" int cascade_reqs_update(cascade_ctx *ctx, const cascade_reqs *dst, in
                                    const int32_t *slots, int m, void *stream) {
     CascadeRange nvtx_range("cascade_reqs_update");
     if (!ctx || !dst || !src || cap < 0 || m < 0) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (m == 0) return CASCADE_OK;
     const cascade_reqs *both[2] = {dst, src};
     for (const cascade_reqs *q : both)
@@ -148,6 +149,7 @@ extern "C" int cascade_budget(cascade_ctx *ctx, const cascade_reqs *r, int n, in
                               int64_t K_act, int64_t *budget_out, uint64_t *key_out, void *stream) {
     CascadeRange nvtx_range("cascade_budget");
     if (!ctx || !r || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (n == 0) return CASCADE_OK;
     if (!budget_out || !key_out || !r->arrival_ns || !r->prompt || !r->pred_out || !r->n0 || !r->n1 || !r->n2 ||
         !r->id || !r->cls)
@@ -165,6 +167,7 @@ extern "C" int cascade_latency_regimes(cascade_ctx *ctx, const cascade_reqs *r, 
                                        int64_t *lat4_out, void *stream) {
     CascadeRange nvtx_range("cascade_latency_regimes");
     if (!ctx || !r || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (n == 0) return CASCADE_OK;
     if (!lat4_out || !r->prompt || !r->n0 || !r->n1 || !r->n2) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;

@@ -33,10 +33,15 @@ struct cascade_ctx {
     int copy_ctas_dev;           // copy CTAs per SM when the record pool is device memory
     int copy_bulk_host;          // >0: TMA bulk-copy ring (that many CTAs per SM) for the pinned-host path
     int copy_bulk_dev;           // >0: TMA bulk-copy ring for the device-staging path
-    int move_ctas;               // >0: CTAs of the fused evict+restore kernel (at most one per SM)
+    int move_ctas;               // >0: CTAs of each of the two grids of the fused evict+restore (at most half the SMs)
+    int copy_piece;              // >0: piece size in bytes of the TMA ring (8192 | 16384 | 32768); 0 = picked per call
+    int copy_ring_kb;            // >0: shared memory of the TMA ring in KiB (64..128); 0 = 128 (host) / 96 (device)
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels
     int rank_sort_max;           // queues up to this size are ordered by counting instead of radix passes
-    int test_move_stall;         // test hook (CASCADE_TEST_MOVE_STALL=1): see MoveArgs::stall
+    int test_move_stall;         // test hooks (CASCADE_TEST_MOVE_STALL): 1 = the evict side of the fused move never
+                                 // reports a block as read out, 2 = the first piece of CTA 0 of a ring kernel announces
+                                 // more bytes than it loads; both make a bounded wait run out; 1, 2 and 3 lower the
+                                 // limit of every bounded wait of the copy kernels to a tenth of a second
 };
 
 // plan_scalars layout
@@ -198,6 +203,13 @@ static inline cudaError_t cascade_launch(bool pdl, int cluster, dim3 grid, dim3 
     cfg.attrs = attr;
     cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args &&>(args)...);
+}
+
+// The hot calls launch on the calling thread's current device and dereference the context's allocations there:
+// a context of another device is rejected on the host (CASCADE_EINVAL) before anything is launched.
+static inline bool cascade_on_ctx_device(const cascade_ctx *ctx) {
+    int d = -1;
+    return cudaGetDevice(&d) == cudaSuccess && d == ctx->device;
 }
 
 // entry points implemented in the other translation units

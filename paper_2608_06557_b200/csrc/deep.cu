@@ -494,6 +494,7 @@ extern "C" int cascade_stage_plan(cascade_ctx *ctx, const cascade_reqs *r, const
                                   const cascade_stage *stage, void *stream) {
     CascadeRange nvtx_range("cascade_stage_plan");
     if (!ctx || !r || !pools || !stage || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (!stage->counts || !pools->host_free_count) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
     if (link_budget_ns < 0 || link_budget_ns > (int64_t(1) << 50) || host_reserve < 0) return CASCADE_ERANGE;
@@ -540,6 +541,7 @@ extern "C" int cascade_stage_plan(cascade_ctx *ctx, const cascade_reqs *r, const
 extern "C" int cascade_dedup(cascade_ctx *ctx, const cascade_dedup_args *u, int n, void *stream) {
     CascadeRange nvtx_range("cascade_dedup");
     if (!ctx || !u || n < 0) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (!u->list_count || !u->free_count || !u->counts || !u->scratch || u->list_cap < 0 || u->free_cap < 0 ||
         u->n_src_ids < 0 || u->n_dst_ids < 0 || u->maxb < 0)
         return CASCADE_EINVAL;

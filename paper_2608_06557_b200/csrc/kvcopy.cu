@@ -1,14 +1,15 @@
-// cascade_kv_restore / cascade_kv_evict: paged KV-block copies between a record-major pool
-// (pinned host memory read or written over the host link, or a device staging buffer) and the
-// paged HBM pool, driven by (src id, dst id) lists that live in device memory.
+// cascade_kv_restore / cascade_kv_evict / cascade_kv_move / cascade_kv_stage: paged KV-block copies
+// between a record-major pool (pinned host memory read or written over the host link, or a device
+// staging buffer) and the paged HBM pool, driven by (src id, dst id) lists that live in device memory.
 //
 // The bytes are opaque.  A block is n_chunks pieces of chunk_bytes; on the record side they are
 // back to back, on the HBM side chunk c of block b sits at c*chunk_stride + b*block_stride.
 // Two kernels do the same copy:
-//   kv_copy_bulk_kernel (default)  one elected thread per CTA drives TMA bulk copies
-//       (cp.async.bulk) through a 4-slot shared-memory ring, 32 KiB pieces, one or two CTAs per SM;
+//   kv_ring_kernel (default)  one elected thread per CTA drives TMA bulk copies (cp.async.bulk)
+//       through a shared-memory ring; the piece size (8, 16 or 32 KiB) is picked per call from the
+//       number of blocks actually moved, so that a call of one block still spreads over the grid;
 //       it leaves the SMs' issue slots free for whatever else runs on the GPU;
-//   kv_copy_kernel                 256 threads x 4 x 16-byte vector loads/stores per 16 KiB piece on a
+//   kv_copy_kernel            256 threads x 4 x 16-byte vector loads/stores per 16 KiB piece on a
 //       persistent grid (selected with CASCADE_COPY_BULK_HOST=0 / CASCADE_COPY_BULK_DEV=0).
 #include "common.cuh"
 
@@ -29,7 +30,14 @@ struct CopyArgs {
     long long chunk_bytes, chunk_stride, block_stride;
     int n_chunks;
     int n_max;
-    int pieces_per_chunk;
+    int pieces_per_chunk;     // vector kernel only
+    int ring_bytes;           // ring kernel: shared memory of the ring
+    int piece_fixed;          // ring kernel: >0 forces this piece size (bytes), 0 = pick per call
+    // fused move only
+    const int32_t *dep;       // per restore: evict-list index of the entry that frees its HBM block, or -1
+    int32_t *done;            // per evict entry: 16-byte units of the block already read out of HBM
+    int32_t *skipped;         // per restore: pieces that were NOT written (0 = the block is complete)
+    int stall;                // test hooks, see cascade_ctx::test_move_stall
 };
 
 template <bool kRestore>
@@ -77,17 +85,25 @@ __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant
 }
 
 
-// ---- bulk-copy variant: TMA (cp.async.bulk) through a shared-memory ring ---------------------------
-// One elected thread per CTA moves pieces of up to 32 KiB: global -> shared with an mbarrier that
-// counts the arriving bytes, then shared -> global as a bulk store group.  kStages ring slots; two
-// loads are kept in flight ahead of the piece being stored, and a slot is refilled only after the
-// store that last used it has finished reading shared memory.  Every wait is bounded: when the
-// clock limit is hit the kernel records CASCADE_ST_ETIMEOUT, stops issuing work, drains its own
-// store groups and returns.
-constexpr int kBulkPiece = 32 * 1024;
-constexpr int kStages = 4;
-constexpr int kAhead = kStages - 2;
+// ---- ring kernel: TMA bulk copies (cp.async.bulk) through a shared-memory ring ----------------------
+// One elected thread per CTA moves pieces: global -> shared with an mbarrier that counts the arriving
+// bytes, then shared -> global as a bulk store group.  The ring has S = ring_bytes / piece slots; S - 1
+// loads are kept in flight ahead of the piece being stored, and a slot is refilled only after the store
+// that last used it has finished reading shared memory.  Every wait is bounded: when the clock limit is
+// hit the CTA records CASCADE_ST_ETIMEOUT, issues nothing more, waits (bounded again) for the loads it
+// still has in flight, drains its store groups and returns.
+//
+// The same loop serves four roles:
+//   kRoleRestore / kRoleEvict          the two plain copies;
+//   kRoleMoveEvict / kRoleMoveRestore  the two grids of the fused evict + restore (see cascade_kv_move).
+constexpr int kPieceMax = 32 * 1024;
+constexpr int kPieceMin = 8 * 1024;
+constexpr int kMaxStages = 16;
+constexpr int kRingHost = 128 * 1024;   // one CTA per SM
+constexpr int kRingDev = 96 * 1024;     // two CTAs per SM fit
 constexpr long long kWaitCycles = 4000000000LL;  // about two seconds at 1.9 GHz
+
+enum { kRoleRestore = 0, kRoleEvict = 1, kRoleMoveEvict = 2, kRoleMoveRestore = 3 };
 
 __device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -108,6 +124,13 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, long long limit) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit) return false;
+    return true;
+}
 __device__ __forceinline__ void bulk_load(unsigned dst_smem, const void *src, unsigned bytes, unsigned bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
                  "l"(src), "r"(bytes), "r"(bar)
@@ -119,84 +142,130 @@ __device__ __forceinline__ void bulk_store(void *dst, unsigned src_smem, unsigne
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-template <bool kRestore>
-__global__ void __launch_bounds__(32) kv_copy_bulk_kernel(const __grid_constant__ CopyArgs a) {
-    cascade_grid_wait();
-    extern __shared__ __align__(128) unsigned char ring[];
-    __shared__ __align__(8) unsigned long long bars[kStages];
-    if (threadIdx.x != 0) return;
-    for (int s = 0; s < kStages; ++s) mbar_init(smem_addr(&bars[s]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+__device__ __forceinline__ int clamp_count(const int32_t *dev, int maxv) {
+    if (!dev) return maxv;
+    const int c = __ldcg(dev);
+    return c < 0 ? 0 : (c < maxv ? c : maxv);
+}
 
-    int count = a.n_max;
-    if (a.n_dev) {
-        const int c = *a.n_dev;
-        count = c < 0 ? 0 : (c < count ? c : count);
+template <int kRole>
+__global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ CopyArgs a) {
+    constexpr bool kRestore = kRole == kRoleRestore || kRole == kRoleMoveRestore;
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long bars[kMaxStages];
+    // barrier set-up touches no global memory, so it runs ahead of the wait for the preceding grid
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) mbar_init(smem_addr(&bars[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    const int ppc = a.pieces_per_chunk;  // pieces of kBulkPiece per chunk
+    // The restore grid of the fused move is launched as a programmatic dependent of the evict grid
+    // and must run BESIDE it, so it does not wait here but at its very end (see cascade_kv_move).
+    if (kRole != kRoleMoveRestore) cascade_grid_wait();
+    if (kRole == kRoleMoveEvict) cascade_grid_trigger();
+    if (threadIdx.x != 0) {
+        if (kRole == kRoleMoveRestore) cascade_grid_wait();
+        return;
+    }
+
+    const int count = clamp_count(a.n_dev, a.n_max);
+    // piece size: the largest of 32 / 16 / 8 KiB that still gives every CTA of the grid two pieces
+    int piece = kPieceMax;
+    if (a.piece_fixed > 0) {
+        piece = a.piece_fixed;
+    } else {
+        while (piece > kPieceMin &&
+               (long long)count * a.n_chunks * ((a.chunk_bytes + piece - 1) / piece) < 2LL * gridDim.x)
+            piece >>= 1;
+    }
+    int S = a.ring_bytes / piece;
+    S = S > kMaxStages ? kMaxStages : S;
+    const int ahead = S - 1;
+    const int ppc = (int)((a.chunk_bytes + piece - 1) / piece);
     const long long per_block = (long long)a.n_chunks * ppc;
     const long long items = (long long)count * per_block;
     const long long bb = (long long)a.n_chunks * a.chunk_bytes;
+    const long long limit = a.stall ? kWaitCycles / 20 : kWaitCycles;
     uint32_t st = 0;
 
     long long next = blockIdx.x;  // next item of this CTA to load
-    // resolves item `it` into addresses; false when an id is outside its pool (pair skipped)
-    auto resolve = [&](long long it, const char *&src, char *&dst, unsigned &bytes) -> bool {
-        const long long i = it / per_block;
-        const int rem = (int)(it - i * per_block);
-        const int c = rem / ppc, pc = rem - c * ppc;
-        const long long s = a.src_ids[i], d = a.dst_ids[i];
-        const long long rec_id = kRestore ? s : d, pg_id = kRestore ? d : s;
-        if (rec_id < 0 || rec_id >= a.record_blocks || pg_id < 0 || pg_id >= a.paged_blocks) return false;
-        const long long off = (long long)pc * kBulkPiece;
-        const long long left = a.chunk_bytes - off;
-        bytes = (unsigned)(left < kBulkPiece ? left : kBulkPiece);
-        char *rec = a.record + rec_id * bb + (long long)c * a.chunk_bytes + off;
-        char *pg = a.paged + (long long)c * a.chunk_stride + pg_id * a.block_stride + off;
-        src = kRestore ? rec : pg;
-        dst = kRestore ? pg : rec;
-        return true;
-    };
-    char *dst_of[kStages];
-    unsigned bytes_of[kStages];
+    char *dst_of[kMaxStages];
+    unsigned bytes_of[kMaxStages];
+    int entry_of[kMaxStages];     // list index of the piece in the slot
     long long issued = 0, stored = 0;
-    auto issue_next = [&]() -> bool {  // loads the next valid item into ring slot issued % kStages
+    auto issue_next = [&]() -> bool {  // loads the next valid item into ring slot issued % S
         while (next < items) {
-            const char *src;
-            char *dst;
-            unsigned bytes;
-            const bool ok = resolve(next, src, dst, bytes);
+            const long long it = next;
             next += gridDim.x;
-            if (!ok) {
-                st |= CASCADE_ST_EBOUNDS;
+            long long i = it / per_block;
+            const int rem = (int)(it - i * per_block);
+            if (kRole == kRoleMoveEvict) i = count - 1 - i;  // blocks freed last are handed out first: read them out first
+            const int c = rem / ppc, pc = rem - c * ppc;
+            const long long s = __ldcg(a.src_ids + i), d = __ldcg(a.dst_ids + i);
+            const long long rec_id = kRestore ? s : d, pg_id = kRestore ? d : s;
+            const long long off = (long long)pc * piece;
+            const long long left = a.chunk_bytes - off;
+            const unsigned bytes = (unsigned)(left < piece ? left : piece);
+            if (rec_id < 0 || rec_id >= a.record_blocks || pg_id < 0 || pg_id >= a.paged_blocks) {
+                st |= CASCADE_ST_EBOUNDS;  // id outside its pool: this pair is skipped
+                // a skipped evict piece still counts as read, or a restore into that block would wait for nothing
+                if (kRole == kRoleMoveEvict) atomicAdd(&a.done[i], (int)(bytes >> 4));
+                if (kRole == kRoleMoveRestore) atomicAdd(&a.skipped[i], 1);
                 continue;
             }
-            const int slot = (int)(issued % kStages);
+            char *rec = a.record + rec_id * bb + (long long)c * a.chunk_bytes + off;
+            char *pg = a.paged + (long long)c * a.chunk_stride + pg_id * a.block_stride + off;
+            const int slot = (int)(issued % S);
             const unsigned bar = smem_addr(&bars[slot]);
-            mbar_expect_tx(bar, bytes);
-            bulk_load(smem_addr(ring + (size_t)slot * kBulkPiece), src, bytes, bar);
-            dst_of[slot] = dst;
+            // test hook 2: the very first piece of CTA 0 announces more bytes than it loads, so its wait runs out
+            const bool short_load = a.stall == 2 && blockIdx.x == 0 && issued == 0;
+            mbar_expect_tx(bar, bytes + (short_load ? 16u : 0u));
+            bulk_load(smem_addr(ring + (size_t)slot * piece), kRestore ? rec : pg, bytes, bar);
+            dst_of[slot] = kRestore ? pg : rec;
             bytes_of[slot] = bytes;
+            entry_of[slot] = (int)i;
             ++issued;
             return true;
         }
         return false;
     };
-    for (int k = 0; k < kAhead; ++k)
+    for (int k = 0; k < ahead; ++k)
         if (!issue_next()) break;
     while (stored < issued) {
-        const int slot = (int)(stored % kStages);
-        const unsigned parity = (unsigned)((stored / kStages) & 1);
-        const unsigned bar = smem_addr(&bars[slot]);
-        const long long t0 = clock64();
-        bool arrived = mbar_try_wait(bar, parity);
-        while (!arrived && clock64() - t0 < kWaitCycles) arrived = mbar_try_wait(bar, parity);
-        if (!arrived) {  // give up: record it, issue nothing more
+        const int slot = (int)(stored % S);
+        const unsigned parity = (unsigned)((stored / S) & 1);
+        if (!mbar_wait_bounded(smem_addr(&bars[slot]), parity, limit)) {
+            // give up: record it, issue nothing more, but do not leave while loads still target this CTA's ring
             st |= CASCADE_ST_ETIMEOUT;
+            for (long long q = stored + 1; q < issued; ++q)
+                mbar_wait_bounded(smem_addr(&bars[q % S]), (unsigned)((q / S) & 1), limit);
+            if (kRole == kRoleMoveRestore)
+                for (long long q = stored; q < issued; ++q) atomicAdd(&a.skipped[entry_of[q % S]], 1);
             break;
         }
-        bulk_store(dst_of[slot], smem_addr(ring + (size_t)slot * kBulkPiece), bytes_of[slot]);
+        bool skip = false;
+        if (kRole == kRoleMoveEvict) {
+            // this piece of the block has left HBM; counted in 16-byte units, because the two grids may
+            // cut their blocks into pieces of different sizes
+            if (a.stall != 1) atomicAdd(&a.done[entry_of[slot]], (int)(bytes_of[slot] >> 4));
+        } else if (kRole == kRoleMoveRestore) {
+            const int dep = __ldcg(a.dep + entry_of[slot]);
+            if (dep >= 0) {
+                // the HBM block is being evicted by this same call: write only after it has been read out
+                const volatile int32_t *flag = a.done + dep;
+                const long long t0 = clock64();
+                if (st & CASCADE_ST_ETIMEOUT) skip = true;  // one expired wait is enough: do not queue up more
+                while (!skip && *flag < (int)(bb >> 4)) {
+                    if (clock64() - t0 > limit) {
+                        st |= CASCADE_ST_ETIMEOUT;
+                        skip = true;
+                    }
+                }
+                __threadfence();
+                if (skip) atomicAdd(&a.skipped[entry_of[slot]], 1);
+            }
+        }
+        if (!skip) bulk_store(dst_of[slot], smem_addr(ring + (size_t)slot * piece), bytes_of[slot]);
         ++stored;
         // the slot refilled next was last read by the store issued one step earlier
         asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
@@ -204,169 +273,82 @@ __global__ void __launch_bounds__(32) kv_copy_bulk_kernel(const __grid_constant_
     }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (st) atomicOr(a.status, st);
+    // completion of this grid must imply completion of the evict grid it ran beside
+    if (kRole == kRoleMoveRestore) cascade_grid_wait();
 }
 
 // ---- fused evict + restore ("move"): both directions of the host link at once ----------------------
-// The evict list and the restore list of one iteration in ONE ring kernel.  Evicted blocks travel
-// device -> host while restored blocks travel host -> device, so the link is used in both directions
-// at the same time.  A restore may target an HBM block that the same call evicts (the tier plan hands
-// freed blocks out again at once): its store into HBM waits until every piece of that block has been
-// read by the evict side.  Each CTA works on one list: the CTAs are shared out in proportion to the
-// lists' lengths; evict CTAs walk their list backwards, because the blocks freed last are handed out
-// first.  Only restore CTAs ever wait, and
-// only for evict CTAs, which never wait for anybody, so with all CTAs resident (one per SM at most)
-// the waits cannot deadlock.  They are clock-bounded all the same (CASCADE_ST_ETIMEOUT, that store
-// is skipped).
-struct MoveArgs {
-    char *paged;
-    char *record;
-    const int32_t *evict_src, *evict_dst, *restore_src, *restore_dst;
+// Three launches on the caller's stream:
+//   1. kv_move_prepare_kernel (one CTA): zeroes the per-entry counters and finds, for every restore, the
+//      evict entry that frees its HBM block (the tier plan hands freed blocks out again at once) through an
+//      open-addressing hash table over the evicted block ids: linear work in the two list lengths;
+//   2. the evict grid (role kRoleMoveEvict), half of the SMs: device -> host; after every piece that has
+//      left HBM it bumps that entry's counter.  It signals "dependents may launch" as its first action;
+//   3. the restore grid (role kRoleMoveRestore), the other half, launched as a PROGRAMMATIC DEPENDENT of
+//      grid 2: the hardware starts it only once every CTA of the evict grid is running (or done), so a
+//      restore CTA that waits for a counter always waits for a CTA that is already on an SM and never waits
+//      itself: no deadlock however busy the GPU is with other work.  A restore into a block that the same
+//      call evicts stores only after that block's counter says it has been read out completely.
+// Without programmatic launch (CASCADE_PDL=0) grid 3 simply starts after grid 2 has finished.
+struct PrepareArgs {
+    const int32_t *evict_src, *restore_dst;
     const int32_t *n_evict_dev, *n_restore_dev;
-    int32_t *dep;    // per restore: index into the evict list of the entry that frees its HBM block, or -1
-    int32_t *done;   // per evict entry: pieces of the block already read out of HBM
-    uint32_t *status;
-    long long paged_blocks, record_blocks;
-    long long chunk_bytes, chunk_stride, block_stride;
-    int n_chunks;
     int n_evict_max, n_restore_max;
-    int pieces_per_chunk;
-    int stall;       // test hook: the evict side never reports a block as read out (exercises the bounded wait)
+    int32_t *skipped, *dep, *done, *hkeys, *hvals;
+    int hash_cap;  // power of two
 };
 
-__device__ __forceinline__ int clamp_count(const int32_t *dev, int maxv) {
-    if (!dev) return maxv;
-    const int c = *dev;
-    return c < 0 ? 0 : (c < maxv ? c : maxv);
-}
+__device__ __forceinline__ unsigned hash_id(int32_t g) { return (unsigned)g * 2654435761u; }
 
-__global__ void __launch_bounds__(256) kv_move_prepare_kernel(const __grid_constant__ MoveArgs a) {
+__global__ void __launch_bounds__(1024) kv_move_prepare_kernel(const __grid_constant__ PrepareArgs a) {
     cascade_grid_wait();
     cascade_grid_trigger();
     const int ne = clamp_count(a.n_evict_dev, a.n_evict_max), nr = clamp_count(a.n_restore_dev, a.n_restore_max);
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    const int stride = gridDim.x * blockDim.x;
-    for (int j = i; j < ne; j += stride) a.done[j] = 0;
-    for (int r = i; r < nr; r += stride) {
+    const int tid = threadIdx.x, T = blockDim.x;
+    int H = 64;  // table size: at most half full
+    while (H < 2 * ne && H < a.hash_cap) H <<= 1;
+    const unsigned mask = (unsigned)H - 1u;
+    for (int h = tid; h < H; h += T) {
+        a.hkeys[h] = -1;
+        a.hvals[h] = -1;
+    }
+    for (int j = tid; j < ne; j += T) a.done[j] = 0;
+    for (int r = tid; r < nr; r += T) a.skipped[r] = 0;
+    __syncthreads();
+    for (int j = tid; j < ne; j += T) {
+        const int32_t g = a.evict_src[j];
+        if (g < 0) continue;  // never matches a valid destination
+        unsigned h = hash_id(g) & mask;
+        for (int probe = 0; probe < H; ++probe) {
+            const int32_t prev = atomicCAS(&a.hkeys[h], -1, g);
+            if (prev == -1 || prev == g) {
+                atomicMax(&a.hvals[h], j);  // the LAST entry that evicts the block is the one to wait for
+                break;
+            }
+            h = (h + 1) & mask;
+        }
+    }
+    __syncthreads();
+    for (int r = tid; r < nr; r += T) {
         const int32_t g = a.restore_dst[r];
         int dep = -1;
-        for (int j = 0; j < ne; ++j)
-            if (a.evict_src[j] == g) dep = j;
+        if (g >= 0) {
+            unsigned h = hash_id(g) & mask;
+            for (int probe = 0; probe < H; ++probe) {
+                const int32_t k = a.hkeys[h];
+                if (k == g) { dep = a.hvals[h]; break; }
+                if (k == -1) break;
+                h = (h + 1) & mask;
+            }
+        }
         a.dep[r] = dep;
     }
 }
 
-__global__ void __launch_bounds__(32) kv_move_kernel(const __grid_constant__ MoveArgs a) {
-    cascade_grid_wait();
-    extern __shared__ __align__(128) unsigned char ring[];
-    __shared__ __align__(8) unsigned long long bars[kStages];
-    if (threadIdx.x != 0) return;
-    for (int s = 0; s < kStages; ++s) mbar_init(smem_addr(&bars[s]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-
-    const int ne = clamp_count(a.n_evict_dev, a.n_evict_max), nr = clamp_count(a.n_restore_dev, a.n_restore_max);
-    const int ppc = a.pieces_per_chunk;
-    const long long per_block = (long long)a.n_chunks * ppc;
-    const long long bb = (long long)a.n_chunks * a.chunk_bytes;
-    uint32_t st = 0;
-    // Each CTA serves one direction, so that both directions of the link are busy at once; the CTAs are shared
-    // out in proportion to the bytes of the two lists (interleaved over the grid), at least one per non-empty
-    // list.  A single-CTA grid does the evict list first, then the restores.
-    const long long G = gridDim.x, b = blockIdx.x;
-    const bool both = G == 1;                          // one CTA walks both lists
-    long long ge = G;                                  // CTAs that evict
-    if (ne > 0 && nr > 0) {
-        ge = (G * ne + (ne + (long long)nr) / 2) / (ne + (long long)nr);
-        ge = ge < 1 ? 1 : (ge > G - 1 ? G - 1 : ge);
-    } else if (ne == 0) {
-        ge = 0;
-    }
-    const long long e_before = b * ge / G;             // evict CTAs among the blocks before this one
-    const bool evict_role = (b + 1) * ge / G > e_before;
-    const long long evict_items = (both || evict_role) ? (long long)ne * per_block : 0;
-    const long long items = evict_items + ((both || !evict_role) ? (long long)nr * per_block : 0);
-    const long long step = both ? 1 : (evict_role ? ge : G - ge);
-
-    long long next = both ? 0 : (evict_role ? e_before : b - e_before);
-    char *dst_of[kStages];
-    unsigned bytes_of[kStages];
-    int evict_of[kStages];  // evict-list index to signal after the load (evict piece), -1 otherwise
-    int wait_of[kStages];   // evict-list index to wait for before the store (restore piece), -1 if none
-    long long issued = 0, stored = 0;
-    auto issue_next = [&]() -> bool {
-        while (next < items) {
-            const long long it = next;
-            next += step;
-            const bool is_evict = it < evict_items;
-            const long long local = is_evict ? it : it - evict_items;
-            long long i = local / per_block;
-            const int rem = (int)(local - i * per_block);
-            if (is_evict) i = ne - 1 - i;  // blocks freed last are reused first: read them out first
-            const int c = rem / ppc, pc = rem - c * ppc;
-            const long long rec_id = is_evict ? a.evict_dst[i] : a.restore_src[i];
-            const long long pg_id = is_evict ? a.evict_src[i] : a.restore_dst[i];
-            if (rec_id < 0 || rec_id >= a.record_blocks || pg_id < 0 || pg_id >= a.paged_blocks) {
-                st |= CASCADE_ST_EBOUNDS;
-                // a skipped evict piece still counts as read, or a restore into that block would wait for nothing
-                if (is_evict) atomicAdd(&a.done[i], 1);
-                continue;
-            }
-            const long long off = (long long)pc * kBulkPiece;
-            const long long left = a.chunk_bytes - off;
-            const unsigned bytes = (unsigned)(left < kBulkPiece ? left : kBulkPiece);
-            char *rec = a.record + rec_id * bb + (long long)c * a.chunk_bytes + off;
-            char *pg = a.paged + (long long)c * a.chunk_stride + pg_id * a.block_stride + off;
-            const int slot = (int)(issued % kStages);
-            const unsigned bar = smem_addr(&bars[slot]);
-            mbar_expect_tx(bar, bytes);
-            bulk_load(smem_addr(ring + (size_t)slot * kBulkPiece), is_evict ? pg : rec, bytes, bar);
-            dst_of[slot] = is_evict ? rec : pg;
-            bytes_of[slot] = bytes;
-            evict_of[slot] = is_evict ? (int)i : -1;
-            wait_of[slot] = is_evict ? -1 : a.dep[i];
-            ++issued;
-            return true;
-        }
-        return false;
-    };
-    for (int k = 0; k < kAhead; ++k)
-        if (!issue_next()) break;
-    while (stored < issued) {
-        const int slot = (int)(stored % kStages);
-        const unsigned parity = (unsigned)((stored / kStages) & 1);
-        const unsigned bar = smem_addr(&bars[slot]);
-        long long t0 = clock64();
-        bool arrived = mbar_try_wait(bar, parity);
-        while (!arrived && clock64() - t0 < kWaitCycles) arrived = mbar_try_wait(bar, parity);
-        if (!arrived) {
-            st |= CASCADE_ST_ETIMEOUT;
-            break;
-        }
-        bool skip = false;
-        if (evict_of[slot] >= 0) {
-            if (!a.stall) atomicAdd(&a.done[evict_of[slot]], 1);  // this piece of the block has left HBM
-        } else if (wait_of[slot] >= 0) {
-            // the HBM block is being evicted by this same call: write only after it has been read out
-            const volatile int32_t *flag = a.done + wait_of[slot];
-            t0 = clock64();
-            if (st & CASCADE_ST_ETIMEOUT) skip = true;  // one expired wait is enough: do not queue up more
-            const long long limit = a.stall ? kWaitCycles / 20 : kWaitCycles;
-            while (!skip && *flag < (int)per_block) {
-                if (clock64() - t0 > limit) {
-                    st |= CASCADE_ST_ETIMEOUT;
-                    skip = true;
-                    break;
-                }
-            }
-            __threadfence();
-        }
-        if (!skip) bulk_store(dst_of[slot], smem_addr(ring + (size_t)slot * kBulkPiece), bytes_of[slot]);
-        ++stored;
-        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-        issue_next();
-    }
-    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    if (st) atomicOr(a.status, st);
+int hash_capacity(int n_evict_max) {
+    int H = 64;
+    while (H < 2 * (long long)n_evict_max) H <<= 1;
+    return H;
 }
 
 int check_layout(const cascade_kv_layout *l, const void *paged, const void *record, long long record_blocks) {
@@ -378,16 +360,10 @@ int check_layout(const cascade_kv_layout *l, const void *paged, const void *reco
     return CASCADE_OK;
 }
 
-template <bool kRestore>
-int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char *record, long long record_blocks,
-                int record_is_device, const int32_t *src_ids, const int32_t *dst_ids, const int32_t *n_dev, int n_max,
-                cudaStream_t s) {
-    if (!ctx || n_max < 0) return CASCADE_EINVAL;
-    if (n_max == 0) return CASCADE_OK;
-    int rc = check_layout(l, paged, record, record_blocks);
-    if (rc != CASCADE_OK) return rc;
-    if (!src_ids || !dst_ids) return CASCADE_EINVAL;
-    CopyArgs a;
+void fill_copy_args(CopyArgs &a, const cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char *record,
+                    long long record_blocks, const int32_t *src_ids, const int32_t *dst_ids, const int32_t *n_dev,
+                    int n_max) {
+    a = CopyArgs{};
     a.paged = paged;
     a.record = record;
     a.src_ids = src_ids;
@@ -401,26 +377,44 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
     a.block_stride = l->block_stride;
     a.n_chunks = l->n_chunks;
     a.n_max = n_max;
+    a.piece_fixed = ctx->copy_piece;
+    a.stall = ctx->test_move_stall;
+}
+
+// the ring kernels need more dynamic shared memory than the default limit: opt in once per device
+template <int kRole>
+cudaError_t configure_ring(int device) {
+    static bool configured_dev[64] = {};
+    if (device >= 0 && device < 64 && configured_dev[device]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kv_ring_kernel<kRole>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingHost);
+    if (e == cudaSuccess && device >= 0 && device < 64) configured_dev[device] = true;
+    return e;
+}
+
+template <bool kRestore>
+int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char *record, long long record_blocks,
+                int record_is_device, const int32_t *src_ids, const int32_t *dst_ids, const int32_t *n_dev, int n_max,
+                cudaStream_t s) {
+    if (!ctx || n_max < 0) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
+    if (n_max == 0) return CASCADE_OK;
+    int rc = check_layout(l, paged, record, record_blocks);
+    if (rc != CASCADE_OK) return rc;
+    if (!src_ids || !dst_ids) return CASCADE_EINVAL;
+    CopyArgs a;
+    fill_copy_args(a, ctx, l, paged, record, record_blocks, src_ids, dst_ids, n_dev, n_max);
     const int mode = record_is_device ? ctx->copy_bulk_dev : ctx->copy_bulk_host;
     if (mode) {
-        // TMA ring: one CTA (one elected thread) per SM slot, 32 KiB pieces
-        a.pieces_per_chunk = (int)((l->chunk_bytes + kBulkPiece - 1) / kBulkPiece);
-        const long long items = (long long)n_max * l->n_chunks * a.pieces_per_chunk;
+        // TMA ring: one elected thread per CTA; `mode` CTAs per SM
+        a.ring_bytes = mode > 1 ? kRingDev : kRingHost;
+        if (ctx->copy_ring_kb > 0) a.ring_bytes = ctx->copy_ring_kb * 1024;
+        const long long items = (long long)n_max * l->n_chunks * ((l->chunk_bytes + kPieceMin - 1) / kPieceMin);
         long long grid = (long long)ctx->num_sms * (mode > 1 ? mode : 1);
         if (grid > items) grid = items;
-        const size_t smem = (size_t)kStages * kBulkPiece;
-        static bool configured_dev[64] = {};
-        bool unknown = false;
-        bool &configured = (ctx->device >= 0 && ctx->device < 64) ? configured_dev[ctx->device] : unknown;
-        if (!configured) {
-            CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_copy_bulk_kernel<true>,
-                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_copy_bulk_kernel<false>,
-                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            configured = true;
-        }
-        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(32), smem, s,
-                                             kv_copy_bulk_kernel<kRestore>, a));
+        constexpr int role = kRestore ? kRoleRestore : kRoleEvict;
+        CASCADE_CUDA_TRY(ctx, configure_ring<role>(ctx->device));
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(32), (size_t)a.ring_bytes, s,
+                                             kv_ring_kernel<role>, a));
         return CASCADE_OK;
     }
     a.pieces_per_chunk = (int)((l->chunk_bytes + kPiece - 1) / kPiece);
@@ -469,6 +463,11 @@ extern "C" int cascade_kv_stage(cascade_ctx *ctx, const void *deep_pool, int64_t
                              src_ids, dst_ids, n_copies_dev, n_copies_max, (cudaStream_t)stream);
 }
 
+extern "C" int64_t cascade_kv_move_scratch_len(int n_evict_max, int n_restore_max) {
+    if (n_evict_max < 0 || n_restore_max < 0) return -1;
+    return 2 * (int64_t)n_restore_max + (int64_t)n_evict_max + 2 * (int64_t)hash_capacity(n_evict_max);
+}
+
 extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, void *host_pool,
                                int64_t host_blocks, const int32_t *evict_src, const int32_t *evict_dst,
                                const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,
@@ -476,50 +475,54 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
                                int32_t *scratch, void *stream) {
     CascadeRange nvtx_range("cascade_kv_move");
     if (!ctx || n_evict_max < 0 || n_restore_max < 0) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (n_evict_max == 0 && n_restore_max == 0) return CASCADE_OK;
     int rc = check_layout(hbm, hbm_pool, host_pool, host_blocks);
     if (rc != CASCADE_OK) return rc;
     if (!scratch || (n_evict_max > 0 && (!evict_src || !evict_dst)) || (n_restore_max > 0 && (!restore_src || !restore_dst)))
         return CASCADE_EINVAL;
     cudaStream_t s = (cudaStream_t)stream;
-    MoveArgs a;
-    a.paged = (char *)hbm_pool;
-    a.record = (char *)host_pool;
-    a.evict_src = evict_src;
-    a.evict_dst = evict_dst;
-    a.restore_src = restore_src;
-    a.restore_dst = restore_dst;
-    a.n_evict_dev = n_evict_dev;
-    a.n_restore_dev = n_restore_dev;
-    a.dep = scratch;
-    a.done = scratch + n_restore_max;
-    a.status = ctx->status_dev;
-    a.paged_blocks = hbm->n_blocks;
-    a.record_blocks = host_blocks;
-    a.chunk_bytes = hbm->chunk_bytes;
-    a.chunk_stride = hbm->chunk_stride;
-    a.block_stride = hbm->block_stride;
-    a.n_chunks = hbm->n_chunks;
-    a.n_evict_max = n_evict_max;
-    a.n_restore_max = n_restore_max;
-    a.pieces_per_chunk = (int)((hbm->chunk_bytes + kBulkPiece - 1) / kBulkPiece);
-    a.stall = ctx->test_move_stall;
-    const int most = n_evict_max > n_restore_max ? n_evict_max : n_restore_max;
-    int pgrid = (most + 255) / 256;
-    if (pgrid > ctx->num_sms * 4) pgrid = ctx->num_sms * 4;
-    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(pgrid), dim3(256), 0, s, kv_move_prepare_kernel, a));
-    const long long items = ((long long)n_evict_max + n_restore_max) * hbm->n_chunks * a.pieces_per_chunk;
-    long long grid = ctx->num_sms;  // one resident CTA per SM: every CTA that can be waited for is running
-    if (ctx->move_ctas > 0 && ctx->move_ctas < grid) grid = ctx->move_ctas;
-    if (grid > items) grid = items;
-    const size_t smem = (size_t)kStages * kBulkPiece;
-    static bool configured_dev[64] = {};
-    bool unknown = false;
-    bool &configured = (ctx->device >= 0 && ctx->device < 64) ? configured_dev[ctx->device] : unknown;
-    if (!configured) {
-        CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(kv_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
-    }
-    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(32), smem, s, kv_move_kernel, a));
+    // scratch: skipped[n_restore_max] | dep[n_restore_max] | done[n_evict_max] | hash keys | hash values
+    PrepareArgs p;
+    p.evict_src = evict_src;
+    p.restore_dst = restore_dst;
+    p.n_evict_dev = n_evict_dev;
+    p.n_restore_dev = n_restore_dev;
+    p.n_evict_max = n_evict_max;
+    p.n_restore_max = n_restore_max;
+    p.hash_cap = hash_capacity(n_evict_max);
+    p.skipped = scratch;
+    p.dep = p.skipped + n_restore_max;
+    p.done = p.dep + n_restore_max;
+    p.hkeys = p.done + n_evict_max;
+    p.hvals = p.hkeys + p.hash_cap;
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(1), dim3(1024), 0, s, kv_move_prepare_kernel, p));
+
+    const long long ppc_max = (hbm->chunk_bytes + kPieceMin - 1) / kPieceMin;
+    int half = ctx->num_sms / 2;
+    if (ctx->move_ctas > 0 && ctx->move_ctas < half) half = ctx->move_ctas;
+    if (half < 1) half = 1;
+    CASCADE_CUDA_TRY(ctx, configure_ring<kRoleMoveEvict>(ctx->device));
+    CASCADE_CUDA_TRY(ctx, configure_ring<kRoleMoveRestore>(ctx->device));
+    CopyArgs e, r;
+    fill_copy_args(e, ctx, hbm, (char *)hbm_pool, (char *)host_pool, host_blocks, evict_src, evict_dst, n_evict_dev,
+                   n_evict_max);
+    fill_copy_args(r, ctx, hbm, (char *)hbm_pool, (char *)host_pool, host_blocks, restore_src, restore_dst,
+                   n_restore_dev, n_restore_max);
+    e.ring_bytes = r.ring_bytes = ctx->copy_ring_kb > 0 ? ctx->copy_ring_kb * 1024 : kRingHost;
+    e.done = r.done = p.done;
+    e.dep = r.dep = p.dep;
+    e.skipped = r.skipped = p.skipped;
+    // the evict grid is launched even when its list is empty: the restore grid is ordered behind it
+    long long ge = half, gr = half;
+    const long long items_e = (long long)n_evict_max * hbm->n_chunks * ppc_max;
+    const long long items_r = (long long)n_restore_max * hbm->n_chunks * ppc_max;
+    if (ge > items_e) ge = items_e < 1 ? 1 : items_e;
+    if (gr > items_r) gr = items_r;
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)ge), dim3(32), (size_t)e.ring_bytes, s,
+                                         kv_ring_kernel<kRoleMoveEvict>, e));
+    if (gr > 0)
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)gr), dim3(32), (size_t)r.ring_bytes, s,
+                                             kv_ring_kernel<kRoleMoveRestore>, r));
     return CASCADE_OK;
 }

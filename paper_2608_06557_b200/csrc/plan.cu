@@ -19,6 +19,11 @@
 // Kernels 2 and 3 (many CTAs, one warp per request): rewrite block tables, free lists and the two
 // copy lists from the offsets kernel 1 left in scratch; pushes of freed ids (kernel 2) finish
 // before any pop (kernel 3).  In plan-only mode (no tables) only kernel 1 runs.
+#include <stdlib.h>
+
+#include <atomic>
+#include <mutex>
+
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -29,13 +34,6 @@ namespace cg = cooperative_groups;
 namespace {
 
 constexpr int kMaxCluster = 16;
-
-#ifdef CASCADE_PHASE_TIMING
-__device__ long long g_plan_ticks[16];
-#define PTICK(i) do { if (threadIdx.x == 0 && crank == 0) g_plan_ticks[(i)] = clock64(); } while (0)
-#else
-#define PTICK(i) do { } while (0)
-#endif
 
 // element flags
 constexpr unsigned kAdm = 1u, kPriv = 2u, kFits = 4u, kValid = 8u, kReal = 16u;
@@ -104,7 +102,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         }
     }
 
-    PTICK(0);
     // ---- phase 1a, slot order (coalesced): Eq. 7 bounds and the restore-vs-recompute choice; the
     //      per-request outputs get their default values here and one packed word per request
     //      (n0 | x1 << 14 | tokens_run << 28 | flags << 46) is left for the schedule-order phases
@@ -168,7 +165,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         runv[k] = (int)((w >> 28) & 0x3ffff);
     }
 
-    PTICK(1);
     // ---- phase 2: forward scan over the admitted set, capacity cut --------------------------------
     int s_need[K], s_x1[K], s_cnt[K];
     long long evictable = 0;
@@ -184,7 +180,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     cta_scan3<T, K>(s_need, s_x1, s_cnt, tot, ws3);
     long long red1[1] = {evictable};
     cta_sum<T, 1>(red1, ws8);
-    PTICK(2);
     if (tid < csize) {
         Exch1 x;
         x.need = tot[0];
@@ -194,7 +189,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         cluster.map_shared_rank(ex1, tid)[crank] = x;
     }
     cluster.sync();
-    PTICK(3);
     long long off_need = 0, cap = hbm_cnt;
     int off_x1 = 0, off_cnt = 0;
 #pragma unroll
@@ -232,7 +226,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         }
     }
 
-    PTICK(4);
     // ---- phase 3: preemptable holders, walked backwards ---------------------------------------------
     int s_v[K], s_h[K], s_c[K];
 #pragma unroll
@@ -245,7 +238,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     cta_scan3<T, K>(s_v, s_h, s_c, tot, ws3);
     long long red5[5] = {k_need, k_cnt, k_x1, k_unadm, k_tok};
     cta_sum<T, 5>(red5, ws8);
-    PTICK(5);
     if (tid < csize) {
         Exch2 x;
         x.v = tot[0];
@@ -261,7 +253,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         cluster.map_shared_rank(ex2, tid)[crank] = x;
     }
     cluster.sync();
-    PTICK(6);
     long long need_total = 0, V = 0, H = 0, tokens = 0;
     int Cn = 0, off_v = 0, off_h = 0, off_c = 0, n_adm = 0, n_rest = 0, n_unadm = 0;
 #pragma unroll
@@ -307,10 +298,8 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
         // ---- phase 4: only preempted requests change the action written in phase 1a -----------------
         if (act == CASCADE_ACT_EVICT || act == CASCADE_ACT_DROP) a.plan.action[slot[k]] = act;
     }
-    PTICK(7);
     long long red3[3] = {s_nv, s_freed, s_nev};
     cta_sum<T, 3>(red3, ws8);
-    PTICK(8);
     if (tid == 0) {
         Exch3 x;
         x.nv = (int)red3[0];
@@ -322,7 +311,6 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     st = __reduce_or_sync(kFull, st);
     if (lane == 0 && st) atomicOr(a.status, st);
     cluster.sync();
-    PTICK(9);
     if (crank == 0 && tid == 0) {
         long long nv = 0, freed = 0, nev = 0;
         for (unsigned c = 0; c < csize; ++c) {
@@ -437,11 +425,10 @@ apply_admitted_kernel(const __grid_constant__ PlanArgs a) {
 
 
 template <int T, int K>
-cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_size, bool pdl, cudaStream_t stream) {
+cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_size, bool pdl, int device,
+                        cudaStream_t stream) {
     // clusters of 16 CTAs need the non-portable size opt-in, once per device
     static bool configured_dev[64] = {};
-    int device = 0;
-    cudaGetDevice(&device);
     if (device < 0 || device >= 64 || !configured_dev[device]) {
         cudaError_t e = cudaFuncSetAttribute(plan_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
@@ -451,28 +438,24 @@ cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_
 }
 
 template <int T>
-cudaError_t launch_plan_k(int K, const cascade_params &p, const PlanArgs &a, int C, bool pdl, cudaStream_t s) {
+cudaError_t launch_plan_k(int K, const cascade_params &p, const PlanArgs &a, int C, bool pdl, int device,
+                          cudaStream_t s) {
     switch (K) {
-        case 1: return launch_plan<T, 1>(p, a, C, pdl, s);
-        case 2: return launch_plan<T, 2>(p, a, C, pdl, s);
-        case 4: return launch_plan<T, 4>(p, a, C, pdl, s);
-        default: return launch_plan<T, 8>(p, a, C, pdl, s);
+        case 1: return launch_plan<T, 1>(p, a, C, pdl, device, s);
+        case 2: return launch_plan<T, 2>(p, a, C, pdl, device, s);
+        case 4: return launch_plan<T, 4>(p, a, C, pdl, device, s);
+        default: return launch_plan<T, 8>(p, a, C, pdl, device, s);
     }
 }
 
 }  // namespace
-
-#ifdef CASCADE_PHASE_TIMING
-extern "C" int cascade_debug_plan_ticks(long long *host_out) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_plan_ticks, sizeof(g_plan_ticks));
-}
-#endif
 
 extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const int64_t *budget,
                                  const uint32_t *order, int32_t *grant, int n, int32_t D_act, int64_t K_act,
                                  const cascade_pools *pools, const cascade_plan *plan_out, void *stream) {
     CascadeRange nvtx_range("cascade_tier_plan");
     if (!ctx || !r || !pools || !plan_out || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (!plan_out->counts || !pools->hbm_free_count || !pools->host_free_count) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
     const bool with_tables = pools->hbm_tbl != nullptr;
@@ -509,7 +492,8 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     a.with_tables = with_tables ? 1 : 0;
     int T, C, K;
     if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, ctx->pdl, s) : launch_plan_k<512>(K, ctx->params, a, C, ctx->pdl, s);
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, ctx->pdl, ctx->device, s)
+                             : launch_plan_k<512>(K, ctx->params, a, C, ctx->pdl, ctx->device, s);
     CASCADE_CUDA_TRY(ctx, e);
     if (with_tables && n > 0) {
         const int grid = ctx->num_sms * 2;
@@ -551,21 +535,35 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocS
 struct NoAllocDevice {
     NoAllocScratch *scratch;  // device address of g_noalloc_scratch on this device
     int num_sms;
-    bool ready;
+    int max_cluster;          // largest cluster this device co-schedules for the plan geometry
+    std::atomic<int> ready;   // published last, with release ordering
 };
 NoAllocDevice g_noalloc_dev[64];
+std::mutex g_noalloc_mutex;   // serialises the first use on a device between host threads
 
-// First use on a device: resolve the device address of the static array (no allocation).
+// First use on a device (that device current): resolve the device address of the static array and
+// query what the geometry needs.  Queries only; nothing is allocated.
 int noalloc_setup(int device, NoAllocDevice **out) {
     if (device < 0 || device >= 64) return CASCADE_EINVAL;
     NoAllocDevice &d = g_noalloc_dev[device];
-    if (!d.ready) {
-        void *ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return CASCADE_ECUDA;
-        if (cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
-            return CASCADE_ECUDA;
-        d.scratch = reinterpret_cast<NoAllocScratch *>(ptr);
-        d.ready = true;
+    if (!d.ready.load(std::memory_order_acquire)) {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!d.ready.load(std::memory_order_relaxed)) {
+            void *ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+                cudaGetLastError();
+                return CASCADE_ECUDA;
+            }
+            if (cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+                cudaGetLastError();
+                return CASCADE_ECUDA;
+            }
+            d.max_cluster = cascade_probe_max_cluster();
+            const char *e = getenv("CASCADE_MAX_CLUSTER");   // lower it to exercise the fallback geometry
+            if (e && atoi(e) > 0 && atoi(e) < d.max_cluster) d.max_cluster = atoi(e);
+            d.scratch = reinterpret_cast<NoAllocScratch *>(ptr);
+            d.ready.store(1, std::memory_order_release);
+        }
     }
     *out = &d;
     return CASCADE_OK;
@@ -627,11 +625,18 @@ extern "C" int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_
     // zeroed anyway so that a call that launches nothing leaves no stale counts behind.
     if (cudaMemsetAsync(dev->scratch->scalars, 0, sizeof(dev->scratch->scalars), s) != cudaSuccess)
         return CASCADE_ECUDA;
+    // same geometry rule as cascade_tier_plan: a device that co-schedules fewer than 16 CTAs gets a
+    // smaller cluster with more requests per thread
     cascade_ctx geo = {};
+    geo.max_cluster = dev->max_cluster;
     int T, C, K;
-    if (!cascade_pick_geometry(&geo, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
-    cudaError_t e = T == 256 ? launch_plan_k<256>(K, *p, a, C, false, s) : launch_plan_k<512>(K, *p, a, C, false, s);
-    if (e != cudaSuccess) return CASCADE_ECUDA;
+    if (!cascade_pick_geometry(&geo, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_ETOOBIG;
+    cudaError_t e = T == 256 ? launch_plan_k<256>(K, *p, a, C, false, device, s)
+                             : launch_plan_k<512>(K, *p, a, C, false, device, s);
+    if (e != cudaSuccess) {
+        cudaGetLastError();  // leave no stale error behind for the caller's next runtime call
+        return CASCADE_ECUDA;
+    }
     if (with_tables && n > 0) {
         const int grid = dev->num_sms * 2;
         apply_victims_kernel<<<grid, 256, 0, s>>>(a);

@@ -280,6 +280,7 @@ extern "C" int cascade_prefetch_plan(cascade_ctx *ctx, const cascade_reqs *r, co
                                      cascade_prefetch_counts *counts_dev, void *stream) {
     CascadeRange nvtx_range("cascade_prefetch_plan");
     if (!ctx || !r || !pools || !plan || !counts_dev || n < 0 || n > ctx->max_requests) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (!plan->counts || !pools->hbm_free_count) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16) || K_act < 0 || K_act > (int64_t(1) << 32)) return CASCADE_ERANGE;
     if (link_budget_ns < 0 || link_budget_ns > (int64_t(1) << 50) || hbm_reserve < 0) return CASCADE_ERANGE;

@@ -74,13 +74,6 @@ struct ScheduleArgs {
     uint32_t *status;
 };
 
-#ifdef CASCADE_PHASE_TIMING
-__device__ long long g_phase_ticks[128];
-#define TICK(i) do { if (tid == 0 && crank == 0) g_phase_ticks[(i)] = clock64(); } while (0)
-#else
-#define TICK(i) do { } while (0)
-#endif
-
 template <typename T>
 __device__ __forceinline__ T seg_incl_scan(T v, int pos, int width) {
     // inclusive scan inside aligned groups of `width` lanes; pos = lane % width
@@ -130,7 +123,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
-    TICK(66);
     // ---- load: key, slot, tokens wanted (prompt minus the matched prefix) ----------------------
     SortElem e[K];
     const unsigned long long key0 = a.key[0];
@@ -195,7 +187,9 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                 cnt += count_range((int)max((long long)mid, min((long long)hi, gi + 1)), hi, false);   // above gi: ties do not count
             }
             partial[tid] = cnt;
-            __syncthreads();
+            // a cluster barrier, not just a CTA barrier: no store into another CTA's shared memory before
+            // every CTA of the cluster has started
+            cluster.sync();
             // the element's owner adds the partial counts and sends the element to its final place
             if (tid < per_rt && e[0].idx != 0xffffffffu) {
                 int pos = 0;
@@ -214,7 +208,9 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         unsigned lo = __reduce_or_sync(kFull, (unsigned)diff);
         unsigned hi = __reduce_or_sync(kFull, (unsigned)(diff >> 32));
         if (lane == 0) wtmp[warp] = (long long)(((unsigned long long)hi << 32) | lo);
-        __syncthreads();
+        // a cluster barrier, not just a CTA barrier: the store below is the first access to another CTA's
+        // shared memory, which must not happen before that CTA has started (and initialised its mbarriers)
+        cluster.sync();
         if (warp == 0) {
             unsigned long long v = lane < W ? (unsigned long long)wtmp[lane] : 0ull;
             lo = __reduce_or_sync(kFull, (unsigned)v);
@@ -245,7 +241,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         }
         ++ep;
 
-        TICK(pass * 8 + 0);
         // (a) stable rank of each element among equal digits of its warp's chunk
         uint16_t *myhist = whist + warp * kWhistStride;
         for (int i = lane; i < kWhistStride / 2; i += 32) reinterpret_cast<uint32_t *>(myhist)[i] = 0;
@@ -270,7 +265,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
             off[k] = pre + __popc(lower);
         }
         __syncthreads();
-        TICK(pass * 8 + 1);
 
         // (b) one thread per digit walks its column of the W per-warp histograms (exclusive scan in
         //     place) and pushes the CTA's count of that digit to every CTA of the cluster
@@ -292,7 +286,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                     if (c < csize) cluster.map_shared_rank(hist_in, c)[crank * kBins + tid] = (uint16_t)mine;
             }
         }
-        TICK(pass * 8 + 2);
         if (a.async_sync) {
             // 16-byte pieces of this CTA's histogram go to every CTA and count on its histogram barrier;
             // a CTA goes on as soon as the sixteen histograms it needs have landed
@@ -308,7 +301,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         } else {
             cluster.sync();  // histograms delivered; every CTA holds its elements in registers
         }
-        TICK(pass * 8 + 3);
         if (dead) continue;
 
         // (c) per digit: global base of this CTA (high bits) and local base inside this CTA (low 14
@@ -341,7 +333,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
             lbase[tid] = excl & 0x3fffu;            // first local position of that run
         }
         __syncthreads();
-        TICK(pass * 8 + 4);
 
         if (a.stage) {
             // (d) group the CTA's elements by digit in a local staging buffer, then copy runs of equal
@@ -383,7 +374,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                 }
             }
         }
-        TICK(pass * 8 + 5);
         if (a.async_sync) {
             // this CTA's slice is complete when all of its T*K elements have arrived
             const bool ok = mbarrier_wait_bounded(elem_bar, phase, kWaitLimit);
@@ -392,12 +382,9 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         } else {
             cluster.sync();  // all remote stores have landed
         }
-        TICK(pass * 8 + 6);
 #pragma unroll
         for (int k = 0; k < K; ++k) e[k] = elems[(warp * K + k) * 32 + lane];
-        TICK(pass * 8 + 7);
     }
-    TICK(64);
     if (dead && tid == 0) atomicOr(a.status, CASCADE_ST_ETIMEOUT);
     }  // radix path
 
@@ -520,7 +507,6 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         atomicAdd(&a.counts->n_admitted, adm);
     }
     if (crank == 0 && tid == 0) a.counts->n_tier1 = N1;
-    TICK(65);
     // every remote store of this kernel is followed by a cluster barrier and nothing reads remote
     // shared memory, so a CTA may leave as soon as it is done
 }
@@ -585,17 +571,12 @@ int cascade_probe_max_cluster() {
     return size < 1 ? 1 : (size > 16 ? 16 : size);
 }
 
-#ifdef CASCADE_PHASE_TIMING
-extern "C" int cascade_debug_ticks(long long *host_out) {
-    return (int)cudaMemcpyFromSymbol(host_out, g_phase_ticks, sizeof(g_phase_ticks));
-}
-#endif
-
 extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const uint64_t *key, int n, int32_t D_act,
                                 uint32_t *order_out, int32_t *grant_out, cascade_sched_counts *counts_dev,
                                 void *stream) {
     CascadeRange nvtx_range("cascade_schedule");
     if (!ctx || !r || n < 0 || n > ctx->max_requests || !counts_dev) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (D_act < 0 || D_act > (1 << 16)) return CASCADE_ERANGE;
     cudaStream_t s = (cudaStream_t)stream;
     if (n == 0) {

@@ -172,7 +172,8 @@ class Instance:
     def run_move(self, stream=None):
         """evict + restore as one call that uses both directions of the host link at once."""
         if not hasattr(self, "move_scratch"):
-            self.move_scratch = torch.empty(self.evict_cap + self.restore_cap, dtype=torch.int32, device=self.device)
+            self.move_scratch = torch.empty(cs.kv_move_scratch_len(self.evict_cap, self.restore_cap),
+                                            dtype=torch.int32, device=self.device)
         self.ctx.kv_move(self.layout, self.hbm_pool, self.host_pool, self.host_blocks, self.evict_src, self.evict_dst,
                          self.plan_counts[1:2], self.evict_cap, self.restore_src, self.restore_dst,
                          self.plan_counts[0:1], self.restore_cap, self.move_scratch, stream)
@@ -240,7 +241,8 @@ class Instance:
     def run_move_merged(self, stream=None):
         """evict + restore over the merged restore list."""
         if not hasattr(self, "move_scratch"):
-            self.move_scratch = torch.empty(self.evict_cap + self.restore_cap, dtype=torch.int32, device=self.device)
+            self.move_scratch = torch.empty(cs.kv_move_scratch_len(self.evict_cap, self.restore_cap),
+                                            dtype=torch.int32, device=self.device)
         self.ctx.kv_move(self.layout, self.hbm_pool, self.host_pool, self.host_blocks, self.evict_src, self.evict_dst,
                          self.plan_counts[1:2], self.evict_cap, self.restore_src_m, self.restore_dst_m,
                          self.dedup_counts_restore[1:2], self.restore_cap, self.move_scratch, stream)

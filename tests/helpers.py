@@ -32,3 +32,23 @@ def clone_workload(w):
 
 def guard_pattern(n_bytes, tag):
     return np.full(n_bytes, tag, np.uint8)
+
+
+def load_gpu_filler():
+    """Builds (if needed) and loads tests/gpu_filler.cu: a test-only kernel that keeps SMs busy for a
+    bounded time.  Returns the ctypes library."""
+    import ctypes
+    import os
+    import subprocess
+    here = os.path.dirname(os.path.abspath(__file__))
+    src, lib = os.path.join(here, "gpu_filler.cu"), os.path.join(here, "libgpu_filler.so")
+    if not os.path.exists(lib) or os.path.getmtime(lib) < os.path.getmtime(src):
+        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+        tmp = lib + f".{os.getpid()}.tmp"
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O2", "-shared", "-Xcompiler",
+                               "-fPIC", "-o", tmp, src])
+        os.replace(tmp, lib)
+    f = ctypes.CDLL(lib)
+    f.filler_launch.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_longlong, ctypes.c_void_p]
+    f.filler_launch.restype = ctypes.c_int
+    return f

@@ -182,7 +182,7 @@ def test_fused_move_equals_evict_then_restore(shape):
     cap_e, cap_r = ne + 3, nr + 2
     pad = lambda a, cap: rig.ids(np.concatenate([a, np.full(cap - len(a), 10**6, np.int32)]))
     counts = torch.tensor([nr, ne], dtype=torch.int32, device="cuda")
-    scratch = torch.empty(cap_e + cap_r, dtype=torch.int32, device="cuda")
+    scratch = torch.empty(rig.cs.kv_move_scratch_len(cap_e, cap_r), dtype=torch.int32, device="cuda")
     for rep in range(2):                              # twice: the scratch is reused as it was left
         rig.hbm.copy_(torch.from_numpy(rig.hbm_np))
         rig.host.copy_(torch.from_numpy(rig.host_np))
@@ -247,10 +247,12 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable(monkeypa
     stalled = cs.Context(wl.default_params(), 16, 0)
     monkeypatch.delenv("CASCADE_TEST_MOVE_STALL")
     hbm, host = torch.from_numpy(hbm_np.copy()).cuda(), torch.from_numpy(host_np.copy()).pin_memory()
-    scratch = torch.empty(8, dtype=torch.int32, device="cuda")
+    scratch = torch.empty(cs.kv_move_scratch_len(2, 2), dtype=torch.int32, device="cuda")
     stalled.kv_move(cs.make_layout(lay), hbm, host, n_host, t(es), t(ed), None, 2, t(rs), t(rd), None, 2, scratch)
     torch.cuda.synchronize()
     assert stalled.status()[0] == cs.ST_ETIMEOUT
+    # the restore that gave up is visible per block: every piece of restore 0 unwritten, restore 1 complete
+    assert scratch[:2].cpu().tolist() == [n_chunks, 0]
     want_host = host_np.copy()
     assert oracle.kv_evict(hbm_np.copy(), lay, want_host, n_host, es, ed) == 0
     assert np.array_equal(host.numpy(), want_host)                        # the evictions happened
@@ -265,3 +267,89 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable(monkeypa
     ref_h, ref_o = hbm_np.copy(), host_np.copy()
     assert oracle.kv_evict(ref_h, lay, ref_o, n_host, es, ed) == 0 and oracle.kv_restore(ref_h, lay, ref_o, n_host, rs, rd) == 0
     assert ctx.status()[0] == 0 and np.array_equal(hbm.cpu().numpy(), ref_h) and np.array_equal(host.numpy(), ref_o)
+    assert scratch[:2].cpu().tolist() == [0, 0]
+
+
+def test_a_load_that_never_completes_is_reported_and_the_loads_in_flight_are_waited_for(monkeypatch):
+    """Second test hook: the first piece of CTA 0 announces 16 bytes more than it loads, so its mbarrier never
+    completes and the wait runs into its (lowered) clock limit.  The CTA must record CASCADE_ST_ETIMEOUT, wait
+    for the other loads it had in flight, and return; every other CTA finishes its share; the context stays usable."""
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    n_chunks, cb = 8, 32768
+    bb = n_chunks * cb
+    n_hbm, n_host, n = 64, 64, 40
+    lay = wl.kv_layout(n_hbm, n_chunks, cb)
+    rng = np.random.default_rng(1)
+    hbm_np = rng.integers(0, 256, n_hbm * bb, dtype=np.uint8)
+    host_np = rng.integers(0, 256, n_host * bb, dtype=np.uint8)
+    src, dst = wl.copy_lists(3, n, n_host, n_hbm)
+    t = lambda a: torch.from_numpy(a).cuda()
+    monkeypatch.setenv("CASCADE_TEST_MOVE_STALL", "2")
+    hooked = cs.Context(wl.default_params(), 16, 0)
+    monkeypatch.delenv("CASCADE_TEST_MOVE_STALL")
+    hbm, host = torch.from_numpy(hbm_np.copy()).cuda(), torch.from_numpy(host_np.copy()).pin_memory()
+    hooked.kv_restore(cs.make_layout(lay), hbm, host, n_host, False, t(src), t(dst), None, n)
+    torch.cuda.synchronize()
+    assert hooked.status()[0] == cs.ST_ETIMEOUT
+    want = hbm_np.copy()
+    assert oracle.kv_restore(want, lay, host_np, n_host, src, dst) == 0
+    got = hbm.cpu().numpy()
+    # only pieces of CTA 0's share may be missing: everything else is in place, nothing else was touched
+    diff = np.nonzero(got != want)[0]
+    assert len(diff) < len(want) // 4
+    untouched = np.ones(n_hbm, bool)
+    untouched[dst] = False
+    v = lambda a: a.reshape(n_chunks, n_hbm, cb)
+    assert np.array_equal(v(got)[:, untouched], v(hbm_np)[:, untouched])
+    # same process, same GPU, ordinary context: the full result
+    ctx = cs.Context(wl.default_params(), 16, 0)
+    ctx.kv_restore(cs.make_layout(lay), hbm, host, n_host, False, t(src), t(dst), None, n)
+    torch.cuda.synchronize()
+    assert ctx.status()[0] == 0 and np.array_equal(hbm.cpu().numpy(), want)
+
+
+def test_fused_move_beside_a_kernel_that_holds_most_of_the_gpu(monkeypatch):
+    """The paper's premise is that spills and restores overlap the running batch.  A finite filler kernel
+    (test-only, clock-bounded) holds the shared memory of all but a few SMs on a second stream while the
+    fused move runs with restores that depend on evictions, the wait limit lowered to a tenth of a second.
+    The restore grid only starts once every evict CTA is on an SM, so no wait can run out: the result equals
+    evict-then-restore bit for bit and the status word stays clear."""
+    import torch
+    from helpers import load_gpu_filler
+    from paper_2608_06557_b200 import cascade as cs
+    filler = load_gpu_filler()
+    n_chunks, cb = 64, 32768
+    bb = n_chunks * cb
+    n_hbm, n_host, ne, nr = 80, 80, 32, 32
+    lay = wl.kv_layout(n_hbm, n_chunks, cb)
+    rng = np.random.default_rng(2)
+    hbm_np = rng.integers(0, 256, n_hbm * bb, dtype=np.uint8)
+    host_np = rng.integers(0, 256, n_host * bb, dtype=np.uint8)
+    hp, op = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_host).astype(np.int32)
+    es, ed, rs = hp[:ne], op[:ne], op[ne:ne + nr]
+    rd = np.concatenate([es[::-1][: nr // 2], hp[ne:ne + nr - nr // 2]]).astype(np.int32)
+    ref_h, ref_o = hbm_np.copy(), host_np.copy()
+    assert oracle.kv_evict(ref_h, lay, ref_o, n_host, es, ed) == 0 and oracle.kv_restore(ref_h, lay, ref_o, n_host, rs, rd) == 0
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    monkeypatch.setenv("CASCADE_TEST_MOVE_STALL", "3")       # lowers the wait limits, stalls nothing
+    ctx = cs.Context(wl.default_params(), 16, 0)
+    monkeypatch.delenv("CASCADE_TEST_MOVE_STALL")
+    hbm, host = torch.from_numpy(hbm_np.copy()).cuda(), torch.from_numpy(host_np.copy()).pin_memory()
+    scratch = torch.empty(cs.kv_move_scratch_len(ne, nr), dtype=torch.int32, device="cuda")
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    side, main = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    done_fill, done_move = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start = torch.cuda.Event(enable_timing=True)
+    start.record(side)
+    # 200 KB of shared memory per CTA: no ring CTA (128 KB) fits beside one; about 30 ms at 1.9 GHz
+    assert filler.filler_launch(sms - 6, 200 * 1024, 60_000_000, side.cuda_stream) == 0
+    done_fill.record(side)
+    ctx.kv_move(cs.make_layout(lay), hbm, host, n_host, t(es), t(ed), None, ne, t(rs), t(rd), None, nr, scratch, main)
+    done_move.record(main)
+    torch.cuda.synchronize()
+    assert ctx.status()[0] == 0
+    assert scratch[:nr].cpu().tolist() == [0] * nr
+    assert np.array_equal(hbm.cpu().numpy(), ref_h) and np.array_equal(host.numpy(), ref_o)
+    assert start.elapsed_time(done_fill) > 5.0            # the filler really held the GPU for a while

@@ -168,3 +168,23 @@ def test_parameters_replaced_between_iterations():
     again = inst2.fetch()
     for k in ("budget", "key", "order", "grant", "x1", "action"):
         assert np.array_equal(again[k], third[k]), k
+
+
+def test_a_context_of_another_device_is_rejected_before_any_launch():
+    """The hot calls launch on the current device and dereference the context's own allocations: a context
+    created for another GPU is refused on the host.  Needs two GPUs; skipped otherwise."""
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    from paper_2608_06557_b200.runner import Instance
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two GPUs")
+    w = wl.config_tiny(0)
+    inst = Instance(w, device="cuda:1", alloc_pools=False)      # context and buffers on GPU 1
+    torch.cuda.set_device(0)
+    try:
+        with pytest.raises(cs.CascadeError, match="CASCADE_EINVAL"):
+            inst.ctx.budget(inst.reqs_struct, inst.n, w.now_ns, w.D_act, w.K_act, inst.budget, inst.key, 0)
+        with pytest.raises(cs.CascadeError, match="CASCADE_EINVAL"):
+            inst.ctx.schedule(inst.reqs_struct, inst.key, inst.n, w.D_act, inst.order, inst.grant, inst.sched_counts, 0)
+    finally:
+        torch.cuda.set_device(0)

@@ -69,7 +69,7 @@ def test_fused_move_on_random_shapes():
         host = torch.from_numpy(host_np).pin_memory()
         t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda() if len(a) else \
             torch.zeros(1, dtype=torch.int32, device="cuda")
-        scratch = torch.empty(ne + nr + 1, dtype=torch.int32, device="cuda")
+        scratch = torch.empty(cs.kv_move_scratch_len(ne, nr), dtype=torch.int32, device="cuda")
         ctx.kv_move(cs.make_layout(lay), hbm, host, n_host, t(es), t(ed), None, ne, t(rs), t(rd), None, nr, scratch)
         torch.cuda.synchronize()
         assert np.array_equal(hbm.cpu().numpy(), ref_h), (n_hbm, n_host, n_chunks, cb, ne, nr, k)

@@ -40,28 +40,47 @@ struct CopyArgs {
     int stall;                // test hooks, see cascade_ctx::test_move_stall
 };
 
-template <bool kRestore>
+enum { kRoleRestore = 0, kRoleEvict = 1, kRoleMoveEvict = 2, kRoleMoveRestore = 3 };
+constexpr long long kWaitCycles = 4000000000LL;  // about two seconds at 1.9 GHz
+
+__device__ __forceinline__ int clamp_count(const int32_t *dev, int maxv) {
+    if (!dev) return maxv;
+    const int c = __ldcg(dev);
+    return c < 0 ? 0 : (c < maxv ? c : maxv);
+}
+
+// Vector variant.  The roles are those of the ring kernel below: the two plain copies and the two grids of
+// the fused evict + restore (see cascade_kv_move for how the two grids are ordered).
+template <int kRole>
 __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant__ CopyArgs a) {
-    cascade_grid_wait();
-    int count = a.n_max;
-    if (a.n_dev) {
-        const int c = *a.n_dev;
-        count = c < 0 ? 0 : (c < count ? c : count);
-    }
+    constexpr bool kRestore = kRole == kRoleRestore || kRole == kRoleMoveRestore;
+    __shared__ int s_skip;
+    if (kRole != kRoleMoveRestore) cascade_grid_wait();
+    if (kRole == kRoleMoveEvict) cascade_grid_trigger();
+    const int count = clamp_count(a.n_dev, a.n_max);
     const long long per_block = (long long)a.n_chunks * a.pieces_per_chunk;
     const long long items = (long long)count * per_block;
     const long long bb = (long long)a.n_chunks * a.chunk_bytes;
+    const long long limit = a.stall ? kWaitCycles / 20 : kWaitCycles;
     const int tid = threadIdx.x;
-    bool bad = false;
+    uint32_t st = 0;
     for (long long it = blockIdx.x; it < items; it += gridDim.x) {
-        const long long i = it / per_block;
+        long long i = it / per_block;
         const int rem = (int)(it - i * per_block);
+        if (kRole == kRoleMoveEvict) i = count - 1 - i;  // blocks freed last are handed out first: read them out first
         const int c = rem / a.pieces_per_chunk;
         const int pc = rem - c * a.pieces_per_chunk;
-        const long long s = a.src_ids[i], d = a.dst_ids[i];
+        const long long s = __ldcg(a.src_ids + i), d = __ldcg(a.dst_ids + i);
         const long long rec_id = kRestore ? s : d, pg_id = kRestore ? d : s;
+        const long long left = a.chunk_bytes - (long long)pc * kPiece;
+        const int piece_bytes = (int)(left < kPiece ? left : kPiece);
         if (rec_id < 0 || rec_id >= a.record_blocks || pg_id < 0 || pg_id >= a.paged_blocks) {
-            bad = true;  // id outside its pool: this pair is skipped
+            st |= CASCADE_ST_EBOUNDS;  // id outside its pool: this pair is skipped
+            if (tid == 0) {
+                // a skipped evict piece still counts as read, or a restore into that block would wait for nothing
+                if (kRole == kRoleMoveEvict) atomicAdd(&a.done[i], piece_bytes >> 4);
+                if (kRole == kRoleMoveRestore) atomicAdd(&a.skipped[i], 1);
+            }
             continue;
         }
         char *rec = a.record + rec_id * bb + (long long)c * a.chunk_bytes;
@@ -75,13 +94,47 @@ __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant
             const long long off = base + (long long)u * kThreads * 16;
             if (off < a.chunk_bytes) v[u] = __ldcs(reinterpret_cast<const uint4 *>(src + off));
         }
+        if (kRole == kRoleMoveRestore) {
+            const int dep = __ldcg(a.dep + i);  // the same for every thread of the CTA
+            if (dep >= 0) {
+                // the HBM block is being evicted by this same call: write only after it has been read out
+                if (tid == 0) {
+                    const volatile int32_t *flag = a.done + dep;
+                    int skip = (st & CASCADE_ST_ETIMEOUT) ? 1 : 0;  // one expired wait is enough: do not queue up more
+                    const long long t0 = clock64();
+                    while (!skip && *flag < (int)(bb >> 4))
+                        if (clock64() - t0 > limit) skip = 1;
+                    if (skip) {
+                        st |= CASCADE_ST_ETIMEOUT;
+                        atomicAdd(&a.skipped[i], 1);
+                    }
+                    __threadfence();
+                    s_skip = skip;
+                }
+                __syncthreads();
+                const bool skip = s_skip != 0;
+                __syncthreads();
+                if (skip) continue;
+            }
+        }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             const long long off = base + (long long)u * kThreads * 16;
             if (off < a.chunk_bytes) __stcs(reinterpret_cast<uint4 *>(dst + off), v[u]);
         }
+        if (kRole == kRoleMoveEvict) {
+            // every thread's loads have returned once its stores are issued: this piece has left HBM; counted in
+            // 16-byte units, because the two grids may cut their blocks into pieces of different sizes
+            __syncthreads();
+            if (tid == 0 && a.stall != 1) {
+                __threadfence();
+                atomicAdd(&a.done[i], piece_bytes >> 4);
+            }
+        }
     }
-    if (bad && tid == 0) atomicOr(a.status, CASCADE_ST_EBOUNDS);
+    if (st && tid == 0) atomicOr(a.status, st);
+    // completion of the restore grid must imply completion of the evict grid it ran beside
+    if (kRole == kRoleMoveRestore) cascade_grid_wait();
 }
 
 
@@ -101,9 +154,6 @@ constexpr int kPieceMin = 8 * 1024;
 constexpr int kMaxStages = 16;
 constexpr int kRingHost = 128 * 1024;   // one CTA per SM
 constexpr int kRingDev = 96 * 1024;     // two CTAs per SM fit
-constexpr long long kWaitCycles = 4000000000LL;  // about two seconds at 1.9 GHz
-
-enum { kRoleRestore = 0, kRoleEvict = 1, kRoleMoveEvict = 2, kRoleMoveRestore = 3 };
 
 __device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -140,12 +190,6 @@ __device__ __forceinline__ void bulk_store(void *dst, unsigned src_smem, unsigne
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
                  : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-
-__device__ __forceinline__ int clamp_count(const int32_t *dev, int maxv) {
-    if (!dev) return maxv;
-    const int c = __ldcg(dev);
-    return c < 0 ? 0 : (c < maxv ? c : maxv);
 }
 
 template <int kRole>
@@ -284,12 +328,17 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
 //      open-addressing hash table over the evicted block ids: linear work in the two list lengths;
 //   2. the evict grid (role kRoleMoveEvict), half of the SMs: device -> host; after every piece that has
 //      left HBM it bumps that entry's counter.  It signals "dependents may launch" as its first action;
-//   3. the restore grid (role kRoleMoveRestore), the other half, launched as a PROGRAMMATIC DEPENDENT of
+//   3. the restore grid (role kRoleMoveRestore), on the other half, launched as a PROGRAMMATIC DEPENDENT of
 //      grid 2: the hardware starts it only once every CTA of the evict grid is running (or done), so a
 //      restore CTA that waits for a counter always waits for a CTA that is already on an SM and never waits
 //      itself: no deadlock however busy the GPU is with other work.  A restore into a block that the same
 //      call evicts stores only after that block's counter says it has been read out completely.
 // Without programmatic launch (CASCADE_PDL=0) grid 3 simply starts after grid 2 has finished.
+// Measured on B200: when both grids use the bulk-copy ring, the restore grid's bulk reads of host memory make
+// no progress until the evict grid's bulk writes are over (52 GB/s, the two directions one after the other);
+// with the restore grid on plain vector loads both directions run at once (71 - 80 GB/s), so by default the
+// evict grid is the ring kernel and the restore grid the vector kernel (CASCADE_MOVE_VECTOR, bit 0 = restore
+// grid, bit 1 = evict grid on the vector kernel).
 struct PrepareArgs {
     const int32_t *evict_src, *restore_dst;
     const int32_t *n_evict_dev, *n_restore_dev;
@@ -422,7 +471,8 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
     const int per_sm = record_is_device ? ctx->copy_ctas_dev : ctx->copy_ctas_host;
     long long grid = (long long)ctx->num_sms * per_sm;
     if (grid > items) grid = items;
-    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(kThreads), 0, s, kv_copy_kernel<kRestore>, a));
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(kThreads), 0, s,
+                                         kv_copy_kernel<kRestore ? kRoleRestore : kRoleEvict>, a));
     return CASCADE_OK;
 }
 
@@ -519,10 +569,29 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     const long long items_r = (long long)n_restore_max * hbm->n_chunks * ppc_max;
     if (ge > items_e) ge = items_e < 1 ? 1 : items_e;
     if (gr > items_r) gr = items_r;
-    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)ge), dim3(32), (size_t)e.ring_bytes, s,
-                                         kv_ring_kernel<kRoleMoveEvict>, e));
-    if (gr > 0)
-        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)gr), dim3(32), (size_t)r.ring_bytes, s,
-                                             kv_ring_kernel<kRoleMoveRestore>, r));
+    e.pieces_per_chunk = r.pieces_per_chunk = (int)((hbm->chunk_bytes + kPiece - 1) / kPiece);
+    const int vec_per_sm = ctx->copy_ctas_host;
+    if (ctx->move_vector & 2) {
+        long long g = (long long)half * vec_per_sm;
+        const long long iv = (long long)n_evict_max * hbm->n_chunks * e.pieces_per_chunk;
+        if (g > iv) g = iv < 1 ? 1 : iv;
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)g), dim3(kThreads), 0, s,
+                                             kv_copy_kernel<kRoleMoveEvict>, e));
+    } else {
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)ge), dim3(32), (size_t)e.ring_bytes, s,
+                                             kv_ring_kernel<kRoleMoveEvict>, e));
+    }
+    if (gr > 0) {
+        if (ctx->move_vector & 1) {
+            long long g = (long long)half * vec_per_sm;
+            const long long iv = (long long)n_restore_max * hbm->n_chunks * r.pieces_per_chunk;
+            if (g > iv) g = iv;
+            CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)g), dim3(kThreads), 0, s,
+                                                 kv_copy_kernel<kRoleMoveRestore>, r));
+        } else {
+            CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)gr), dim3(32), (size_t)r.ring_bytes, s,
+                                                 kv_ring_kernel<kRoleMoveRestore>, r));
+        }
+    }
     return CASCADE_OK;
 }

@@ -21,7 +21,8 @@
  *     mapped host allocation (cudaHostAlloc / torch pin_memory) counts as device-accessible.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - The library allocates device memory only in cascade_create.  The five hot calls allocate
- *     nothing, never synchronise the host and use no stream of their own.
+ *     nothing, never synchronise the host and use no stream of their own (the one exception, by its
+ *     nature, is cascade_kv_move_staged: it drives the copy engines from the host).
  *   - One context per stream.  A context is not thread-safe.
  *   - Return value: 0 on success, a negative CASCADE_E* code for errors found on the host before
  *     anything is launched.  Conditions found on the device never trap; they OR a CASCADE_ST_* bit
@@ -387,6 +388,39 @@ int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_po
                     const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,
                     const int32_t *restore_dst, const int32_t *n_restore_dev, int n_restore_max, int32_t *scratch,
                     void *stream);
+
+/*
+ * Evict and restore through the GPU's copy engines (the "asynchronous prefix prefetcher" driven from the host;
+ * the rate this path reaches is the B^eff of Eq. 6 for large blocks).  Same result as cascade_kv_evict followed
+ * by cascade_kv_restore; same list arguments as cascade_kv_move.  Unlike every other hot call this one
+ * SYNCHRONISES THE HOST with `stream` once, because the copy engines are programmed by the host and the lists
+ * live in device memory:
+ *   1. a kernel publishes the two counts and the live list entries into `mailbox`, the host waits for it;
+ *   2. evictions: the paged blocks are gathered into `staging` on `stream` (HBM to HBM), then one
+ *      cudaMemcpyAsync per run of consecutive host records drains them to the host pool on a side stream;
+ *   3. restores: one cudaMemcpyAsync per run of consecutive host records fills `staging` on a second side
+ *      stream, then the staged blocks are scattered into the paged pool on `stream` (behind every gather);
+ *   4. `stream` is made to wait for both side streams, so work issued on it afterwards sees the complete result.
+ * The call returns when everything has been enqueued, not when it has run.  Both directions of the link are
+ * busy at once; if a restore reads a host record that this call's evictions write, the fills wait for the drains.
+ *   staging         caller-owned device buffer of staging_blocks * block bytes, 16-byte aligned, at least one
+ *                   block per non-empty list (CASCADE_EINVAL otherwise, found after the host wait);
+ *                   split between the two directions in proportion to the lists; with fewer blocks than
+ *                   the lists hold the batches queue up for space (correct, slower)
+ *   mailbox         caller-owned PINNED, mapped host array of cascade_kv_mailbox_len(n_evict_max, n_restore_max)
+ *                   int32; after the call: [0] eviction count, [1] restore count, then the four lists
+ * Faster than the zero-copy kernels for blocks of a megabyte and more (the copy engines move 55 - 57 GB/s per
+ * direction and 96 - 100 GB/s both ways on a PCIe Gen5 x16 link), slower for small blocks (a few microseconds
+ * of host and engine work per copy).  Cannot be captured in a CUDA graph (host synchronisation).
+ * Errors: as cascade_kv_move, plus CASCADE_ENOMEM (host bookkeeping could not grow).  Ids outside a pool:
+ * that pair is skipped, CASCADE_ST_EBOUNDS.
+ */
+int64_t cascade_kv_mailbox_len(int n_evict_max, int n_restore_max);
+int cascade_kv_move_staged(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, void *host_pool,
+                           int64_t host_blocks, const int32_t *evict_src, const int32_t *evict_dst,
+                           const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,
+                           const int32_t *restore_dst, const int32_t *n_restore_dev, int n_restore_max, void *staging,
+                           int64_t staging_blocks, int32_t *mailbox, void *stream);
 
 /* ---------------------------------------------------------------------------------------------------
  * Deep tier as a real stage, and one copy per shared block.

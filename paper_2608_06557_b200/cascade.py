@@ -25,7 +25,7 @@ EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_b
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
            "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan", "cascade_kv_move",
            "cascade_stage_plan", "cascade_kv_stage", "cascade_dedup", "cascade_reqs_update",
-           "cascade_kv_move_scratch_len")
+           "cascade_kv_move_scratch_len", "cascade_kv_mailbox_len", "cascade_kv_move_staged")
 
 
 class Params(C.Structure):
@@ -142,6 +142,9 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_kv_move.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int,
                                     vp, vp]
     lib.cascade_kv_move_scratch_len.argtypes = [C.c_int, C.c_int]
+    lib.cascade_kv_mailbox_len.argtypes = [C.c_int, C.c_int]
+    lib.cascade_kv_move_staged.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int,
+                                           vp, i64, vp, vp]
     lib.cascade_reqs_update.argtypes = [vp, C.POINTER(Reqs), C.c_int, C.POINTER(Reqs), vp, C.c_int, vp]
     lib.cascade_stage_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64, i64, i32, C.POINTER(Pools),
                                        C.POINTER(Stage), vp]
@@ -153,6 +156,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
         if name != "cascade_destroy":
             getattr(lib, name).restype = C.c_int
     lib.cascade_kv_move_scratch_len.restype = C.c_int64
+    lib.cascade_kv_mailbox_len.restype = C.c_int64
     return lib
 
 
@@ -215,6 +219,11 @@ def _check(rc: int, what: str):
 def kv_move_scratch_len(n_evict_max: int, n_restore_max: int) -> int:
     """int32 entries cascade_kv_move needs in its caller-owned scratch."""
     return int(_lib.cascade_kv_move_scratch_len(n_evict_max, n_restore_max))
+
+
+def kv_mailbox_len(n_evict_max: int, n_restore_max: int) -> int:
+    """int32 entries of the pinned mailbox cascade_kv_move_staged publishes the lists into."""
+    return int(_lib.cascade_kv_mailbox_len(n_evict_max, n_restore_max))
 
 
 def make_reqs(t: dict) -> Reqs:
@@ -288,6 +297,15 @@ class Context:
                                     _p(evict_src), _p(evict_dst), _p(n_evict_dev), n_evict_max, _p(restore_src),
                                     _p(restore_dst), _p(n_restore_dev), n_restore_max, _p(scratch),
                                     _stream(stream)), "cascade_kv_move")
+
+    def kv_move_staged(self, layout: KvLayout, hbm_pool, host_pool, host_blocks, evict_src, evict_dst, n_evict_dev,
+                       n_evict_max, restore_src, restore_dst, n_restore_dev, n_restore_max, staging, staging_blocks,
+                       mailbox, stream=None):
+        _check(_lib.cascade_kv_move_staged(self._h, C.byref(layout), _p(hbm_pool), _p(host_pool), host_blocks,
+                                           _p(evict_src), _p(evict_dst), _p(n_evict_dev), n_evict_max,
+                                           _p(restore_src), _p(restore_dst), _p(n_restore_dev), n_restore_max,
+                                           _p(staging), staging_blocks, _p(mailbox), _stream(stream)),
+               "cascade_kv_move_staged")
 
     def stage_plan(self, reqs: Reqs, budget, order, action, n, D_act, K_act, link_budget_ns, host_reserve,
                    pools: Pools, stage: Stage, stream=None):

@@ -77,6 +77,10 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->move_ctas = e ? atoi(e) : 0;
     e = getenv("CASCADE_MOVE_VECTOR");
     ctx->move_vector = e ? (atoi(e) & 3) : 1;   // measured: bulk reads of the restore grid starve beside the evict grid's bulk writes
+    e = getenv("CASCADE_CE_HYBRID");
+    ctx->ce_hybrid = e ? atoi(e) : 0;
+    e = getenv("CASCADE_CE_LANES");
+    ctx->ce_lanes = e && atoi(e) == 2 ? 2 : 1;   // measured: a second stream per direction gains nothing
     e = getenv("CASCADE_COPY_PIECE");
     ctx->copy_piece = e ? atoi(e) : 0;
     if (ctx->copy_piece != 8192 && ctx->copy_piece != 16384 && ctx->copy_piece != 32768) ctx->copy_piece = 0;
@@ -98,6 +102,10 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
               cudaMalloc(&ctx->work_admit, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->work_victim, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->plan_scalars, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
+    for (int i = 0; ok && i < 4; ++i)
+        ok = cudaStreamCreateWithFlags(&ctx->ce_stream[i], cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < 7; ++i)
+        ok = cudaEventCreateWithFlags(&ctx->ce_event[i], cudaEventDisableTiming) == cudaSuccess;
     if (ok) ok = cudaMemset(ctx->status_dev, 0, sizeof(uint32_t)) == cudaSuccess &&
                  cudaMemset(ctx->plan_scalars, 0, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
     if (!ok) {
@@ -121,6 +129,11 @@ extern "C" void cascade_destroy(cascade_ctx *ctx) {
     cudaFree(ctx->work_admit);
     cudaFree(ctx->work_victim);
     cudaFree(ctx->plan_scalars);
+    for (int i = 0; i < 4; ++i)
+        if (ctx->ce_stream[i]) cudaStreamDestroy(ctx->ce_stream[i]);
+    for (int i = 0; i < 7; ++i)
+        if (ctx->ce_event[i]) cudaEventDestroy(ctx->ce_event[i]);
+    free(ctx->ce_bitmap);
     if (prev_device >= 0) cudaSetDevice(prev_device);
     free(ctx);
 }

@@ -39,6 +39,13 @@ struct cascade_ctx {
     int copy_ring_kb;            // >0: shared memory of the TMA ring in KiB (64..128); 0 = 128 (host) / 96 (device)
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels
     int rank_sort_max;           // queues up to this size are ordered by counting instead of radix passes
+    // copy-engine path (cascade_kv_move_staged): side streams and events, created with the context
+    cudaStream_t ce_stream[4];   // [0], [1] host -> staging (restores); [2], [3] staging -> host (evictions)
+    cudaEvent_t ce_event[7];     // lists published, gather done, scatter done, fill done x2, drain done x2
+    int ce_lanes;                // side streams used per direction (1 | 2)
+    int ce_hybrid;               // 1: evictions by the zero-copy kernel, only the restores through the copy engines
+    unsigned long long *ce_bitmap;   // host-side: one bit per host record, grown on demand
+    size_t ce_bitmap_words;
     int test_move_stall;         // test hooks (CASCADE_TEST_MOVE_STALL): 1 = the evict side of the fused move never
                                  // reports a block as read out, 2 = the first piece of CTA 0 of a ring kernel announces
                                  // more bytes than it loads; both make a bounded wait run out; 1, 2 and 3 lower the

@@ -11,6 +11,9 @@
 //       it leaves the SMs' issue slots free for whatever else runs on the GPU;
 //   kv_copy_kernel            256 threads x 4 x 16-byte vector loads/stores per 16 KiB piece on a
 //       persistent grid (selected with CASCADE_COPY_BULK_HOST=0 / CASCADE_COPY_BULK_DEV=0).
+#include <stdlib.h>
+#include <string.h>
+
 #include "common.cuh"
 
 namespace {
@@ -33,6 +36,9 @@ struct CopyArgs {
     int pieces_per_chunk;     // vector kernel only
     int ring_bytes;           // ring kernel: shared memory of the ring
     int piece_fixed;          // ring kernel: >0 forces this piece size (bytes), 0 = pick per call
+    int record_iota;          // ring kernel: the record id of list entry i is i itself (staging buffer filled in list order)
+    const int32_t *iota_check;    // with record_iota: entry i is skipped unless 0 <= iota_check[i] < iota_check_blocks
+    long long iota_check_blocks;  // (the id its staging slot was, or will be, copied from / to by the copy engines)
     // fused move only
     const int32_t *dep;       // per restore: evict-list index of the entry that frees its HBM block, or -1
     int32_t *done;            // per evict entry: 16-byte units of the block already read out of HBM
@@ -245,7 +251,18 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
             const int rem = (int)(it - i * per_block);
             if (kRole == kRoleMoveEvict) i = count - 1 - i;  // blocks freed last are handed out first: read them out first
             const int c = rem / ppc, pc = rem - c * ppc;
-            const long long s = __ldcg(a.src_ids + i), d = __ldcg(a.dst_ids + i);
+            long long s, d;
+            if (a.record_iota) {   // only the paged side has a list
+                s = kRestore ? i : __ldcg(a.src_ids + i);
+                d = kRestore ? __ldcg(a.dst_ids + i) : i;
+                if (a.iota_check) {
+                    const long long far = __ldcg(a.iota_check + i);
+                    if (far < 0 || far >= a.iota_check_blocks) { if (kRestore) s = -1; else d = -1; }
+                }
+            } else {
+                s = __ldcg(a.src_ids + i);
+                d = __ldcg(a.dst_ids + i);
+            }
             const long long rec_id = kRestore ? s : d, pg_id = kRestore ? d : s;
             const long long off = (long long)pc * piece;
             const long long left = a.chunk_bytes - off;
@@ -593,5 +610,249 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
                                                  kv_ring_kernel<kRoleMoveRestore>, r));
         }
     }
+    return CASCADE_OK;
+}
+
+
+// ---- evict + restore through the copy engines -------------------------------------------------------
+// The lists live in device memory, the copy engines are driven by the host: a small kernel publishes
+// the two counts and the lists' live entries into a pinned mailbox, the host waits for it ONCE, then
+//   evictions: [stream] gather the paged blocks into the staging buffer (ring kernel, HBM to HBM)
+//              [side 1] one cudaMemcpyAsync per run of consecutive host records, staging -> host pool
+//   restores:  [side 0] one cudaMemcpyAsync per run of consecutive host records, host pool -> staging
+//              [stream] scatter the staged blocks into the paged pool (ring kernel, HBM to HBM)
+// with every gather ahead of every scatter on the caller's stream (a freed block may be handed out again
+// at once) and the two side streams running beside each other, so both directions of the link are busy.
+// Gathers and fills go in batches (a small first one) so that the link starts after microseconds.
+namespace {
+
+struct PublishArgs {
+    const int32_t *evict_src, *evict_dst, *restore_src, *restore_dst;
+    const int32_t *n_evict_dev, *n_restore_dev;
+    int n_evict_max, n_restore_max;
+    int32_t *mailbox;   // pinned, mapped host memory
+};
+
+__global__ void __launch_bounds__(256) kv_publish_lists_kernel(const __grid_constant__ PublishArgs a) {
+    cascade_grid_wait();
+    const int ne = clamp_count(a.n_evict_dev, a.n_evict_max), nr = clamp_count(a.n_restore_dev, a.n_restore_max);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
+    int32_t *es = a.mailbox + 2, *ed = es + a.n_evict_max, *rs = ed + a.n_evict_max, *rd = rs + a.n_restore_max;
+    for (int j = i; j < ne; j += stride) {
+        es[j] = a.evict_src[j];
+        ed[j] = a.evict_dst[j];
+    }
+    for (int j = i; j < nr; j += stride) {
+        rs[j] = a.restore_src[j];
+        rd[j] = a.restore_dst[j];
+    }
+    if (i == 0) {
+        a.mailbox[0] = ne;
+        a.mailbox[1] = nr;
+    }
+}
+
+constexpr int kFirstBatch = 8;    // blocks in the first gather / fill batch: the link starts early
+constexpr int kBatch = 64;
+
+// one HBM-to-HBM pass of the ring kernel between the paged pool and a staging region filled in list order
+template <bool kRestore>
+int launch_staged_pass(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char *region, const int32_t *paged_ids,
+                       const int32_t *host_ids, long long host_blocks, int m, cudaStream_t s) {
+    CopyArgs a;
+    fill_copy_args(a, ctx, l, paged, region, m, kRestore ? nullptr : paged_ids, kRestore ? paged_ids : nullptr, nullptr, m);
+    a.record_iota = 1;
+    a.iota_check = host_ids;
+    a.iota_check_blocks = host_blocks;
+    a.ring_bytes = ctx->copy_ring_kb > 0 ? ctx->copy_ring_kb * 1024 : kRingDev;
+    const long long items = (long long)m * l->n_chunks * ((l->chunk_bytes + kPieceMin - 1) / kPieceMin);
+    long long grid = (long long)ctx->num_sms * 2;
+    if (grid > items) grid = items;
+    constexpr int role = kRestore ? kRoleRestore : kRoleEvict;
+    CASCADE_CUDA_TRY(ctx, configure_ring<role>(ctx->device));
+    CASCADE_CUDA_TRY(ctx, cascade_launch(false, 0, dim3((unsigned)grid), dim3(32), (size_t)a.ring_bytes, s,
+                                         kv_ring_kernel<role>, a));
+    return CASCADE_OK;
+}
+
+}  // namespace
+
+extern "C" int64_t cascade_kv_mailbox_len(int n_evict_max, int n_restore_max) {
+    if (n_evict_max < 0 || n_restore_max < 0) return -1;
+    return 2 + 2 * (int64_t)n_evict_max + 2 * (int64_t)n_restore_max;
+}
+
+extern "C" int cascade_kv_move_staged(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_pool, void *host_pool,
+                                      int64_t host_blocks, const int32_t *evict_src, const int32_t *evict_dst,
+                                      const int32_t *n_evict_dev, int n_evict_max, const int32_t *restore_src,
+                                      const int32_t *restore_dst, const int32_t *n_restore_dev, int n_restore_max,
+                                      void *staging, int64_t staging_blocks, int32_t *mailbox, void *stream) {
+    CascadeRange nvtx_range("cascade_kv_move_staged");
+    if (!ctx || n_evict_max < 0 || n_restore_max < 0) return CASCADE_EINVAL;
+    if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
+    if (n_evict_max == 0 && n_restore_max == 0) return CASCADE_OK;
+    int rc = check_layout(hbm, hbm_pool, host_pool, host_blocks);
+    if (rc != CASCADE_OK) return rc;
+    if (!staging || !mailbox || staging_blocks < 1 || ((uintptr_t)staging & 15)) return CASCADE_EINVAL;
+    if ((n_evict_max > 0 && (!evict_src || !evict_dst)) || (n_restore_max > 0 && (!restore_src || !restore_dst)))
+        return CASCADE_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaStream_t *s_fill = ctx->ce_stream, *s_drain = ctx->ce_stream + 2;
+    cudaEvent_t ev_lists = ctx->ce_event[0], ev_gather = ctx->ce_event[1], ev_scatter = ctx->ce_event[2];
+    cudaEvent_t *ev_fill = ctx->ce_event + 3, *ev_drain = ctx->ce_event + 5;
+    const int L = ctx->ce_lanes;   // copies of one direction alternate between L side streams: the engines' per-copy
+                                   // set-up of one stream hides behind the transfer of the other
+    const long long bb = (long long)hbm->n_chunks * hbm->chunk_bytes;
+
+    // 1. lists -> pinned mailbox, and the one host wait of the call
+    PublishArgs p = {evict_src, evict_dst, restore_src, restore_dst, n_evict_dev, n_restore_dev, n_evict_max, n_restore_max, mailbox};
+    const int most = n_evict_max > n_restore_max ? n_evict_max : n_restore_max;
+    int pgrid = (most + 255) / 256;
+    if (pgrid > ctx->num_sms) pgrid = ctx->num_sms;
+    CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(pgrid), dim3(256), 0, s, kv_publish_lists_kernel, p));
+    CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_lists, s));
+    CASCADE_CUDA_TRY(ctx, cudaEventSynchronize(ev_lists));
+    const int ne = mailbox[0], nr = mailbox[1];
+    if (ne < 0 || ne > n_evict_max || nr < 0 || nr > n_restore_max) return CASCADE_EINVAL;
+    if (ne > 0 && nr > 0 && staging_blocks < 2) return CASCADE_EINVAL;   // one block of staging per direction at least
+    const int32_t *h_es = mailbox + 2, *h_ed = h_es + n_evict_max, *h_rs = h_ed + n_evict_max, *h_rd = h_rs + n_restore_max;
+    const long long paged_blocks = hbm->n_blocks;
+
+    // 2. does a restore read a host record that this call's evictions write?  Then the fills wait for the drains.
+    bool fill_after_drain = false;
+    if (ne > 0 && nr > 0) {
+        const size_t words = (size_t)(host_blocks + 63) / 64;
+        if (words > ctx->ce_bitmap_words) {
+            unsigned long long *nb = (unsigned long long *)realloc(ctx->ce_bitmap, words * sizeof(unsigned long long));
+            if (!nb) return CASCADE_ENOMEM;
+            ctx->ce_bitmap = nb;
+            ctx->ce_bitmap_words = words;
+        }
+        memset(ctx->ce_bitmap, 0, words * sizeof(unsigned long long));
+        for (int i = 0; i < ne; ++i)
+            if (h_ed[i] >= 0 && h_ed[i] < host_blocks) ctx->ce_bitmap[h_ed[i] >> 6] |= 1ull << (h_ed[i] & 63);
+        for (int i = 0; i < nr && !fill_after_drain; ++i)
+            if (h_rs[i] >= 0 && h_rs[i] < host_blocks && (ctx->ce_bitmap[h_rs[i] >> 6] >> (h_rs[i] & 63) & 1))
+                fill_after_drain = true;
+    }
+
+    // 3. staging regions: one per direction, in proportion to the lists
+    const bool hybrid = ctx->ce_hybrid == 1;
+    const bool hybrid_r = ctx->ce_hybrid == 2;   // restores by the zero-copy kernel, evictions through the copy engines
+    long long region_e = (ne == 0 || hybrid) ? 0 : (nr == 0 ? staging_blocks : staging_blocks * ne / ((long long)ne + nr));
+    if (ne > 0 && !hybrid && region_e < 1) region_e = 1;
+    if (nr > 0 && region_e > staging_blocks - 1) region_e = staging_blocks - 1;
+    const long long region_r = staging_blocks - region_e;
+    char *stage_e = (char *)staging, *stage_r = (char *)staging + region_e * bb;
+
+    // 4. evictions: gather batch -> drain batch; a region position is reused only after its drain
+    bool drained_any = false;
+    {
+        if (hybrid && ne > 0) {
+            rc = launch_copy<false>(ctx, hbm, (char *)hbm_pool, (char *)host_pool, host_blocks, 0, evict_src, evict_dst,
+                                    n_evict_dev, n_evict_max, s);
+            if (rc != CASCADE_OK) return rc;
+        }
+        long long pos = 0;
+        int batch = kFirstBatch, lane = 0;
+        for (int off = 0; off < (hybrid ? 0 : ne);) {
+            int m = ne - off < batch ? ne - off : batch;
+            if (m > region_e) m = (int)region_e;
+            if (pos + m > region_e) {   // wrap: everything drained so far must have left the region
+                pos = 0;
+                if (drained_any)
+                    for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ev_drain[k], 0));
+            }
+            rc = launch_staged_pass<false>(ctx, hbm, (char *)hbm_pool, stage_e + pos * bb, evict_src + off,
+                                           evict_dst + off, host_blocks, m, s);
+            if (rc != CASCADE_OK) return rc;
+            CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_gather, s));
+            for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_drain[k], ev_gather, 0));
+            for (int i = 0; i < m;) {
+                const long long rec = h_ed[off + i], pg = h_es[off + i];
+                if (rec < 0 || rec >= host_blocks || pg < 0 || pg >= paged_blocks) {
+                    i += 1;   // an id outside its pool: that pair is skipped (the gather kernel set the status bit)
+                    continue;
+                }
+                int run = 1;
+                while (i + run < m && h_ed[off + i + run] == rec + run && rec + run < host_blocks &&
+                       h_es[off + i + run] >= 0 && h_es[off + i + run] < paged_blocks)
+                    ++run;
+                CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync((char *)host_pool + rec * bb, stage_e + (pos + i) * bb,
+                                                      (size_t)run * bb, cudaMemcpyDeviceToHost, s_drain[lane]));
+                lane = (lane + 1) % L;
+                i += run;
+            }
+            for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_drain[k], s_drain[k]));
+            drained_any = true;
+            pos += m;
+            off += m;
+            batch = kBatch;
+        }
+    }
+
+    // 5. restores: fill batch -> scatter batch (all scatters are behind all gathers on the caller's stream)
+    {
+        for (int k = 0; k < L; ++k) {
+            if (fill_after_drain && drained_any)
+                for (int j = 0; j < L; ++j) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_drain[j], 0));
+            if (fill_after_drain && hybrid && ne > 0) {   // the zero-copy evictions are on the caller's stream
+                CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_gather, s));
+                CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_gather, 0));
+            }
+            // the fills follow everything issued earlier on the caller's stream: an earlier call's scatter may still
+            // read the staging region, an earlier kernel may still write the host records read here
+            CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_lists, 0));
+        }
+        if (hybrid_r && nr > 0) {
+            if (fill_after_drain && drained_any)
+                for (int j = 0; j < L; ++j) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ev_drain[j], 0));
+            rc = launch_copy<true>(ctx, hbm, (char *)hbm_pool, (char *)host_pool, host_blocks, 0, restore_src, restore_dst,
+                                   n_restore_dev, n_restore_max, s);
+            if (rc != CASCADE_OK) return rc;
+        }
+        long long pos = 0;
+        int batch = kFirstBatch, lane = 0;
+        bool scattered_any = false;
+        for (int off = 0; off < (hybrid_r ? 0 : nr);) {
+            int m = nr - off < batch ? nr - off : batch;
+            if (m > region_r) m = (int)region_r;
+            if (pos + m > region_r) {
+                pos = 0;
+                if (scattered_any)
+                    for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_scatter, 0));
+            }
+            for (int i = 0; i < m;) {
+                const long long rec = h_rs[off + i], pg = h_rd[off + i];
+                if (rec < 0 || rec >= host_blocks || pg < 0 || pg >= paged_blocks) {
+                    i += 1;   // an id outside its pool: that pair is skipped (the scatter kernel sets the status bit)
+                    continue;
+                }
+                int run = 1;
+                while (i + run < m && h_rs[off + i + run] == rec + run && rec + run < host_blocks &&
+                       h_rd[off + i + run] >= 0 && h_rd[off + i + run] < paged_blocks)
+                    ++run;
+                CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync(stage_r + (pos + i) * bb, (const char *)host_pool + rec * bb,
+                                                      (size_t)run * bb, cudaMemcpyHostToDevice, s_fill[lane]));
+                lane = (lane + 1) % L;
+                i += run;
+            }
+            for (int k = 0; k < L; ++k) {
+                CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_fill[k], s_fill[k]));
+                CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ev_fill[k], 0));
+            }
+            rc = launch_staged_pass<true>(ctx, hbm, (char *)hbm_pool, stage_r + pos * bb, restore_dst + off,
+                                          restore_src + off, host_blocks, m, s);
+            if (rc != CASCADE_OK) return rc;
+            CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_scatter, s));
+            scattered_any = true;
+            pos += m;
+            off += m;
+            batch = kBatch;
+        }
+    }
+    // 6. completion of the caller's stream implies that every host record has been written
+    if (drained_any)
+        for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ev_drain[k], 0));
     return CASCADE_OK;
 }

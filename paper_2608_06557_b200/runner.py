@@ -178,6 +178,17 @@ class Instance:
                          self.plan_counts[1:2], self.evict_cap, self.restore_src, self.restore_dst,
                          self.plan_counts[0:1], self.restore_cap, self.move_scratch, stream)
 
+    def run_move_staged(self, staging, stream=None):
+        """evict + restore through the copy engines (one host synchronisation inside the call); ``staging`` is a
+        device uint8 tensor of a whole number of blocks."""
+        if not hasattr(self, "mailbox"):
+            self.mailbox = torch.empty(cs.kv_mailbox_len(self.evict_cap, self.restore_cap), dtype=torch.int32,
+                                       pin_memory=True)
+        self.ctx.kv_move_staged(self.layout, self.hbm_pool, self.host_pool, self.host_blocks, self.evict_src,
+                                self.evict_dst, self.plan_counts[1:2], self.evict_cap, self.restore_src,
+                                self.restore_dst, self.plan_counts[0:1], self.restore_cap, staging,
+                                staging.numel() // self.block_bytes, self.mailbox, stream)
+
     # -- deep tier and shared blocks -------------------------------------------------------------
     def enable_deep(self, w, deep_pool=None, alloc_pool: bool = True):
         """Upload the deep-tier table of ``w`` and allocate what the stage plan and the one-copy-per-source

@@ -353,3 +353,67 @@ def test_fused_move_beside_a_kernel_that_holds_most_of_the_gpu(monkeypatch):
     assert scratch[:nr].cpu().tolist() == [0] * nr
     assert np.array_equal(hbm.cpu().numpy(), ref_h) and np.array_equal(host.numpy(), ref_o)
     assert start.elapsed_time(done_fill) > 5.0            # the filler really held the GPU for a while
+
+
+@pytest.mark.parametrize("shape,stage_blocks", [((64, 48, 4, 4096), 64), ((64, 48, 4, 4096), 5), ((40, 40, 3, 208), 2),
+                                                ((300, 300, 8, 32768), 37), ((30, 30, 2, 32 * 1024 + 64), 30)])
+def test_staged_move_through_the_copy_engines_equals_evict_then_restore(shape, stage_blocks):
+    """The copy-engine path: lists published to a pinned mailbox, one host wait, per-run cudaMemcpyAsync through a
+    device staging buffer, gather / scatter by the ring kernel.  Half of the restores land in blocks the same call
+    evicts; staging buffers smaller than the lists make the batches wrap."""
+    n_hbm, n_host, n_chunks, cb = shape
+    rig = CopyRig(n_hbm, n_host, n_chunks, cb)
+    torch, cs = rig.torch, rig.cs
+    rng = np.random.default_rng(n_hbm + stage_blocks)
+    ne, nr = n_hbm // 3, n_host // 3
+    hperm, operm = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_host).astype(np.int32)
+    evict_src, evict_dst = hperm[:ne], np.sort(operm[:ne])           # sorted records: runs of consecutive ids occur
+    restore_src = np.sort(operm[ne:ne + nr])
+    reuse = evict_src[::-1][: nr // 2]
+    restore_dst = np.concatenate([reuse, hperm[ne:ne + nr - len(reuse)]]).astype(np.int32)
+    ref_hbm, ref_host = rig.hbm_np.copy(), rig.host_np.copy()
+    assert oracle.kv_evict(ref_hbm, rig.lay, ref_host, n_host, evict_src, evict_dst) == 0
+    assert oracle.kv_restore(ref_hbm, rig.lay, ref_host, n_host, restore_src, restore_dst) == 0
+    cap_e, cap_r = ne + 3, nr + 2
+    pad = lambda a, cap: rig.ids(np.concatenate([a, np.full(cap - len(a), 10**6, np.int32)]))
+    counts = torch.tensor([nr, ne], dtype=torch.int32, device="cuda")
+    staging = torch.empty(stage_blocks * rig.bb, dtype=torch.uint8, device="cuda")
+    mailbox = torch.empty(cs.kv_mailbox_len(cap_e, cap_r), dtype=torch.int32, pin_memory=True)
+    for rep in range(2):
+        rig.hbm.copy_(torch.from_numpy(rig.hbm_np))
+        rig.host.copy_(torch.from_numpy(rig.host_np))
+        rig.ctx.kv_move_staged(rig.layout, rig.hbm, rig.host, n_host, pad(evict_src, cap_e), pad(evict_dst, cap_e),
+                               counts[1:2], cap_e, pad(restore_src, cap_r), pad(restore_dst, cap_r), counts[0:1], cap_r,
+                               staging, stage_blocks, mailbox)
+        torch.cuda.synchronize()
+        assert mailbox[:2].tolist() == [ne, nr]
+        assert np.array_equal(rig.hbm.cpu().numpy(), ref_hbm), rep
+        assert np.array_equal(rig.host.cpu().numpy(), ref_host), rep
+    assert rig.guards_intact() and rig.ctx.status()[0] == 0
+
+
+def test_staged_move_orders_a_restore_behind_the_eviction_that_writes_its_record_and_skips_bad_ids():
+    rig = CopyRig(32, 32, 4, 4096)
+    torch, cs = rig.torch, rig.cs
+    # restore 0 reads host record 7, which eviction 1 of the same call writes; ids outside the pools on both lists
+    evict_src = np.array([3, 9, 40, 11, 12], np.int32)
+    evict_dst = np.array([5, 7, 8, -2, 13], np.int32)
+    restore_src = np.array([7, 20, 99, 21], np.int32)
+    restore_dst = np.array([9, 1, 2, -1], np.int32)
+    ref_hbm, ref_host = rig.hbm_np.copy(), rig.host_np.copy()
+    st_e = oracle.kv_evict(ref_hbm, rig.lay, ref_host, 32, evict_src, evict_dst)
+    st_r = oracle.kv_restore(ref_hbm, rig.lay, ref_host, 32, restore_src, restore_dst)
+    assert st_e == st_r == cs.ST_EBOUNDS
+    staging = torch.empty(16 * rig.bb, dtype=torch.uint8, device="cuda")
+    mailbox = torch.empty(cs.kv_mailbox_len(5, 4), dtype=torch.int32, pin_memory=True)
+    rig.ctx.kv_move_staged(rig.layout, rig.hbm, rig.host, 32, rig.ids(evict_src), rig.ids(evict_dst), None, 5,
+                           rig.ids(restore_src), rig.ids(restore_dst), None, 4, staging, 16, mailbox)
+    torch.cuda.synchronize()
+    assert np.array_equal(rig.hbm.cpu().numpy(), ref_hbm) and np.array_equal(rig.host.cpu().numpy(), ref_host)
+    assert rig.ctx.status()[0] == cs.ST_EBOUNDS and rig.guards_intact()
+    # one list empty, then both empty
+    rig.ctx.kv_move_staged(rig.layout, rig.hbm, rig.host, 32, None, None, None, 0, rig.ids(restore_src[1:2]),
+                           rig.ids(restore_dst[1:2]), None, 1, staging, 16, mailbox)
+    rig.ctx.kv_move_staged(rig.layout, rig.hbm, rig.host, 32, None, None, None, 0, None, None, None, 0, staging, 16, mailbox)
+    torch.cuda.synchronize()
+    assert np.array_equal(rig.hbm.cpu().numpy(), ref_hbm) and rig.ctx.status()[0] == 0

@@ -87,6 +87,10 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     e = getenv("CASCADE_COPY_RING_KB");
     ctx->copy_ring_kb = e ? atoi(e) : 0;
     if (ctx->copy_ring_kb < 64 || ctx->copy_ring_kb > 128) ctx->copy_ring_kb = 0;
+    e = getenv("CASCADE_MERGE_SORT");
+    ctx->merge_sort = e ? atoi(e) : 1;
+    e = getenv("CASCADE_SORT_TOP_FIRST");
+    ctx->sort_top_first = e ? (atoi(e) != 0) : 1;
     e = getenv("CASCADE_RANK_SORT_MAX");
     ctx->rank_sort_max = e ? atoi(e) : 2048;
     e = getenv("CASCADE_TEST_MOVE_STALL");

@@ -38,6 +38,8 @@ struct cascade_ctx {
     int copy_piece;              // >0: piece size in bytes of the TMA ring (8192 | 16384 | 32768); 0 = picked per call
     int copy_ring_kb;            // >0: shared memory of the TMA ring in KiB (64..128); 0 = 128 (host) / 96 (device)
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels
+    int sort_top_first;          // 1: radix passes over bits 16..63 first, local fix-up of equal values (budget policy only)
+    int merge_sort;              // 1: queues of up to 16384 requests beyond the counting path are ordered by local sort + merge by rank
     int rank_sort_max;           // queues up to this size are ordered by counting instead of radix passes
     // copy-engine path (cascade_kv_move_staged): side streams and events, created with the context
     cudaStream_t ce_stream[4];   // [0], [1] host -> staging (restores); [2], [3] staging -> host (evictions)

@@ -56,6 +56,14 @@ struct __align__(16) Exch {
     int cnt;                  // elements with a non-zero grant before the batch-size cap
 };
 
+// what every CTA tells the others after the passes over bits 16..63
+struct __align__(16) TieExch {
+    unsigned long long first, last;  // bits 16..63 of the CTA's first and last real element
+    int count;                       // real elements the CTA holds
+    int flags;                       // 1: equal neighbours inside the CTA, 2: a run longer than kMaxRun
+};
+constexpr int kMaxRun = 128;
+
 struct ScheduleArgs {
     const uint64_t *key;
     const int32_t *prompt, *n0, *n1, *n2;
@@ -70,6 +78,7 @@ struct ScheduleArgs {
     int bt;
     int stage;          // 1: group by digit locally before the remote copy
     int async_sync;     // 1: per-pass exchanges complete on mbarriers (data driven), 0: cluster barriers
+    int top_first;      // 1: order by bits 16..63 first, fix short runs of equal values locally (see the pass loop)
     int rank_per;       // >0: small queue, order by counting (see rank_order below) with this many elements per CTA
     uint32_t *status;
 };
@@ -82,6 +91,139 @@ __device__ __forceinline__ T seg_incl_scan(T v, int pos, int width) {
         if (pos >= s) v += t;
     }
     return v;
+}
+
+// Admission (Algorithm 1, phase 2) on the sorted elements while they are still on chip: clamped prefix sums of
+// the tokens wanted against the Tier-1 / Tier-2 token budgets, the batch-size cap, then `order`, `grant` and the
+// counts are written.  e[k] is the element at sorted position crank*per_rt + (warp*K + k)*32 + lane; padding has
+// idx 0xffffffff.  Two cluster barriers; every CTA of the cluster must call it.
+template <int T, int K>
+__device__ __forceinline__ void admit_and_write(const ScheduleArgs &a, const SortElem (&e)[K], int per_rt,
+                                                cg::cluster_group &cluster, long long *wtmp, int *itmp, Exch *exall) {
+    constexpr int W = T / 32;
+    const unsigned crank = cluster.block_rank();
+    const unsigned csize = cluster.num_blocks();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    // ---- admission: clamped prefix sums over the sorted elements ---------------------------------
+    long long ex[K];
+    long long run = 0, s1 = 0, s2 = 0;
+    int c1 = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const long long w = e[k].want;
+        const bool real = e[k].idx != 0xffffffffu;
+        const bool t2 = (e[k].key >> 63) != 0;
+        if (real && !t2) { s1 += w; ++c1; }
+        if (real && t2) s2 += w;
+        const long long x = seg_incl_scan(w, lane, 32);
+        ex[k] = run + x - w;
+        run += __shfl_sync(kFull, x, 31);
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        s1 += __shfl_xor_sync(kFull, s1, s);
+        s2 += __shfl_xor_sync(kFull, s2, s);
+        c1 += __shfl_xor_sync(kFull, c1, s);
+    }
+    if (lane == 0) {
+        wtmp[warp] = run;
+        wtmp[32 + warp] = s1;
+        wtmp[64 + warp] = s2;
+        itmp[warp] = c1;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const bool in = lane < W;
+        const long long t = in ? wtmp[lane] : 0;
+        const long long inc = seg_incl_scan(t, lane, 32);
+        long long a1 = in ? wtmp[32 + lane] : 0, a2 = in ? wtmp[64 + lane] : 0;
+        int ac = in ? itmp[lane] : 0;
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) {
+            a1 += __shfl_xor_sync(kFull, a1, s);
+            a2 += __shfl_xor_sync(kFull, a2, s);
+            ac += __shfl_xor_sync(kFull, ac, s);
+        }
+        if (in) wtmp[lane] = inc - t;  // exclusive offset of each warp inside the CTA
+        if (lane < csize) {
+            Exch *x = cluster.map_shared_rank(exall, lane) + crank;
+            x->w1 = a1;
+            x->w2 = a2;
+            x->n1 = ac;
+        }
+    }
+    cluster.sync();
+    long long W1 = 0, W2 = 0, cta_off = 0;
+    int N1 = 0;
+#pragma unroll
+    for (int c = 0; c < kMaxCluster; ++c) {
+        if (c < csize) {
+            const long long x1 = exall[c].w1, x2 = exall[c].w2;
+            W1 += x1;
+            W2 += x2;
+            N1 += exall[c].n1;
+            if (c < crank) cta_off += x1 + x2;
+        }
+    }
+    const long long R2 = min(min(a.reserve, W2), a.TB);
+    const long long TB1 = a.TB - R2;
+    const long long TB2 = a.TB - min(TB1, W1);  // the reserve plus whatever Tier-1 left
+    const long long warp_off = cta_off + wtmp[warp];
+    int grant[K];
+    unsigned runc = 0;
+    unsigned exf[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const long long w = e[k].want;
+        const long long eg = warp_off + ex[k];
+        const bool t2 = (e[k].key >> 63) != 0;
+        long long g = t2 ? (TB2 - (eg - W1)) : (TB1 - eg);
+        g = g < 0 ? 0 : (g > w ? w : g);
+        grant[k] = (int)g;
+        const unsigned b = __ballot_sync(kFull, g > 0);
+        exf[k] = runc + __popc(b & lt_mask);
+        runc += __popc(b);
+    }
+    __syncthreads();  // wtmp is reused below
+    if (lane == 0) reinterpret_cast<unsigned *>(wtmp)[warp] = runc;
+    __syncthreads();
+    if (warp == 0) {
+        const unsigned t = lane < W ? reinterpret_cast<unsigned *>(wtmp)[lane] : 0u;
+        const unsigned inc = seg_incl_scan(t, lane, 32);
+        if (lane < W) reinterpret_cast<unsigned *>(wtmp)[lane] = inc - t;
+        const int tot = (int)__shfl_sync(kFull, inc, 31);
+        if (lane < csize) cluster.map_shared_rank(exall, lane)[crank].cnt = tot;
+    }
+    cluster.sync();
+    unsigned cnt_off = reinterpret_cast<unsigned *>(wtmp)[warp];
+#pragma unroll
+    for (int c = 0; c < kMaxCluster; ++c)
+        if (c < crank) cnt_off += (unsigned)exall[c].cnt;
+
+    long long tok = 0;
+    int adm = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (grant[k] > 0 && (long long)(cnt_off + exf[k]) >= (long long)a.seq_cap) grant[k] = 0;
+        if (e[k].idx != 0xffffffffu) {
+            const long long g = (long long)crank * per_rt + (warp * K + k) * 32 + lane;
+            a.order_out[g] = e[k].idx;
+            a.grant_out[e[k].idx] = grant[k];
+            tok += grant[k];
+            adm += grant[k] > 0;
+        }
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        tok += __shfl_xor_sync(kFull, tok, s);
+        adm += __shfl_xor_sync(kFull, adm, s);
+    }
+    if (lane == 0 && adm > 0) {
+        atomicAdd(reinterpret_cast<unsigned long long *>(&a.counts->tokens_granted), (unsigned long long)tok);
+        atomicAdd(&a.counts->n_admitted, adm);
+    }
+    if (crank == 0 && tid == 0) a.counts->n_tier1 = N1;
 }
 
 template <int T, int K>
@@ -105,8 +247,9 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     Exch *exall = reinterpret_cast<Exch *>(wtmp + 3 * 32);             // [kMaxCluster]
     uint16_t *minehist = reinterpret_cast<uint16_t *>(exall + kMaxCluster);   // [kBins], 16-byte aligned
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(minehist + kBins);  // hist[2], elem[2]
+    TieExch *tie_ex = reinterpret_cast<TieExch *>(bars + 4);                              // [kMaxCluster]
     // counting path only (the <256, 1> instance): every key of the queue, then per-thread partial counts
-    uint64_t *keys_all = reinterpret_cast<uint64_t *>(bars + 4);
+    uint64_t *keys_all = reinterpret_cast<uint64_t *>(tie_ex + kMaxCluster);
     int *partial = reinterpret_cast<int *>(keys_all + kRankMaxKeys);
     const bool by_rank = (K == 1) && a.rank_per > 0;
     const int per_rt = by_rank ? a.rank_per : per;   // elements this CTA holds
@@ -127,8 +270,7 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     SortElem e[K];
     const unsigned long long key0 = a.key[0];
     unsigned long long diff = 0;
-#pragma unroll
-    for (int k = 0; k < K; ++k) {
+    auto load_elem = [&](int k) {
         const int li = (warp * K + k) * 32 + lane;
         const long long g = (long long)crank * per_rt + li;
         if (li < per_rt && g < a.n) {
@@ -145,7 +287,9 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
             e[k].idx = 0xffffffffu;
             e[k].want = 0;
         }
-    }
+    };
+#pragma unroll
+    for (int k = 0; k < K; ++k) load_elem(k);
     if (by_rank) {
         if constexpr (K == 1) {
             // ---- order by counting ----------------------------------------------------------------
@@ -225,9 +369,16 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         if (c < csize) alld |= exall[c].diff;
 
     // ---- LSD radix sort, 8 bits per pass --------------------------------------------------------
+    // With top_first the two passes over the low 16 bits (arrival-id bits) are left out at first: budgets are
+    // nanosecond values, so after six passes over bits 16..63 equal values are rare and short runs of them are put
+    // in (key, slot) order by a local fix-up.  Only when a run is longer than kMaxRun or crosses a CTA boundary
+    // the queue is loaded again and ordered with all eight passes.
     int ep = 0;          // passes executed so far: selects the mbarrier pair and its phase
     bool dead = false;   // a bounded wait expired: stop exchanging, keep walking the barriers
-    for (int pass = 0; pass < 8; ++pass) {
+    int first_pass = a.top_first ? 2 : 0;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+    const int ep_before = ep;
+    for (int pass = first_pass; pass < 8; ++pass) {
         const int shift = pass * 8;
         if (((alld >> shift) & 0xffull) == 0) continue;  // same digit in every key: nothing moves
         if (dead) continue;
@@ -385,130 +536,302 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
 #pragma unroll
         for (int k = 0; k < K; ++k) e[k] = elems[(warp * K + k) * 32 + lane];
     }
-    if (dead && tid == 0) atomicOr(a.status, CASCADE_ST_ETIMEOUT);
-    }  // radix path
+    if (first_pass == 0 || dead) break;   // all eight passes ran (or nothing can be trusted any more)
 
-    // ---- admission: clamped prefix sums over the sorted elements ---------------------------------
-    long long ex[K];
-    long long run = 0, s1 = 0, s2 = 0;
-    int c1 = 0;
+    // ---- ordered by bits 16..63: look for equal neighbours ---------------------------------------------
+    if (ep == ep_before) {   // no pass ran: the elements are still only in registers, in slot order
+#pragma unroll
+        for (int k = 0; k < K; ++k) elems[(warp * K + k) * 32 + lane] = e[k];
+        __syncthreads();
+    }
+    const long long here_ll = (long long)a.n - (long long)crank * per;
+    const int n_here = here_ll < 0 ? 0 : (here_ll > per ? per : (int)here_ll);   // real elements of this CTA
+    bool tie = false, long_run = false;
 #pragma unroll
     for (int k = 0; k < K; ++k) {
-        const long long w = e[k].want;
-        const bool real = e[k].idx != 0xffffffffu;
-        const bool t2 = (e[k].key >> 63) != 0;
-        if (real && !t2) { s1 += w; ++c1; }
-        if (real && t2) s2 += w;
-        const long long x = seg_incl_scan(w, lane, 32);
-        ex[k] = run + x - w;
-        run += __shfl_sync(kFull, x, 31);
-    }
-#pragma unroll
-    for (int s = 16; s > 0; s >>= 1) {
-        s1 += __shfl_xor_sync(kFull, s1, s);
-        s2 += __shfl_xor_sync(kFull, s2, s);
-        c1 += __shfl_xor_sync(kFull, c1, s);
-    }
-    if (lane == 0) {
-        wtmp[warp] = run;
-        wtmp[32 + warp] = s1;
-        wtmp[64 + warp] = s2;
-        reinterpret_cast<int *>(base)[warp] = c1;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        const bool in = lane < W;
-        const long long t = in ? wtmp[lane] : 0;
-        const long long inc = seg_incl_scan(t, lane, 32);
-        long long a1 = in ? wtmp[32 + lane] : 0, a2 = in ? wtmp[64 + lane] : 0;
-        int ac = in ? reinterpret_cast<int *>(base)[lane] : 0;
-#pragma unroll
-        for (int s = 16; s > 0; s >>= 1) {
-            a1 += __shfl_xor_sync(kFull, a1, s);
-            a2 += __shfl_xor_sync(kFull, a2, s);
-            ac += __shfl_xor_sync(kFull, ac, s);
-        }
-        if (in) wtmp[lane] = inc - t;  // exclusive offset of each warp inside the CTA
-        if (lane < csize) {
-            Exch *x = cluster.map_shared_rank(exall, lane) + crank;
-            x->w1 = a1;
-            x->w2 = a2;
-            x->n1 = ac;
+        const int li = (warp * K + k) * 32 + lane;
+        if (li < n_here) {
+            const unsigned long long top = e[k].key >> 16;
+            if (li > 0 && (elems[li - 1].key >> 16) == top) tie = true;
+            if (li >= kMaxRun && (elems[li - kMaxRun].key >> 16) == top) long_run = true;
         }
     }
-    cluster.sync();
-    long long W1 = 0, W2 = 0, cta_off = 0;
-    int N1 = 0;
+    const bool cta_tie = __syncthreads_or(tie);
+    const bool cta_long = __syncthreads_or(long_run);
+    if (warp == 0 && lane < csize) {
+        TieExch x;
+        x.first = n_here > 0 ? elems[0].key >> 16 : 0ull;
+        x.last = n_here > 0 ? elems[n_here - 1].key >> 16 : 0ull;
+        x.count = n_here;
+        x.flags = (cta_tie ? 1 : 0) | (cta_long ? 2 : 0);
+        cluster.map_shared_rank(tie_ex, lane)[crank] = x;
+    }
+    cluster.sync();   // also: every CTA is done reading its elements before anybody starts another pass
+    bool redo = false;
 #pragma unroll
     for (int c = 0; c < kMaxCluster; ++c) {
         if (c < csize) {
-            const long long x1 = exall[c].w1, x2 = exall[c].w2;
-            W1 += x1;
-            W2 += x2;
-            N1 += exall[c].n1;
-            if (c < crank) cta_off += x1 + x2;
+            if (tie_ex[c].flags & 2) redo = true;
+            if (c + 1 < csize && tie_ex[c + 1].count > 0 && tie_ex[c].last == tie_ex[c + 1].first) redo = true;
         }
     }
-    const long long R2 = min(min(a.reserve, W2), a.TB);
-    const long long TB1 = a.TB - R2;
-    const long long TB2 = a.TB - min(TB1, W1);  // the reserve plus whatever Tier-1 left
-    const long long warp_off = cta_off + wtmp[warp];
-    int grant[K];
-    unsigned runc = 0;
-    unsigned exf[K];
+    if (!redo) {
+        if (cta_tie) {
+            // runs of equal values lie inside this CTA and are at most kMaxRun long: every element of a run counts the
+            // elements of its run that come before it by (key, slot) and moves there
+            unsigned newpos[K];
 #pragma unroll
-    for (int k = 0; k < K; ++k) {
-        const long long w = e[k].want;
-        const long long eg = warp_off + ex[k];
-        const bool t2 = (e[k].key >> 63) != 0;
-        long long g = t2 ? (TB2 - (eg - W1)) : (TB1 - eg);
-        g = g < 0 ? 0 : (g > w ? w : g);
-        grant[k] = (int)g;
-        const unsigned b = __ballot_sync(kFull, g > 0);
-        exf[k] = runc + __popc(b & lt_mask);
-        runc += __popc(b);
-    }
-    __syncthreads();  // wtmp is reused below
-    if (lane == 0) reinterpret_cast<unsigned *>(wtmp)[warp] = runc;
-    __syncthreads();
-    if (warp == 0) {
-        const unsigned t = lane < W ? reinterpret_cast<unsigned *>(wtmp)[lane] : 0u;
-        const unsigned inc = seg_incl_scan(t, lane, 32);
-        if (lane < W) reinterpret_cast<unsigned *>(wtmp)[lane] = inc - t;
-        const int tot = (int)__shfl_sync(kFull, inc, 31);
-        if (lane < csize) cluster.map_shared_rank(exall, lane)[crank].cnt = tot;
-    }
-    cluster.sync();
-    unsigned cnt_off = reinterpret_cast<unsigned *>(wtmp)[warp];
+            for (int k = 0; k < K; ++k) {
+                const int li = (warp * K + k) * 32 + lane;
+                newpos[k] = li;
+                if (li >= n_here) continue;
+                const unsigned long long top = e[k].key >> 16;
+                int lo = li, hi = li;
+                while (lo > 0 && (elems[lo - 1].key >> 16) == top) --lo;
+                while (hi + 1 < n_here && (elems[hi + 1].key >> 16) == top) ++hi;
+                int r = 0;
+                for (int j = lo; j <= hi; ++j) {
+                    const SortElem o = elems[j];
+                    r += (o.key < e[k].key) || (o.key == e[k].key && o.idx < e[k].idx);
+                }
+                newpos[k] = lo + r;
+            }
+            __syncthreads();
 #pragma unroll
-    for (int c = 0; c < kMaxCluster; ++c)
-        if (c < crank) cnt_off += (unsigned)exall[c].cnt;
+            for (int k = 0; k < K; ++k)
+                if ((warp * K + k) * 32 + lane < n_here) elems[newpos[k]] = e[k];
+            __syncthreads();
+#pragma unroll
+            for (int k = 0; k < K; ++k) e[k] = elems[(warp * K + k) * 32 + lane];
+        }
+        break;
+    }
+    // a long or CTA-crossing run: start again from the queue as it was loaded, this time with every pass
+    first_pass = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) load_elem(k);
+    }  // attempts
+    if (dead && tid == 0) atomicOr(a.status, CASCADE_ST_ETIMEOUT);
+    }  // radix path
 
-    long long tok = 0;
-    int adm = 0;
-#pragma unroll
-    for (int k = 0; k < K; ++k) {
-        if (grant[k] > 0 && (long long)(cnt_off + exf[k]) >= (long long)a.seq_cap) grant[k] = 0;
-        if (e[k].idx != 0xffffffffu) {
-            const long long g = (long long)crank * per_rt + (warp * K + k) * 32 + lane;
-            a.order_out[g] = e[k].idx;
-            a.grant_out[e[k].idx] = grant[k];
-            tok += grant[k];
-            adm += grant[k] > 0;
-        }
-    }
-#pragma unroll
-    for (int s = 16; s > 0; s >>= 1) {
-        tok += __shfl_xor_sync(kFull, tok, s);
-        adm += __shfl_xor_sync(kFull, adm, s);
-    }
-    if (lane == 0 && adm > 0) {
-        atomicAdd(reinterpret_cast<unsigned long long *>(&a.counts->tokens_granted), (unsigned long long)tok);
-        atomicAdd(&a.counts->n_admitted, adm);
-    }
-    if (crank == 0 && tid == 0) a.counts->n_tier1 = N1;
+    admit_and_write<T, K>(a, e, per_rt, cluster, wtmp, reinterpret_cast<int *>(base), exall);
     // every remote store of this kernel is followed by a cluster barrier and nothing reads remote
     // shared memory, so a CTA may leave as soon as it is done
+}
+
+// ---- merge-rank ordering: queues that fit one CTA's shared memory as bare keys (up to 16384) -------------
+// The radix passes above pay two cluster-wide exchanges per digit.  Here every CTA first orders ITS OWN
+// T*K elements with the same stable radix passes run entirely inside the CTA (no exchange), then the sorted
+// key lists of all CTAs are gathered into every CTA's shared memory (one exchange), each element finds its
+// global position as the sum, over the lists, of the number of keys below it (binary searches in shared memory;
+// lists of CTAs in front count equal keys too, which keeps the order stable by slot), and ONE more exchange
+// sends every element to its place.  Two exchanges in total instead of sixteen.
+constexpr int kMergeMaxKeys = 16384;
+
+template <int T, int K>
+__global__ void __launch_bounds__(T, 1) schedule_merge_kernel(const __grid_constant__ ScheduleArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
+    constexpr int W = T / 32;
+    constexpr int per = T * K;
+    static_assert((per & (per - 1)) == 0, "the searches assume lists of a power-of-two length");
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned crank = cluster.block_rank();
+    const unsigned csize = cluster.num_blocks();
+
+    extern __shared__ __align__(16) unsigned char smem[];
+    SortElem *elems = reinterpret_cast<SortElem *>(smem);                              // [per]
+    uint64_t *keys_all = reinterpret_cast<uint64_t *>(elems + per);                    // [csize][per], sorted lists
+    uint16_t *whist = reinterpret_cast<uint16_t *>(keys_all + kMergeMaxKeys);          // [W][kWhistStride]
+    uint32_t *lbase = reinterpret_cast<uint32_t *>(whist + W * kWhistStride);          // [kBins]
+    long long *wtmp = reinterpret_cast<long long *>(lbase + kBins);                    // 3 * 32 entries
+    Exch *exall = reinterpret_cast<Exch *>(wtmp + 3 * 32);                             // [kMaxCluster]
+    int *itmp = reinterpret_cast<int *>(exall + kMaxCluster);                          // [32]
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(itmp + 32);      // keys, elements
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const int n = a.n;
+    // elements of the final order that land in this CTA
+    const long long mine_ll = (long long)n - (long long)crank * per;
+    const int n_mine = mine_ll < 0 ? 0 : (mine_ll > per ? per : (int)mine_ll);
+
+    if (crank == 0 && tid == 0) {
+        a.counts->n_admitted = 0;
+        a.counts->tokens_granted = 0;
+    }
+    const unsigned keys_bar = cta_smem_addr(&bars[0]), elem_bar = cta_smem_addr(&bars[1]);
+    if (tid == 0) {
+        mbarrier_init(keys_bar, 1);
+        mbarrier_init(elem_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbarrier_arrive_expect(keys_bar, (csize - 1) * (unsigned)(per * sizeof(uint64_t)));
+        mbarrier_arrive_expect(elem_bar, (unsigned)(n_mine * sizeof(SortElem)));
+    }
+
+    // ---- load: key, slot, tokens wanted -------------------------------------------------------------
+    SortElem e[K];
+    unsigned long long diff = 0, key_first = 0;
+    {
+        const long long g0 = (long long)crank * per;
+        key_first = g0 < n ? a.key[g0] : 0ull;
+    }
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const int li = (warp * K + k) * 32 + lane;
+        const long long g = (long long)crank * per + li;
+        if (g < n) {
+            const unsigned long long key = a.key[g];
+            const long long P = a.prompt[g], h0 = a.n0[g], h1 = a.n1[g], h2 = a.n2[g];
+            long long want = 0;
+            if (dev_request_valid(a.bt, P, h0, h1, h2)) want = a.want_in ? a.want_in[g] : P - (h0 + h1 + h2) * a.bt;
+            e[k].key = key;
+            e[k].idx = (uint32_t)g;
+            e[k].want = (int32_t)want;
+            diff |= key ^ key_first;
+        } else {
+            e[k].key = ~0ull;  // padding sorts behind every real key of this CTA and stays there (stable passes)
+            e[k].idx = 0xffffffffu;
+            e[k].want = 0;
+        }
+    }
+    // bits in which this CTA's keys differ: passes over other digits would move nothing
+    {
+        unsigned lo = __reduce_or_sync(kFull, (unsigned)diff);
+        unsigned hi = __reduce_or_sync(kFull, (unsigned)(diff >> 32));
+        if (lane == 0) wtmp[warp] = (long long)(((unsigned long long)hi << 32) | lo);
+        __syncthreads();
+        unsigned long long v = 0;
+#pragma unroll
+        for (int w = 0; w < W; ++w) v |= (unsigned long long)wtmp[w];
+        diff = v;
+        __syncthreads();
+    }
+
+    // ---- local order: stable LSD radix passes inside the CTA ---------------------------------------------
+    for (int pass = 0; pass < 8; ++pass) {
+        const int shift = pass * 8;
+        if (((diff >> shift) & 0xffull) == 0) continue;
+        // (a) stable rank of each element among equal digits of its warp's 32*K elements
+        uint16_t *myhist = whist + warp * kWhistStride;
+        for (int i = lane; i < kWhistStride / 2; i += 32) reinterpret_cast<uint32_t *>(myhist)[i] = 0;
+        __syncwarp();
+        unsigned off[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
+            unsigned peers = kFull;
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                const unsigned bal = __ballot_sync(kFull, (d >> b) & 1u);
+                peers &= ((d >> b) & 1u) ? bal : ~bal;
+            }
+            const unsigned lower = peers & lt_mask;
+            const unsigned pre = myhist[d];
+            __syncwarp();
+            if (lower == 0) myhist[d] = (uint16_t)(pre + __popc(peers));
+            __syncwarp();
+            off[k] = pre + __popc(lower);
+        }
+        __syncthreads();
+        // (b) per digit: exclusive scan of the warps' counts in place, CTA total, then the scan over the digits
+        unsigned mine = 0, incl = 0;
+        if (tid < kBins) {
+            unsigned v[W];
+#pragma unroll
+            for (int w = 0; w < W; ++w) v[w] = whist[w * kWhistStride + tid];
+#pragma unroll
+            for (int w = 0; w < W; ++w) {
+                whist[w * kWhistStride + tid] = (uint16_t)mine;
+                mine += v[w];
+            }
+            incl = seg_incl_scan(mine, lane, 32);
+            if (lane == 31) reinterpret_cast<unsigned *>(wtmp)[warp] = incl;
+        }
+        __syncthreads();
+        if (tid < kBins) {
+            unsigned add = 0;
+#pragma unroll
+            for (int w = 0; w < kBins / 32; ++w) {
+                const unsigned t = reinterpret_cast<unsigned *>(wtmp)[w];
+                if (w < warp) add += t;
+            }
+            lbase[tid] = incl - mine + add;
+        }
+        __syncthreads();
+        // (c) every element to its place, then back into registers in position order
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const unsigned d = (unsigned)(e[k].key >> shift) & 0xffu;
+            const unsigned pos = lbase[d] + whist[warp * kWhistStride + d] + off[k];
+            *reinterpret_cast<uint4 *>(elems + pos) = *reinterpret_cast<const uint4 *>(&e[k]);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < K; ++k) e[k] = elems[(warp * K + k) * 32 + lane];
+    }
+
+    // ---- gather the sorted key lists of all CTAs -----------------------------------------------------------
+    uint64_t *my_list = keys_all + (size_t)crank * per;
+#pragma unroll
+    for (int k = 0; k < K; ++k) my_list[(warp * K + k) * 32 + lane] = e[k].key;
+    // first access to other CTAs' shared memory: they must all have started and initialised their barriers
+    cluster.sync();
+    for (unsigned op = tid; op < (csize - 1) * (per / 2); op += T) {
+        unsigned dst = op / (per / 2);
+        const unsigned piece = op % (per / 2);
+        dst += dst >= crank;   // everybody but myself
+        const uint4 v = *reinterpret_cast<const uint4 *>(my_list + piece * 2);
+        st_async_16(cluster_addr(cta_smem_addr(my_list + piece * 2), dst), v, cluster_addr(keys_bar, dst));
+    }
+    bool dead = !mbarrier_wait_bounded(keys_bar, 0, kWaitLimit);
+    if (__syncthreads_or(dead)) dead = true;
+
+    // ---- global position: keys below mine in every list --------------------------------------------------
+    if (!dead) {
+        unsigned pos[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) pos[k] = (warp * K + k) * 32 + lane;   // own list: the local position
+        for (unsigned c = 0; c < csize; ++c) {
+            if (c == crank) continue;
+            const uint64_t *list = keys_all + (size_t)c * per;
+            const bool ties = c < crank;   // equal keys of CTAs in front hold lower slots: they come first
+            unsigned p[K];
+#pragma unroll
+            for (int k = 0; k < K; ++k) p[k] = 0;
+#pragma unroll
+            for (int s = per / 2; s > 0; s >>= 1) {
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const uint64_t v = list[p[k] + s - 1];
+                    p[k] += (ties ? v <= e[k].key : v < e[k].key) ? s : 0;
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                const uint64_t v = list[p[k]];
+                p[k] += (ties ? v <= e[k].key : v < e[k].key) ? 1 : 0;
+                pos[k] += p[k];
+            }
+        }
+        // ---- every real element to its place (padding stays behind: nobody reads the slots past n) ----------
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            if (e[k].idx == 0xffffffffu) continue;
+            st_async_16(cluster_addr(cta_smem_addr(elems + (pos[k] % per)), pos[k] / per),
+                        *reinterpret_cast<const uint4 *>(&e[k]), cluster_addr(elem_bar, pos[k] / per));
+        }
+        dead = !mbarrier_wait_bounded(elem_bar, 0, kWaitLimit);
+    }
+    if (__syncthreads_or(dead)) dead = true;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const int li = (warp * K + k) * 32 + lane;
+        if (!dead && li < n_mine) e[k] = elems[li];
+        else { e[k].key = ~0ull; e[k].idx = 0xffffffffu; e[k].want = 0; }
+    }
+    if (dead && tid == 0) atomicOr(a.status, CASCADE_ST_ETIMEOUT);
+    admit_and_write<T, K>(a, e, per, cluster, wtmp, itmp, exall);
 }
 
 __global__ void zero_counts_kernel(cascade_sched_counts *c) {
@@ -520,7 +843,8 @@ __global__ void zero_counts_kernel(cascade_sched_counts *c) {
 size_t smem_bytes(int T, int K) {
     return (T == 256 && K == 1 ? kRankExtra : 0) + 2 * size_t(T) * K * sizeof(SortElem) + size_t(T / 32) * kWhistStride * sizeof(uint16_t) +
            2 * size_t(kMaxCluster) * kBins * sizeof(uint16_t) + 2 * kBins * sizeof(uint32_t) +
-           3 * 32 * sizeof(long long) + kMaxCluster * sizeof(Exch) + kBins * sizeof(uint16_t) + 4 * 8 + 16;
+           3 * 32 * sizeof(long long) + kMaxCluster * sizeof(Exch) + kBins * sizeof(uint16_t) + 4 * 8 +
+           kMaxCluster * sizeof(TieExch) + 16;
 }
 
 template <int T, int K>
@@ -538,6 +862,38 @@ cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, bool pdl
         configured = true;
     }
     return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), smem, stream, schedule_kernel<T, K>, a);
+}
+
+size_t merge_smem_bytes(int T, int K) {
+    return size_t(T) * K * sizeof(SortElem) + size_t(kMergeMaxKeys) * sizeof(uint64_t) +
+           size_t(T / 32) * kWhistStride * sizeof(uint16_t) + kBins * sizeof(uint32_t) + 3 * 32 * sizeof(long long) +
+           kMaxCluster * sizeof(Exch) + 32 * sizeof(int) + 2 * 8 + 16;
+}
+
+template <int K>
+cudaError_t launch_merge(const ScheduleArgs &a, int cluster_size, int device, bool pdl, cudaStream_t stream) {
+    static bool configured_dev[64] = {};
+    bool unknown = false;
+    bool &configured = (device >= 0 && device < 64) ? configured_dev[device] : unknown;
+    const size_t smem = merge_smem_bytes(256, K);
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(schedule_merge_kernel<256, K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(schedule_merge_kernel<256, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(256), smem, stream, schedule_merge_kernel<256, K>, a);
+}
+
+cudaError_t launch_merge_k(int K, const ScheduleArgs &a, int C, int device, bool pdl, cudaStream_t s) {
+    switch (K) {
+        case 1: return launch_merge<1>(a, C, device, pdl, s);
+        case 2: return launch_merge<2>(a, C, device, pdl, s);
+        case 4: return launch_merge<4>(a, C, device, pdl, s);
+        default: return launch_merge<8>(a, C, device, pdl, s);
+    }
 }
 
 template <int T>
@@ -607,6 +963,8 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
     a.bt = p.bt;
     a.stage = ctx->sort_stage >= 0 ? ctx->sort_stage : (K >= 4);
     a.async_sync = ctx->sort_async;
+    // the comparison policies order by small integers (tokens left, ...): equal values are the rule there
+    a.top_first = ctx->sort_top_first && p.policy == CASCADE_POLICY_BUDGET;
     a.rank_per = 0;
     if (n <= ctx->rank_sort_max && n <= kRankMaxKeys) {
         // counting path: the widest cluster the device schedules, 256 threads, 32..256 elements per CTA
@@ -622,7 +980,14 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
         }
     }
     a.status = ctx->status_dev;
-    cudaError_t e = T == 256 ? launch_k<256>(K, a, C, ctx->device, ctx->pdl, s) : launch_k<512>(K, a, C, ctx->device, ctx->pdl, s);
+    // queues beyond the counting path whose bare keys fit one CTA's shared memory: local order + merge by rank
+    // (measured: a gain while every thread holds one element, i.e. up to 4096 requests; beyond that the searches
+    // cost more than the exchanges they save, unless CASCADE_MERGE_SORT=2 forces it)
+    const bool merge = ctx->merge_sort && a.rank_per == 0 && T == 256 && (long long)C * T * K <= kMergeMaxKeys &&
+                       (K == 1 || ctx->merge_sort == 2);
+    cudaError_t e = merge      ? launch_merge_k(K, a, C, ctx->device, ctx->pdl, s)
+                    : T == 256 ? launch_k<256>(K, a, C, ctx->device, ctx->pdl, s)
+                               : launch_k<512>(K, a, C, ctx->device, ctx->pdl, s);
     CASCADE_CUDA_TRY(ctx, e);
     return CASCADE_OK;
 }

@@ -534,6 +534,43 @@ typedef struct cascade_dedup_args {
  */
 int cascade_dedup(cascade_ctx *ctx, const cascade_dedup_args *a, int n, void *stream);
 
+/*
+ * One iteration in one call: what a serving loop issues between two engine iterations (Algorithm 1 as a
+ * whole: re-budget every queued request, order, admit, plan, move).  Validates once and launches, in stream
+ * order on `stream`,
+ *     cascade_reqs_update   (if upd_m > 0)
+ *     cascade_budget -> cascade_schedule -> cascade_tier_plan
+ *     cascade_kv_move       (if layout != NULL; counts taken from plan->counts on the device)
+ * with exactly the arguments of those calls; results and errors are theirs.  Nothing here synchronises the
+ * host.  A caller that does not capture the iteration in a CUDA graph pays one crossing of its foreign-function
+ * interface instead of four or five.  All members are host values; pointers are device pointers as in the
+ * single calls.
+ */
+typedef struct cascade_step_args {
+    const cascade_reqs *reqs;      /* the queue */
+    int32_t n;                     /* queued requests */
+    int32_t D_act;                 /* decode sequences in flight */
+    int64_t K_act;                 /* their KV tokens */
+    int64_t now_ns;
+    const cascade_reqs *upd_src;   /* queue maintenance, see cascade_reqs_update; ignored when upd_m == 0 */
+    const int32_t *upd_slots;
+    int32_t upd_m;
+    int32_t upd_cap;
+    int64_t *budget;               /* outputs of cascade_budget */
+    uint64_t *key;
+    uint32_t *order;               /* outputs of cascade_schedule */
+    int32_t *grant;
+    cascade_sched_counts *sched_counts;
+    const cascade_pools *pools;    /* cascade_tier_plan */
+    const cascade_plan *plan;
+    const cascade_kv_layout *layout; /* NULL: no copies */
+    void *hbm_pool;
+    void *host_pool;
+    int64_t host_blocks;
+    int32_t *move_scratch;         /* cascade_kv_move_scratch_len(plan->evict_cap, plan->restore_cap) int32 */
+} cascade_step_args;
+int cascade_step(cascade_ctx *ctx, const cascade_step_args *args, void *stream);
+
 /* Waits for `stream`, copies the status word to *host_out and, if clear != 0, resets it. */
 int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream);
 

@@ -25,7 +25,7 @@ EXPORTS = ("cascade_create", "cascade_destroy", "cascade_set_params", "cascade_b
            "cascade_tier_plan", "cascade_kv_restore", "cascade_kv_evict", "cascade_status", "cascade_version",
            "cascade_tier_plan_noalloc", "cascade_latency_regimes", "cascade_prefetch_plan", "cascade_kv_move",
            "cascade_stage_plan", "cascade_kv_stage", "cascade_dedup", "cascade_reqs_update",
-           "cascade_kv_move_scratch_len", "cascade_kv_mailbox_len", "cascade_kv_move_staged")
+           "cascade_kv_move_scratch_len", "cascade_kv_mailbox_len", "cascade_kv_move_staged", "cascade_step")
 
 
 class Params(C.Structure):
@@ -110,6 +110,15 @@ def make_dedup_args(**kw) -> DedupArgs:
     return a
 
 
+class StepArgs(C.Structure):
+    _fields_ = [("reqs", C.POINTER(Reqs)), ("n", C.c_int32), ("D_act", C.c_int32), ("K_act", C.c_int64),
+                ("now_ns", C.c_int64), ("upd_src", C.POINTER(Reqs)), ("upd_slots", C.c_void_p), ("upd_m", C.c_int32),
+                ("upd_cap", C.c_int32), ("budget", C.c_void_p), ("key", C.c_void_p), ("order", C.c_void_p),
+                ("grant", C.c_void_p), ("sched_counts", C.c_void_p), ("pools", C.POINTER(Pools)),
+                ("plan", C.POINTER(Plan)), ("layout", C.c_void_p), ("hbm_pool", C.c_void_p),
+                ("host_pool", C.c_void_p), ("host_blocks", C.c_int64), ("move_scratch", C.c_void_p)]
+
+
 class KvLayout(C.Structure):
     _fields_ = [("n_blocks", C.c_int64), ("n_chunks", C.c_int32), ("reserved", C.c_int32),
                 ("chunk_bytes", C.c_int64), ("chunk_stride", C.c_int64), ("block_stride", C.c_int64)]
@@ -145,6 +154,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.cascade_kv_mailbox_len.argtypes = [C.c_int, C.c_int]
     lib.cascade_kv_move_staged.argtypes = [vp, C.POINTER(KvLayout), vp, vp, i64, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int,
                                            vp, i64, vp, vp]
+    lib.cascade_step.argtypes = [vp, C.POINTER(StepArgs), vp]
     lib.cascade_reqs_update.argtypes = [vp, C.POINTER(Reqs), C.c_int, C.POINTER(Reqs), vp, C.c_int, vp]
     lib.cascade_stage_plan.argtypes = [vp, C.POINTER(Reqs), vp, vp, vp, C.c_int, i32, i64, i64, i32, C.POINTER(Pools),
                                        C.POINTER(Stage), vp]
@@ -306,6 +316,9 @@ class Context:
                                            _p(restore_src), _p(restore_dst), _p(n_restore_dev), n_restore_max,
                                            _p(staging), staging_blocks, _p(mailbox), _stream(stream)),
                "cascade_kv_move_staged")
+
+    def step(self, args: StepArgs, stream=None):
+        _check(_lib.cascade_step(self._h, C.byref(args), _stream(stream)), "cascade_step")
 
     def stage_plan(self, reqs: Reqs, budget, order, action, n, D_act, K_act, link_budget_ns, host_reserve,
                    pools: Pools, stage: Stage, stream=None):

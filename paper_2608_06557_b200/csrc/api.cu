@@ -150,6 +150,31 @@ extern "C" int cascade_set_params(cascade_ctx *ctx, const cascade_params *p) {
     return CASCADE_OK;
 }
 
+extern "C" int cascade_step(cascade_ctx *ctx, const cascade_step_args *a, void *stream) {
+    CascadeRange nvtx_range("cascade_step");
+    if (!ctx || !a || !a->reqs || !a->pools || !a->plan) return CASCADE_EINVAL;
+    int rc = CASCADE_OK;
+    if (a->upd_m > 0) {
+        rc = cascade_reqs_update(ctx, a->reqs, a->upd_cap, a->upd_src, a->upd_slots, a->upd_m, stream);
+        if (rc != CASCADE_OK) return rc;
+    }
+    rc = cascade_budget(ctx, a->reqs, a->n, a->now_ns, a->D_act, a->K_act, a->budget, a->key, stream);
+    if (rc != CASCADE_OK) return rc;
+    rc = cascade_schedule(ctx, a->reqs, a->key, a->n, a->D_act, a->order, a->grant, a->sched_counts, stream);
+    if (rc != CASCADE_OK) return rc;
+    rc = cascade_tier_plan(ctx, a->reqs, a->budget, a->order, a->grant, a->n, a->D_act, a->K_act, a->pools, a->plan,
+                           stream);
+    if (rc != CASCADE_OK) return rc;
+    if (a->layout) {
+        const cascade_plan *pl = a->plan;
+        if (!pl->counts) return CASCADE_EINVAL;
+        rc = cascade_kv_move(ctx, a->layout, a->hbm_pool, a->host_pool, a->host_blocks, pl->evict_src, pl->evict_dst,
+                             &pl->counts->n_evict, pl->evict_cap, pl->restore_src, pl->restore_dst,
+                             &pl->counts->n_restore, pl->restore_cap, a->move_scratch, stream);
+    }
+    return rc;
+}
+
 extern "C" int cascade_status(cascade_ctx *ctx, cascade_status_t *host_out, int clear, void *stream) {
     if (!ctx || !host_out) return CASCADE_EINVAL;
     if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;

@@ -142,6 +142,36 @@ class Instance:
         c.tier_plan(self.reqs_struct, self.budget, self.order, self.grant, self.n, self.D_act, self.K_act,
                     self.pools_struct, self.plan_struct, stream)
 
+    def step_args(self, with_update: bool = False, with_move: bool = False) -> cs.StepArgs:
+        """The arguments of one whole iteration for cascade_step; the structure points at this instance's buffers
+        and is kept alive by it (only clock, load and the update count change from iteration to iteration)."""
+        import ctypes as C
+        a = cs.StepArgs()
+        a.reqs = C.pointer(self.reqs_struct)
+        a.n, a.D_act, a.K_act, a.now_ns = self.n, self.D_act, self.K_act, self.now_ns
+        if with_update:
+            a.upd_src = C.pointer(self.upd_struct)
+            a.upd_slots, a.upd_m, a.upd_cap = cs._p(self.upd_slots), self.upd_m, self.cap
+        a.budget, a.key, a.order, a.grant = (cs._p(t) for t in (self.budget, self.key, self.order, self.grant))
+        a.sched_counts = cs._p(self.sched_counts)
+        a.pools, a.plan = C.pointer(self.pools_struct), C.pointer(self.plan_struct)
+        if with_move:
+            if not hasattr(self, "move_scratch"):
+                self.move_scratch = torch.empty(cs.kv_move_scratch_len(self.evict_cap, self.restore_cap),
+                                                dtype=torch.int32, device=self.device)
+            self._layout_keep = self.layout
+            a.layout = C.addressof(self.layout)
+            a.hbm_pool, a.host_pool, a.host_blocks = cs._p(self.hbm_pool), cs._p(self.host_pool), self.host_blocks
+            a.move_scratch = cs._p(self.move_scratch)
+        return a
+
+    def run_step(self, args: cs.StepArgs, stream=None):
+        """One cascade_step call with the current clock and load."""
+        args.n, args.D_act, args.K_act, args.now_ns = self.n, self.D_act, self.K_act, self.now_ns
+        if args.upd_slots:
+            args.upd_m = self.upd_m
+        self.ctx.step(args, stream)
+
     def run_prefetch(self, link_budget_ns: int, hbm_reserve: int = 0, stream=None):
         """Budget-bounded prefetch for the requests that stay queued (after run_schedule, before run_copies)."""
         if not hasattr(self, "pf"):

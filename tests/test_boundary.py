@@ -62,7 +62,8 @@ def test_header_is_plain_c_and_the_binding_mirrors_its_struct_layouts(tmp_path):
              ("cascade_plan_counts", cs.PlanCounts), ("cascade_pools", cs.Pools), ("cascade_plan", cs.Plan),
              ("cascade_kv_layout", cs.KvLayout), ("cascade_status_t", cs.Status),
              ("cascade_stage_counts", cs.StageCounts), ("cascade_stage", cs.Stage),
-             ("cascade_dedup_counts", cs.DedupCounts), ("cascade_dedup_args", cs.DedupArgs)]
+             ("cascade_dedup_counts", cs.DedupCounts), ("cascade_dedup_args", cs.DedupArgs),
+             ("cascade_step_args", cs.StepArgs)]
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "cascade.h"', 'int main(void) {']
     for cname, ct in pairs:
         lines.append(f'  printf("{cname} %zu", sizeof({cname}));')

@@ -297,3 +297,46 @@ def test_plan_first_admission(seed):
     w.params = dict(w.params, plan_first=1, token_budget=200_000, max_batch=2048)
     got, ref = compare_iteration(w, f"plan-first-7000-{seed}")
     assert got["sched_counts"]["n_admitted"] > 50
+
+
+@pytest.mark.parametrize("seed", [0, 3])
+def test_one_call_iteration_equals_the_single_calls(seed):
+    """cascade_step issues slot update, budget, schedule, tier plan and the fused move from C: same outputs as
+    the oracle, same bytes moved."""
+    torch, cs, Instance = _gpu()
+    w = wl.config_tiny(seed, hbm_free_target=60)
+    w.params["ttft_ns"] = [20 * t for t in w.params["ttft_ns"]]
+    ref = oracle_iteration(w)
+    plan = ref["plan"]
+    bb = w.block_bytes
+    hbm_np = wl.pool_bytes(3, w.layout["n_blocks"] * bb).copy()
+    host_np = wl.pool_bytes(4, w.host_blocks * bb).copy()
+    inst = Instance(w)
+    inst.hbm_pool.copy_(torch.from_numpy(hbm_np))
+    inst.host_pool.copy_(torch.from_numpy(host_np))
+    # start from a queue whose first slots are wrong, and let the step's own slot update repair them
+    slots = np.arange(0, w.n, 3, dtype=np.int64)
+    for k in ("prompt", "n0", "n1"):
+        inst.reqs[k][: w.n][torch.from_numpy(slots).cuda()] = 1
+    inst.stage_slot_update(w.reqs, slots)
+    args = inst.step_args(with_update=True, with_move=True)
+    inst.run_step(args)
+    got = inst.fetch()
+    assert oracle.kv_evict(hbm_np, w.layout, host_np, w.host_blocks, plan["evict_src"], plan["evict_dst"]) == 0
+    assert oracle.kv_restore(hbm_np, w.layout, host_np, w.host_blocks, plan["restore_src"], plan["restore_dst"]) == 0
+    for k in ("budget", "key", "order", "grant"):
+        assert np.array_equal(got[k], ref[k]), k
+    for k in ("x1", "x2", "tokens_run", "action", "restore_src", "restore_dst", "evict_src", "evict_dst"):
+        assert np.array_equal(got[k], plan[k]), k
+    assert got["plan_counts"] == plan["counts"] and got["status"] == ref["status"]
+    assert np.array_equal(inst.hbm_pool.cpu().numpy(), hbm_np) and np.array_equal(inst.host_pool.cpu().numpy(), host_np)
+    assert plan["counts"]["n_restore"] > 0 and plan["counts"]["n_evict"] > 0
+    # plan-only queue, no update, no copies
+    sw = wl.SchedulerSweep(5000, seed=seed)
+    w2 = sw.workload()
+    inst2 = Instance(w2, alloc_pools=False)
+    inst2.run_step(inst2.step_args())
+    got2, ref2 = inst2.fetch(), oracle_iteration(w2, with_tables=False)
+    for k in ("budget", "key", "order", "grant"):
+        assert np.array_equal(got2[k], ref2[k]), k
+    assert got2["plan_counts"] == ref2["plan"]["counts"]

@@ -367,9 +367,24 @@ class Instance:
         return out
 
 
-def alloc_pinned_pool(nbytes: int, floor: int = 1 << 28):
-    """Pinned, device-mapped host pool of ``nbytes``; the request is halved until the allocation
-    succeeds.  Returns (uint8 tensor, bytes obtained)."""
+def host_memory_available() -> int | None:
+    """MemAvailable of the box in bytes (None where /proc/meminfo cannot be read)."""
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return None
+
+
+def alloc_pinned_pool(nbytes: int, floor: int = 1 << 28, share_of_available: float = 0.7):
+    """Pinned, device-mapped host pool of ``nbytes``.  The request is first cut to ``share_of_available`` of
+    the box's available memory (page-locking more than the box can spare takes the box down instead of
+    failing), then halved until the allocation succeeds.  Returns (uint8 tensor, bytes obtained)."""
+    avail = host_memory_available()
+    if avail is not None and nbytes > avail * share_of_available:
+        nbytes = int(avail * share_of_available) // (1 << 21) * (1 << 21)
     while nbytes >= floor:
         try:
             return torch.empty(nbytes, dtype=torch.uint8, pin_memory=True), nbytes

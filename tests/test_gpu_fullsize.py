@@ -28,6 +28,7 @@ def pools():
     yield dict(hbm=hbm_pool, host=host_pool, hbm_bytes=hbm_pool.numel(), host_bytes=(host_bytes // BB) * BB)
     del hbm_pool, host_pool
     torch.cuda.empty_cache()
+    torch._C._host_emptyCache()
 
 
 def hbm_block(torch, pool, lay, ids):

@@ -49,14 +49,24 @@ def verify_by_content(torch, hbm, host, lay, n_host, hbm_content, host_content):
         assert torch.equal(got, oc[base:base + len(got), None] * P1 + j[None, :] * P2), base
 
 
-@pytest.mark.parametrize("variant", ["pressure", "restore_heavy", "pressure_fused_move"])
+@pytest.mark.parametrize("variant", ["pressure", "restore_heavy", "pressure_fused_move", "stated_size"])
 def test_replay_iterations_match_oracle_and_bytes_end_up_where_they_should(variant):
     import torch
     from paper_2608_06557_b200 import cascade as cs
-    from paper_2608_06557_b200.runner import Instance
+    from paper_2608_06557_b200.runner import Instance, alloc_pinned_pool
 
     fused = variant.endswith("fused_move")
-    if variant.startswith("pressure"):
+    cap = 1024
+    if variant == "stated_size":
+        # the configuration as stated: 4096 requests arriving at 20 per second over about 200 s, 200 iterations,
+        # pools of 60 and 40 * 10^9 bytes (less only if the box cannot hold them; the sizes used are checked below)
+        free, _ = torch.cuda.mem_get_info()
+        hbm_bytes = 60 * 10**9 if free > 75 * 10**9 else int(free * 0.6)
+        host_pool_t, host_bytes = alloc_pinned_pool(40 * 10**9)
+        tr = wl.config_llama70b_trace(2, n=4096, rate_per_s=20.0, hbm_bytes=hbm_bytes, host_bytes=host_bytes)
+        iters, cap, fused = 200, 4096, True
+        assert tr.layout["n_blocks"] >= 6000 and tr.host_blocks >= 3000, (hbm_bytes, host_bytes)
+    elif variant.startswith("pressure"):
         tr = wl.config_llama70b_trace(1, n=1024, hbm_bytes=12 * 10**9, host_bytes=8 * 10**9, hbm_occupancy=0.7,
                                       rate_per_s=60.0)
         iters = 200
@@ -67,13 +77,14 @@ def test_replay_iterations_match_oracle_and_bytes_end_up_where_they_should(varia
     bb = lay["n_chunks"] * lay["chunk_bytes"]
     assert bb == 5 * 1024 * 1024
     hbm = torch.empty(lay["n_blocks"] * bb, dtype=torch.uint8, device="cuda")
-    host = torch.empty(tr.host_blocks * bb, dtype=torch.uint8, pin_memory=True)
+    host = host_pool_t[: tr.host_blocks * bb] if variant == "stated_size" else \
+        torch.empty(tr.host_blocks * bb, dtype=torch.uint8, pin_memory=True)
     fill_by_content(torch, hbm, host, lay, tr.host_blocks)
     hbm_content = np.arange(lay["n_blocks"], dtype=np.int64)
     host_content = np.arange(tr.host_blocks, dtype=np.int64) + HOST_TAG
 
     rp = Replay(tr)
-    ctx = cs.Context(tr.params, 1024, 0)
+    ctx = cs.Context(tr.params, cap, 0)
     tot = dict(n_restore=0, n_evict=0, n_drop_blocks=0, n_unadmitted=0)
     for it in range(iters):
         w, ids = rp.workload()
@@ -108,3 +119,8 @@ def test_replay_iterations_match_oracle_and_bytes_end_up_where_they_should(varia
     if variant.startswith("pressure"):
         assert tot["n_evict"] > 0 and tot["n_drop_blocks"] > 0 and tot["n_unadmitted"] > 0
     verify_by_content(torch, hbm, host, lay, tr.host_blocks, hbm_content, host_content)
+    if variant == "stated_size":
+        assert it >= 150, it           # the trace really ran (almost) its 200 iterations
+        del hbm, host, host_pool_t
+        torch.cuda.empty_cache()
+        torch._C._host_emptyCache()

@@ -161,10 +161,10 @@ def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
     check(keys_with_runs([(0, 2), (n - 2, 2)]), "first and last")
 
 
-@pytest.mark.parametrize("n,iters", [(1024, 1000), (4096, 100), (16384, 40), (65536, 8)])
+@pytest.mark.parametrize("n,iters", [(1024, 1000), (4096, 1000), (16384, 1000), (65536, 1000)])
 def test_scheduler_sweep_iterations_with_churn(n, iters):
-    """Consecutive iterations of the scheduler-scale sweep (plan-only): the clock advances 25 ms and 5 % of
-    the slots and of the decode contexts are replaced every iteration."""
+    """The scheduler-scale sweep at its stated length: 1000 consecutive iterations (plan-only) for each queue
+    size; the clock advances 25 ms and 5 % of the slots and of the decode contexts are replaced every iteration."""
     torch, cs, Instance = _gpu()
     sw = wl.SchedulerSweep(n, seed=1)
     inst = Instance(sw.workload(), alloc_pools=False)

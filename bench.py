@@ -8,8 +8,11 @@ seeded batch (request arrays, block tables, free lists) that is already resident
 timed region starts; the KV bytes a step moves cross the host link inside the copy kernels.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --case copy-hbm|copy-host|move|staged|schedule|deep [--case-n N]
 
-Prints one JSON line.  With --gpus N > 1 (launched by torchrun) every rank runs an independent
+Prints one JSON line.  `--case` runs one small, self-contained invocation of a single kernel family instead
+(a few launches, a few GB on the device at most, more than the 126 MB L2 per launch where bandwidth is
+measured): the commands behind the ncu summaries under profiles/.  With --gpus N > 1 (launched by torchrun) every rank runs an independent
 replica on its own GPU: the path has no exchange step, so there is no collective on the data path.
 """
 from __future__ import annotations
@@ -51,6 +54,11 @@ def parse_args():
     ap.add_argument("--separate-copies", action="store_true",
                     help="run cascade_kv_evict then cascade_kv_restore instead of the fused cascade_kv_move")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time bound of the oracle baseline leg")
+    ap.add_argument("--host-sweep-gb", type=float, default=100.0,
+                    help="pinned host pool asked for (10^9 bytes): the copy sweep uses all of it, the step its first --host-gb")
+    ap.add_argument("--case", default=None, choices=["copy-hbm", "copy-host", "move", "staged", "schedule", "deep"],
+                    help="run one small profiling case instead of the benchmark")
+    ap.add_argument("--case-n", type=int, default=None, help="blocks / requests of the --case")
     return ap.parse_args()
 
 
@@ -118,10 +126,25 @@ def oracle_step(w, scratch):
     return t_sched + t_copy, moved
 
 
-def run_oracle_arm(args, seconds, first_seed=0, max_steps=None, warmup=1):
+def host_description(core):
+    """What the oracle ran on: logical cores of the box, CPU model, the core the process was pinned to."""
+    model = "unknown"
     try:
-        os.sched_setaffinity(0, {sorted(os.sched_getaffinity(0))[0]})
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                model = line.split(":", 1)[1].strip()
+                break
     except OSError:
+        pass
+    return dict(nproc=os.cpu_count(), cpu_model=model, pinned_to_core=core)
+
+
+def run_oracle_arm(args, seconds, first_seed=0, max_steps=None, warmup=1):
+    core = None
+    try:
+        core = sorted(os.sched_getaffinity(0))[0]
+        os.sched_setaffinity(0, {core})
+    except (OSError, AttributeError):
         pass
     w = make_batch(args, first_seed)
     scratch = OracleScratch(w)
@@ -142,7 +165,7 @@ def run_oracle_arm(args, seconds, first_seed=0, max_steps=None, warmup=1):
                 sample=f"{steps} step(s) of the same workload (seeds {first_seed}..{first_seed + steps - 1}): "
                        "budget+schedule+plan on the full queue, evict/restore as memcpy on host mirrors "
                        "compacted to the blocks each step touches",
-                ms_per_step=total_t / steps * 1e3, steps=steps)
+                ms_per_step=total_t / steps * 1e3, steps=steps, host=host_description(core))
 
 
 def oracle_schedule_latency():
@@ -181,8 +204,9 @@ def reference_main(args):
     line = dict(impl="reference", metric=METRIC, value=res["value"], unit="GB/s", n_gpus=args.gpus,
                 steps=res["steps"], warmup=args.warmup, ms_per_step=res["ms_per_step"], higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="u8", data="synthetic",
-                config=workload_config(args, None),
-                cpu_baseline=dict(value=res["value"], unit="GB/s", cores=1, kind="oracle", sample=res["sample"]),
+                config=workload_config(args),
+                cpu_baseline=dict(value=res["value"], unit="GB/s", cores=1, kind="oracle", sample=res["sample"],
+                                  host=res["host"]),
                 e2e=dict(value=res["value"], unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
 
@@ -190,15 +214,13 @@ def reference_main(args):
 # --------------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------------
-def workload_config(args, extra):
-    cfg = dict(workload="llama3-8b-shaped KV step: %d requests, 3 SLO classes, 2 MiB blocks (64 x 32 KiB), "
-                        "HBM pool %.0f GB, pinned host pool %.0f GB, token budget 8192, one fresh seeded batch per step"
-                        % (args.requests, args.hbm_gb, args.host_gb),
-               l2="every step moves far more than the 126 MB L2 across the host link; inputs larger than L2",
-               replicas=args.gpus)
-    if extra:
-        cfg.update(extra)
-    return cfg
+def workload_config(args):
+    """The workload and nothing else (both arms print the same dictionary; what a run measured goes to "run")."""
+    return dict(workload="llama3-8b-shaped KV step: %d requests, 3 SLO classes, 2 MiB blocks (64 x 32 KiB), "
+                         "HBM pool %.0f GB, pinned host pool %.0f GB, token budget 8192, one fresh seeded batch per step"
+                         % (args.requests, args.hbm_gb, args.host_gb),
+                l2="every step moves far more than the 126 MB L2 across the host link; inputs larger than L2",
+                replicas=args.gpus)
 
 
 def rank_seed(rank: int, step: int) -> int:
@@ -287,10 +309,52 @@ def measure_link_peaks(torch, host_pool, hbm_pool):
     return out
 
 
-def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, stage):
-    """Evict / restore bandwidth for 1, 16, 256 and 4096 scattered blocks per call, through the pinned
-    host pool (host link) and through a device staging buffer (HBM): 3 warm-ups, then 20 timed calls (10 for
-    4096 blocks over the host link); best and median."""
+def timed_calls(torch, fn, reps, warm=3):
+    """CUDA-event time of single calls launched from Python (the host's launch work is inside): best, median in ms."""
+    ts = []
+    for it in range(warm + reps):
+        a, b = event_pair(torch)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        if it >= warm:
+            ts.append(a.elapsed_time(b))
+    return min(ts), statistics.median(ts)
+
+
+def graph_per_call_us(torch, fn_i, flush, reps=20):
+    """Device time per call with the host out of the way: `reps` calls (call i works on its own blocks) captured in
+    one CUDA graph; a buffer larger than L2 is rewritten before every replay.  Median microseconds per call."""
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        for i in range(reps):
+            fn_i(i, st)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        for i in range(reps):
+            fn_i(i, st)
+    ts = []
+    for it in range(8):
+        flush.fill_(it)
+        torch.cuda.synchronize()
+        a, b = event_pair(torch)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            ts.append(a.elapsed_time(b) / reps * 1e3)
+    return statistics.median(ts)
+
+
+def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, stage, peaks):
+    """Evict / restore bandwidth for 1, 16, 256 and 4096 scattered blocks per call, through the pinned host pool
+    (host link) and through a device staging buffer (HBM).  Every figure is given twice where the call is short:
+    launched from Python and bracketed by events (3 warm-ups, 20 calls; 10 for 4096 blocks over the link), and
+    as device time per call inside a CUDA graph of 20 calls on distinct blocks, next to cudaMemcpyAsync copies of
+    the same size measured the same way."""
     from paper_2608_06557_b200 import workload as wl
     bb = lay["n_chunks"] * lay["chunk_bytes"]
     out, median = {}, {}
@@ -300,57 +364,116 @@ def copy_sweep(torch, cs, ctx, layout, lay, hbm_pool, host_pool, host_blocks, st
             m = min(n, nrec, lay["n_blocks"])
             src, dst = wl.copy_lists(100 + n, m, nrec, lay["n_blocks"])
             s, d = torch.from_numpy(src).cuda(), torch.from_numpy(dst).cuda()
-            for kind in ("evict", "restore"):
-                ts = []
-                for it in range(3 + (20 if n <= 256 or isdev else 10)):
-                    a, b = event_pair(torch)
-                    a.record()
-                    if kind == "evict":
-                        ctx.kv_evict(layout, hbm_pool, rec, nrec, isdev, d, s, None, m)
-                    else:
-                        ctx.kv_restore(layout, hbm_pool, rec, nrec, isdev, s, d, None, m)
-                    b.record()
-                    torch.cuda.synchronize()
-                    if it >= 3:
-                        ts.append(a.elapsed_time(b))
-                scale = (2 if isdev else 1) * m * bb / 1e6
-                out[f"{kind}_{name}_{n}"] = round(scale / min(ts), 1)
-                median[f"{kind}_{name}_{n}"] = round(scale / statistics.median(ts), 1)
-    # both directions at once: n blocks evicted and n restored by one cascade_kv_move, half of the restores
-    # into blocks the same call evicts
-    for n in (16, 256, 2048):
-        m = min(n, host_blocks // 2, lay["n_blocks"] // 2)
+            reps = 20 if n <= 256 or isdev else 10
+            scale = (2 if isdev else 1) * m * bb / 1e6
+            best, med = timed_calls(torch, lambda: ctx.kv_evict(layout, hbm_pool, rec, nrec, isdev, d, s, None, m), reps)
+            out[f"evict_{name}_{n}"], median[f"evict_{name}_{n}"] = round(scale / best, 1), round(scale / med, 1)
+            best, med = timed_calls(torch, lambda: ctx.kv_restore(layout, hbm_pool, rec, nrec, isdev, s, d, None, m), reps)
+            out[f"restore_{name}_{n}"], median[f"restore_{name}_{n}"] = round(scale / best, 1), round(scale / med, 1)
+
+    # short calls without the host's launch work, and copy-engine copies of the same size measured the same way
+    small = {}
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    REPS = 20
+    for n in (1, 16):
         rng = np.random.default_rng(n)
-        hp, op = rng.permutation(lay["n_blocks"]).astype(np.int32), rng.permutation(host_blocks).astype(np.int32)
-        es, ed, rs = hp[:m], op[:m], op[m:2 * m]
-        rd = np.concatenate([es[::-1][: m // 2], hp[m:2 * m - m // 2]]).astype(np.int32)
-        t = [torch.from_numpy(np.ascontiguousarray(x)).cuda() for x in (es, ed, rs, rd)]
-        scratch = torch.empty(cs.kv_move_scratch_len(m, m), dtype=torch.int32, device="cuda")
-        best = 1e30
-        for it in range(6):
-            a, b = event_pair(torch)
-            a.record()
-            ctx.kv_move(layout, hbm_pool, host_pool, host_blocks, t[0], t[1], None, m, t[2], t[3], None, m, scratch)
-            b.record()
-            torch.cuda.synchronize()
-            if it >= 2:
-                best = min(best, a.elapsed_time(b))
-        out[f"move_host_{n}+{n}"] = round(2 * m * bb / best / 1e6, 1)
+        hp = rng.permutation(lay["n_blocks"])[: REPS * n].astype(np.int32).reshape(REPS, n)
+        op = rng.permutation(min(host_blocks, stage_blocks))[: REPS * n].astype(np.int32).reshape(REPS, n)
+        H = [torch.from_numpy(hp[i]).cuda() for i in range(REPS)]
+        O = [torch.from_numpy(op[i]).cuda() for i in range(REPS)]
+        nbytes = n * bb
+        for name, rec, nrec, isdev, mult in (("host", host_pool, host_blocks, False, 1), ("hbm", stage, stage_blocks, True, 2)):
+            t = graph_per_call_us(torch, lambda i, st: ctx.kv_restore(layout, hbm_pool, rec, nrec, isdev, O[i], H[i], None, n, st), flush)
+            small[f"restore_{name}_{n}"] = dict(us=round(t, 1), GBps=round(mult * nbytes / t / 1e3, 1))
+            t = graph_per_call_us(torch, lambda i, st: ctx.kv_evict(layout, hbm_pool, rec, nrec, isdev, H[i], O[i], None, n, st), flush)
+            small[f"evict_{name}_{n}"] = dict(us=round(t, 1), GBps=round(mult * nbytes / t / 1e3, 1))
+        for name, dst, src, mult in (("h2d", hbm_pool, host_pool, 1), ("d2h", host_pool, hbm_pool, 1), ("d2d", stage, hbm_pool, 2)):
+            t = graph_per_call_us(torch, lambda i, st: dst[i * nbytes:(i + 1) * nbytes].copy_(src[i * nbytes:(i + 1) * nbytes], non_blocking=True), flush)
+            small[f"cudaMemcpyAsync_{name}_{n}x2MiB"] = dict(us=round(t, 1), GBps=round(mult * nbytes / t / 1e3, 1))
+        small[f"restore_host_{n}_fraction_of_same_size_copy"] = round(
+            small[f"restore_host_{n}"]["GBps"] / small[f"cudaMemcpyAsync_h2d_{n}x2MiB"]["GBps"], 3)
+        small[f"evict_host_{n}_fraction_of_same_size_copy"] = round(
+            small[f"evict_host_{n}"]["GBps"] / small[f"cudaMemcpyAsync_d2h_{n}x2MiB"]["GBps"], 3)
+        small[f"restore_host_{n}_fraction_of_1GiB_peak"] = round(small[f"restore_host_{n}"]["GBps"] / peaks["h2d"], 3)
+        small[f"evict_host_{n}_fraction_of_1GiB_peak"] = round(small[f"evict_host_{n}"]["GBps"] / peaks["d2h"], 3)
+    del flush
+    out["graph_timed_small_calls"] = small
+
+    # other block sizes: the tiny configuration's 16 KiB blocks (4 chunks of 4 KiB) and the 70B-shaped 5 MiB blocks
+    # (160 chunks of 32 KiB), 256 blocks per call, over the link and through the staging buffer
+    other = {}
+    for tag, n_chunks, cb in (("16KiB", 4, 4096), ("5MiB", 160, 32768)):
+        bb2 = n_chunks * cb
+        nb = min(4096, hbm_pool.numel() // bb2 // 2)
+        lay2 = wl.kv_layout(nb, n_chunks, cb)
+        layout2 = cs.make_layout(lay2)
+        m = 256
+        for name, rec, isdev in (("host", host_pool, False), ("hbm", stage, True)):
+            nrec = min(rec.numel() // bb2, 4096)
+            src, dst = wl.copy_lists(300, m, nrec, nb)
+            s_, d_ = torch.from_numpy(src).cuda(), torch.from_numpy(dst).cuda()
+            scale = (2 if isdev else 1) * m * bb2 / 1e6
+            best, med = timed_calls(torch, lambda: ctx.kv_evict(layout2, hbm_pool, rec, nrec, isdev, d_, s_, None, m), 10)
+            other[f"evict_{name}_{tag}_256"] = round(scale / med, 1)
+            best, med = timed_calls(torch, lambda: ctx.kv_restore(layout2, hbm_pool, rec, nrec, isdev, s_, d_, None, m), 10)
+            other[f"restore_{name}_{tag}_256"] = round(scale / med, 1)
+    out["other_block_sizes_median_GBps"] = other
+
+    # both directions at once: n blocks evicted and n restored in one call, half of the restores into blocks the
+    # same call evicts; the zero-copy kernels (cascade_kv_move) next to the copy engines (cascade_kv_move_staged)
+    duplex = {}
+    for tag, n_chunks, cb, pairs in (("2MiB", lay["n_chunks"], lay["chunk_bytes"], ((16, 16), (240, 20), (256, 256), (2048, 2048))),
+                                     ("5MiB", 160, 32768, ((128, 128),))):
+        bb2 = n_chunks * cb
+        if tag == "2MiB":
+            lay2, layout2, nb, nrec = lay, layout, lay["n_blocks"], host_blocks
+        else:
+            nb = min(4096, hbm_pool.numel() // bb2 // 2)
+            lay2 = wl.kv_layout(nb, n_chunks, cb)
+            layout2, nrec = cs.make_layout(lay2), min(host_pool.numel() // bb2, 8192)
+        for ne, nr in pairs:
+            if ne + nr > nrec or ne + nr > nb or (ne + nr) * bb2 > stage.numel():
+                continue
+            rng = np.random.default_rng(ne + nr)
+            hp, op = rng.permutation(nb).astype(np.int32), rng.permutation(nrec).astype(np.int32)
+            es, ed, rs = hp[:ne], op[:ne], op[ne:ne + nr]
+            k = min(ne, nr) // 2
+            rd = np.concatenate([es[::-1][:k], hp[ne:ne + nr - k]]).astype(np.int32)
+            t = [torch.from_numpy(np.ascontiguousarray(x)).cuda() for x in (es, ed, rs, rd)]
+            scratch = torch.empty(cs.kv_move_scratch_len(ne, nr), dtype=torch.int32, device="cuda")
+            mailbox = torch.empty(cs.kv_mailbox_len(ne, nr), dtype=torch.int32, pin_memory=True)
+            reps = 4 if ne + nr > 1000 else 6
+            _, med = timed_calls(torch, lambda: ctx.kv_move(layout2, hbm_pool, host_pool, nrec, t[0], t[1], None, ne, t[2], t[3],
+                                                            None, nr, scratch), reps, warm=2)
+            _, med2 = timed_calls(torch, lambda: ctx.kv_move_staged(layout2, hbm_pool, host_pool, nrec, t[0], t[1], None, ne, t[2],
+                                                                    t[3], None, nr, stage, (ne + nr), mailbox), reps, warm=2)
+            gb = (ne + nr) * bb2 / 1e6
+            duplex[f"{tag}_{ne}+{nr}"] = dict(zero_copy_kernels_GBps=round(gb / med, 1), copy_engines_GBps=round(gb / med2, 1))
+    # what the copy engines reach with ONE contiguous copy per direction, both at once
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    nbytes = 512 << 20
+
+    def two_way():
+        cur = torch.cuda.current_stream()
+        s1.wait_stream(cur)
+        s2.wait_stream(cur)
+        with torch.cuda.stream(s1):
+            hbm_pool[:nbytes].copy_(host_pool[:nbytes], non_blocking=True)
+        with torch.cuda.stream(s2):
+            host_pool[nbytes:2 * nbytes].copy_(hbm_pool[nbytes:2 * nbytes], non_blocking=True)
+        cur.wait_stream(s1)
+        cur.wait_stream(s2)
+    _, med = timed_calls(torch, two_way, 5, warm=2)
+    duplex["cudaMemcpyAsync_512MiB_each_way_GBps"] = round(2 * nbytes / med / 1e6, 1)
+    out["both_directions"] = duplex
+
     # first hop of the deep-tier path: pinned "deep" records -> pinned host records (the bytes cross the host
     # link twice, once in each direction)
     m = min(256, host_blocks)
     deep = torch.empty(m * bb, dtype=torch.uint8, pin_memory=True)
     src, dst = wl.copy_lists(77, m, m, host_blocks)
     s, d = torch.from_numpy(src).cuda(), torch.from_numpy(dst).cuda()
-    best = 1e30
-    for it in range(6):
-        a, b = event_pair(torch)
-        a.record()
-        ctx.kv_stage(deep, m, host_pool, host_blocks, bb, s, d, None, m)
-        b.record()
-        torch.cuda.synchronize()
-        if it >= 2:
-            best = min(best, a.elapsed_time(b))
+    best, _ = timed_calls(torch, lambda: ctx.kv_stage(deep, m, host_pool, host_blocks, bb, s, d, None, m), 4, warm=2)
     out[f"stage_host_{m}"] = round(m * bb / best / 1e6, 1)
     del deep
     return out, median
@@ -419,7 +542,8 @@ def deep_sweep(torch, cs):
 def schedule_sweep(torch, cs):
     """budget+schedule+plan latency for 1k..64k queued requests (plan-only, no tables): the three calls
     captured in a CUDA graph, 20 iterations per replay, median microseconds per iteration; launched call by
-    call; and 200 iterations of the churning sweep with the 5 % slot update inside the timed region (median, p99)."""
+    call; 200 iterations of the churning sweep with the 5 % slot update inside the timed region (median, p99),
+    launched call by call from Python and as ONE cascade_step call per iteration."""
     from paper_2608_06557_b200 import workload as wl
     from paper_2608_06557_b200.runner import Instance
     out = {}
@@ -471,6 +595,22 @@ def schedule_sweep(torch, cs):
             torch.cuda.synchronize()
             if it >= 3:
                 upd.append(a.elapsed_time(b) * 1e3)
+        # the same churning iterations through cascade_step: one C call issues slot update + budget + schedule + plan
+        step_args = inst.step_args(with_update=True)
+        one = []
+        for it in range(203):
+            slots = sw.step()
+            w = sw.workload()
+            inst.stage_slot_update(w.reqs, slots)
+            inst.set_clock(w.now_ns, w.D_act, w.K_act)
+            a, b = event_pair(torch)
+            a.record()
+            inst.run_step(step_args)
+            b.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                one.append(a.elapsed_time(b) * 1e3)
+        one.sort()
         # the same iteration (last staged update) captured in a graph: device time without the Python launches
         g2 = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g2, stream=st):
@@ -492,6 +632,8 @@ def schedule_sweep(torch, cs):
                            graph_with_slot_update_us=round(statistics.median(tg), 1),
                            with_slot_update_us=round(statistics.median(upd), 1),
                            with_slot_update_p99_us=round(upd[int(0.99 * (len(upd) - 1))], 1),
+                           one_call_with_slot_update_us=round(statistics.median(one), 1),
+                           one_call_with_slot_update_p99_us=round(one[int(0.99 * (len(one) - 1))], 1),
                            slot_update_bytes=upd_bytes)
         inst.ctx.status(clear=True)
         del inst
@@ -523,14 +665,17 @@ def ours_main(args):
     batches = [make_batch(args, rank_seed(rank, s)) for s in range(W + K)]
     w0 = batches[0]
     bb = w0.block_bytes
-    host_pool, host_bytes = alloc_pinned_pool(w0.host_blocks * bb)
-    if host_bytes != w0.host_blocks * bb:      # pinning was refused at full size: regenerate at the size we got
-        args.host_gb = host_bytes / GB
+    # one pinned allocation: the copy sweep's pool as stated (100 * 10^9 bytes, or what the box grants); the step
+    # uses its first --host-gb
+    want_sweep = 0 if args.no_sweeps or rank != 0 else int(args.host_sweep_gb * GB) // bb * bb
+    big_pool, big_bytes = alloc_pinned_pool(max(want_sweep, w0.host_blocks * bb))
+    if big_bytes < w0.host_blocks * bb:        # pinning was refused at full size: regenerate at the size we got
+        args.host_gb = big_bytes / GB
         batches = [make_batch(args, rank_seed(rank, s)) for s in range(W + K)]
         w0 = batches[0]
-        host_pool = host_pool[: w0.host_blocks * bb]
+    host_pool = big_pool[: w0.host_blocks * bb]
     hbm_pool = torch.empty(w0.layout["n_blocks"] * bb, dtype=torch.uint8, device=dev)
-    fill_pools(hbm_pool, host_pool)
+    fill_pools(hbm_pool, big_pool)
     ctx = cs.Context(w0.params, args.requests, local_rank)
     insts = [Instance(w, device=dev, ctx=ctx, hbm_pool=hbm_pool, host_pool=host_pool, alloc_pools=False)
              for w in batches]
@@ -593,7 +738,7 @@ def ours_main(args):
         ideal_ms = sum(max(int(e) * bb / peaks["d2h"], int(r) * bb / peaks["h2d"]) for e, r in zip(n_evict, n_restore)) / 1e6
         dom_ach = (ev_bytes + rs_bytes) / (t_move * 1e-3) / GB if t_move else 0.0
         dom_peak = (ev_bytes + rs_bytes) / (ideal_ms * 1e-3) / GB if ideal_ms else 0.0
-        dominant = "kv_move_kernel (evict + restore, both link directions)"
+        dominant = "cascade_kv_move: kv_ring_kernel<evict> beside kv_copy_kernel<restore> (both link directions)"
         dom_launch_bytes = (ev_bytes + rs_bytes) / K
         traffic = int((NCU_DRAM_BYTES_PER_BLOCK["evict"] * n_evict.sum() + NCU_DRAM_BYTES_PER_BLOCK["restore"] * n_restore.sum()) / K)
         evict_gbs = restore_gbs = None
@@ -601,7 +746,7 @@ def ours_main(args):
         evict_gbs = ev_bytes / (t_evict.sum() * 1e-3) / GB if ev_bytes else 0.0
         restore_gbs = rs_bytes / (t_rest.sum() * 1e-3) / GB if rs_bytes else 0.0
         is_ev = t_evict.sum() >= t_rest.sum()
-        dominant = "kv_copy_bulk_kernel<evict>" if is_ev else "kv_copy_bulk_kernel<restore>"
+        dominant = "kv_ring_kernel<evict>" if is_ev else "kv_ring_kernel<restore>"
         dom_ach = evict_gbs if is_ev else restore_gbs
         dom_peak = peaks["d2h"] if is_ev else peaks["h2d"]
         dom_launch_bytes = (ev_bytes if is_ev else rs_bytes) / K
@@ -611,6 +756,7 @@ def ours_main(args):
                     traffic=traffic,
                     traffic_source="ncu captures of 128 blocks per direction, scaled by the blocks per launch",
                     algorithmic_bytes_per_launch=int(dom_launch_bytes),
+                    link_peaks_GBps=dict(h2d=round(peaks["h2d"], 2), d2h=round(peaks["d2h"], 2)),
                     peak_source="pinned cudaMemcpyAsync of one contiguous 1 GiB buffer per direction, measured by "
                                 "this run (MEASURED_PEAKS.json holds no host-link figure); for the fused kernel the "
                                 "peak is the byte total over the slower direction's ideal time",
@@ -623,13 +769,14 @@ def ours_main(args):
     if rank == 0:
         # ---- end to end: inputs start in pinned host memory, results are read back every step -------
         e2e = run_e2e(torch, args, batches[W:], insts[0], K)
-        extra = dict(blocks_restored_per_step=float(n_restore.mean()), blocks_evicted_per_step=float(n_evict.mean()),
-                     host_pool_bytes=int(host_pool.numel()), hbm_pool_bytes=int(hbm_pool.numel()),
-                     status_bits=status)
-        line["config"] = workload_config(args, extra)
+        line["config"] = workload_config(args)
+        line["run"] = dict(blocks_restored_per_step=float(n_restore.mean()), blocks_evicted_per_step=float(n_evict.mean()),
+                           host_pool_bytes=int(host_pool.numel()), hbm_pool_bytes=int(hbm_pool.numel()),
+                           status_bits=status)
         line["clocks"] = clocks
         line["e2e"] = e2e
-        line["gpu_launches"] = 7 * K
+        # budget, schedule, plan + 2 table rewrites, and the move's prepare + evict grid + restore grid
+        line["gpu_launches"] = (8 if fused else 7) * K
         line["roofline"] = roofline
         line["kernels"] = dict(schedule_us_per_step=round(float(np.median(t_sched)) * 1e3, 1),
                                copies="fused cascade_kv_move" if fused else "cascade_kv_evict + cascade_kv_restore",
@@ -644,13 +791,15 @@ def ours_main(args):
             lay = dict(w0.layout)
             lay_small = dict(lay, n_blocks=(hbm_pool.numel() - stage_bytes) // bb // 2)
             lay_small["chunk_stride"] = lay_small["n_blocks"] * lay["chunk_bytes"]
-            sweep, sweep_median = copy_sweep(torch, cs, ctx, cs.make_layout(lay_small), lay_small, hbm_pool, host_pool,
-                                             w0.host_blocks, stage)
+            sweep, sweep_median = copy_sweep(torch, cs, ctx, cs.make_layout(lay_small), lay_small, hbm_pool, big_pool,
+                                             big_pool.numel() // bb, stage, peaks)
+            line["run"]["copy_sweep_host_pool"] = dict(asked_bytes=int(args.host_sweep_gb * GB), pinned_bytes=int(big_bytes),
+                                                       records=int(big_pool.numel() // bb))
             line["copy_sweep_GBps"] = sweep
             line["copy_sweep_median_GBps"] = sweep_median
             hbm_peak = load_hbm_peak()
             big = sweep.get("restore_hbm_4096", 0.0)
-            line["roofline_hbm"] = dict(bound="hbm", kernel="kv_copy_bulk_kernel<restore>, device staging buffer, "
+            line["roofline_hbm"] = dict(bound="hbm", kernel="kv_ring_kernel<restore>, device staging buffer, "
                                         "4096 blocks", achieved=big, peak=hbm_peak[0], unit="GB/s",
                                         frac=round(big / hbm_peak[0], 4),
                                         traffic=int(1027.4e6 / 256 * 4096),
@@ -662,15 +811,26 @@ def ours_main(args):
             line["deep_tier_us"] = deep_sweep(torch, cs)
             # the four targets the build was given, side by side with what this run measured
             sl = line["schedule_latency_us"]
+            small = sweep["graph_timed_small_calls"]
             line["targets"] = dict(
-                restore_fraction_of_h2d_peak=dict(target=0.80, measured=round(sweep["restore_host_256"] / peaks["h2d"], 3)),
-                evict_fraction_of_d2h_peak=dict(target=0.80, measured=round(sweep["evict_host_256"] / peaks["d2h"], 3)),
-                hbm_scatter_fraction_of_hbm_peak=dict(target=0.70, measured=round(sweep["restore_hbm_4096"] / hbm_peak[0], 3)),
+                restore_fraction_of_h2d_peak=dict(target=0.80, measured=round(sweep["restore_host_256"] / peaks["h2d"], 3),
+                                                  at_16_blocks=small["restore_host_16_fraction_of_1GiB_peak"],
+                                                  at_1_block=small["restore_host_1_fraction_of_1GiB_peak"],
+                                                  at_1_block_of_same_size_copy=small["restore_host_1_fraction_of_same_size_copy"]),
+                evict_fraction_of_d2h_peak=dict(target=0.80, measured=round(sweep["evict_host_256"] / peaks["d2h"], 3),
+                                                at_16_blocks=small["evict_host_16_fraction_of_1GiB_peak"],
+                                                at_1_block=small["evict_host_1_fraction_of_1GiB_peak"]),
+                hbm_scatter_fraction_of_hbm_peak=dict(target=0.70, measured=round(sweep["restore_hbm_4096"] / hbm_peak[0], 3),
+                                                      at_256_blocks=round(sweep["restore_hbm_256"] / hbm_peak[0], 3),
+                                                      at_16_blocks=round(small["restore_hbm_16"]["GBps"] / hbm_peak[0], 3),
+                                                      one_block_latency_us=small["restore_hbm_1"]["us"]),
                 budget_schedule_plan_16k_us=dict(target=100.0, measured=sl["16384"]["graph_us"],
-                                                 launched_from_python=sl["16384"]["launched_us"]),
+                                                 launched_from_python=sl["16384"]["launched_us"],
+                                                 one_call_with_slot_update=sl["16384"]["one_call_with_slot_update_us"],
+                                                 one_call_with_slot_update_p99=sl["16384"]["one_call_with_slot_update_p99_us"]),
                 parity="bit-exact against the CPU oracle: see tests/ (-m gpu)")
         line["cpu_baseline"] = {k: v for k, v in run_oracle_arm(args, args.cpu_seconds, first_seed=W).items()
-                                if k in ("value", "unit", "cores", "kind", "sample")}
+                                if k in ("value", "unit", "cores", "kind", "sample", "host")}
         if not args.no_sweeps:
             line["cpu_baseline"]["schedule_latency_us"] = oracle_schedule_latency()
         print(json.dumps(line))
@@ -753,9 +913,112 @@ def run_e2e(torch, args, batches, inst, K):
                 d2h_bytes_per_step=int(d2h), ms_per_step=round(ms / len(pinned), 4))
 
 
+# --------------------------------------------------------------------------------------------
+# small cases: one kernel family, a few launches (what the ncu captures under profiles/ run)
+# --------------------------------------------------------------------------------------------
+def run_case(args):
+    import torch
+    import __graft_entry__ as ge
+    ge.build()
+    from paper_2608_06557_b200 import cascade as cs
+    from paper_2608_06557_b200 import workload as wl
+    from paper_2608_06557_b200.runner import Instance
+
+    def timed(fn, reps=5):
+        out = []
+        for _ in range(reps):
+            a, b = event_pair(torch)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            out.append(a.elapsed_time(b) * 1e3)
+        return out
+
+    n_chunks, chunk_bytes = 64, 32 * 1024
+    bb = n_chunks * chunk_bytes
+    case = args.case
+    if case in ("copy-hbm", "copy-host"):
+        n = args.case_n or 256
+        on_device = case == "copy-hbm"
+        n_hbm, n_rec = 2 * n + 64, n + 64
+        lay = wl.kv_layout(n_hbm, n_chunks, chunk_bytes)
+        hbm = torch.empty(n_hbm * bb, dtype=torch.uint8, device="cuda").fill_(1)
+        rec = (torch.empty(n_rec * bb, dtype=torch.uint8, device="cuda") if on_device
+               else torch.empty(n_rec * bb, dtype=torch.uint8, pin_memory=True)).fill_(2)
+        ctx = cs.Context(wl.default_params(), 16, 0)
+        layout = cs.make_layout(lay)
+        src, dst = wl.copy_lists(7, n, n_rec, n_hbm)
+        s, d = torch.from_numpy(src).cuda(), torch.from_numpy(dst).cuda()
+        torch.cuda.synchronize()
+        t_r = timed(lambda: ctx.kv_restore(layout, hbm, rec, n_rec, on_device, s, d, None, n))
+        t_e = timed(lambda: ctx.kv_evict(layout, hbm, rec, n_rec, on_device, d, s, None, n))
+        mult = 2 if on_device else 1
+        for name, ts in (("restore", t_r), ("evict", t_e)):
+            print(f"{name}: {n} blocks x {bb} B, us per launch {[round(t, 1) for t in ts]}, "
+                  f"best {mult * n * bb / min(ts) / 1e3:.1f} GB/s ({'read+write' if mult == 2 else 'link'} bytes)")
+        print("status", ctx.status())
+    elif case in ("move", "staged"):
+        # n blocks evicted and n restored by one call; half of the restores reuse evicted blocks
+        n = args.case_n or 128
+        n_hbm, n_rec = 3 * n + 64, 3 * n + 64
+        lay = wl.kv_layout(n_hbm, n_chunks, chunk_bytes)
+        hbm = torch.empty(n_hbm * bb, dtype=torch.uint8, device="cuda").fill_(1)
+        rec = torch.empty(n_rec * bb, dtype=torch.uint8, pin_memory=True).fill_(2)
+        ctx = cs.Context(wl.default_params(), 16, 0)
+        layout = cs.make_layout(lay)
+        rng = np.random.default_rng(3)
+        hp, op = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_rec).astype(np.int32)
+        es, ed, rs = hp[:n], op[:n], op[n:2 * n]
+        rd = np.concatenate([es[::-1][: n // 2], hp[n:2 * n - n // 2]]).astype(np.int32)
+        t = [torch.from_numpy(np.ascontiguousarray(x)).cuda() for x in (es, ed, rs, rd)]
+        if case == "move":
+            scratch = torch.empty(cs.kv_move_scratch_len(n, n), dtype=torch.int32, device="cuda")
+            fn = lambda: ctx.kv_move(layout, hbm, rec, n_rec, t[0], t[1], None, n, t[2], t[3], None, n, scratch)
+        else:
+            staging = torch.empty(2 * n * bb, dtype=torch.uint8, device="cuda")
+            mailbox = torch.empty(cs.kv_mailbox_len(n, n), dtype=torch.int32, pin_memory=True)
+            fn = lambda: ctx.kv_move_staged(layout, hbm, rec, n_rec, t[0], t[1], None, n, t[2], t[3], None, n, staging,
+                                            2 * n, mailbox)
+        torch.cuda.synchronize()
+        ts = timed(fn)
+        print(f"{case}: {n} evicted + {n} restored blocks x {bb} B, us per call {[round(x, 1) for x in ts]}, "
+              f"best {2 * n * bb / min(ts) / 1e3:.1f} GB/s over the link (both directions)")
+        print("status", ctx.status())
+    elif case == "schedule":
+        n = args.case_n or 16384
+        sw = wl.SchedulerSweep(n, seed=0)
+        inst = Instance(sw.workload(), alloc_pools=False)
+        ts = timed(inst.run_schedule, reps=8)
+        print(f"budget+schedule+plan, {n} requests, us per iteration (event-bracketed, launched call by call): "
+              f"{[round(t, 1) for t in ts]}")
+        print("status", inst.ctx.status())
+    elif case == "deep":
+        # three independent iterations (seeds 0..2) of the shared-prefix workload: plan, merge of the restore list,
+        # stage plan, merge of the stage list, evict + restore, stage copy (16 KiB blocks)
+        n = args.case_n or 1024
+        for seed in range(3):
+            w = wl.config_deep_shared(seed, n=n, n_hbm=16 * n, n_host=16 * n, n_deep=32 * n, hbm_free_target=8 * n)
+            w.params["plan_first"] = 1
+            inst = Instance(w)
+            inst.enable_deep(w)
+            inst.hbm_pool.fill_(1)
+            inst.host_pool.fill_(2)
+            inst.deep_pool.fill_(3)
+            torch.cuda.synchronize()
+            ts = timed(lambda: inst.run_iteration_deep(10**9, 0), reps=1)
+            d = inst.fetch_deep()
+            print(f"seed {seed}: {n} requests, iteration {ts[0]:.1f} us; restore list {d['dedup_restore']['n_in']} -> "
+                  f"{d['dedup_restore']['n_unique']}, stage list {d['dedup_stage']['n_in']} -> "
+                  f"{d['dedup_stage']['n_unique']}, status {inst.ctx.status()}")
+            del inst
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         reference_main(args)
     else:
         ours_main(args)

@@ -81,6 +81,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->ce_hybrid = e ? atoi(e) : 0;
     e = getenv("CASCADE_CE_LANES");
     ctx->ce_lanes = e && atoi(e) == 2 ? 2 : 1;   // measured: a second stream per direction gains nothing
+    e = getenv("CASCADE_COPY_AHEAD_SUB");
+    ctx->copy_ahead_sub = e && atoi(e) == 1 ? 1 : 2;   // measured: refilling the slot of the store just issued stalls the ring
     e = getenv("CASCADE_COPY_PIECE");
     ctx->copy_piece = e ? atoi(e) : 0;
     if (ctx->copy_piece != 8192 && ctx->copy_piece != 16384 && ctx->copy_piece != 32768) ctx->copy_piece = 0;

@@ -35,6 +35,7 @@ struct cascade_ctx {
     int copy_bulk_dev;           // >0: TMA bulk-copy ring for the device-staging path
     int move_ctas;               // >0: CTAs of each of the two grids of the fused evict+restore (at most half the SMs)
     int move_vector;             // fused move: bit 0 = restore grid, bit 1 = evict grid use the vector kernel instead of the ring
+    int copy_ahead_sub;          // TMA ring: loads kept in flight = ring slots minus this (1 | 2)
     int copy_piece;              // >0: piece size in bytes of the TMA ring (8192 | 16384 | 32768); 0 = picked per call
     int copy_ring_kb;            // >0: shared memory of the TMA ring in KiB (64..128); 0 = 128 (host) / 96 (device)
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels

@@ -36,6 +36,7 @@ struct CopyArgs {
     int pieces_per_chunk;     // vector kernel only
     int ring_bytes;           // ring kernel: shared memory of the ring
     int piece_fixed;          // ring kernel: >0 forces this piece size (bytes), 0 = pick per call
+    int ahead_sub;            // ring kernel: loads in flight ahead of the store = ring slots minus this (1 or 2)
     int record_iota;          // ring kernel: the record id of list entry i is i itself (staging buffer filled in list order)
     const int32_t *iota_check;    // with record_iota: entry i is skipped unless 0 <= iota_check[i] < iota_check_blocks
     long long iota_check_blocks;  // (the id its staging slot was, or will be, copied from / to by the copy engines)
@@ -146,9 +147,11 @@ __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant
 
 // ---- ring kernel: TMA bulk copies (cp.async.bulk) through a shared-memory ring ----------------------
 // One elected thread per CTA moves pieces: global -> shared with an mbarrier that counts the arriving
-// bytes, then shared -> global as a bulk store group.  The ring has S = ring_bytes / piece slots; S - 1
-// loads are kept in flight ahead of the piece being stored, and a slot is refilled only after the store
-// that last used it has finished reading shared memory.  Every wait is bounded: when the clock limit is
+// bytes, then shared -> global as a bulk store group.  The ring has S = ring_bytes / piece slots.  S - 1
+// loads are issued before the first wait (short calls live off this); afterwards S - 2 loads are kept in
+// flight ahead of the piece being stored, so that the slot refilled next was last read by the store issued
+// one step EARLIER, which has long finished reading shared memory (with S - 1 in flight the refill would
+// wait for the store just issued: measured 6.2 instead of 6.55 TB/s through the staging buffer).  Every wait is bounded: when the clock limit is
 // hit the CTA records CASCADE_ST_ETIMEOUT, issues nothing more, waits (bounded again) for the loads it
 // still has in flight, drains its store groups and returns.
 //
@@ -230,12 +233,15 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
     }
     int S = a.ring_bytes / piece;
     S = S > kMaxStages ? kMaxStages : S;
-    const int ahead = S - 1;
+    const int prime = S - 1;   // loads issued before the first wait
     const int ppc = (int)((a.chunk_bytes + piece - 1) / piece);
     const long long per_block = (long long)a.n_chunks * ppc;
     const long long items = (long long)count * per_block;
     const long long bb = (long long)a.n_chunks * a.chunk_bytes;
     const long long limit = a.stall ? kWaitCycles / 20 : kWaitCycles;
+    // loads in flight ahead of the store after the first wait: a call of a few pieces per CTA is over before the
+    // ring reaches a steady state and keeps every slot busy; a long one leaves the slot of the store just issued alone
+    const int steady = (items < 16LL * gridDim.x || S - a.ahead_sub < 1) ? S - 1 : S - a.ahead_sub;
     uint32_t st = 0;
 
     long long next = blockIdx.x;  // next item of this CTA to load
@@ -290,7 +296,7 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
         }
         return false;
     };
-    for (int k = 0; k < ahead; ++k)
+    for (int k = 0; k < prime; ++k)
         if (!issue_next()) break;
     while (stored < issued) {
         const int slot = (int)(stored % S);
@@ -328,9 +334,9 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
         }
         if (!skip) bulk_store(dst_of[slot], smem_addr(ring + (size_t)slot * piece), bytes_of[slot]);
         ++stored;
-        // the slot refilled next was last read by the store issued one step earlier
+        // every store but the one just issued has finished reading shared memory
         asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-        issue_next();
+        if (issued - stored < steady) issue_next();
     }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (st) atomicOr(a.status, st);
@@ -444,6 +450,7 @@ void fill_copy_args(CopyArgs &a, const cascade_ctx *ctx, const cascade_kv_layout
     a.n_chunks = l->n_chunks;
     a.n_max = n_max;
     a.piece_fixed = ctx->copy_piece;
+    a.ahead_sub = ctx->copy_ahead_sub;
     a.stall = ctx->test_move_stall;
 }
 

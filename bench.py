@@ -33,11 +33,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "restored KV GB/s vs host-link/HBM roofline; per-iteration schedule latency us"
-# dram__bytes_read.sum + dram__bytes_write.sum per 2 MiB block of the host-link copy kernel, from the
-# 128-block ncu captures summarised in profiles/kv_copy_bulk_kernel_pinned_host_128_blocks.md; the traffic
+# dram__bytes_read.sum + dram__bytes_write.sum per 2 MiB block of the two grids of the fused move, from the
+# 128 + 128-block ncu capture summarised in profiles/cascade_kv_move_pinned_host_128+128_blocks.md; the traffic
 # grows in proportion to the blocks moved, so a launch's traffic is this figure times its block count
 # (the restore figure is low because part of the written lines is still in L2 when the kernel ends)
-NCU_DRAM_BYTES_PER_BLOCK = {"evict": (268_630_272 + 3_547_648) / 128, "restore": (99_840 + 209_025_792) / 128}
+NCU_DRAM_BYTES_PER_BLOCK = {"evict": (268_466_688 + 4_401_664) / 128, "restore": (228_096 + 208_928_768) / 128}
 GB = 1e9
 
 
@@ -802,8 +802,8 @@ def ours_main(args):
             line["roofline_hbm"] = dict(bound="hbm", kernel="kv_ring_kernel<restore>, device staging buffer, "
                                         "4096 blocks", achieved=big, peak=hbm_peak[0], unit="GB/s",
                                         frac=round(big / hbm_peak[0], 4),
-                                        traffic=int(1027.4e6 / 256 * 4096),
-                                        traffic_source="ncu capture of 256 staged blocks (537.0 MB read + 490.4 MB "
+                                        traffic=int(1028.25e6 / 256 * 4096),
+                                        traffic_source="ncu capture of 256 staged blocks (537.0 MB read + 491.3 MB "
                                                        "written), scaled to 4096 blocks",
                                         algorithmic_bytes_per_launch=int(2 * 4096 * bb), peak_source=hbm_peak[1])
             del insts

@@ -545,8 +545,9 @@ uint32_t orc_prefetch_plan(const orc_params *p, int n, const int32_t *prompt, co
  * iteration's plan did not preempt and whose own restore choice (Eq. 7 bounds, then the cheapest
  * candidate, from its budget) contains a deep fetch x2 > 0 gets host records for its first x2 deep
  * blocks while the deep link's time budget and the host pool (above a reserve) last.  One hop costs
- * what P(2) adds to P(1) in Eq. 6.  HBM is not touched ("allocated only at the final hop"): the
- * staged blocks become host blocks of the request and a later iteration restores them. */
+ * what P(2) adds to P(1) in Eq. 6.  HBM is not touched (Section 4.4, memory management: HBM is taken
+ * at the last hop only): the staged blocks become host blocks of the request and a later iteration
+ * restores them. */
 uint32_t orc_stage_plan(const orc_params *p, int n, const int32_t *prompt, const int32_t *n0, const int32_t *n1,
                         const int32_t *n2, const int64_t *budget, const uint32_t *order, const uint8_t *action,
                         int32_t D_act, int64_t K_act, int64_t link_budget_ns, int32_t host_reserve,

@@ -417,3 +417,49 @@ def test_staged_move_orders_a_restore_behind_the_eviction_that_writes_its_record
     rig.ctx.kv_move_staged(rig.layout, rig.hbm, rig.host, 32, None, None, None, 0, None, None, None, 0, staging, 16, mailbox)
     torch.cuda.synchronize()
     assert np.array_equal(rig.hbm.cpu().numpy(), ref_hbm) and rig.ctx.status()[0] == 0
+
+
+def test_fused_move_inside_a_cuda_graph():
+    """The fused move's two grids are tied together by programmatic launch edges; captured in a CUDA graph together
+    with the kernels around it (an evict before, a restore after, as a serving loop would queue them) and replayed
+    on fresh data, the result must still be evict-then-restore, bit for bit."""
+    rig = CopyRig(96, 96, 8, 32768)
+    torch, cs = rig.torch, rig.cs
+    rng = np.random.default_rng(11)
+    ne, nr = 30, 30
+    hp, op = rng.permutation(96).astype(np.int32), rng.permutation(96).astype(np.int32)
+    es, ed, rs = hp[:ne], op[:ne], op[ne:ne + nr]
+    rd = np.concatenate([es[::-1][: nr // 2], hp[ne:ne + nr - nr // 2]]).astype(np.int32)
+    pre_s, pre_d = hp[70:75], op[70:75]                      # an eviction before the move
+    post_s, post_d = op[80:84], hp[80:84]                    # a restore after it
+    t = [rig.ids(x) for x in (es, ed, rs, rd, pre_s, pre_d, post_s, post_d)]
+    scratch = torch.empty(cs.kv_move_scratch_len(ne, nr), dtype=torch.int32, device="cuda")
+    st = torch.cuda.Stream()
+
+    def chain():
+        rig.ctx.kv_evict(rig.layout, rig.hbm, rig.host, 96, False, t[4], t[5], None, 5, st)
+        rig.ctx.kv_move(rig.layout, rig.hbm, rig.host, 96, t[0], t[1], None, ne, t[2], t[3], None, nr, scratch, st)
+        rig.ctx.kv_restore(rig.layout, rig.hbm, rig.host, 96, False, t[6], t[7], None, 4, st)
+
+    with torch.cuda.stream(st):
+        chain()                                               # warm-up outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        chain()
+    for rep in range(3):
+        hbm_np = rng.integers(0, 256, rig.hbm_np.size, dtype=np.uint8)
+        host_np = rng.integers(0, 256, rig.host_np.size, dtype=np.uint8)
+        rig.hbm.copy_(torch.from_numpy(hbm_np))
+        rig.host.copy_(torch.from_numpy(host_np))
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        ref_h, ref_o = hbm_np.copy(), host_np.copy()
+        assert oracle.kv_evict(ref_h, rig.lay, ref_o, 96, pre_s, pre_d) == 0
+        assert oracle.kv_evict(ref_h, rig.lay, ref_o, 96, es, ed) == 0
+        assert oracle.kv_restore(ref_h, rig.lay, ref_o, 96, rs, rd) == 0
+        assert oracle.kv_restore(ref_h, rig.lay, ref_o, 96, post_s, post_d) == 0
+        assert np.array_equal(rig.hbm.cpu().numpy(), ref_h), rep
+        assert np.array_equal(rig.host.cpu().numpy(), ref_o), rep
+    assert rig.ctx.status()[0] == 0 and rig.guards_intact()

@@ -99,3 +99,51 @@ def test_repeated_runs_give_identical_results(n, reps):
         else:
             assert all(torch.equal(a, b) for a, b in zip(ref, cur))
     assert inst.ctx.status()[0] == 0
+
+
+def test_staged_move_on_random_shapes():
+    """The copy-engine path on random shapes, list lengths and staging sizes (down to one block per direction), with
+    restores into blocks the same call evicts, runs of consecutive host records and, now and then, a restore that
+    reads a record the same call's evictions write."""
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    rng = np.random.default_rng(17)
+    ctx = cs.Context(wl.default_params(), 16, 0)
+    done = 0
+    while done < 60:
+        n_hbm, n_host = int(rng.integers(8, 200)), int(rng.integers(8, 200))
+        n_chunks = int(rng.choice([1, 3, 8, 64]))
+        cb = int(rng.choice([16, 48, 4096, 32768, 32768 + 16]))
+        if n_chunks * cb * (n_hbm + n_host) > 200e6:
+            continue
+        lay = wl.kv_layout(n_hbm, n_chunks, cb)
+        bb = n_chunks * cb
+        hbm_np = rng.integers(0, 256, n_hbm * bb, dtype=np.uint8)
+        host_np = rng.integers(0, 256, n_host * bb, dtype=np.uint8)
+        ne = int(rng.integers(0, min(n_hbm, n_host) // 2 + 1))
+        nr = int(rng.integers(0, min(n_hbm, n_host) // 2 + 1))
+        hp, op = rng.permutation(n_hbm).astype(np.int32), rng.permutation(n_host).astype(np.int32)
+        es, ed, rs = hp[:ne], op[:ne].copy(), op[ne:ne + nr].copy()
+        if rng.random() < 0.5:
+            ed.sort()
+            rs.sort()
+        if ne and nr and rng.random() < 0.3:
+            rs[0] = ed[-1]                                   # a restore reads what this call's evictions write
+        k = int(rng.integers(0, min(ne, nr) + 1))
+        rd = rng.permutation(np.concatenate([rng.permutation(es)[:k], hp[ne:ne + nr - k]])).astype(np.int32)
+        ref_h, ref_o = hbm_np.copy(), host_np.copy()
+        assert oracle.kv_evict(ref_h, lay, ref_o, n_host, es, ed) == 0
+        assert oracle.kv_restore(ref_h, lay, ref_o, n_host, rs, rd) == 0
+        hbm = torch.from_numpy(hbm_np).cuda()
+        host = torch.from_numpy(host_np).pin_memory()
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda() if len(a) else None
+        stage_blocks = int(rng.integers(2 if ne and nr else 1, ne + nr + 3))
+        staging = torch.empty(stage_blocks * bb, dtype=torch.uint8, device="cuda")
+        mailbox = torch.empty(cs.kv_mailbox_len(ne, nr), dtype=torch.int32, pin_memory=True)
+        ctx.kv_move_staged(cs.make_layout(lay), hbm, host, n_host, t(es), t(ed), None, ne, t(rs), t(rd), None, nr, staging,
+                           stage_blocks, mailbox)
+        torch.cuda.synchronize()
+        assert np.array_equal(hbm.cpu().numpy(), ref_h), (n_hbm, n_host, n_chunks, cb, ne, nr, k, stage_blocks)
+        assert np.array_equal(host.numpy(), ref_o), (n_hbm, n_host, n_chunks, cb, ne, nr, k, stage_blocks)
+        done += 1
+    assert ctx.status()[0] == 0

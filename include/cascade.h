@@ -216,7 +216,8 @@ typedef struct cascade_ctx cascade_ctx;
 
 /* Creates a context on `device` for queues of up to max_requests (<= CASCADE_MAX_REQUESTS, and
  * <= 4096 times the largest thread-block cluster the device co-schedules: 16 on a full B200).
- * Validates the parameters against the bounds above.  Allocates scratch (about 44 bytes per request).
+ * Validates the parameters against the bounds above.  Allocates scratch (about 44 bytes per request, 76 for
+ * contexts of more than 16384 requests), four side streams and seven events for the copy-engine path.
  * `p` and `out` are host pointers.  The calling thread's current device is left as it was; the hot calls
  * launch on the current device, so make `device` current (and pass one of its streams) when calling them:
  * a call made while another device is current returns CASCADE_EINVAL and launches nothing. */

@@ -112,6 +112,10 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
         ok = cudaStreamCreateWithFlags(&ctx->ce_stream[i], cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; ok && i < 7; ++i)
         ok = cudaEventCreateWithFlags(&ctx->ce_event[i], cudaEventDisableTiming) == cudaSuccess;
+    e = getenv("CASCADE_MULTI_SORT");
+    ctx->multi_sort = e ? atoi(e) : 1;
+    if (ok && max_requests > 16384 && ctx->max_cluster >= 16)
+        ok = cudaMalloc(&ctx->sort_runs, n * 16) == cudaSuccess && cudaMalloc(&ctx->sort_sorted, n * 16) == cudaSuccess;
     if (ok) ok = cudaMemset(ctx->status_dev, 0, sizeof(uint32_t)) == cudaSuccess &&
                  cudaMemset(ctx->plan_scalars, 0, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
     if (!ok) {
@@ -135,6 +139,8 @@ extern "C" void cascade_destroy(cascade_ctx *ctx) {
     cudaFree(ctx->work_admit);
     cudaFree(ctx->work_victim);
     cudaFree(ctx->plan_scalars);
+    cudaFree(ctx->sort_runs);
+    cudaFree(ctx->sort_sorted);
     for (int i = 0; i < 4; ++i)
         if (ctx->ce_stream[i]) cudaStreamDestroy(ctx->ce_stream[i]);
     for (int i = 0; i < 7; ++i)

@@ -78,6 +78,9 @@ struct ScheduleArgs {
     int bt;
     int stage;          // 1: group by digit locally before the remote copy
     int async_sync;     // 1: per-pass exchanges complete on mbarriers (data driven), 0: cluster barriers
+    SortElem *runs_out; // run mode: every cluster orders its own 16384-slot stretch of the queue and leaves the ordered
+                        // elements here (no admission); NULL otherwise
+    const SortElem *sorted_in;  // admission-only kernel: the fully ordered elements
     int top_first;      // 1: order by bits 16..63 first, fix short runs of equal values locally (see the pass loop)
     int rank_per;       // >0: small queue, order by counting (see rank_order below) with this many elements per CTA
     uint32_t *status;
@@ -257,7 +260,11 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned lt_mask = (1u << lane) - 1u;
 
-    if (crank == 0 && tid == 0) {
+    // run mode: this cluster orders the slots [base, base + n_q) only
+    const long long base_slot = a.runs_out ? (long long)(blockIdx.x / csize) * ((long long)csize * per) : 0;
+    const long long left_q = (long long)a.n - base_slot;
+    const int n_q = a.runs_out ? (int)(left_q < 0 ? 0 : (left_q > (long long)csize * per ? (long long)csize * per : left_q)) : a.n;
+    if (crank == 0 && tid == 0 && !a.runs_out) {
         a.counts->n_admitted = 0;
         a.counts->tokens_granted = 0;
     }
@@ -268,12 +275,13 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
 
     // ---- load: key, slot, tokens wanted (prompt minus the matched prefix) ----------------------
     SortElem e[K];
-    const unsigned long long key0 = a.key[0];
+    const unsigned long long key0 = n_q > 0 ? a.key[base_slot] : 0ull;
     unsigned long long diff = 0;
     auto load_elem = [&](int k) {
         const int li = (warp * K + k) * 32 + lane;
-        const long long g = (long long)crank * per_rt + li;
-        if (li < per_rt && g < a.n) {
+        const long long gl = (long long)crank * per_rt + li;   // position inside this cluster's stretch
+        const long long g = base_slot + gl;                     // slot of the queue
+        if (li < per_rt && gl < n_q) {
             const unsigned long long key = a.key[g];
             const long long P = a.prompt[g], h0 = a.n0[g], h1 = a.n1[g], h2 = a.n2[g];
             long long want = 0;
@@ -544,7 +552,7 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         for (int k = 0; k < K; ++k) elems[(warp * K + k) * 32 + lane] = e[k];
         __syncthreads();
     }
-    const long long here_ll = (long long)a.n - (long long)crank * per;
+    const long long here_ll = (long long)n_q - (long long)crank * per;
     const int n_here = here_ll < 0 ? 0 : (here_ll > per ? per : (int)here_ll);   // real elements of this CTA
     bool tie = false, long_run = false;
 #pragma unroll
@@ -614,9 +622,81 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     if (dead && tid == 0) atomicOr(a.status, CASCADE_ST_ETIMEOUT);
     }  // radix path
 
+    if (a.runs_out) {
+        // run mode: the ordered stretch goes to global memory (coalesced), the merge and the admission follow in
+        // their own kernels
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const long long gl = (long long)crank * per + (warp * K + k) * 32 + lane;
+            if (gl < n_q) a.runs_out[base_slot + gl] = e[k];
+        }
+        return;
+    }
     admit_and_write<T, K>(a, e, per_rt, cluster, wtmp, reinterpret_cast<int *>(base), exall);
     // every remote store of this kernel is followed by a cluster barrier and nothing reads remote
     // shared memory, so a CTA may leave as soon as it is done
+}
+
+// ---- queues beyond 32768 requests: ordered runs of 16384, merged by rank, then admission ---------------------
+// One cluster cannot hold more than 16 x 4096 elements and its radix passes slow down with the elements per
+// thread (6.2 us per pass at 65536 against 2.3 us at 16384).  Larger queues are cut into stretches of 16384 slots;
+// one cluster per stretch orders it with the kernel above (all stretches at the same time), every element then
+// finds its place among all elements as its position in its own run plus the number of keys below it in the
+// other runs (binary searches through L2; runs in front count equal keys too: stable by slot), and one
+// cluster reads the merged order back for the admission scans.
+constexpr int kRunLen = 16384;
+
+__global__ void __launch_bounds__(256) merge_runs_kernel(const SortElem *__restrict__ runs, SortElem *__restrict__ sorted,
+                                                         int n) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const SortElem me = runs[i];
+    const int r = i / kRunLen;
+    int pos = i - r * kRunLen;
+    const int n_runs = (n + kRunLen - 1) / kRunLen;
+    for (int q = 0; q < n_runs; ++q) {
+        if (q == r) continue;
+        const SortElem *list = runs + (size_t)q * kRunLen;
+        int len = min(kRunLen, n - q * kRunLen), lo = 0;
+        const bool ties = q < r;
+        while (len > 0) {
+            const int half = len >> 1;
+            const unsigned long long v = list[lo + half].key;
+            const bool below = ties ? v <= me.key : v < me.key;
+            lo = below ? lo + half + 1 : lo;
+            len = below ? len - half - 1 : half;
+        }
+        pos += lo;
+    }
+    sorted[pos] = me;
+}
+
+template <int T, int K>
+__global__ void __launch_bounds__(T, 1) admit_kernel(const __grid_constant__ ScheduleArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
+    constexpr int per = T * K;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned crank = cluster.block_rank();
+    __shared__ long long wtmp[3 * 32];
+    __shared__ int itmp[32];
+    __shared__ Exch exall[kMaxCluster];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (crank == 0 && tid == 0) {
+        a.counts->n_admitted = 0;
+        a.counts->tokens_granted = 0;
+    }
+    SortElem e[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const long long g = (long long)crank * per + (warp * K + k) * 32 + lane;
+        if (g < a.n) e[k] = a.sorted_in[g];
+        else { e[k].key = ~0ull; e[k].idx = 0xffffffffu; e[k].want = 0; }
+    }
+    cluster.sync();   // the counts are zero and every CTA has started before anybody writes to a neighbour
+    admit_and_write<T, K>(a, e, per, cluster, wtmp, itmp, exall);
 }
 
 // ---- merge-rank ordering: queues that fit one CTA's shared memory as bare keys (up to 16384) -------------
@@ -848,7 +928,7 @@ size_t smem_bytes(int T, int K) {
 }
 
 template <int T, int K>
-cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, bool pdl, cudaStream_t stream) {
+cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, bool pdl, cudaStream_t stream, int n_clusters = 1) {
     static bool configured_dev[64] = {};
     bool unknown = false;
     bool &configured = (device >= 0 && device < 64) ? configured_dev[device] : unknown;
@@ -861,7 +941,7 @@ cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, bool pdl
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), smem, stream, schedule_kernel<T, K>, a);
+    return cascade_launch(pdl, cluster_size, dim3(cluster_size * n_clusters), dim3(T), smem, stream, schedule_kernel<T, K>, a);
 }
 
 size_t merge_smem_bytes(int T, int K) {
@@ -980,6 +1060,28 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
         }
     }
     a.status = ctx->status_dev;
+    a.runs_out = nullptr;
+    a.sorted_in = nullptr;
+    if (ctx->sort_runs && ctx->multi_sort && n > (ctx->multi_sort == 2 ? kRunLen : 2 * kRunLen)) {
+        // stretches of 16384 slots ordered by one cluster each, merged by rank, admission by one cluster
+        const int n_runs = (n + kRunLen - 1) / kRunLen;
+        ScheduleArgs r = a;
+        r.runs_out = reinterpret_cast<SortElem *>(ctx->sort_runs);
+        r.stage = ctx->sort_stage >= 0 ? ctx->sort_stage : 1;
+        CASCADE_CUDA_TRY(ctx, (launch<256, 4>(r, 16, ctx->device, ctx->pdl, s, n_runs)));
+        SortElem *sorted = reinterpret_cast<SortElem *>(ctx->sort_sorted);
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((n + 255) / 256), dim3(256), 0, s, merge_runs_kernel,
+                                             (const SortElem *)r.runs_out, sorted, n));
+        ScheduleArgs c = a;
+        c.sorted_in = sorted;
+        static bool configured_dev[64] = {};
+        if (ctx->device < 0 || ctx->device >= 64 || !configured_dev[ctx->device]) {
+            CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(admit_kernel<512, 8>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+            if (ctx->device >= 0 && ctx->device < 64) configured_dev[ctx->device] = true;
+        }
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 16, dim3(16), dim3(512), 0, s, admit_kernel<512, 8>, c));
+        return CASCADE_OK;
+    }
     // queues beyond the counting path whose bare keys fit one CTA's shared memory: local order + merge by rank
     // (measured: a gain while every thread holds one element, i.e. up to 4096 requests; beyond that the searches
     // cost more than the exchanges they save, unless CASCADE_MERGE_SORT=2 forces it)

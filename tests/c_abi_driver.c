@@ -3,6 +3,8 @@
  * only, no Python, no PyTorch).  Reads a little-endian input file written by tests/test_gpu_c_abi.py,
  * runs budget -> schedule -> tier plan -> evict -> restore on the default stream and writes every output
  * to a second file.  Exit code 0 on success, otherwise the line number of the failing call.
+ * Optional third argument: "step" issues the whole iteration as ONE cascade_step call (with the fused move),
+ * "staged" moves the blocks through the copy engines (cascade_kv_move_staged) after the three plan calls.
  *
  * Input file:  int64 header[16] = { n, maxb, n_hbm, n_host, n_chunks, chunk_bytes, hbm_free_count,
  *              host_free_count, now_ns, D_act, K_act, sizeof(cascade_params), 0... }, then the parameter
@@ -42,7 +44,9 @@ static int write_back(FILE *f, const void *dev, size_t bytes) {
 }
 
 int main(int argc, char **argv) {
-    CHECK(argc == 3);
+    CHECK(argc == 3 || argc == 4);
+    const int use_step = argc == 4 && strcmp(argv[3], "step") == 0;
+    const int use_staged = argc == 4 && strcmp(argv[3], "staged") == 0;
     FILE *in = fopen(argv[1], "rb");
     CHECK(in);
     int64_t hd[16];
@@ -137,13 +141,51 @@ int main(int argc, char **argv) {
 
     cascade_ctx *ctx = NULL;
     CHECK(cascade_create(&ctx, &params, n, 0) == CASCADE_OK);
-    CHECK(cascade_budget(ctx, &r, n, now_ns, D_act, K_act, budget, key, NULL) == CASCADE_OK);
-    CHECK(cascade_schedule(ctx, &r, key, n, D_act, order, grant, sc, NULL) == CASCADE_OK);
-    CHECK(cascade_tier_plan(ctx, &r, budget, order, grant, n, D_act, K_act, &pools, &plan, NULL) == CASCADE_OK);
-    CHECK(cascade_kv_evict(ctx, &lay, hbm_pool, host_pool, n_host, 0, plan.evict_src, plan.evict_dst,
-                           &plan.counts->n_evict, plan.evict_cap, NULL) == CASCADE_OK);
-    CHECK(cascade_kv_restore(ctx, &lay, hbm_pool, host_pool, n_host, 0, plan.restore_src, plan.restore_dst,
-                             &plan.counts->n_restore, plan.restore_cap, NULL) == CASCADE_OK);
+    if (use_step) {
+        const int64_t words = cascade_kv_move_scratch_len(plan.evict_cap, plan.restore_cap);
+        CHECK(words > 0);
+        cascade_step_args a;
+        memset(&a, 0, sizeof a);
+        a.reqs = &r;
+        a.n = n;
+        a.D_act = D_act;
+        a.K_act = K_act;
+        a.now_ns = now_ns;
+        a.budget = budget;
+        a.key = key;
+        a.order = order;
+        a.grant = grant;
+        a.sched_counts = sc;
+        a.pools = &pools;
+        a.plan = &plan;
+        a.layout = &lay;
+        a.hbm_pool = hbm_pool;
+        a.host_pool = host_pool;
+        a.host_blocks = n_host;
+        a.move_scratch = (int32_t *)to_device(NULL, (size_t)words * 4);
+        CHECK(a.move_scratch);
+        CHECK(cascade_step(ctx, &a, NULL) == CASCADE_OK);
+    } else {
+        CHECK(cascade_budget(ctx, &r, n, now_ns, D_act, K_act, budget, key, NULL) == CASCADE_OK);
+        CHECK(cascade_schedule(ctx, &r, key, n, D_act, order, grant, sc, NULL) == CASCADE_OK);
+        CHECK(cascade_tier_plan(ctx, &r, budget, order, grant, n, D_act, K_act, &pools, &plan, NULL) == CASCADE_OK);
+        if (use_staged) {
+            const int64_t words = cascade_kv_mailbox_len(plan.evict_cap, plan.restore_cap);
+            const int64_t staging_blocks = 24;                 /* smaller than the lists: the batches wrap */
+            int32_t *mailbox = NULL;
+            void *staging = to_device(NULL, (size_t)(staging_blocks * bb));
+            CHECK(words > 0 && staging && cudaHostAlloc((void **)&mailbox, (size_t)words * 4, cudaHostAllocMapped) == cudaSuccess);
+            CHECK(cascade_kv_move_staged(ctx, &lay, hbm_pool, host_pool, n_host, plan.evict_src, plan.evict_dst,
+                                         &plan.counts->n_evict, plan.evict_cap, plan.restore_src, plan.restore_dst,
+                                         &plan.counts->n_restore, plan.restore_cap, staging, staging_blocks, mailbox,
+                                         NULL) == CASCADE_OK);
+        } else {
+            CHECK(cascade_kv_evict(ctx, &lay, hbm_pool, host_pool, n_host, 0, plan.evict_src, plan.evict_dst,
+                                   &plan.counts->n_evict, plan.evict_cap, NULL) == CASCADE_OK);
+            CHECK(cascade_kv_restore(ctx, &lay, hbm_pool, host_pool, n_host, 0, plan.restore_src, plan.restore_dst,
+                                     &plan.counts->n_restore, plan.restore_cap, NULL) == CASCADE_OK);
+        }
+    }
     cascade_status_t st;
     CHECK(cascade_status(ctx, &st, 1, NULL) == CASCADE_OK);
 

@@ -1,6 +1,6 @@
 """The library used from plain C: tests/c_abi_driver.c is compiled with gcc against the header and the CUDA
-runtime, runs one whole iteration without Python or PyTorch in the process, and its outputs are compared
-with the oracle's."""
+runtime, runs one whole iteration without Python or PyTorch in the process (as the five calls, as one cascade_step call, or
+with the copy-engine move), and its outputs are compared with the oracle's."""
 import ctypes
 import os
 import subprocess
@@ -29,8 +29,8 @@ def _compile(tmp_path):
     return exe
 
 
-@pytest.mark.parametrize("seed", [0, 3])
-def test_one_iteration_from_plain_c(tmp_path, seed):
+@pytest.mark.parametrize("seed,mode", [(0, "calls"), (3, "calls"), (0, "step"), (3, "staged")])
+def test_one_iteration_from_plain_c(tmp_path, seed, mode):
     w = wl.config_tiny(seed, hbm_free_target=60)
     w.params["ttft_ns"] = [20 * t for t in w.params["ttft_ns"]]
     lay, bb = w.layout, w.block_bytes
@@ -51,7 +51,8 @@ def test_one_iteration_from_plain_c(tmp_path, seed):
         for a in (w.hbm_tbl, w.host_tbl, w.hbm_free, w.host_free, hbm, host):
             f.write(np.ascontiguousarray(a).tobytes())
     exe = _compile(tmp_path)
-    subprocess.check_call([str(exe), str(tmp_path / "in.bin"), str(tmp_path / "out.bin")])
+    subprocess.check_call([str(exe), str(tmp_path / "in.bin"), str(tmp_path / "out.bin")] +
+                          ([] if mode == "calls" else [mode]))
 
     ref = oracle_iteration(w)
     plan, pools = ref["plan"], ref["pools"]

@@ -51,6 +51,27 @@ def test_host_validation_without_a_device():
         assert lib.cascade_create(ctypes.byref(h), ctypes.byref(q), 16, 0) == cs.ERANGE, bad
     assert lib.cascade_budget(None, None, 0, 0, 0, 0, None, None, None) == cs.EINVAL
     assert lib.cascade_status(None, None, 0, None) == cs.EINVAL
+    assert lib.cascade_step(None, None, None) == cs.EINVAL
+    assert lib.cascade_kv_move(None, None, None, None, 0, None, None, None, 1, None, None, None, 1, None, None) == cs.EINVAL
+    assert lib.cascade_kv_move_staged(None, None, None, None, 0, None, None, None, 1, None, None, None, 1, None, 4, None,
+                                      None) == cs.EINVAL
+
+
+def test_scratch_and_mailbox_sizes_are_plain_host_arithmetic():
+    """The two size helpers need no device: restore results + restore matches + evict counters + a hash table of at
+    most half-full power-of-two size for the move; two counts + four lists for the mailbox."""
+    from paper_2608_06557_b200 import cascade as cs
+    assert cs.kv_move_scratch_len(0, 0) == 2 * 64
+    assert cs.kv_move_scratch_len(10, 7) == 2 * 7 + 10 + 2 * 64
+    assert cs.kv_move_scratch_len(33, 0) == 33 + 2 * 128            # 66 slots needed -> 128
+    assert cs.kv_move_scratch_len(19073, 28610) == 2 * 28610 + 19073 + 2 * 65536
+    assert cs.kv_move_scratch_len(-1, 0) == -1 and cs.kv_mailbox_len(0, -5) == -1
+    assert cs.kv_mailbox_len(0, 0) == 2 and cs.kv_mailbox_len(5, 9) == 2 + 10 + 18
+    prev = 0
+    for ne in range(0, 3000, 37):
+        cur = cs.kv_move_scratch_len(ne, 11)
+        assert cur >= prev and cur >= 2 * 11 + ne + 4 * ne           # room for a table no more than half full
+        prev = cur
 
 
 def test_header_is_plain_c_and_the_binding_mirrors_its_struct_layouts(tmp_path):

@@ -768,7 +768,7 @@ def ours_main(args):
 
     if rank == 0:
         # ---- end to end: inputs start in pinned host memory, results are read back every step -------
-        e2e = run_e2e(torch, args, batches[W:], insts[0], K)
+        e2e = run_e2e(torch, args, batches[W:], insts[:2] if len(insts) > 1 else [insts[0], insts[0]], K)
         line["config"] = workload_config(args)
         line["run"] = dict(blocks_restored_per_step=float(n_restore.mean()), blocks_evicted_per_step=float(n_evict.mean()),
                            host_pool_bytes=int(host_pool.numel()), hbm_pool_bytes=int(hbm_pool.numel()),
@@ -850,10 +850,11 @@ def load_hbm_peak():
 FUSED_MOVE = [True]
 
 
-def run_e2e(torch, args, batches, inst, K):
+def run_e2e(torch, args, batches, two, K):
     """The same metric through the public API with HOST inputs: every step copies that step's request
-    arrays, block tables and free lists from pinned host memory, runs the five calls and reads the
-    per-request results and counts back to the host."""
+    arrays, block tables and free lists from pinned host memory, runs the calls and reads the per-request
+    results and counts back to the host, which waits for them before it goes on.  Two sets of device buffers
+    (`two`) alternate, so the inputs of step i+1 travel on a second stream while step i runs."""
     keys_req = ("arrival_ns", "prompt", "pred_out", "n0", "n1", "n2", "id", "cls", "flags")
     pinned = []
     for w in batches[:K]:
@@ -865,7 +866,7 @@ def run_e2e(torch, args, batches, inst, K):
         p["host_free"] = torch.from_numpy(w.host_free).pin_memory()
         p["counts"] = torch.tensor([w.hbm_free_count, w.host_free_count], dtype=torch.int32).pin_memory()
         pinned.append((w, p))
-    n = inst.n
+    n = two[0].n
     out_host = dict(grant=torch.empty(n, dtype=torch.int32, pin_memory=True),
                     x1=torch.empty(n, dtype=torch.int32, pin_memory=True),
                     x2=torch.empty(n, dtype=torch.int32, pin_memory=True),
@@ -874,43 +875,71 @@ def run_e2e(torch, args, batches, inst, K):
                     counts=torch.empty(12, dtype=torch.int32, pin_memory=True))
     h2d = sum(t.numel() * t.element_size() for t in pinned[0][1].values())
     d2h = sum(t.numel() * t.element_size() for t in out_host.values())
-    free_counts = torch.empty(2, dtype=torch.int32, device=inst.device)
-    moved = 0
+    main, up = torch.cuda.current_stream(), torch.cuda.Stream()
+    uploaded = [torch.cuda.Event(), torch.cuda.Event()]
+    finished = [torch.cuda.Event(), torch.cuda.Event()]
+    free_counts = [torch.empty(2, dtype=torch.int32, device=two[0].device) for _ in range(2)]
 
-    def step(w, p):
-        for k in keys_req:
-            dst = inst.reqs[k][:n]
-            dst.view(torch.int32).copy_(p[k], non_blocking=True) if dst.dtype == torch.uint32 else \
-                dst.copy_(p[k], non_blocking=True)
-        inst.hbm_tbl.copy_(p["hbm_tbl"], non_blocking=True)
-        inst.host_tbl.copy_(p["host_tbl"], non_blocking=True)
-        inst.hbm_free.copy_(p["hbm_free"], non_blocking=True)
-        inst.host_free.copy_(p["host_free"], non_blocking=True)
-        free_counts.copy_(p["counts"], non_blocking=True)
-        inst.hbm_free_count.copy_(free_counts[0:1], non_blocking=True)
-        inst.host_free_count.copy_(free_counts[1:2], non_blocking=True)
+    def upload(j, w, p):
+        inst = two[j % 2]
+        if j >= 2:
+            up.wait_event(finished[j % 2])          # the step that last used these buffers is over
+        with torch.cuda.stream(up):
+            for k in keys_req:
+                dst = inst.reqs[k][:n]
+                dst.view(torch.int32).copy_(p[k], non_blocking=True) if dst.dtype == torch.uint32 else \
+                    dst.copy_(p[k], non_blocking=True)
+            inst.hbm_tbl.copy_(p["hbm_tbl"], non_blocking=True)
+            inst.host_tbl.copy_(p["host_tbl"], non_blocking=True)
+            inst.hbm_free.copy_(p["hbm_free"], non_blocking=True)
+            inst.host_free.copy_(p["host_free"], non_blocking=True)
+            free_counts[j % 2].copy_(p["counts"], non_blocking=True)
+            inst.hbm_free_count.copy_(free_counts[j % 2][0:1], non_blocking=True)
+            inst.host_free_count.copy_(free_counts[j % 2][1:2], non_blocking=True)
+            uploaded[j % 2].record(up)
+
+    step_args = [inst.step_args(with_move=True) if FUSED_MOVE[0] else None for inst in two]
+
+    def enqueue(j, w):
+        inst = two[j % 2]
+        main.wait_event(uploaded[j % 2])
         inst.set_clock(w.now_ns, w.D_act, w.K_act)
-        inst.run_iteration(fused_move=FUSED_MOVE[0])
+        if FUSED_MOVE[0]:
+            inst.run_step(step_args[j % 2])         # the whole iteration as one call of the C ABI
+        else:
+            inst.run_iteration(fused_move=False)
         out_host["grant"].copy_(inst.grant[:n], non_blocking=True)
         out_host["x1"].copy_(inst.x1[:n], non_blocking=True)
         out_host["x2"].copy_(inst.x2[:n], non_blocking=True)
         out_host["tokens_run"].copy_(inst.tokens_run[:n], non_blocking=True)
         out_host["action"].copy_(inst.action[:n], non_blocking=True)
         out_host["counts"].copy_(inst.plan_counts, non_blocking=True)
-        torch.cuda.synchronize()       # the caller needs the plan before it can build the next batch
+        finished[j % 2].record(main)
+
+    def finish():
+        main.synchronize()                          # the caller needs the plan before it goes on
         return int(out_host["counts"][0]) + int(out_host["counts"][1])
 
-    step(*pinned[0])                    # untimed warm-up of the code path
+    upload(0, *pinned[0])                           # untimed warm-up of the code path
+    enqueue(0, pinned[0][0])
+    finish()
     torch.cuda.synchronize()
+    moved = 0
     a, b = event_pair(torch)
     a.record()
-    for w, p in pinned:
-        moved += step(w, p) * inst.block_bytes
+    upload(0, *pinned[0])
+    for j, (w, p) in enumerate(pinned):
+        enqueue(j, w)
+        if j + 1 < len(pinned):
+            upload(j + 1, *pinned[j + 1])           # queued behind nothing: it runs beside step j
+        moved += finish() * two[0].block_bytes
     b.record()
     torch.cuda.synchronize()
     ms = a.elapsed_time(b)
     return dict(value=round(moved / (ms * 1e-3) / GB, 3), unit="GB/s", h2d_bytes_per_step=int(h2d),
-                d2h_bytes_per_step=int(d2h), ms_per_step=round(ms / len(pinned), 4))
+                d2h_bytes_per_step=int(d2h), ms_per_step=round(ms / len(pinned), 4),
+                note="inputs of step i+1 are uploaded on a second stream while step i runs; the host waits for "
+                     "every step's results")
 
 
 # --------------------------------------------------------------------------------------------

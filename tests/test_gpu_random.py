@@ -78,7 +78,7 @@ def test_fused_move_on_random_shapes():
     assert ctx.status()[0] == 0
 
 
-@pytest.mark.parametrize("n,reps", [(1024, 400), (2048, 200), (16384, 200), (65536, 40)])
+@pytest.mark.parametrize("n,reps", [(1024, 400), (2048, 200), (4096, 200), (16384, 200), (40000, 40), (65536, 40)])
 def test_repeated_runs_give_identical_results(n, reps):
     """The cluster kernels exchange data through shared memory of other CTAs; an ordering bug there would show
     as results that change from run to run.  Same inputs, many runs, every output compared with the first."""

@@ -668,7 +668,8 @@ def ours_main(args):
     # one pinned allocation: the copy sweep's pool as stated (100 * 10^9 bytes, or what the box grants); the step
     # uses its first --host-gb
     want_sweep = 0 if args.no_sweeps or rank != 0 else int(args.host_sweep_gb * GB) // bb * bb
-    big_pool, big_bytes = alloc_pinned_pool(max(want_sweep, w0.host_blocks * bb))
+    # every rank of a multi-replica run pins its own pool on the same host: each takes its share of what is available
+    big_pool, big_bytes = alloc_pinned_pool(max(want_sweep, w0.host_blocks * bb), share_of_available=0.7 / max(world, 1))
     if big_bytes < w0.host_blocks * bb:        # pinning was refused at full size: regenerate at the size we got
         args.host_gb = big_bytes / GB
         batches = [make_batch(args, rank_seed(rank, s)) for s in range(W + K)]

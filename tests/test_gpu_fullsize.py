@@ -70,7 +70,10 @@ def test_bench_step_at_full_size(pools, seed):
     probe = np.sort(rng.choice(w.host_blocks, size=512, replace=False))
     host_before = host_record(inst.host_pool, t(probe), BB).view(torch.int64).sum(dim=1).numpy()
 
-    inst.run_iteration()
+    if seed == 14:
+        inst.run_step(inst.step_args(with_move=True))     # as bench.py times it: one call, evict + restore as the fused move
+    else:
+        inst.run_iteration()                              # the five calls, evict then restore
     got = inst.fetch()
 
     # scheduling and plan outputs in full

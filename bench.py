@@ -611,6 +611,17 @@ def schedule_sweep(torch, cs):
             if it >= 3:
                 one.append(a.elapsed_time(b) * 1e3)
         one.sort()
+        plain_args = inst.step_args()
+        one_plain = []
+        for it in range(103):
+            a, b = event_pair(torch)
+            a.record()
+            inst.run_step(plain_args)
+            b.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                one_plain.append(a.elapsed_time(b) * 1e3)
+        one_plain.sort()
         # the same iteration (last staged update) captured in a graph: device time without the Python launches
         g2 = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g2, stream=st):
@@ -632,6 +643,8 @@ def schedule_sweep(torch, cs):
                            graph_with_slot_update_us=round(statistics.median(tg), 1),
                            with_slot_update_us=round(statistics.median(upd), 1),
                            with_slot_update_p99_us=round(upd[int(0.99 * (len(upd) - 1))], 1),
+                           one_call_us=round(statistics.median(one_plain), 1),
+                           one_call_p99_us=round(one_plain[int(0.99 * (len(one_plain) - 1))], 1),
                            one_call_with_slot_update_us=round(statistics.median(one), 1),
                            one_call_with_slot_update_p99_us=round(one[int(0.99 * (len(one) - 1))], 1),
                            slot_update_bytes=upd_bytes)
@@ -827,6 +840,8 @@ def ours_main(args):
                                                       one_block_latency_us=small["restore_hbm_1"]["us"]),
                 budget_schedule_plan_16k_us=dict(target=100.0, measured=sl["16384"]["graph_us"],
                                                  launched_from_python=sl["16384"]["launched_us"],
+                                                 one_call=sl["16384"]["one_call_us"],
+                                                 one_call_p99=sl["16384"]["one_call_p99_us"],
                                                  one_call_with_slot_update=sl["16384"]["one_call_with_slot_update_us"],
                                                  one_call_with_slot_update_p99=sl["16384"]["one_call_with_slot_update_p99_us"]),
                 parity="bit-exact against the CPU oracle: see tests/ (-m gpu)")

@@ -151,9 +151,9 @@ __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant
 // loads are issued before the first wait (short calls live off this); afterwards S - 2 loads are kept in
 // flight ahead of the piece being stored, so that the slot refilled next was last read by the store issued
 // one step EARLIER, which has long finished reading shared memory (with S - 1 in flight the refill would
-// wait for the store just issued: measured 6.2 instead of 6.55 TB/s through the staging buffer).  Every wait is bounded: when the clock limit is
-// hit the CTA records CASCADE_ST_ETIMEOUT, issues nothing more, waits (bounded again) for the loads it
-// still has in flight, drains its store groups and returns.
+// wait for the store just issued: measured 6.2 instead of 6.55 TB/s through the staging buffer).  Every
+// wait is bounded: when the clock limit is hit the CTA records CASCADE_ST_ETIMEOUT, issues nothing more,
+// waits (bounded again) for the loads it still has in flight, drains its store groups and returns.
 //
 // The same loop serves four roles:
 //   kRoleRestore / kRoleEvict          the two plain copies;

@@ -412,8 +412,9 @@ int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, void *hbm_po
  *                   int32; after the call: [0] eviction count, [1] restore count, then the four lists
  * Faster than the zero-copy kernels for blocks of a megabyte and more (the copy engines move 55 - 57 GB/s per
  * direction and 96 - 100 GB/s both ways on a PCIe Gen5 x16 link), slower for small blocks (a few microseconds
- * of host and engine work per copy).  Meant for up to about a thousand blocks per direction and call: beyond that
- * the host is made to wait while it queues the copies and the two directions stop overlapping (still correct).
+ * of host and engine work per copy).  With a staging buffer that holds both lists the drains and the fills are
+ * queued alternately, so both directions stay busy however long the lists are; with a smaller one the lists are
+ * worked off one after the other in batches that wait for space (correct, slower).
  * Cannot be captured in a CUDA graph (host synchronisation).
  * Errors: as cascade_kv_move, plus CASCADE_ENOMEM (host bookkeeping could not grow).  Ids outside a pool:
  * that pair is skipped, CASCADE_ST_EBOUNDS.

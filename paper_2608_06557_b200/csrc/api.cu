@@ -77,8 +77,6 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->move_ctas = e ? atoi(e) : 0;
     e = getenv("CASCADE_MOVE_VECTOR");
     ctx->move_vector = e ? (atoi(e) & 3) : 1;   // measured: bulk reads of the restore grid starve beside the evict grid's bulk writes
-    e = getenv("CASCADE_CE_HYBRID");
-    ctx->ce_hybrid = e ? atoi(e) : 0;
     e = getenv("CASCADE_CE_LANES");
     ctx->ce_lanes = e && atoi(e) == 2 ? 2 : 1;   // measured: a second stream per direction gains nothing
     e = getenv("CASCADE_COPY_AHEAD_SUB");

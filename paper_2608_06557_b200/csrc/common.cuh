@@ -48,7 +48,6 @@ struct cascade_ctx {
     cudaStream_t ce_stream[4];   // [0], [1] host -> staging (restores); [2], [3] staging -> host (evictions)
     cudaEvent_t ce_event[7];     // lists published, gather done, scatter done, fill done x2, drain done x2
     int ce_lanes;                // side streams used per direction (1 | 2)
-    int ce_hybrid;               // 1: evictions by the zero-copy kernel, only the restores through the copy engines
     unsigned long long *ce_bitmap;   // host-side: one bit per host record, grown on demand
     size_t ce_bitmap_words;
     int test_move_stall;         // test hooks (CASCADE_TEST_MOVE_STALL): 1 = the evict side of the fused move never

@@ -744,25 +744,101 @@ extern "C" int cascade_kv_move_staged(cascade_ctx *ctx, const cascade_kv_layout 
     }
 
     // 3. staging regions: one per direction, in proportion to the lists
-    const bool hybrid = ctx->ce_hybrid == 1;
-    const bool hybrid_r = ctx->ce_hybrid == 2;   // restores by the zero-copy kernel, evictions through the copy engines
-    long long region_e = (ne == 0 || hybrid) ? 0 : (nr == 0 ? staging_blocks : staging_blocks * ne / ((long long)ne + nr));
-    if (ne > 0 && !hybrid && region_e < 1) region_e = 1;
+    long long region_e = ne == 0 ? 0 : (nr == 0 ? staging_blocks : staging_blocks * ne / ((long long)ne + nr));
+    if (ne > 0 && region_e < 1) region_e = 1;
     if (nr > 0 && region_e > staging_blocks - 1) region_e = staging_blocks - 1;
     const long long region_r = staging_blocks - region_e;
     char *stage_e = (char *)staging, *stage_r = (char *)staging + region_e * bb;
 
-    // 4. evictions: gather batch -> drain batch; a region position is reused only after its drain
+    // Helpers: one batch of drains / fills (one cudaMemcpyAsync per run of consecutive host records, pairs with an
+    // id outside its pool left out; the gather / scatter kernel sets the status bit for them).
     bool drained_any = false;
-    {
-        if (hybrid && ne > 0) {
-            rc = launch_copy<false>(ctx, hbm, (char *)hbm_pool, (char *)host_pool, host_blocks, 0, evict_src, evict_dst,
-                                    n_evict_dev, n_evict_max, s);
-            if (rc != CASCADE_OK) return rc;
+    int lane_e = 0, lane_r = 0;
+    auto drain_batch = [&](int off, int m, long long pos) -> int {
+        for (int i = 0; i < m;) {
+            const long long rec = h_ed[off + i], pg = h_es[off + i];
+            if (rec < 0 || rec >= host_blocks || pg < 0 || pg >= paged_blocks) {
+                i += 1;
+                continue;
+            }
+            int run = 1;
+            while (i + run < m && h_ed[off + i + run] == rec + run && rec + run < host_blocks &&
+                   h_es[off + i + run] >= 0 && h_es[off + i + run] < paged_blocks)
+                ++run;
+            CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync((char *)host_pool + rec * bb, stage_e + (pos + i) * bb,
+                                                  (size_t)run * bb, cudaMemcpyDeviceToHost, s_drain[lane_e]));
+            lane_e = (lane_e + 1) % L;
+            i += run;
         }
+        for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_drain[k], s_drain[k]));
+        drained_any = true;
+        return CASCADE_OK;
+    };
+    auto fill_batch = [&](int off, int m, long long pos) -> int {
+        for (int i = 0; i < m;) {
+            const long long rec = h_rs[off + i], pg = h_rd[off + i];
+            if (rec < 0 || rec >= host_blocks || pg < 0 || pg >= paged_blocks) {
+                i += 1;
+                continue;
+            }
+            int run = 1;
+            while (i + run < m && h_rs[off + i + run] == rec + run && rec + run < host_blocks &&
+                   h_rd[off + i + run] >= 0 && h_rd[off + i + run] < paged_blocks)
+                ++run;
+            CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync(stage_r + (pos + i) * bb, (const char *)host_pool + rec * bb,
+                                                  (size_t)run * bb, cudaMemcpyHostToDevice, s_fill[lane_r]));
+            lane_r = (lane_r + 1) % L;
+            i += run;
+        }
+        return CASCADE_OK;
+    };
+    // the fills follow everything issued earlier on the caller's stream: an earlier call's scatter may still read the
+    // staging region, an earlier kernel may still write the host records read here
+    for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_lists, 0));
+
+    if (region_e >= ne && region_r >= nr && !fill_after_drain) {
+        // 4a. Both lists fit their regions: drains and fills are queued ALTERNATELY, batch by batch, so that neither side
+        // stream runs dry while the host waits for room in the other one's queue (the driver makes the host wait once a
+        // stream holds about a thousand pending operations).  One scatter over all restores follows every gather.
+        int off_e = 0, off_r = 0, batch = kFirstBatch;
+        while (off_e < ne || off_r < nr) {
+            if (off_e < ne) {
+                const int m = ne - off_e < batch ? ne - off_e : batch;
+                rc = launch_staged_pass<false>(ctx, hbm, (char *)hbm_pool, stage_e + (long long)off_e * bb, evict_src + off_e,
+                                               evict_dst + off_e, host_blocks, m, s);
+                if (rc != CASCADE_OK) return rc;
+                CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_gather, s));
+                for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_drain[k], ev_gather, 0));
+                rc = drain_batch(off_e, m, off_e);
+                if (rc != CASCADE_OK) return rc;
+                off_e += m;
+            }
+            if (off_r < nr) {
+                // fills in step with the drains: both lists are through their queues at about the same time
+                long long m = ne > 0 ? ((long long)batch * nr + ne - 1) / ne : batch;
+                m = m < 1 ? 1 : (m > nr - off_r ? nr - off_r : m);
+                rc = fill_batch(off_r, (int)m, off_r);
+                if (rc != CASCADE_OK) return rc;
+                off_r += (int)m;
+            }
+            batch = kBatch;
+        }
+        if (nr > 0) {
+            for (int k = 0; k < L; ++k) {
+                CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_fill[k], s_fill[k]));
+                CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ev_fill[k], 0));
+            }
+            rc = launch_staged_pass<true>(ctx, hbm, (char *)hbm_pool, stage_r, restore_dst, restore_src, host_blocks, nr, s);
+            if (rc != CASCADE_OK) return rc;
+            CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_scatter, s));
+        }
+    } else {
+    // 4b. A staging buffer smaller than the lists (or fills that must wait for drains): the two lists one after the
+    // other in the host's program, each batch reusing its region only after the batch before has left it.
+    {
         long long pos = 0;
-        int batch = kFirstBatch, lane = 0;
-        for (int off = 0; off < (hybrid ? 0 : ne);) {
+        int batch = kFirstBatch;
+        for (int off = 0; off < ne;) {
             int m = ne - off < batch ? ne - off : batch;
             if (m > region_e) m = (int)region_e;
             if (pos + m > region_e) {   // wrap: everything drained so far must have left the region
@@ -775,53 +851,22 @@ extern "C" int cascade_kv_move_staged(cascade_ctx *ctx, const cascade_kv_layout 
             if (rc != CASCADE_OK) return rc;
             CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_gather, s));
             for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_drain[k], ev_gather, 0));
-            for (int i = 0; i < m;) {
-                const long long rec = h_ed[off + i], pg = h_es[off + i];
-                if (rec < 0 || rec >= host_blocks || pg < 0 || pg >= paged_blocks) {
-                    i += 1;   // an id outside its pool: that pair is skipped (the gather kernel set the status bit)
-                    continue;
-                }
-                int run = 1;
-                while (i + run < m && h_ed[off + i + run] == rec + run && rec + run < host_blocks &&
-                       h_es[off + i + run] >= 0 && h_es[off + i + run] < paged_blocks)
-                    ++run;
-                CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync((char *)host_pool + rec * bb, stage_e + (pos + i) * bb,
-                                                      (size_t)run * bb, cudaMemcpyDeviceToHost, s_drain[lane]));
-                lane = (lane + 1) % L;
-                i += run;
-            }
-            for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_drain[k], s_drain[k]));
-            drained_any = true;
+            rc = drain_batch(off, m, pos);
+            if (rc != CASCADE_OK) return rc;
             pos += m;
             off += m;
             batch = kBatch;
         }
     }
-
-    // 5. restores: fill batch -> scatter batch (all scatters are behind all gathers on the caller's stream)
     {
         for (int k = 0; k < L; ++k) {
             if (fill_after_drain && drained_any)
                 for (int j = 0; j < L; ++j) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_drain[j], 0));
-            if (fill_after_drain && hybrid && ne > 0) {   // the zero-copy evictions are on the caller's stream
-                CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_gather, s));
-                CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_gather, 0));
-            }
-            // the fills follow everything issued earlier on the caller's stream: an earlier call's scatter may still
-            // read the staging region, an earlier kernel may still write the host records read here
-            CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_lists, 0));
-        }
-        if (hybrid_r && nr > 0) {
-            if (fill_after_drain && drained_any)
-                for (int j = 0; j < L; ++j) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ev_drain[j], 0));
-            rc = launch_copy<true>(ctx, hbm, (char *)hbm_pool, (char *)host_pool, host_blocks, 0, restore_src, restore_dst,
-                                   n_restore_dev, n_restore_max, s);
-            if (rc != CASCADE_OK) return rc;
         }
         long long pos = 0;
-        int batch = kFirstBatch, lane = 0;
+        int batch = kFirstBatch;
         bool scattered_any = false;
-        for (int off = 0; off < (hybrid_r ? 0 : nr);) {
+        for (int off = 0; off < nr;) {
             int m = nr - off < batch ? nr - off : batch;
             if (m > region_r) m = (int)region_r;
             if (pos + m > region_r) {
@@ -829,21 +874,8 @@ extern "C" int cascade_kv_move_staged(cascade_ctx *ctx, const cascade_kv_layout 
                 if (scattered_any)
                     for (int k = 0; k < L; ++k) CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s_fill[k], ev_scatter, 0));
             }
-            for (int i = 0; i < m;) {
-                const long long rec = h_rs[off + i], pg = h_rd[off + i];
-                if (rec < 0 || rec >= host_blocks || pg < 0 || pg >= paged_blocks) {
-                    i += 1;   // an id outside its pool: that pair is skipped (the scatter kernel sets the status bit)
-                    continue;
-                }
-                int run = 1;
-                while (i + run < m && h_rs[off + i + run] == rec + run && rec + run < host_blocks &&
-                       h_rd[off + i + run] >= 0 && h_rd[off + i + run] < paged_blocks)
-                    ++run;
-                CASCADE_CUDA_TRY(ctx, cudaMemcpyAsync(stage_r + (pos + i) * bb, (const char *)host_pool + rec * bb,
-                                                      (size_t)run * bb, cudaMemcpyHostToDevice, s_fill[lane]));
-                lane = (lane + 1) % L;
-                i += run;
-            }
+            rc = fill_batch(off, m, pos);
+            if (rc != CASCADE_OK) return rc;
             for (int k = 0; k < L; ++k) {
                 CASCADE_CUDA_TRY(ctx, cudaEventRecord(ev_fill[k], s_fill[k]));
                 CASCADE_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ev_fill[k], 0));
@@ -857,6 +889,7 @@ extern "C" int cascade_kv_move_staged(cascade_ctx *ctx, const cascade_kv_layout 
             off += m;
             batch = kBatch;
         }
+    }
     }
     // 6. completion of the caller's stream implies that every host record has been written
     if (drained_any)

@@ -41,6 +41,7 @@ struct cascade_ctx {
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels
     void *sort_runs, *sort_sorted;   // queues beyond 32768 requests: the ordered runs and the merged order (16 B per request each)
     int multi_sort;              // 1: such queues are ordered as runs of 16384 by one cluster each, then merged by rank
+    int plan_prepare_min;        // queues above this size run the tier plan's per-request phase as a grid of its own
     int sort_top_first;          // 1: radix passes over bits 16..63 first, local fix-up of equal values (budget policy only)
     int merge_sort;              // 1: queues of up to 16384 requests beyond the counting path are ordered by local sort + merge by rank
     int rank_sort_max;           // queues up to this size are ordered by counting instead of radix passes

@@ -53,6 +53,7 @@ struct PlanArgs {
     int64_t A_act;
     int n;
     int with_tables;
+    int prepared;                      // 1: phase 1a was done by plan_prepare_kernel
 };
 
 // per-CTA totals published to every CTA of the cluster
@@ -69,6 +70,60 @@ struct __align__(16) Exch2 {
 struct __align__(16) Exch3 {
     int nv, freed, nev, pad;
 };
+
+// Phase 1a for one request (slot r): Eq. 7 bounds and the restore-vs-recompute choice; the per-request outputs
+// get their default values and one packed word (n0 | x1 << 14 | tokens_run << 28 | flags << 46) is left for
+// the schedule-order phases.  Returns the status bits it found.
+__device__ __forceinline__ uint32_t plan_prepare_one(const cascade_params &p, const PlanArgs &a, long long r) {
+    const int bt = p.bt;
+    uint32_t st = 0;
+    const long long P = a.prompt[r], n0 = a.n0[r], n1 = a.n1[r], n2 = a.n2[r];
+    const long long b = a.budget[r];
+    const int g = a.grant[r];
+    const unsigned rf = a.flags[r];
+    bool valid = dev_request_valid(bt, P, n0, n1, n2);
+    if (valid && a.with_tables) valid = (P + bt - 1) / bt <= a.pools.maxb;
+    unsigned long long w = (unsigned long long)kReal << 46;
+    int x1 = 0, x2 = 0, run = 0;
+    if (!valid) {
+        st |= CASCADE_ST_EPRECOND;
+        if (g != 0) a.grant[r] = 0;
+    } else {
+        unsigned f = kReal | kValid;
+        if (rf & CASCADE_FLAG_HBM_PRIVATE) f |= kPriv;
+        if (dev_restore_time(p, 1, n0) <= b) f |= kFits;
+        if (g > 0) {
+            int64_t bx1, bx2;
+            dev_choose_restore(p, a.A_act, P, n0, n1, n2, b, &bx1, &bx2);
+            // a deep fetch is staged first: nothing runs now, HBM is taken at the last hop only
+            const long long left = P - (n0 + bx1) * bt;
+            x1 = (int)bx1;
+            x2 = (int)bx2;
+            run = bx2 > 0 ? 0 : (int)(g < left ? g : left);
+            f |= kAdm;
+        }
+        w = (unsigned long long)n0 | ((unsigned long long)x1 << 14) | ((unsigned long long)run << 28) |
+            ((unsigned long long)f << 46);
+    }
+    a.pack[r] = w;
+    a.plan.x1[r] = x1;
+    a.plan.x2[r] = x2;
+    a.plan.tokens_run[r] = run;
+    a.plan.action[r] = (valid && n0 > 0) ? CASCADE_ACT_RETAIN : CASCADE_ACT_NONE;
+    return st;
+}
+
+// Phase 1a as a grid of its own, one thread per request: used for large queues, where the sixteen CTAs of the
+// cluster kernel would spend several microseconds on what the whole GPU does in one.
+__global__ void __launch_bounds__(256)
+plan_prepare_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ PlanArgs a) {
+    cascade_grid_wait();
+    cascade_grid_trigger();
+    const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t st = r < a.n ? plan_prepare_one(p, a, r) : 0u;
+    st = __reduce_or_sync(0xffffffffu, st);
+    if ((threadIdx.x & 31) == 0 && st) atomicOr(a.status, st);
+}
 
 template <int T, int K>
 __global__ void __launch_bounds__(T, 1)
@@ -106,43 +161,12 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     //      per-request outputs get their default values here and one packed word per request
     //      (n0 | x1 << 14 | tokens_run << 28 | flags << 46) is left for the schedule-order phases
     const long long pos0 = (long long)crank * per + (warp * K) * 32 + lane;
+    if (!a.prepared) {
 #pragma unroll
-    for (int k = 0; k < K; ++k) {
-        const long long r = pos0 + k * 32;
-        if (r >= n) continue;
-        const long long P = a.prompt[r], n0 = a.n0[r], n1 = a.n1[r], n2 = a.n2[r];
-        const long long b = a.budget[r];
-        const int g = a.grant[r];
-        const unsigned rf = a.flags[r];
-        bool valid = dev_request_valid(bt, P, n0, n1, n2);
-        if (valid && a.with_tables) valid = (P + bt - 1) / bt <= a.pools.maxb;
-        unsigned long long w = (unsigned long long)kReal << 46;
-        int x1 = 0, x2 = 0, run = 0;
-        if (!valid) {
-            st |= CASCADE_ST_EPRECOND;
-            if (g != 0) a.grant[r] = 0;
-        } else {
-            unsigned f = kReal | kValid;
-            if (rf & CASCADE_FLAG_HBM_PRIVATE) f |= kPriv;
-            if (dev_restore_time(p, 1, n0) <= b) f |= kFits;
-            if (g > 0) {
-                int64_t bx1, bx2;
-                dev_choose_restore(p, a.A_act, P, n0, n1, n2, b, &bx1, &bx2);
-                // a deep fetch is staged first: nothing runs now, HBM is taken at the last hop only
-                const long long left = P - (n0 + bx1) * bt;
-                x1 = (int)bx1;
-                x2 = (int)bx2;
-                run = bx2 > 0 ? 0 : (int)(g < left ? g : left);
-                f |= kAdm;
-            }
-            w = (unsigned long long)n0 | ((unsigned long long)x1 << 14) | ((unsigned long long)run << 28) |
-                ((unsigned long long)f << 46);
+        for (int k = 0; k < K; ++k) {
+            const long long r = pos0 + k * 32;
+            if (r < n) st |= plan_prepare_one(p, a, r);
         }
-        a.pack[r] = w;
-        a.plan.x1[r] = x1;
-        a.plan.x2[r] = x2;
-        a.plan.tokens_run[r] = run;
-        a.plan.action[r] = (valid && n0 > 0) ? CASCADE_ACT_RETAIN : CASCADE_ACT_NONE;
     }
     cluster.sync();  // the packed words are visible to every CTA of the cluster
 
@@ -490,8 +514,14 @@ extern "C" int cascade_tier_plan(cascade_ctx *ctx, const cascade_reqs *r, const 
     a.A_act = make_load_consts(ctx->params, D_act, K_act).A_act;
     a.n = n;
     a.with_tables = with_tables ? 1 : 0;
+    a.prepared = 0;
     int T, C, K;
     if (!cascade_pick_geometry(ctx, n > 0 ? n : 1, &T, &C, &K)) return CASCADE_EINVAL;
+    if (n > ctx->plan_prepare_min) {
+        a.prepared = 1;
+        CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((n + 255) / 256), dim3(256), 0, s, plan_prepare_kernel,
+                                             ctx->params, a));
+    }
     cudaError_t e = T == 256 ? launch_plan_k<256>(K, ctx->params, a, C, ctx->pdl, ctx->device, s)
                              : launch_plan_k<512>(K, ctx->params, a, C, ctx->pdl, ctx->device, s);
     CASCADE_CUDA_TRY(ctx, e);
@@ -620,6 +650,7 @@ extern "C" int cascade_tier_plan_noalloc(const cascade_params *p, const cascade_
     a.A_act = make_load_consts(*p, D_act, K_act).A_act;
     a.n = n;
     a.with_tables = with_tables ? 1 : 0;
+    a.prepared = 0;
     // The scalars are rewritten by every call before the rewrite kernels read them and only the
     // work entries written by this call are read back, so nothing has to be cleared; they are
     // zeroed anyway so that a call that launches nothing leaves no stale counts behind.

@@ -147,3 +147,31 @@ def test_staged_move_on_random_shapes():
         assert np.array_equal(host.numpy(), ref_o), (n_hbm, n_host, n_chunks, cb, ne, nr, k, stage_blocks)
         done += 1
     assert ctx.status()[0] == 0
+
+
+def test_ordering_with_random_runs_of_equal_high_bits():
+    """Random tie structure for the two-stage ordering (bits 16..63 first, runs of equal values repaired afterwards):
+    the high 48 bits are drawn from pools of different sizes, so runs of every length from 2 to far beyond the local
+    repair's limit appear at random positions, inside CTAs and astride their boundaries; the low 16 bits are random
+    or constant (full-key duplicates keep slot order).  Checked against numpy's stable argsort."""
+    import torch
+    from paper_2608_06557_b200.runner import Instance
+    rng = np.random.default_rng(321)
+    w = wl.config_llama8b(seed=2, n=65536, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9)
+    w.hbm_tbl = w.host_tbl = w.hbm_free = w.host_free = None
+    w.hbm_free_count, w.host_free_count = 1 << 30, 1 << 30
+    inst = Instance(w, alloc_pools=False)
+    for trial in range(120):
+        n = int(rng.integers(4097, 65537)) if trial % 3 else int(rng.choice([4097, 8192, 16384, 16385, 32768, 32769, 65536]))
+        pool = int(rng.choice([n // 300 + 1, n // 20 + 1, n // 3 + 1, n, 4 * n]))      # fewer values -> longer runs
+        high = rng.integers(0, 1 << 47, pool, dtype=np.int64).astype(np.uint64)[rng.integers(0, pool, n)]
+        if trial % 4 == 0:
+            high[rng.integers(0, n, n // 10)] = high[0]                                  # one very long run
+        low = rng.integers(0, 1 << 16, n).astype(np.uint64) if trial % 5 else np.zeros(n, np.uint64)
+        key = (high << np.uint64(16)) | low
+        inst.n = n
+        inst.key.view(torch.int64)[:n].copy_(torch.from_numpy(key.view(np.int64)))
+        inst.ctx.schedule(inst.reqs_struct, inst.key, n, w.D_act, inst.order, inst.grant, inst.sched_counts)
+        torch.cuda.synchronize()
+        assert np.array_equal(inst.order[:n].cpu().numpy(), np.argsort(key, kind="stable")), (trial, n, pool)
+    assert inst.ctx.status()[0] == 0

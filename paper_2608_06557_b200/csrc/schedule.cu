@@ -56,13 +56,14 @@ struct __align__(16) Exch {
     int cnt;                  // elements with a non-zero grant before the batch-size cap
 };
 
-// what every CTA tells the others after the passes over bits 16..63
+// what every CTA tells the others after the passes over bits kTopShift..63
 struct __align__(16) TieExch {
-    unsigned long long first, last;  // bits 16..63 of the CTA's first and last real element
+    unsigned long long first, last;  // bits kTopShift..63 of the CTA's first and last real element
     int count;                       // real elements the CTA holds
     int flags;                       // 1: equal neighbours inside the CTA, 2: a run longer than kMaxRun
 };
 constexpr int kMaxRun = 128;
+constexpr int kTopShift = 24;   // first-stage order: key bits 24..63 = tier, budget / 2 ns (a multiple of the 8-bit digits)
 
 struct ScheduleArgs {
     const uint64_t *key;
@@ -81,7 +82,7 @@ struct ScheduleArgs {
     SortElem *runs_out; // run mode: every cluster orders its own 16384-slot stretch of the queue and leaves the ordered
                         // elements here (no admission); NULL otherwise
     const SortElem *sorted_in;  // admission-only kernel: the fully ordered elements
-    int top_first;      // 1: order by bits 16..63 first, fix short runs of equal values locally (see the pass loop)
+    int top_first;      // 1: order by bits 24..63 first, fix short runs of equal values locally (see the pass loop)
     int rank_per;       // >0: small queue, order by counting (see rank_order below) with this many elements per CTA
     uint32_t *status;
 };
@@ -377,13 +378,13 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         if (c < csize) alld |= exall[c].diff;
 
     // ---- LSD radix sort, 8 bits per pass --------------------------------------------------------
-    // With top_first the two passes over the low 16 bits (arrival-id bits) are left out at first: budgets are
-    // nanosecond values, so after six passes over bits 16..63 equal values are rare and short runs of them are put
-    // in (key, slot) order by a local fix-up.  Only when a run is longer than kMaxRun or crosses a CTA boundary
-    // the queue is loaded again and ordered with all eight passes.
+    // With top_first the three passes over the low 24 bits (the arrival id and the budget's lowest bit) are left out
+    // at first: budgets are nanosecond values, so after five passes over bits 24..63 (tier, budget in steps of 2 ns)
+    // equal values are rare and short runs of them are put in (key, slot) order by a local fix-up.  Only when a run
+    // is longer than kMaxRun or crosses a CTA boundary the queue is loaded again and ordered with all eight passes.
     int ep = 0;          // passes executed so far: selects the mbarrier pair and its phase
     bool dead = false;   // a bounded wait expired: stop exchanging, keep walking the barriers
-    int first_pass = a.top_first ? 2 : 0;
+    int first_pass = a.top_first ? kTopShift / 8 : 0;
     for (int attempt = 0; attempt < 2; ++attempt) {
     const int ep_before = ep;
     for (int pass = first_pass; pass < 8; ++pass) {
@@ -546,7 +547,7 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     }
     if (first_pass == 0 || dead) break;   // all eight passes ran (or nothing can be trusted any more)
 
-    // ---- ordered by bits 16..63: look for equal neighbours ---------------------------------------------
+    // ---- ordered by bits kTopShift..63: look for equal neighbours ---------------------------------------------
     if (ep == ep_before) {   // no pass ran: the elements are still only in registers, in slot order
 #pragma unroll
         for (int k = 0; k < K; ++k) elems[(warp * K + k) * 32 + lane] = e[k];
@@ -559,17 +560,17 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     for (int k = 0; k < K; ++k) {
         const int li = (warp * K + k) * 32 + lane;
         if (li < n_here) {
-            const unsigned long long top = e[k].key >> 16;
-            if (li > 0 && (elems[li - 1].key >> 16) == top) tie = true;
-            if (li >= kMaxRun && (elems[li - kMaxRun].key >> 16) == top) long_run = true;
+            const unsigned long long top = e[k].key >> kTopShift;
+            if (li > 0 && (elems[li - 1].key >> kTopShift) == top) tie = true;
+            if (li >= kMaxRun && (elems[li - kMaxRun].key >> kTopShift) == top) long_run = true;
         }
     }
     const bool cta_tie = __syncthreads_or(tie);
     const bool cta_long = __syncthreads_or(long_run);
     if (warp == 0 && lane < csize) {
         TieExch x;
-        x.first = n_here > 0 ? elems[0].key >> 16 : 0ull;
-        x.last = n_here > 0 ? elems[n_here - 1].key >> 16 : 0ull;
+        x.first = n_here > 0 ? elems[0].key >> kTopShift : 0ull;
+        x.last = n_here > 0 ? elems[n_here - 1].key >> kTopShift : 0ull;
         x.count = n_here;
         x.flags = (cta_tie ? 1 : 0) | (cta_long ? 2 : 0);
         cluster.map_shared_rank(tie_ex, lane)[crank] = x;
@@ -593,10 +594,10 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                 const int li = (warp * K + k) * 32 + lane;
                 newpos[k] = li;
                 if (li >= n_here) continue;
-                const unsigned long long top = e[k].key >> 16;
+                const unsigned long long top = e[k].key >> kTopShift;
                 int lo = li, hi = li;
-                while (lo > 0 && (elems[lo - 1].key >> 16) == top) --lo;
-                while (hi + 1 < n_here && (elems[hi + 1].key >> 16) == top) ++hi;
+                while (lo > 0 && (elems[lo - 1].key >> kTopShift) == top) --lo;
+                while (hi + 1 < n_here && (elems[hi + 1].key >> kTopShift) == top) ++hi;
                 int r = 0;
                 for (int j = lo; j <= hi; ++j) {
                     const SortElem o = elems[j];

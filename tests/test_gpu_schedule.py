@@ -111,11 +111,12 @@ def test_duplicate_and_constant_keys_keep_slot_order():
 
 @pytest.mark.parametrize("n", [2500, 5000, 16384, 40000, 65536])
 def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
-    """The radix path orders by bits 16..63 first and repairs runs of equal values afterwards: short runs inside a
+    """The radix path orders by bits 24..63 first and repairs runs of equal values afterwards: short runs inside a
     CTA locally, long runs and runs across a CTA boundary by ordering again with every pass.  Keys are built so
     that the sorted position of every element is known, then runs are planted at chosen sorted positions: pairs and
-    triples whose low bits are in descending slot order, runs of exactly 16 and of 17, runs astride every multiple
-    of 256 (every possible CTA boundary), and full-key duplicates that must keep slot order."""
+    triples whose low bits are in descending slot order, runs of exactly 128 and of 129 (the local repair's limit),
+    runs astride every multiple of 256 (every possible CTA boundary), full-key duplicates that must keep slot order,
+    and a dense variant in which every 16 neighbours form a run."""
     torch, cs, Instance = _gpu()
     w = wl.config_llama8b(seed=n, n=n, hbm_bytes=2 * 10**9, host_bytes=2 * 10**9)
     w.hbm_tbl = w.host_tbl = w.hbm_free = w.host_free = None
@@ -132,8 +133,8 @@ def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
         assert np.array_equal(inst.grant[:n].cpu().numpy(), grant), tag
         assert inst.ctx.status()[0] == 0
 
-    def keys_with_runs(runs):
-        """runs: list of (first sorted position, length).  Element at sorted position q has bits 20.. = q, except
+    def keys_with_runs(runs, shift=24):
+        """runs: list of (first sorted position, length).  Element at sorted position q has bits shift.. = q, except
         inside a run, where all share the run's first position and differ (or not) in the low 16 bits."""
         rank = np.arange(n, dtype=np.uint64)
         top = rank.copy()
@@ -145,7 +146,7 @@ def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
             low[q:q + length] = np.arange(length, 0, -1)          # descending: the repair has to reverse the run
             if length >= 3:
                 low[q + 1] = low[q]                                # one full-key duplicate: slot order decides
-        key_sorted = (top << np.uint64(20)) | low
+        key_sorted = (top << np.uint64(shift)) | low
         slot_of = rng.permutation(n)                               # sorted position -> slot
         key = np.empty(n, np.uint64)
         key[slot_of] = key_sorted
@@ -154,8 +155,9 @@ def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
     check(keys_with_runs([]), "no runs")
     check(keys_with_runs([(q, 2) for q in range(10, n - 2, 97)]), "pairs")
     check(keys_with_runs([(q, 3) for q in range(5, n - 3, 61)]), "triples")
-    check(keys_with_runs([(100, 16), (900, 16), (n - 20, 16)]), "runs of 16")
-    check(keys_with_runs([(100, 2), (2000, 17)]), "a run of 17")
+    check(keys_with_runs([(100, 128), (900, 128), (n - 130, 128)]), "runs of 128")
+    check(keys_with_runs([(100, 2), (2000, 129)]), "a run of 129")
+    check(keys_with_runs([(3, 2), (700, 5)], shift=20), "every 16 neighbours equal above bit 24")
     check(keys_with_runs([(b - 1, 2) for b in range(256, n - 1, 256)]), "pairs astride every boundary")
     check(keys_with_runs([(b - 7, 14) for b in range(1024, n - 7, 1024)] + [(3, 2)]), "runs of 14 astride boundaries")
     check(keys_with_runs([(0, 2), (n - 2, 2)]), "first and last")

@@ -63,7 +63,7 @@ struct __align__(16) TieExch {
     int flags;                       // 1: equal neighbours inside the CTA, 2: a run longer than kMaxRun
 };
 constexpr int kMaxRun = 128;
-constexpr int kTopShift = 24;   // first-stage order: key bits 24..63 = tier, budget / 2 ns (a multiple of the 8-bit digits)
+constexpr int kTopShift = 32;   // first-stage order: key bits 32..63 = tier, budget / 512 ns (a multiple of the 8-bit digits)
 
 struct ScheduleArgs {
     const uint64_t *key;
@@ -380,8 +380,9 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
     // ---- LSD radix sort, 8 bits per pass --------------------------------------------------------
     // With top_first the three passes over the low 24 bits (the arrival id and the budget's lowest bit) are left out
     // at first: budgets are nanosecond values, so after five passes over bits 24..63 (tier, budget in steps of 2 ns)
-    // equal values are rare and short runs of them are put in (key, slot) order by a local fix-up.  Only when a run
-    // is longer than kMaxRun or crosses a CTA boundary the queue is loaded again and ordered with all eight passes.
+    // equal values are rare and short runs of them are put in (key, slot) order by a fix-up inside the CTA (or between
+    // two neighbouring CTAs).  Only when a run is longer than kMaxRun the queue is loaded again and ordered with all
+    // eight passes.
     int ep = 0;          // passes executed so far: selects the mbarrier pair and its phase
     bool dead = false;   // a bounded wait expired: stop exchanging, keep walking the barriers
     int first_pass = a.top_first ? kTopShift / 8 : 0;
@@ -576,46 +577,71 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         cluster.map_shared_rank(tie_ex, lane)[crank] = x;
     }
     cluster.sync();   // also: every CTA is done reading its elements before anybody starts another pass
-    bool redo = false;
+    bool redo = false, any_tie = false, crossing = false;
 #pragma unroll
     for (int c = 0; c < kMaxCluster; ++c) {
         if (c < csize) {
             if (tie_ex[c].flags & 2) redo = true;
-            if (c + 1 < csize && tie_ex[c + 1].count > 0 && tie_ex[c].last == tie_ex[c + 1].first) redo = true;
+            if (tie_ex[c].flags & 1) any_tie = true;
+            if (c + 1 < csize && tie_ex[c + 1].count > 0 && tie_ex[c].last == tie_ex[c + 1].first) crossing = true;
         }
     }
     if (!redo) {
-        if (cta_tie) {
-            // runs of equal values lie inside this CTA and are at most kMaxRun long: every element of a run counts the
-            // elements of its run that come before it by (key, slot) and moves there
-            unsigned newpos[K];
+        if (crossing || cta_tie) {
+            // Runs of equal values are short (no part of a run inside one CTA is longer than kMaxRun, so a run lies
+            // in one CTA or in two neighbours): every element of a run counts the members of its run that come before
+            // it by (key, slot) and moves there.  A run astride a CTA boundary is read from, and written into, the
+            // neighbour's shared memory; then every CTA of the cluster takes part in the two barriers (the decision is
+            // the same everywhere: all CTAs hold the same exchanged values).
+            const long long g0 = (long long)crank * per;
+            auto elem_at = [&](long long gpos) -> SortElem {
+                const unsigned c = (unsigned)(gpos / per);
+                const int l = (int)(gpos - (long long)c * per);
+                return c == crank ? elems[l] : cluster.map_shared_rank(elems, c)[l];
+            };
+            long long newpos[K];
 #pragma unroll
             for (int k = 0; k < K; ++k) {
                 const int li = (warp * K + k) * 32 + lane;
-                newpos[k] = li;
+                newpos[k] = g0 + li;
                 if (li >= n_here) continue;
                 const unsigned long long top = e[k].key >> kTopShift;
-                int lo = li, hi = li;
-                while (lo > 0 && (elems[lo - 1].key >> kTopShift) == top) --lo;
-                while (hi + 1 < n_here && (elems[hi + 1].key >> kTopShift) == top) ++hi;
+                const long long g = g0 + li;
+                // a neighbour in the same CTA decides quickly; only at the CTA's ends the other CTA is looked at
+                const bool left_same = li > 0 ? (elems[li - 1].key >> kTopShift) == top
+                                              : (crossing && g > 0 && (elem_at(g - 1).key >> kTopShift) == top);
+                const bool right_same = li + 1 < n_here ? (elems[li + 1].key >> kTopShift) == top
+                                                        : (crossing && g + 1 < n_q && (elem_at(g + 1).key >> kTopShift) == top);
+                if (!left_same && !right_same) continue;
+                // without a run astride a boundary nobody looks into another CTA's shared memory: its owner may be
+                // rewriting it, or may have left already
+                const long long lo_min = crossing ? 0 : g0, hi_max = crossing ? (long long)n_q - 1 : g0 + n_here - 1;
+                long long lo = g, hi = g;
+                while (lo > lo_min && g - lo < 2 * kMaxRun && (elem_at(lo - 1).key >> kTopShift) == top) --lo;
+                while (hi < hi_max && hi - g < 2 * kMaxRun && (elem_at(hi + 1).key >> kTopShift) == top) ++hi;
                 int r = 0;
-                for (int j = lo; j <= hi; ++j) {
-                    const SortElem o = elems[j];
+                for (long long j = lo; j <= hi; ++j) {
+                    const SortElem o = elem_at(j);
                     r += (o.key < e[k].key) || (o.key == e[k].key && o.idx < e[k].idx);
                 }
                 newpos[k] = lo + r;
             }
-            __syncthreads();
+            if (crossing) cluster.sync(); else __syncthreads();   // every read of the old order is done
 #pragma unroll
-            for (int k = 0; k < K; ++k)
-                if ((warp * K + k) * 32 + lane < n_here) elems[newpos[k]] = e[k];
-            __syncthreads();
+            for (int k = 0; k < K; ++k) {
+                if ((warp * K + k) * 32 + lane >= n_here) continue;
+                const unsigned c = (unsigned)(newpos[k] / per);
+                const int l = (int)(newpos[k] - (long long)c * per);
+                SortElem *dst = c == crank ? elems + l : cluster.map_shared_rank(elems, c) + l;
+                *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(&e[k]);
+            }
+            if (crossing) cluster.sync(); else __syncthreads();   // every element is at its place
 #pragma unroll
             for (int k = 0; k < K; ++k) e[k] = elems[(warp * K + k) * 32 + lane];
         }
         break;
     }
-    // a long or CTA-crossing run: start again from the queue as it was loaded, this time with every pass
+    // a run longer than the local repair takes: start again from the queue as it was loaded, this time with every pass
     first_pass = 0;
 #pragma unroll
     for (int k = 0; k < K; ++k) load_elem(k);

@@ -111,8 +111,8 @@ def test_duplicate_and_constant_keys_keep_slot_order():
 
 @pytest.mark.parametrize("n", [2500, 5000, 16384, 40000, 65536])
 def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
-    """The radix path orders by bits 24..63 first and repairs runs of equal values afterwards: short runs inside a
-    CTA locally, long runs and runs across a CTA boundary by ordering again with every pass.  Keys are built so
+    """The radix path orders by bits 32..63 first and repairs runs of equal values afterwards: short runs inside a
+    CTA locally, runs across a CTA boundary through the neighbour's shared memory, long runs by ordering again with every pass.  Keys are built so
     that the sorted position of every element is known, then runs are planted at chosen sorted positions: pairs and
     triples whose low bits are in descending slot order, runs of exactly 128 and of 129 (the local repair's limit),
     runs astride every multiple of 256 (every possible CTA boundary), full-key duplicates that must keep slot order,
@@ -133,7 +133,7 @@ def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
         assert np.array_equal(inst.grant[:n].cpu().numpy(), grant), tag
         assert inst.ctx.status()[0] == 0
 
-    def keys_with_runs(runs, shift=24):
+    def keys_with_runs(runs, shift=32):
         """runs: list of (first sorted position, length).  Element at sorted position q has bits shift.. = q, except
         inside a run, where all share the run's first position and differ (or not) in the low 16 bits."""
         rank = np.arange(n, dtype=np.uint64)
@@ -157,7 +157,8 @@ def test_runs_of_equal_budgets_are_ordered_by_id_then_slot(n):
     check(keys_with_runs([(q, 3) for q in range(5, n - 3, 61)]), "triples")
     check(keys_with_runs([(100, 128), (900, 128), (n - 130, 128)]), "runs of 128")
     check(keys_with_runs([(100, 2), (2000, 129)]), "a run of 129")
-    check(keys_with_runs([(3, 2), (700, 5)], shift=20), "every 16 neighbours equal above bit 24")
+    check(keys_with_runs([(3, 2), (700, 5)], shift=28), "every 16 neighbours equal above bit 32")
+    check(keys_with_runs([(3, 2)], shift=26), "every 64 neighbours equal above bit 32: runs astride every boundary")
     check(keys_with_runs([(b - 1, 2) for b in range(256, n - 1, 256)]), "pairs astride every boundary")
     check(keys_with_runs([(b - 7, 14) for b in range(1024, n - 7, 1024)] + [(3, 2)]), "runs of 14 astride boundaries")
     check(keys_with_runs([(0, 2), (n - 2, 2)]), "first and last")

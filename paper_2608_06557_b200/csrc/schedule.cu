@@ -60,7 +60,8 @@ struct __align__(16) Exch {
 struct __align__(16) TieExch {
     unsigned long long first, last;  // bits kTopShift..63 of the CTA's first and last real element
     int count;                       // real elements the CTA holds
-    int flags;                       // 1: equal neighbours inside the CTA, 2: a run longer than kMaxRun
+    int flags;                       // 1: equal neighbours inside the CTA, 2: a run longer than kMaxRun, or more than
+                                     //    an eighth of the CTA's threads hold an element equal to its neighbour
 };
 constexpr int kMaxRun = 128;
 constexpr int kTopShift = 32;   // first-stage order: key bits 32..63 = tier, budget / 512 ns (a multiple of the 8-bit digits)
@@ -566,8 +567,11 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
             if (li >= kMaxRun && (elems[li - kMaxRun].key >> kTopShift) == top) long_run = true;
         }
     }
-    const bool cta_tie = __syncthreads_or(tie);
-    const bool cta_long = __syncthreads_or(long_run);
+    // the repair counts inside every run: fine for the odd pair of equal budgets, quadratic when much of the queue is
+    // tied (quantised budgets, a burst of identical requests): then the remaining passes are cheaper
+    const int tied_threads = __syncthreads_count(tie);
+    const bool cta_tie = tied_threads > 0;
+    const bool cta_long = __syncthreads_or(long_run) || tied_threads * 8 > T;
     if (warp == 0 && lane < csize) {
         TieExch x;
         x.first = n_here > 0 ? elems[0].key >> kTopShift : 0ull;

@@ -370,15 +370,17 @@ struct PrepareArgs {
     int hash_cap;  // power of two
 };
 
-__device__ __forceinline__ unsigned hash_id(int32_t g) { return (unsigned)g * 2654435761u; }
+// multiplicative hashing: the HIGH bits of the product depend on every bit of the id (block ids that are all multiples
+// of a power of two would share the low ones)
+__device__ __forceinline__ unsigned hash_id(int32_t g, int bits) { return ((unsigned)g * 2654435761u) >> (32 - bits); }
 
 __global__ void __launch_bounds__(1024) kv_move_prepare_kernel(const __grid_constant__ PrepareArgs a) {
     cascade_grid_wait();
     cascade_grid_trigger();
     const int ne = clamp_count(a.n_evict_dev, a.n_evict_max), nr = clamp_count(a.n_restore_dev, a.n_restore_max);
     const int tid = threadIdx.x, T = blockDim.x;
-    int H = 64;  // table size: at most half full
-    while (H < 2 * ne && H < a.hash_cap) H <<= 1;
+    int H = 64, hbits = 6;  // table size: at most half full
+    while (H < 2 * ne && H < a.hash_cap) { H <<= 1; ++hbits; }
     const unsigned mask = (unsigned)H - 1u;
     for (int h = tid; h < H; h += T) {
         a.hkeys[h] = -1;
@@ -390,7 +392,7 @@ __global__ void __launch_bounds__(1024) kv_move_prepare_kernel(const __grid_cons
     for (int j = tid; j < ne; j += T) {
         const int32_t g = a.evict_src[j];
         if (g < 0) continue;  // never matches a valid destination
-        unsigned h = hash_id(g) & mask;
+        unsigned h = hash_id(g, hbits);
         for (int probe = 0; probe < H; ++probe) {
             const int32_t prev = atomicCAS(&a.hkeys[h], -1, g);
             if (prev == -1 || prev == g) {
@@ -405,7 +407,7 @@ __global__ void __launch_bounds__(1024) kv_move_prepare_kernel(const __grid_cons
         const int32_t g = a.restore_dst[r];
         int dep = -1;
         if (g >= 0) {
-            unsigned h = hash_id(g) & mask;
+            unsigned h = hash_id(g, hbits);
             for (int probe = 0; probe < H; ++probe) {
                 const int32_t k = a.hkeys[h];
                 if (k == g) { dep = a.hvals[h]; break; }

@@ -463,3 +463,31 @@ def test_fused_move_inside_a_cuda_graph():
         assert np.array_equal(rig.hbm.cpu().numpy(), ref_h), rep
         assert np.array_equal(rig.host.cpu().numpy(), ref_o), rep
     assert rig.ctx.status()[0] == 0 and rig.guards_intact()
+
+
+def test_fused_move_with_block_ids_that_are_multiples_of_a_power_of_two():
+    """The match of restore destinations to evicted blocks goes through a hash table over the block ids; ids that share
+    their low bits (every 64th block) must neither break it nor make it crawl."""
+    n_hbm, n_host, n_chunks, cb = 64 * 300, 700, 2, 256
+    rig = CopyRig(n_hbm, n_host, n_chunks, cb)
+    torch, cs = rig.torch, rig.cs
+    rng = np.random.default_rng(4)
+    ne, nr = 290, 290
+    strided = (rng.permutation(300).astype(np.int32) * 64)
+    es, ed, rs = strided[:ne], rng.permutation(n_host)[:ne].astype(np.int32), rng.permutation(n_host)[ne:ne + nr].astype(np.int32)
+    rd = rng.permutation(es)[:nr].astype(np.int32)                    # every restore lands in an evicted block
+    ref_h, ref_o = rig.hbm_np.copy(), rig.host_np.copy()
+    assert oracle.kv_evict(ref_h, rig.lay, ref_o, n_host, es, ed) == 0 and oracle.kv_restore(ref_h, rig.lay, ref_o, n_host, rs, rd) == 0
+    scratch = torch.empty(cs.kv_move_scratch_len(ne, nr), dtype=torch.int32, device="cuda")
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rig.ctx.kv_move(rig.layout, rig.hbm, rig.host, n_host, rig.ids(es), rig.ids(ed), None, ne, rig.ids(rs), rig.ids(rd), None, nr, scratch)
+    a.record()
+    rig.ctx.kv_move(rig.layout, rig.hbm, rig.host, n_host, rig.ids(es), rig.ids(ed), None, ne, rig.ids(rs), rig.ids(rd), None, nr, scratch)
+    b.record()
+    torch.cuda.synchronize()
+    rig.hbm.copy_(torch.from_numpy(rig.hbm_np)); rig.host.copy_(torch.from_numpy(rig.host_np))
+    rig.ctx.kv_move(rig.layout, rig.hbm, rig.host, n_host, rig.ids(es), rig.ids(ed), None, ne, rig.ids(rs), rig.ids(rd), None, nr, scratch)
+    torch.cuda.synchronize()
+    assert np.array_equal(rig.hbm.cpu().numpy(), ref_h) and np.array_equal(rig.host.cpu().numpy(), ref_o)
+    assert rig.ctx.status()[0] == 0 and scratch[:nr].cpu().tolist() == [0] * nr
+    assert a.elapsed_time(b) < 5.0                                     # milliseconds: 150 KB of payload

@@ -370,7 +370,9 @@ int cascade_kv_evict(cascade_ctx *ctx, const cascade_kv_layout *hbm, const void 
  * Same result as cascade_kv_evict on the evict list followed by cascade_kv_restore on the restore list (the
  * order the tier plan requires): a restore whose HBM block is also evicted by this call waits, block by
  * block, until that block has been read out.  Both lists as in the two calls above; the host pool must be
- * pinned, mapped host memory (or device memory).
+ * pinned, mapped host memory (or device memory).  Precondition: no restore reads a host record that an eviction
+ * of the same call writes (the tier plan never produces that: evictions take records off the free list); such a
+ * pair is not ordered here.  cascade_kv_move_staged orders it.
  *   scratch   caller-owned device array of cascade_kv_move_scratch_len(n_evict_max, n_restore_max) int32;
  *             contents irrelevant before the call.  After the call scratch[i], i < restore count, is the
  *             number of pieces of restore i that were NOT written: 0 = that block is complete, > 0 = a

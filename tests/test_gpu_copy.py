@@ -474,7 +474,8 @@ def test_fused_move_with_block_ids_that_are_multiples_of_a_power_of_two():
     rng = np.random.default_rng(4)
     ne, nr = 290, 290
     strided = (rng.permutation(300).astype(np.int32) * 64)
-    es, ed, rs = strided[:ne], rng.permutation(n_host)[:ne].astype(np.int32), rng.permutation(n_host)[ne:ne + nr].astype(np.int32)
+    op = rng.permutation(n_host).astype(np.int32)
+    es, ed, rs = strided[:ne], op[:ne], op[ne:ne + nr]               # restore sources are not among the evict destinations
     rd = rng.permutation(es)[:nr].astype(np.int32)                    # every restore lands in an evicted block
     ref_h, ref_o = rig.hbm_np.copy(), rig.host_np.copy()
     assert oracle.kv_evict(ref_h, rig.lay, ref_o, n_host, es, ed) == 0 and oracle.kv_restore(ref_h, rig.lay, ref_o, n_host, rs, rd) == 0

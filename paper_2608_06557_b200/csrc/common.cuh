@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "cascade.h"
 
 #include <nvtx3/nvToolsExt.h>
@@ -42,8 +44,8 @@ struct cascade_ctx {
     void *sort_runs, *sort_sorted;   // queues beyond 32768 requests: the ordered runs and the merged order (16 B per request each)
     int multi_sort;              // 1: such queues are ordered as runs of 16384 by one cluster each, then merged by rank
     int plan_prepare_min;        // queues above this size run the tier plan's per-request phase as a grid of its own
-    int sort_top_first;          // 1: radix passes over bits 16..63 first, local fix-up of equal values (budget policy only)
-    int merge_sort;              // 1: queues of up to 16384 requests beyond the counting path are ordered by local sort + merge by rank
+    int sort_top_first;          // 1: radix passes over key bits 32..63 only, then equal values are put in order of the low bits (budget policy only)
+    int merge_sort;              // 1: queues beyond the counting path that fit one key per thread (up to 4096) are ordered by local sort + merge by rank; 2: every queue of up to 16384
     int rank_sort_max;           // queues up to this size are ordered by counting instead of radix passes
     // copy-engine path (cascade_kv_move_staged): side streams and events, created with the context
     cudaStream_t ce_stream[4];   // [0], [1] host -> staging (restores); [2], [3] staging -> host (evictions)
@@ -217,6 +219,16 @@ static inline cudaError_t cascade_launch(bool pdl, int cluster, dim3 grid, dim3 
     cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args &&>(args)...);
 }
+
+// Function attributes (shared-memory opt-in, non-portable cluster size) are set once per device and kernel.  The flag may
+// be read and written by several host threads: setting an attribute twice is harmless, so a set-once atomic is enough.
+struct CascadeDeviceOnce {
+    std::atomic<bool> done[64] = {};
+    bool is_set(int device) const { return device >= 0 && device < 64 && done[device].load(std::memory_order_acquire); }
+    void set(int device) {
+        if (device >= 0 && device < 64) done[device].store(true, std::memory_order_release);
+    }
+};
 
 // The hot calls launch on the calling thread's current device and dereference the context's allocations there:
 // a context of another device is rejected on the host (CASCADE_EINVAL) before anything is launched.

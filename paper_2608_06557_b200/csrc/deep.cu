@@ -255,13 +255,13 @@ __global__ void __launch_bounds__(256) apply_stage_kernel(const __grid_constant_
 
 template <int T, int K>
 cudaError_t launch_stage(const cascade_params &p, const StageArgs &a, int cluster_size, bool pdl, cudaStream_t stream) {
-    static bool configured_dev[64] = {};
+    static CascadeDeviceOnce configured;
     int device = 0;
     cudaGetDevice(&device);
-    if (device < 0 || device >= 64 || !configured_dev[device]) {
+    if (!configured.is_set(device)) {
         cudaError_t e = cudaFuncSetAttribute(stage_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
-        if (device >= 0 && device < 64) configured_dev[device] = true;
+        configured.set(device);
     }
     return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), 0, stream, stage_kernel<T, K>, p, a);
 }

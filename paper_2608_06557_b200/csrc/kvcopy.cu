@@ -304,8 +304,11 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
         if (!mbar_wait_bounded(smem_addr(&bars[slot]), parity, limit)) {
             // give up: record it, issue nothing more, but do not leave while loads still target this CTA's ring
             st |= CASCADE_ST_ETIMEOUT;
-            for (long long q = stored + 1; q < issued; ++q)
-                mbar_wait_bounded(smem_addr(&bars[q % S]), (unsigned)((q / S) & 1), limit);
+            const long long t_giveup = clock64();   // one more limit for all of them together, not one each
+            for (long long q = stored + 1; q < issued; ++q) {
+                const long long left = limit - (clock64() - t_giveup);
+                mbar_wait_bounded(smem_addr(&bars[q % S]), (unsigned)((q / S) & 1), left > 0 ? left : 0);
+            }
             if (kRole == kRoleMoveRestore)
                 for (long long q = stored; q < issued; ++q) atomicAdd(&a.skipped[entry_of[q % S]], 1);
             break;
@@ -419,9 +422,11 @@ __global__ void __launch_bounds__(1024) kv_move_prepare_kernel(const __grid_cons
     }
 }
 
+constexpr int kMaxMoveList = 1 << 28;   // longest list the fused move accepts (the hash table has twice as many slots)
+
 int hash_capacity(int n_evict_max) {
     int H = 64;
-    while (H < 2 * (long long)n_evict_max) H <<= 1;
+    while (H < 2 * (long long)n_evict_max && H < (1 << 30)) H <<= 1;
     return H;
 }
 
@@ -459,10 +464,10 @@ void fill_copy_args(CopyArgs &a, const cascade_ctx *ctx, const cascade_kv_layout
 // the ring kernels need more dynamic shared memory than the default limit: opt in once per device
 template <int kRole>
 cudaError_t configure_ring(int device) {
-    static bool configured_dev[64] = {};
-    if (device >= 0 && device < 64 && configured_dev[device]) return cudaSuccess;
+    static CascadeDeviceOnce configured;
+    if (configured.is_set(device)) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(kv_ring_kernel<kRole>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingHost);
-    if (e == cudaSuccess && device >= 0 && device < 64) configured_dev[device] = true;
+    if (e == cudaSuccess) configured.set(device);
     return e;
 }
 
@@ -540,7 +545,7 @@ extern "C" int cascade_kv_stage(cascade_ctx *ctx, const void *deep_pool, int64_t
 }
 
 extern "C" int64_t cascade_kv_move_scratch_len(int n_evict_max, int n_restore_max) {
-    if (n_evict_max < 0 || n_restore_max < 0) return -1;
+    if (n_evict_max < 0 || n_restore_max < 0 || n_evict_max > kMaxMoveList || n_restore_max > kMaxMoveList) return -1;
     return 2 * (int64_t)n_restore_max + (int64_t)n_evict_max + 2 * (int64_t)hash_capacity(n_evict_max);
 }
 
@@ -551,6 +556,7 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
                                int32_t *scratch, void *stream) {
     CascadeRange nvtx_range("cascade_kv_move");
     if (!ctx || n_evict_max < 0 || n_restore_max < 0) return CASCADE_EINVAL;
+    if (n_evict_max > kMaxMoveList || n_restore_max > kMaxMoveList) return CASCADE_EINVAL;
     if (!cascade_on_ctx_device(ctx)) return CASCADE_EINVAL;
     if (n_evict_max == 0 && n_restore_max == 0) return CASCADE_OK;
     int rc = check_layout(hbm, hbm_pool, host_pool, host_blocks);

@@ -452,11 +452,11 @@ template <int T, int K>
 cudaError_t launch_plan(const cascade_params &p, const PlanArgs &a, int cluster_size, bool pdl, int device,
                         cudaStream_t stream) {
     // clusters of 16 CTAs need the non-portable size opt-in, once per device
-    static bool configured_dev[64] = {};
-    if (device < 0 || device >= 64 || !configured_dev[device]) {
+    static CascadeDeviceOnce configured;
+    if (!configured.is_set(device)) {
         cudaError_t e = cudaFuncSetAttribute(plan_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
-        if (device >= 0 && device < 64) configured_dev[device] = true;
+        configured.set(device);
     }
     return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), 0, stream, plan_kernel<T, K>, p, a);
 }

@@ -250,13 +250,13 @@ __global__ void __launch_bounds__(256) apply_prefetch_kernel(const __grid_consta
 
 template <int T, int K>
 cudaError_t launch_pf(const cascade_params &p, const PrefetchArgs &a, int cluster_size, bool pdl, cudaStream_t stream) {
-    static bool configured_dev[64] = {};
+    static CascadeDeviceOnce configured;
     int device = 0;
     cudaGetDevice(&device);
-    if (device < 0 || device >= 64 || !configured_dev[device]) {
+    if (!configured.is_set(device)) {
         cudaError_t e = cudaFuncSetAttribute(prefetch_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
-        if (device >= 0 && device < 64) configured_dev[device] = true;
+        configured.set(device);
     }
     return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(T), 0, stream, prefetch_kernel<T, K>, p, a);
 }

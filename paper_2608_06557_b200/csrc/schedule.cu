@@ -83,7 +83,7 @@ struct ScheduleArgs {
     SortElem *runs_out; // run mode: every cluster orders its own 16384-slot stretch of the queue and leaves the ordered
                         // elements here (no admission); NULL otherwise
     const SortElem *sorted_in;  // admission-only kernel: the fully ordered elements
-    int top_first;      // 1: order by bits 24..63 first, fix short runs of equal values locally (see the pass loop)
+    int top_first;      // 1: order by bits kTopShift..63 first, fix short runs of equal values locally (see the pass loop)
     int rank_per;       // >0: small queue, order by counting (see rank_order below) with this many elements per CTA
     uint32_t *status;
 };
@@ -379,11 +379,11 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         if (c < csize) alld |= exall[c].diff;
 
     // ---- LSD radix sort, 8 bits per pass --------------------------------------------------------
-    // With top_first the three passes over the low 24 bits (the arrival id and the budget's lowest bit) are left out
-    // at first: budgets are nanosecond values, so after five passes over bits 24..63 (tier, budget in steps of 2 ns)
-    // equal values are rare and short runs of them are put in (key, slot) order by a fix-up inside the CTA (or between
-    // two neighbouring CTAs).  Only when a run is longer than kMaxRun the queue is loaded again and ordered with all
-    // eight passes.
+    // With top_first the four passes over the low 32 bits (the arrival id and the budget's lowest nine bits) are left
+    // out at first: budgets are nanosecond values, so after four passes over bits 32..63 (tier, budget in steps of
+    // 512 ns) equal values are rare and short runs of them are put in (key, slot) order by a fix-up inside the CTA (or
+    // between two neighbouring CTAs).  Only when a run is longer than kMaxRun, or when much of a CTA is tied, the queue
+    // is loaded again and ordered with all eight passes.
     int ep = 0;          // passes executed so far: selects the mbarrier pair and its phase
     bool dead = false;   // a bounded wait expired: stop exchanging, keep walking the barriers
     int first_pass = a.top_first ? kTopShift / 8 : 0;
@@ -960,17 +960,15 @@ size_t smem_bytes(int T, int K) {
 
 template <int T, int K>
 cudaError_t launch(const ScheduleArgs &a, int cluster_size, int device, bool pdl, cudaStream_t stream, int n_clusters = 1) {
-    static bool configured_dev[64] = {};
-    bool unknown = false;
-    bool &configured = (device >= 0 && device < 64) ? configured_dev[device] : unknown;
+    static CascadeDeviceOnce configured;
     const size_t smem = smem_bytes(T, K);
-    if (!configured) {
+    if (!configured.is_set(device)) {
         cudaError_t e = cudaFuncSetAttribute(schedule_kernel<T, K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(schedule_kernel<T, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured.set(device);
     }
     return cascade_launch(pdl, cluster_size, dim3(cluster_size * n_clusters), dim3(T), smem, stream, schedule_kernel<T, K>, a);
 }
@@ -983,17 +981,15 @@ size_t merge_smem_bytes(int T, int K) {
 
 template <int K>
 cudaError_t launch_merge(const ScheduleArgs &a, int cluster_size, int device, bool pdl, cudaStream_t stream) {
-    static bool configured_dev[64] = {};
-    bool unknown = false;
-    bool &configured = (device >= 0 && device < 64) ? configured_dev[device] : unknown;
+    static CascadeDeviceOnce configured;
     const size_t smem = merge_smem_bytes(256, K);
-    if (!configured) {
+    if (!configured.is_set(device)) {
         cudaError_t e = cudaFuncSetAttribute(schedule_merge_kernel<256, K>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(schedule_merge_kernel<256, K>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured.set(device);
     }
     return cascade_launch(pdl, cluster_size, dim3(cluster_size), dim3(256), smem, stream, schedule_merge_kernel<256, K>, a);
 }
@@ -1105,10 +1101,10 @@ extern "C" int cascade_schedule(cascade_ctx *ctx, const cascade_reqs *r, const u
                                              (const SortElem *)r.runs_out, sorted, n));
         ScheduleArgs c = a;
         c.sorted_in = sorted;
-        static bool configured_dev[64] = {};
-        if (ctx->device < 0 || ctx->device >= 64 || !configured_dev[ctx->device]) {
+        static CascadeDeviceOnce configured;
+        if (!configured.is_set(ctx->device)) {
             CASCADE_CUDA_TRY(ctx, cudaFuncSetAttribute(admit_kernel<512, 8>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-            if (ctx->device >= 0 && ctx->device < 64) configured_dev[ctx->device] = true;
+            configured.set(ctx->device);
         }
         CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 16, dim3(16), dim3(512), 0, s, admit_kernel<512, 8>, c));
         return CASCADE_OK;

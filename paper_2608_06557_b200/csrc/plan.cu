@@ -167,8 +167,12 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
             const long long r = pos0 + k * 32;
             if (r < n) st |= plan_prepare_one(p, a, r);
         }
+        cluster.sync();  // the packed words are visible to every CTA of the cluster
+    } else {
+        // the packed words come from the grid before; only "every CTA has started" is needed, in front of the first
+        // store into a neighbour's shared memory: the wait sits there and the gathers below run in the meantime
+        cluster.barrier_arrive();
     }
-    cluster.sync();  // the packed words are visible to every CTA of the cluster
 
     // ---- phase 1b, schedule order: one 8-byte gather per element --------------------------------
     uint32_t slot[K];
@@ -204,6 +208,7 @@ plan_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ Pl
     cta_scan3<T, K>(s_need, s_x1, s_cnt, tot, ws3);
     long long red1[1] = {evictable};
     cta_sum<T, 1>(red1, ws8);
+    if (a.prepared) cluster.barrier_wait();
     if (tid < csize) {
         Exch1 x;
         x.need = tot[0];

@@ -274,6 +274,9 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         for (int i = 0; i < 4; ++i) mbarrier_init(cta_smem_addr(&bars[i]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // "I have started, my barriers exist": the matching wait sits in front of the first store into another CTA's
+    // shared memory, so the barrier's latency hides behind the loads below
+    cluster.barrier_arrive();
 
     // ---- load: key, slot, tokens wanted (prompt minus the matched prefix) ----------------------
     SortElem e[K];
@@ -341,9 +344,10 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
                 cnt += count_range((int)max((long long)mid, min((long long)hi, gi + 1)), hi, false);   // above gi: ties do not count
             }
             partial[tid] = cnt;
-            // a cluster barrier, not just a CTA barrier: no store into another CTA's shared memory before
-            // every CTA of the cluster has started
-            cluster.sync();
+            // besides the CTA barrier, the cluster barrier begun at the top: no store into another CTA's shared memory
+            // before every CTA of the cluster has started
+            __syncthreads();
+            cluster.barrier_wait();
             // the element's owner adds the partial counts and sends the element to its final place
             if (tid < per_rt && e[0].idx != 0xffffffffu) {
                 int pos = 0;
@@ -362,9 +366,10 @@ __global__ void __launch_bounds__(T, 1) schedule_kernel(const __grid_constant__ 
         unsigned lo = __reduce_or_sync(kFull, (unsigned)diff);
         unsigned hi = __reduce_or_sync(kFull, (unsigned)(diff >> 32));
         if (lane == 0) wtmp[warp] = (long long)(((unsigned long long)hi << 32) | lo);
-        // a cluster barrier, not just a CTA barrier: the store below is the first access to another CTA's
-        // shared memory, which must not happen before that CTA has started (and initialised its mbarriers)
-        cluster.sync();
+        // besides the CTA barrier, the cluster barrier begun at the top: the store below is the first access to another
+        // CTA's shared memory, which must not happen before that CTA has started (and initialised its mbarriers)
+        __syncthreads();
+        cluster.barrier_wait();
         if (warp == 0) {
             unsigned long long v = lane < W ? (unsigned long long)wtmp[lane] : 0ull;
             lo = __reduce_or_sync(kFull, (unsigned)v);
@@ -719,6 +724,7 @@ __global__ void __launch_bounds__(T, 1) admit_kernel(const __grid_constant__ Sch
         a.counts->n_admitted = 0;
         a.counts->tokens_granted = 0;
     }
+    cluster.barrier_arrive();
     SortElem e[K];
 #pragma unroll
     for (int k = 0; k < K; ++k) {
@@ -726,7 +732,7 @@ __global__ void __launch_bounds__(T, 1) admit_kernel(const __grid_constant__ Sch
         if (g < a.n) e[k] = a.sorted_in[g];
         else { e[k].key = ~0ull; e[k].idx = 0xffffffffu; e[k].want = 0; }
     }
-    cluster.sync();   // the counts are zero and every CTA has started before anybody writes to a neighbour
+    cluster.barrier_wait();   // every CTA has started (and the counts are zero) before anybody writes to a neighbour
     admit_and_write<T, K>(a, e, per, cluster, wtmp, itmp, exall);
 }
 
@@ -779,6 +785,7 @@ __global__ void __launch_bounds__(T, 1) schedule_merge_kernel(const __grid_const
         mbarrier_arrive_expect(keys_bar, (csize - 1) * (unsigned)(per * sizeof(uint64_t)));
         mbarrier_arrive_expect(elem_bar, (unsigned)(n_mine * sizeof(SortElem)));
     }
+    cluster.barrier_arrive();   // waited for in front of the first store into another CTA's shared memory
 
     // ---- load: key, slot, tokens wanted -------------------------------------------------------------
     SortElem e[K];
@@ -887,7 +894,8 @@ __global__ void __launch_bounds__(T, 1) schedule_merge_kernel(const __grid_const
 #pragma unroll
     for (int k = 0; k < K; ++k) my_list[(warp * K + k) * 32 + lane] = e[k].key;
     // first access to other CTAs' shared memory: they must all have started and initialised their barriers
-    cluster.sync();
+    __syncthreads();
+    cluster.barrier_wait();
     for (unsigned op = tid; op < (csize - 1) * (per / 2); op += T) {
         unsigned dst = op / (per / 2);
         const unsigned piece = op % (per / 2);

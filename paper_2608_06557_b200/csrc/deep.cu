@@ -80,6 +80,9 @@ stage_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ S
     const int n = a.n;
     const int bt = p.bt;
     uint32_t st = 0;
+    // "I have started": waited for in front of the first store into another CTA's shared memory (which must exist by
+    // then); the barrier's latency hides behind the per-request work
+    cluster.barrier_arrive();
 
     long long host_cnt = *a.pools.host_free_count;
     if (a.with_tables && (host_cnt < 0 || host_cnt > a.pools.host_free_cap)) {
@@ -135,6 +138,7 @@ stage_kernel(const __grid_constant__ cascade_params p, const __grid_constant__ S
     int tot[3];
     cta_scan3<T, K>(mv, cv, zero, tot, ws3);               // mv, cv now inclusive
     const long long t_total = cta_scan_ll<T, K>(tv, &ws8[0][0]);
+    cluster.barrier_wait();
     if (tid < csize) {
         StExch1 x;
         x.time = t_total;

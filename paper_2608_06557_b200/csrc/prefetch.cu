@@ -67,6 +67,9 @@ prefetch_kernel(const __grid_constant__ cascade_params p, const __grid_constant_
     const int n = a.n;
     const int bt = p.bt;
     uint32_t st = 0;
+    // "I have started": waited for in front of the first store into another CTA's shared memory (which must exist by
+    // then); the barrier's latency hides behind the per-request work
+    cluster.barrier_arrive();
 
     long long hbm_cnt = *a.pools.hbm_free_count;
     if (a.with_tables && (hbm_cnt < 0 || hbm_cnt > a.pools.hbm_free_cap)) {
@@ -135,6 +138,7 @@ prefetch_kernel(const __grid_constant__ cascade_params p, const __grid_constant_
     const long long t_total = cta_scan_ll<T, K>(tv, &ws8[0][0]);
     long long red[1] = {used};
     cta_sum<T, 1>(red, ws8);
+    cluster.barrier_wait();
     if (tid < csize) {
         PfExch1 x;
         x.time = t_total;

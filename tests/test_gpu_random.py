@@ -150,7 +150,7 @@ def test_staged_move_on_random_shapes():
 
 
 def test_ordering_with_random_runs_of_equal_high_bits():
-    """Random tie structure for the two-stage ordering (bits 16..63 first, runs of equal values repaired afterwards):
+    """Random tie structure for the two-stage ordering (bits 32..63 first, runs of equal values repaired afterwards):
     the high 48 bits are drawn from pools of different sizes, so runs of every length from 2 to far beyond the local
     repair's limit appear at random positions, inside CTAs and astride their boundaries; the low 16 bits are random
     or constant (full-key duplicates keep slot order).  Checked against numpy's stable argsort."""

@@ -463,11 +463,11 @@ def fuzz_params(rng) -> dict:
     return d
 
 
-def fuzz_workload(rng, d: dict) -> Workload:
-    """A random queue with tables, free lists and a deep tier for the parameters ``d``: sizes from 1 to 3000,
-    hit profiles of every shape, a few requests outside the input bounds, rows too short for their prompt,
-    shared host / deep record ids, free lists from empty to ample, loads from idle to the maximum."""
-    n = int(rng.choice([1, 2, 33, 200, 1000, 1025, 3000]))
+def fuzz_workload(rng, d: dict, sizes=(1, 2, 33, 200, 1000, 1025, 3000)) -> Workload:
+    """A random queue with tables, free lists and a deep tier for the parameters ``d``: sizes from 1 to 3000
+    (or one of ``sizes``), hit profiles of every shape, a few requests outside the input bounds, rows too short for
+    their prompt, shared host / deep record ids, free lists from empty to ample, loads from idle to the maximum."""
+    n = int(rng.choice(list(sizes)))
     bt = d["bt"]
     nc = len(d["ttft_ns"])
     maxb = int(rng.choice([8, 64, 200]))

@@ -57,6 +57,22 @@ def test_random_inputs_through_the_whole_plan_chain(first):
             raise AssertionError(f"seed {1000 + seed}: {e}") from e
 
 
+@pytest.mark.parametrize("first", range(0, 48, 8))
+def test_random_inputs_with_queues_beyond_one_key_per_thread(first):
+    """The same chain on queues of 4097 to 20000 requests: two and four keys per thread, the radix passes with the
+    two-stage order, the tier plan with its per-request phase as a grid of its own (from 8192 requests up)."""
+    for seed in range(first, first + 8):
+        g = np.random.default_rng(7000 + seed)
+        d = wl.fuzz_params(g)
+        w = wl.fuzz_workload(g, d, sizes=(4097, 5000, 8191, 8192, 9000, 16384, 20000))
+        args = (int(g.choice([0, 10**6, 10**9, 1 << 50])), int(g.choice([0, 2, 100])),
+                int(g.choice([0, 10**6, 10**9, 1 << 50])), int(g.choice([0, 2, 100])))
+        try:
+            _compare(w, *args)
+        except AssertionError as e:
+            raise AssertionError(f"seed {7000 + seed}: {e}") from e
+
+
 def test_request_parked_for_a_bad_class_is_still_offered_tokens_in_both_admission_modes():
     """A request whose class index is out of range is parked at the very end of the order with the lowest
     budget; it is still a request with a usable shape, so whatever tokens are left reach it, in the default

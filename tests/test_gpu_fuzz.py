@@ -9,14 +9,17 @@ from paper_2608_06557_b200 import workload as wl
 pytestmark = pytest.mark.gpu
 
 
-def _compare(w, link, hbm_reserve, stage_link, host_reserve):
+def _compare(w, link, hbm_reserve, stage_link, host_reserve, one_call=False):
     from paper_2608_06557_b200.runner import Instance
     out = oracle_chain(w, link, hbm_reserve, stage_link, host_reserve)
     res, pf, dr, st, ds = out["res"], out["pf"], out["dr"], out["st"], out["ds"]
     pools, plan = res["pools"], res["plan"]
     inst = Instance(w, alloc_pools=False)
     inst.enable_deep(w, alloc_pool=False)
-    inst.run_schedule()
+    if one_call:
+        inst.run_step(inst.step_args())     # one cascade_step call
+    else:
+        inst.run_schedule()                 # the three calls
     inst.run_prefetch(link, hbm_reserve)
     inst.run_dedup_restore()
     inst.run_stage_plan(stage_link, host_reserve)
@@ -52,7 +55,7 @@ def test_random_inputs_through_the_whole_plan_chain(first):
         args = (int(g.choice([0, 10**6, 10**9, 1 << 50])), int(g.choice([0, 2, 100])),
                 int(g.choice([0, 10**6, 10**9, 1 << 50])), int(g.choice([0, 2, 100])))
         try:
-            _compare(w, *args)
+            _compare(w, *args, one_call=seed % 2 == 1)
         except AssertionError as e:
             raise AssertionError(f"seed {1000 + seed}: {e}") from e
 
@@ -68,7 +71,7 @@ def test_random_inputs_with_queues_beyond_one_key_per_thread(first):
         args = (int(g.choice([0, 10**6, 10**9, 1 << 50])), int(g.choice([0, 2, 100])),
                 int(g.choice([0, 10**6, 10**9, 1 << 50])), int(g.choice([0, 2, 100])))
         try:
-            _compare(w, *args)
+            _compare(w, *args, one_call=seed % 2 == 1)
         except AssertionError as e:
             raise AssertionError(f"seed {7000 + seed}: {e}") from e
 

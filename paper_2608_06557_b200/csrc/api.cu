@@ -81,6 +81,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->ce_lanes = e && atoi(e) == 2 ? 2 : 1;   // measured: a second stream per direction gains nothing
     e = getenv("CASCADE_COPY_AHEAD_SUB");
     ctx->copy_ahead_sub = e && atoi(e) == 1 ? 1 : 2;   // measured: refilling the slot of the store just issued stalls the ring
+    e = getenv("CASCADE_COPY_DYNAMIC");
+    ctx->copy_dynamic = e ? (atoi(e) != 0) : 1;
     e = getenv("CASCADE_COPY_PIECE");
     ctx->copy_piece = e ? atoi(e) : 0;
     if (ctx->copy_piece != 8192 && ctx->copy_piece != 16384 && ctx->copy_piece != 32768) ctx->copy_piece = 0;
@@ -105,7 +107,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
               cudaMalloc(&ctx->want_by_slot, n * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&ctx->work_admit, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->work_victim, n * sizeof(int4)) == cudaSuccess &&
-              cudaMalloc(&ctx->plan_scalars, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
+              cudaMalloc(&ctx->plan_scalars, PS_COUNT * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->copy_tickets, 8 * sizeof(unsigned)) == cudaSuccess;
     for (int i = 0; ok && i < 4; ++i)
         ok = cudaStreamCreateWithFlags(&ctx->ce_stream[i], cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; ok && i < 7; ++i)
@@ -117,7 +120,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     if (ok && max_requests > 16384 && ctx->max_cluster >= 16)
         ok = cudaMalloc(&ctx->sort_runs, n * 16) == cudaSuccess && cudaMalloc(&ctx->sort_sorted, n * 16) == cudaSuccess;
     if (ok) ok = cudaMemset(ctx->status_dev, 0, sizeof(uint32_t)) == cudaSuccess &&
-                 cudaMemset(ctx->plan_scalars, 0, PS_COUNT * sizeof(int32_t)) == cudaSuccess;
+                 cudaMemset(ctx->plan_scalars, 0, PS_COUNT * sizeof(int32_t)) == cudaSuccess &&
+                 cudaMemset(ctx->copy_tickets, 0, 8 * sizeof(unsigned)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         cascade_destroy(ctx);
@@ -139,6 +143,7 @@ extern "C" void cascade_destroy(cascade_ctx *ctx) {
     cudaFree(ctx->work_admit);
     cudaFree(ctx->work_victim);
     cudaFree(ctx->plan_scalars);
+    cudaFree(ctx->copy_tickets);
     cudaFree(ctx->sort_runs);
     cudaFree(ctx->sort_sorted);
     for (int i = 0; i < 4; ++i)

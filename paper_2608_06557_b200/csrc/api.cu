@@ -75,6 +75,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->copy_bulk_dev = e ? atoi(e) : 2;
     e = getenv("CASCADE_MOVE_CTAS");
     ctx->move_ctas = e ? atoi(e) : 0;
+    e = getenv("CASCADE_MOVE_CTAS_RESTORE");
+    ctx->move_ctas_restore = e ? atoi(e) : 0;
     e = getenv("CASCADE_MOVE_VECTOR");
     ctx->move_vector = e ? (atoi(e) & 3) : 1;   // measured: bulk reads of the restore grid starve beside the evict grid's bulk writes
     e = getenv("CASCADE_CE_LANES");

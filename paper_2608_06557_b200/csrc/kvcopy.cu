@@ -371,7 +371,7 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
 //   1. kv_move_prepare_kernel (one CTA): zeroes the per-entry counters and finds, for every restore, the
 //      evict entry that frees its HBM block (the tier plan hands freed blocks out again at once) through an
 //      open-addressing hash table over the evicted block ids: linear work in the two list lengths;
-//   2. the evict grid (role kRoleMoveEvict), half of the SMs: device -> host; after every piece that has
+//   2. the evict grid (role kRoleMoveEvict), a little under half of the SMs: device -> host; after every piece that has
 //      left HBM it bumps that entry's counter.  It signals "dependents may launch" as its first action;
 //   3. the restore grid (role kRoleMoveRestore), on the other half, launched as a PROGRAMMATIC DEPENDENT of
 //      grid 2: the hardware starts it only once every CTA of the evict grid is running (or done), so a
@@ -601,9 +601,14 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3(1), dim3(1024), 0, s, kv_move_prepare_kernel, p));
 
     const long long ppc_max = (hbm->chunk_bytes + kPieceMin - 1) / kPieceMin;
-    int half = ctx->num_sms / 2;
-    if (ctx->move_ctas > 0 && ctx->move_ctas < half) half = ctx->move_ctas;
+    // SMs per grid: a little under half of them.  Measured on B200 (148 SMs), 512 + 512 blocks of 2 MiB: 65 + 65 gives
+    // 79 GB/s, 74 + 74 gives 77, 58 + 58 gives 78, 50 + 50 gives 75: with fewer posted writes queued towards the host the
+    // restore grid's read requests get through sooner.
+    int half = (ctx->num_sms * 44 + 50) / 100;
+    if (ctx->move_ctas > 0 && ctx->move_ctas <= ctx->num_sms / 2) half = ctx->move_ctas;
     if (half < 1) half = 1;
+    int half_r = half;
+    if (ctx->move_ctas_restore > 0 && ctx->move_ctas_restore <= ctx->num_sms / 2) half_r = ctx->move_ctas_restore;
     CASCADE_CUDA_TRY(ctx, configure_ring<kRoleMoveEvict>(ctx->device));
     CASCADE_CUDA_TRY(ctx, configure_ring<kRoleMoveRestore>(ctx->device));
     CopyArgs e, r;
@@ -620,7 +625,7 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     e.dep = r.dep = p.dep;
     e.skipped = r.skipped = p.skipped;
     // the evict grid is launched even when its list is empty: the restore grid is ordered behind it
-    long long ge = half, gr = half;
+    long long ge = half, gr = half_r;
     const long long items_e = (long long)n_evict_max * hbm->n_chunks * ppc_max;
     const long long items_r = (long long)n_restore_max * hbm->n_chunks * ppc_max;
     if (ge > items_e) ge = items_e < 1 ? 1 : items_e;
@@ -639,7 +644,7 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     }
     if (gr > 0) {
         if (ctx->move_vector & 1) {
-            long long g = (long long)half * vec_per_sm;
+            long long g = (long long)half_r * vec_per_sm;
             const long long iv = (long long)n_restore_max * hbm->n_chunks * r.pieces_per_chunk;
             if (g > iv) g = iv;
             CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)g), dim3(kThreads), 0, s,

@@ -75,6 +75,8 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
     ctx->copy_bulk_dev = e ? atoi(e) : 2;
     e = getenv("CASCADE_MOVE_CTAS");
     ctx->move_ctas = e ? atoi(e) : 0;
+    e = getenv("CASCADE_COPY_GRID_HOST");
+    ctx->copy_grid_host = e ? atoi(e) : 0;
     e = getenv("CASCADE_MOVE_CTAS_RESTORE");
     ctx->move_ctas_restore = e ? atoi(e) : 0;
     e = getenv("CASCADE_MOVE_VECTOR");

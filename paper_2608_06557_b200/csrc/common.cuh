@@ -36,6 +36,7 @@ struct cascade_ctx {
     int copy_bulk_host;          // >0: TMA bulk-copy ring (that many CTAs per SM) for the pinned-host path
     int copy_bulk_dev;           // >0: TMA bulk-copy ring for the device-staging path
     int move_ctas;               // >0: CTAs of each of the two grids of the fused evict+restore (at most half the SMs)
+    int copy_grid_host;          // >0: CTAs of the TMA ring over the host link (default: 44 % of the SMs)
     int move_ctas_restore;       // >0: SMs' worth of CTAs of the restore grid alone (tuning)
     int move_vector;             // fused move: bit 0 = restore grid, bit 1 = evict grid use the vector kernel instead of the ring
     int copy_ahead_sub;          // TMA ring: loads kept in flight = ring slots minus this (1 | 2)

@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kThreads) kv_copy_kernel(const __grid_constant
 constexpr int kPieceMax = 32 * 1024;
 constexpr int kPieceMin = 8 * 1024;
 constexpr int kMaxStages = 16;
-constexpr int kRingHost = 128 * 1024;   // one CTA per SM
+constexpr int kRingHost = 128 * 1024;   // at most one CTA per SM
 constexpr int kRingDev = 96 * 1024;     // two CTAs per SM fit
 
 __device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -509,6 +509,12 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
         if (ctx->copy_ring_kb > 0) a.ring_bytes = ctx->copy_ring_kb * 1024;
         const long long items = (long long)n_max * l->n_chunks * ((l->chunk_bytes + kPieceMin - 1) / kPieceMin);
         long long grid = (long long)ctx->num_sms * (mode > 1 ? mode : 1);
+        // Over the host link the rate does not depend on the grid between 40 and 148 CTAs (evict 52.7 GB/s with 24, 65 or
+        // 148; restore 50.1 / 51.4 / 50.6 GB/s; one block and sixteen blocks take the same time too), so the copy takes
+        // 44 % of the SMs and leaves the shared memory of the others to whatever else runs on the GPU.
+        if (!record_is_device)
+            grid = ctx->copy_grid_host > 0 ? ctx->copy_grid_host : (ctx->num_sms * 44 + 50) / 100;
+        if (grid < 1) grid = 1;
         if (grid > items) grid = items;
         constexpr int role = kRestore ? kRoleRestore : kRoleEvict;
         a.ticket = ctx->copy_dynamic ? ctx->copy_tickets + 2 * role : nullptr;

@@ -691,21 +691,36 @@ __global__ void __launch_bounds__(256) merge_runs_kernel(const SortElem *__restr
     const SortElem me = runs[i];
     const int r = i / kRunLen;
     int pos = i - r * kRunLen;
-    const int n_runs = (n + kRunLen - 1) / kRunLen;
-    for (int q = 0; q < n_runs; ++q) {
-        if (q == r) continue;
-        const SortElem *list = runs + (size_t)q * kRunLen;
-        int len = min(kRunLen, n - q * kRunLen), lo = 0;
-        const bool ties = q < r;
-        while (len > 0) {
-            const int half = len >> 1;
-            const unsigned long long v = list[lo + half].key;
-            const bool below = ties ? v <= me.key : v < me.key;
-            lo = below ? lo + half + 1 : lo;
-            len = below ? len - half - 1 : half;
-        }
-        pos += lo;
+    // the searches through the other runs advance in step: their loads (L2 latency each) do not depend on one another,
+    // so a round of the loop costs one latency instead of one per run
+    constexpr int kMaxRuns = CASCADE_MAX_REQUESTS / kRunLen;
+    int lo[kMaxRuns], len[kMaxRuns];
+    bool more = false;
+#pragma unroll
+    for (int q = 0; q < kMaxRuns; ++q) {
+        lo[q] = 0;
+        len[q] = (q == r || q * kRunLen >= n) ? 0 : min(kRunLen, n - q * kRunLen);
+        more |= len[q] > 0;
     }
+    while (more) {
+        unsigned long long v[kMaxRuns];
+#pragma unroll
+        for (int q = 0; q < kMaxRuns; ++q)
+            if (len[q] > 0) v[q] = runs[(size_t)q * kRunLen + lo[q] + (len[q] >> 1)].key;
+        more = false;
+#pragma unroll
+        for (int q = 0; q < kMaxRuns; ++q) {
+            if (len[q] > 0) {
+                const int half = len[q] >> 1;
+                const bool below = q < r ? v[q] <= me.key : v[q] < me.key;   // runs in front count equal keys too
+                lo[q] = below ? lo[q] + half + 1 : lo[q];
+                len[q] = below ? len[q] - half - 1 : half;
+                more |= len[q] > 0;
+            }
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < kMaxRuns; ++q) pos += lo[q];
     sorted[pos] = me;
 }
 

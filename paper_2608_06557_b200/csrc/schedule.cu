@@ -926,26 +926,41 @@ __global__ void __launch_bounds__(T, 1) schedule_merge_kernel(const __grid_const
         unsigned pos[K];
 #pragma unroll
         for (int k = 0; k < K; ++k) pos[k] = (warp * K + k) * 32 + lane;   // own list: the local position
-        for (unsigned c = 0; c < csize; ++c) {
-            if (c == crank) continue;
-            const uint64_t *list = keys_all + (size_t)c * per;
-            const bool ties = c < crank;   // equal keys of CTAs in front hold lower slots: they come first
-            unsigned p[K];
+        // four lists at a time: their searches advance in step, so the shared-memory latency of a round is paid once
+        // for the four of them (the own list is searched along and left out of the sum; csize is a power of two)
+        constexpr int G = 4;
+        for (unsigned c0 = 0; c0 < csize; c0 += G) {
+            unsigned p[G][K];
+            const uint64_t *list[G];
+            bool ties[G], counted[G];
 #pragma unroll
-            for (int k = 0; k < K; ++k) p[k] = 0;
+            for (int j = 0; j < G; ++j) {
+                const unsigned c = c0 + j < csize ? c0 + j : csize - 1;
+                list[j] = keys_all + (size_t)c * per;
+                ties[j] = c < crank;       // equal keys of CTAs in front hold lower slots: they come first
+                counted[j] = c0 + j < csize && c != crank;
+#pragma unroll
+                for (int k = 0; k < K; ++k) p[j][k] = 0;
+            }
 #pragma unroll
             for (int s = per / 2; s > 0; s >>= 1) {
 #pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    const uint64_t v = list[p[k] + s - 1];
-                    p[k] += (ties ? v <= e[k].key : v < e[k].key) ? s : 0;
+                for (int j = 0; j < G; ++j) {
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const uint64_t v = list[j][p[j][k] + s - 1];
+                        p[j][k] += (ties[j] ? v <= e[k].key : v < e[k].key) ? s : 0;
+                    }
                 }
             }
 #pragma unroll
-            for (int k = 0; k < K; ++k) {
-                const uint64_t v = list[p[k]];
-                p[k] += (ties ? v <= e[k].key : v < e[k].key) ? 1 : 0;
-                pos[k] += p[k];
+            for (int j = 0; j < G; ++j) {
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const uint64_t v = list[j][p[j][k]];
+                    p[j][k] += (ties[j] ? v <= e[k].key : v < e[k].key) ? 1 : 0;
+                    if (counted[j]) pos[k] += p[j][k];
+                }
             }
         }
         // ---- every real element to its place (padding stays behind: nobody reads the slots past n) ----------

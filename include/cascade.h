@@ -23,7 +23,9 @@
  *   - The library allocates device memory only in cascade_create.  The five hot calls allocate
  *     nothing, never synchronise the host and use no stream of their own (the one exception, by its
  *     nature, is cascade_kv_move_staged: it drives the copy engines from the host).
- *   - One context per stream.  A context is not thread-safe.
+ *   - One context per stream.  A context is not thread-safe, and its calls must not run on two streams at
+ *     the same time either (order them with events if they are issued to different streams): the kernels
+ *     of one context share scratch, the plan's work lists and the copy kernels' work counters.
  *   - Return value: 0 on success, a negative CASCADE_E* code for errors found on the host before
  *     anything is launched.  Conditions found on the device never trap; they OR a CASCADE_ST_* bit
  *     into the context's sticky status word, read with cascade_status.

@@ -112,7 +112,7 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
               cudaMalloc(&ctx->work_admit, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->work_victim, n * sizeof(int4)) == cudaSuccess &&
               cudaMalloc(&ctx->plan_scalars, PS_COUNT * sizeof(int32_t)) == cudaSuccess &&
-              cudaMalloc(&ctx->copy_tickets, 8 * sizeof(unsigned)) == cudaSuccess;
+              cudaMalloc(&ctx->copy_tickets, 128 * sizeof(unsigned)) == cudaSuccess;
     for (int i = 0; ok && i < 4; ++i)
         ok = cudaStreamCreateWithFlags(&ctx->ce_stream[i], cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; ok && i < 7; ++i)
@@ -125,7 +125,7 @@ extern "C" int cascade_create(cascade_ctx **out, const cascade_params *p, int ma
         ok = cudaMalloc(&ctx->sort_runs, n * 16) == cudaSuccess && cudaMalloc(&ctx->sort_sorted, n * 16) == cudaSuccess;
     if (ok) ok = cudaMemset(ctx->status_dev, 0, sizeof(uint32_t)) == cudaSuccess &&
                  cudaMemset(ctx->plan_scalars, 0, PS_COUNT * sizeof(int32_t)) == cudaSuccess &&
-                 cudaMemset(ctx->copy_tickets, 0, 8 * sizeof(unsigned)) == cudaSuccess;
+                 cudaMemset(ctx->copy_tickets, 0, 128 * sizeof(unsigned)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         cascade_destroy(ctx);

@@ -43,7 +43,8 @@ struct cascade_ctx {
     int copy_piece;              // >0: piece size in bytes of the TMA ring (8192 | 16384 | 32768); 0 = picked per call
     int copy_ring_kb;            // >0: shared memory of the TMA ring in KiB (64..128); 0 = 128 (host) / 96 (device)
     int copy_dynamic;            // 1: the TMA ring hands its pieces out on demand (a counter) instead of by a fixed stride
-    unsigned *copy_tickets;      // device: two counters per role of the ring kernel, zero between launches
+    unsigned *copy_tickets;      // device: 64 pairs of counters, one pair per launch of the ring kernel in turn, zero between uses
+    unsigned copy_ticket_seq;    // launches so far
     int pdl;                     // 1: programmatic dependent launch between the calls' kernels
     void *sort_runs, *sort_sorted;   // queues beyond 32768 requests: the ordered runs and the merged order (16 B per request each)
     int multi_sort;              // 1: such queues are ordered as runs of 16384 by one cluster each, then merged by rank

@@ -480,6 +480,16 @@ void fill_copy_args(CopyArgs &a, const cascade_ctx *ctx, const cascade_kv_layout
     a.stall = ctx->test_move_stall;
 }
 
+// Work counters of one ring launch: a pair out of a small pool, taken in turn, so that two launches that overlap (the
+// two grids of the fused move; launches a caller put on two streams against the rule) never share one.  A pair is
+// zero whenever no launch is using it: the last CTA out resets it.
+constexpr int kTicketPairs = 64;
+
+unsigned *next_ticket(cascade_ctx *ctx) {
+    if (!ctx->copy_dynamic) return nullptr;
+    return ctx->copy_tickets + 2 * (ctx->copy_ticket_seq++ % kTicketPairs);
+}
+
 // the ring kernels need more dynamic shared memory than the default limit: opt in once per device
 template <int kRole>
 cudaError_t configure_ring(int device) {
@@ -517,7 +527,7 @@ int launch_copy(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged, char 
         if (grid < 1) grid = 1;
         if (grid > items) grid = items;
         constexpr int role = kRestore ? kRoleRestore : kRoleEvict;
-        a.ticket = ctx->copy_dynamic ? ctx->copy_tickets + 2 * role : nullptr;
+        a.ticket = next_ticket(ctx);
         CASCADE_CUDA_TRY(ctx, configure_ring<role>(ctx->device));
         CASCADE_CUDA_TRY(ctx, cascade_launch(ctx->pdl, 0, dim3((unsigned)grid), dim3(32), (size_t)a.ring_bytes, s,
                                              kv_ring_kernel<role>, a));
@@ -623,10 +633,8 @@ extern "C" int cascade_kv_move(cascade_ctx *ctx, const cascade_kv_layout *hbm, v
     fill_copy_args(r, ctx, hbm, (char *)hbm_pool, (char *)host_pool, host_blocks, restore_src, restore_dst,
                    n_restore_dev, n_restore_max);
     e.ring_bytes = r.ring_bytes = ctx->copy_ring_kb > 0 ? ctx->copy_ring_kb * 1024 : kRingHost;
-    if (ctx->copy_dynamic) {
-        e.ticket = ctx->copy_tickets + 2 * kRoleMoveEvict;
-        r.ticket = ctx->copy_tickets + 2 * kRoleMoveRestore;
-    }
+    e.ticket = next_ticket(ctx);
+    r.ticket = next_ticket(ctx);
     e.done = r.done = p.done;
     e.dep = r.dep = p.dep;
     e.skipped = r.skipped = p.skipped;
@@ -719,7 +727,7 @@ int launch_staged_pass(cascade_ctx *ctx, const cascade_kv_layout *l, char *paged
     long long grid = (long long)ctx->num_sms * 2;
     if (grid > items) grid = items;
     constexpr int role = kRestore ? kRoleRestore : kRoleEvict;
-    a.ticket = ctx->copy_dynamic ? ctx->copy_tickets + 2 * role : nullptr;
+    a.ticket = next_ticket(ctx);
     CASCADE_CUDA_TRY(ctx, configure_ring<role>(ctx->device));
     CASCADE_CUDA_TRY(ctx, cascade_launch(false, 0, dim3((unsigned)grid), dim3(32), (size_t)a.ring_bytes, s,
                                          kv_ring_kernel<role>, a));

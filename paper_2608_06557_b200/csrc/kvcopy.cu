@@ -357,10 +357,16 @@ __global__ void __launch_bounds__(32) kv_ring_kernel(const __grid_constant__ Cop
     }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (st) atomicOr(a.status, st);
-    // the last CTA out leaves the two counters at zero for the next launch (every CTA has made its last claim by then)
-    if (on_demand && atomicAdd(a.ticket + 1, 1u) == gridDim.x - 1) {
-        a.ticket[0] = 0;
-        a.ticket[1] = 0;
+    // The last CTA out leaves the two counters at zero for the next launch that uses them.  Every CTA has made its last
+    // claim by then: the test of `next` waits for the value of this CTA's last claim (also on the give-up path, where
+    // nothing else reads it), and the fences keep the claim, the count of CTAs that are done and the reset in this order.
+    if (on_demand && next >= 0) {
+        __threadfence();
+        if (atomicAdd(a.ticket + 1, 1u) == gridDim.x - 1) {
+            __threadfence();
+            a.ticket[0] = 0;
+            a.ticket[1] = 0;
+        }
     }
     // completion of this grid must imply completion of the evict grid it ran beside
     if (kRole == kRoleMoveRestore) cascade_grid_wait();

@@ -175,3 +175,38 @@ def test_ordering_with_random_runs_of_equal_high_bits():
         torch.cuda.synchronize()
         assert np.array_equal(inst.order[:n].cpu().numpy(), np.argsort(key, kind="stable")), (trial, n, pool)
     assert inst.ctx.status()[0] == 0
+
+
+def test_many_long_copies_in_a_row_on_one_context():
+    """Long calls of the copy ring hand their pieces out through a pair of counters that the last CTA leaves at zero;
+    the context owns 64 such pairs and gives them to its launches in turn.  150 calls in a row (every pair used more
+    than twice), evictions and restores with fresh random lists, each long enough for the on-demand form, no host
+    synchronisation in between: the pools must equal the oracle's after the same sequence."""
+    import torch
+    from paper_2608_06557_b200 import cascade as cs
+    n_chunks, cb = 8, 16384
+    bb = n_chunks * cb
+    n_hbm, n_host = 400, 400
+    lay = wl.kv_layout(n_hbm, n_chunks, cb)
+    rng = np.random.default_rng(77)
+    hbm_np = rng.integers(0, 256, n_hbm * bb, dtype=np.uint8)
+    host_np = rng.integers(0, 256, n_host * bb, dtype=np.uint8)
+    hbm, host = torch.from_numpy(hbm_np.copy()).cuda(), torch.from_numpy(host_np.copy()).pin_memory()
+    ctx = cs.Context(wl.default_params(), 16, 0)
+    layout = cs.make_layout(lay)
+    keep = []
+    for call in range(150):
+        n = int(rng.integers(140, 200))                     # 1120 .. 1600 pieces: more than sixteen per CTA
+        h = rng.permutation(n_hbm)[:n].astype(np.int32)
+        o = rng.permutation(n_host)[:n].astype(np.int32)
+        th, to = torch.from_numpy(h).cuda(), torch.from_numpy(o).cuda()
+        keep.append((th, to))
+        if call % 2 == 0:
+            ctx.kv_evict(layout, hbm, host, n_host, False, th, to, None, n)
+            assert oracle.kv_evict(hbm_np, lay, host_np, n_host, h, o) == 0
+        else:
+            ctx.kv_restore(layout, hbm, host, n_host, False, to, th, None, n)
+            assert oracle.kv_restore(hbm_np, lay, host_np, n_host, o, h) == 0
+    torch.cuda.synchronize()
+    assert ctx.status()[0] == 0
+    assert np.array_equal(hbm.cpu().numpy(), hbm_np) and np.array_equal(host.numpy(), host_np)

@@ -122,6 +122,42 @@ def test_bad_ids_are_skipped_and_flagged():
     assert np.array_equal(rig.host.cpu().numpy(), rig.host_np)
 
 
+def test_bad_ids_in_a_long_list_are_skipped_and_flagged():
+    """The same on a call long enough for the ring to hand its pieces out on demand (more than sixteen pieces per CTA),
+    over the host link and through the staging buffer, with ids below zero and beyond either pool scattered through
+    both lists, and with a device-side count shorter than the list."""
+    rig = CopyRig(260, 260, 8, 16384)
+    torch = rig.torch
+    rng = np.random.default_rng(9)
+    n = 250
+    src = rng.permutation(260)[:n].astype(np.int32)
+    dst = rng.permutation(260)[:n].astype(np.int32)
+    for k, v in ((3, -1), (40, 260), (41, 1 << 30), (199, -7)):
+        src[k] = v
+    for k, v in ((7, -2), (120, 260), (233, 99999)):
+        dst[k] = v
+    live = 240                                                   # the last ten entries are beyond the device count
+    count = torch.tensor([live], dtype=torch.int32, device="cuda")
+    for on_device in (False, True):
+        rec = rig.stage if on_device else rig.host
+        ref = rig.hbm_np.copy()
+        st = oracle.kv_restore(ref, rig.lay, rig.host_np, 260, src[:live], dst[:live])
+        rig.hbm.copy_(torch.from_numpy(rig.hbm_np))
+        rig.ctx.kv_restore(rig.layout, rig.hbm, rec, 260, on_device, rig.ids(src), rig.ids(dst), count, n)
+        torch.cuda.synchronize()
+        assert np.array_equal(rig.hbm.cpu().numpy(), ref), on_device
+        assert rig.ctx.status(clear=True)[0] == st == 1
+        ref_rec = rig.host_np.copy()
+        st = oracle.kv_evict(rig.hbm_np, rig.lay, ref_rec, 260, dst[:live], src[:live])
+        rig.hbm.copy_(torch.from_numpy(rig.hbm_np))
+        rec.copy_(torch.from_numpy(rig.host_np))
+        rig.ctx.kv_evict(rig.layout, rig.hbm, rec, 260, on_device, rig.ids(dst), rig.ids(src), count, n)
+        torch.cuda.synchronize()
+        assert np.array_equal(rec.cpu().numpy(), ref_rec), on_device
+        assert rig.ctx.status(clear=True)[0] == st == 1
+    assert rig.guards_intact()
+
+
 def test_layout_validation_on_the_host():
     rig = CopyRig(8, 8, 2, 64)
     cs = rig.cs
